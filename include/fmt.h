@@ -1,0 +1,200 @@
+/*
+ * fmt - vocabulary masking for grammar-constrained decoding on one NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-step token mask of "Earley-Driven Dynamic Pruning for
+ * Efficient Structured Decoding" (ZapFormat / Formatron): every vocabulary token's bytes are
+ * fed through each sequence's pruned Earley chart and the token is valid iff the chart stays
+ * non-empty (Sections 3.2, 3.3, 4.1, 4.2 of the paper).
+ *
+ * Conventions
+ *  - Every function returns fmt_status (FMT_OK = 0).  No exception crosses this boundary.
+ *    fmt_last_error() gives a thread-local message for the last non-OK return.
+ *  - Pointers named *_dev are DEVICE pointers, all others are HOST pointers.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All device
+ *    work is enqueued on it; unless stated otherwise a call does not synchronize.
+ *  - Handles (fmt_grammar, fmt_state) are owned by the library and freed by the matching
+ *    destroy.  Caller buffers are never freed or kept beyond the stream work of the call.
+ *  - Per-row problems (a rejected token, a finished row, a capacity overflow) are data: they
+ *    are written to the caller's status array and the call itself still returns FMT_OK.
+ *  - One fmt_state must be used from one stream at a time.
+ *
+ * Grammar text (Section 3.1: rules A -> alpha over terminals and non-terminals; terminals here
+ * are single bytes or byte classes, i.e. the grammar is scannerless):
+ *     name ::= alternative ( "|" alternative )*
+ *     items: "literal"  [class]  [^negated]  name  ( group )  postfix * + ?   # comment
+ *     escapes: \xHH \n \r \t \\ \" \] \- \^ ; "" is the empty string
+ *
+ * Mask format (Section 3.3): ceil(V/32) uint32 words per row; bit (t & 31) of word (t >> 5)
+ * is 1 iff token t may come next; padding bits are 0.  The EOS token is valid iff the bytes so
+ * far form a complete sentence.  Any other token with no bytes is never valid.
+ */
+#ifndef FMT_H_
+#define FMT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FMT_OK = 0,
+  FMT_ERR_INVALID_ARG = 1,
+  FMT_ERR_GRAMMAR_SYNTAX = 2,
+  FMT_ERR_UNDEFINED_SYMBOL = 3,
+  FMT_ERR_EMPTY_LANGUAGE = 4,
+  FMT_ERR_OOM = 5,
+  FMT_ERR_CUDA = 6,
+  FMT_ERR_CAPACITY = 7,       /* a chart, set or table outgrew its configured capacity */
+  FMT_ERR_TOKEN_REJECTED = 8, /* per row: the token is not valid in the current state */
+  FMT_ERR_FINISHED = 9        /* per row: EOS was already taken */
+} fmt_status;
+
+typedef enum { FMT_BF16 = 0, FMT_FP32 = 1 } fmt_dtype;
+
+typedef struct fmt_grammar fmt_grammar;
+typedef struct fmt_state fmt_state;
+
+/* Options of fmt_compile.  Zero-initialise, then set what you need; 0 means "default". */
+typedef struct {
+  uint32_t host_only;        /* 1: build the tables on the host only (no device needed; the
+                                grammar can be inspected but no state can be created) */
+  uint32_t unit_max_nodes;   /* trie subtrees larger than this are split into several work
+                                units (default 192) */
+  uint32_t reserved[6];
+} fmt_compile_options;
+
+/* Options of fmt_state_create.  Zero-initialise; 0 means "default". */
+typedef struct {
+  uint32_t cache_disable;     /* 1: no state cache: every fill recomputes its mask */
+  uint32_t max_states;        /* state-cache entries (default 65536) */
+  uint32_t max_mask_rows;     /* cached mask rows (default 8192) */
+  uint32_t chart_words;       /* capacity of one row's chart in uint32 words (default 65536) */
+  uint64_t pool_words;        /* uint32 words of chart storage for the cache (default 64 Mi) */
+  uint32_t reserved[6];
+} fmt_state_options;
+
+typedef struct {
+  uint32_t n_nonterminals;   /* after useless-rule removal, including the augmented start */
+  uint32_t n_rules;          /* productions kept (empty ones are folded into nullability) */
+  uint32_t n_dotted;         /* dotted-rule positions D */
+  uint32_t n_classes;        /* distinct byte classes */
+  uint32_t n_nullable;       /* nullable non-terminals */
+  uint32_t vocab_size;       /* V */
+  uint32_t mask_words;       /* ceil(V/32) */
+  uint32_t trie_nodes;       /* T, including the root */
+  uint32_t trie_depth;       /* longest token in bytes */
+  uint32_t n_units;          /* work units of the mask kernel */
+  uint32_t n_empty_tokens;   /* tokens with no bytes (EOS included) */
+  uint32_t start_nullable;   /* 1 if the empty string is a sentence */
+} fmt_grammar_info;
+
+typedef struct {
+  uint64_t steps_advanced;     /* row-advances that changed a chart */
+  uint64_t fills;              /* rows asked for a mask */
+  uint64_t fills_computed;     /* rows whose mask was computed by the trie walk */
+  uint64_t fills_from_cache;   /* rows served from a cached mask */
+  uint64_t fills_shared;       /* rows that shared another row's mask computed in the same call */
+  uint64_t states_cached;      /* distinct pruned charts held by the cache */
+  uint64_t mask_rows_cached;
+  uint64_t pool_words_used;
+  uint64_t chart_items_max;    /* largest pruned chart seen (items) */
+  uint64_t chart_sets_max;     /* most live Earley sets seen in one chart */
+  uint64_t capacity_errors;
+  uint64_t big_mode_units;     /* work units redone with the large scratch area */
+} fmt_stats;
+
+/*
+ * Build the device tables of a grammar and the byte trie of a vocabulary.
+ * Paper: Section 3.1 (CFG), Section 4.5 (useless rules removed, null rules folded into the
+ * prediction tables), Section 4.1 (the vocabulary is what is checked every step).
+ *   ebnf, ebnf_len    grammar text (host), need not be NUL-terminated
+ *   start_rule        NUL-terminated name of the start rule
+ *   vocab_bytes       concatenated token bytes (host); vocab_offsets has V+1 entries, token t
+ *                     is vocab_bytes[vocab_offsets[t] .. vocab_offsets[t+1])
+ *   eos_token_id      id of the end-of-sequence token, or -1 for none
+ *   opt               may be NULL
+ * Errors: INVALID_ARG, GRAMMAR_SYNTAX, UNDEFINED_SYMBOL, EMPTY_LANGUAGE (the start rule derives
+ * no string), CAPACITY (more than 65535 dotted rules, more than 4096 non-terminals, or a token
+ * longer than 32 bytes), OOM, CUDA.
+ * The grammar is immutable and may be shared by any number of states.
+ */
+fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule, const uint8_t* vocab_bytes,
+                       const uint64_t* vocab_offsets, uint32_t V, int32_t eos_token_id,
+                       const fmt_compile_options* opt, fmt_grammar** out);
+void fmt_grammar_destroy(fmt_grammar* g);
+
+/* Sizes of the compiled grammar (host data; works for host_only grammars too). */
+fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out);
+
+/*
+ * Copy one host-side table of the compiled grammar, for inspection and tests.
+ *   which: 0 trie child_off [T+1] u32   1 trie node_byte [T] u8    2 trie parent [T] u32
+ *          3 trie tok_off [T+1] u32     4 trie tok_ids u32         5 unit_node [U] u32
+ *          6 nullable flags [N] u8      7 item info [D] u32        8 item lhs [D] u16
+ *          9 unit_kind [U] u8 (0 = whole subtree, 1 = the node alone)
+ * Writes min(cap_bytes, size) bytes to `out` (may be NULL) and the full size to *size_bytes.
+ */
+fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, size_t cap_bytes, size_t* size_bytes);
+
+/*
+ * Create `batch` sequences, all at the start of the grammar (Earley set S[0], Section 3.2).
+ * Runs a small kernel on `stream` and synchronizes it once.  opt may be NULL.
+ */
+fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_state_options* opt, void* stream,
+                            fmt_state** out);
+void fmt_state_destroy(fmt_state* s);
+
+/* Put rows `rows_dev[0..n)` (DEVICE array of row indices; NULL = rows 0..n-1) back to the start. */
+fmt_status fmt_state_reset(fmt_state* s, const uint32_t* rows_dev, uint32_t n, void* stream);
+
+/*
+ * Advance every row by its chosen token (Section 3.2 scan / complete / predict per byte, with
+ * the Compact step of Section 4.2.3 between complete and predict; the resulting pruned chart
+ * is looked up in the state cache, Section 5.2 "state cache").
+ *   token_ids_dev  [batch] int32 on the device; -1 leaves the row alone
+ *   status_dev     [batch] int32 on the device or NULL; receives FMT_OK, FMT_ERR_TOKEN_REJECTED
+ *                  (row unchanged), FMT_ERR_FINISHED, FMT_ERR_INVALID_ARG (id out of range) or
+ *                  FMT_ERR_CAPACITY (row unchanged; its later masks are all-zero)
+ * Taking EOS in an accepting state finishes the row: its mask is then the EOS bit alone.
+ */
+fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t* status_dev, void* stream);
+
+/*
+ * Write the mask of every row (Sections 3.3, 4.1): mask_dev[row * stride_words + w].
+ * stride_words >= ceil(V/32).  Rows whose pruned chart is in the state cache copy the cached
+ * mask; the others walk the vocabulary trie.
+ */
+fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, void* stream);
+
+/*
+ * Section 3.3: set the logits of invalid tokens to -inf (bf16 0xFF80, fp32 0xFF800000); valid
+ * entries keep their bits.  logits_dev[row * row_stride_elems + t], t < V.
+ */
+fmt_status fmt_apply_mask(const uint32_t* mask_dev, size_t stride_words, void* logits_dev, fmt_dtype dtype,
+                          uint32_t batch, uint32_t V, size_t row_stride_elems, void* stream);
+
+/* fmt_fill_mask followed by fmt_apply_mask without a second pass over the mask in HBM:
+ * the logits are masked straight from the cached mask rows.  mask_dev may be NULL. */
+fmt_status fmt_fill_and_apply(fmt_state* s, uint32_t* mask_dev_or_null, size_t stride_words, void* logits_dev,
+                              fmt_dtype dtype, size_t row_stride_elems, void* stream);
+
+/* Forget every cached chart and mask (rows keep their current charts). */
+fmt_status fmt_state_cache_clear(fmt_state* s, void* stream);
+
+/* Per-row summary, written to host arrays (any may be NULL); synchronizes `stream`.
+ *   accepting[batch] u8, finished[batch] u8 (1 finished, 2 broken by a capacity error),
+ *   n_sets[batch] u32, n_items[batch] u32, state_id[batch] i32 (-1 = not in the cache) */
+fmt_status fmt_state_query(fmt_state* s, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets,
+                           uint32_t* n_items, int32_t* state_id, void* stream);
+
+/* Counters since creation; synchronizes `stream`. */
+fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream);
+
+const char* fmt_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FMT_H_ */

@@ -1,0 +1,587 @@
+// Grammar text -> reduced grammar -> flat tables; vocabulary -> CSR byte trie and work units.
+//
+// Follows the paper's Section 3.1 (rules A -> alpha), Section 4.5 (remove useless rules; handle
+// rules deriving the empty string once, at compile time) and Section 4.1 (the whole vocabulary
+// is checked each step, hence the trie).  Repetition is desugared into LEFT recursion so that
+// the pruned chart of a list does not grow with the list's length (rules of the form A -> B a
+// are the ones whose history can be dropped, Section 4.1).
+#include <algorithm>
+#include <array>
+#include <cctype>
+#include <cstring>
+#include <map>
+
+#include "../../include/fmt.h"
+#include "host_tables.h"
+
+namespace fmt {
+namespace {
+
+using Bits256 = std::array<uint32_t, 8>;
+
+// ------------------------------------------------------------------------------------ lexer
+
+enum class Tok { Ident, Define, Bar, LParen, RParen, Star, Plus, Question, Literal, Class, End };
+
+struct Lexeme {
+  Tok kind;
+  std::string text;  // Ident name / Literal bytes
+  Bits256 cls;       // Class
+  size_t pos;
+};
+
+class Lexer {
+ public:
+  Lexer(const char* s, size_t n) : s_(s), n_(n) {}
+
+  std::vector<Lexeme> run() {
+    std::vector<Lexeme> out;
+    for (;;) {
+      blank();
+      if (p_ >= n_) break;
+      size_t at = p_;
+      unsigned char c = (unsigned char)s_[p_];
+      if (c == ':' && p_ + 2 < n_ && s_[p_ + 1] == ':' && s_[p_ + 2] == '=') {
+        p_ += 3;
+        out.push_back(simple(Tok::Define, at));
+      } else if (c == '|') {
+        ++p_, out.push_back(simple(Tok::Bar, at));
+      } else if (c == '(') {
+        ++p_, out.push_back(simple(Tok::LParen, at));
+      } else if (c == ')') {
+        ++p_, out.push_back(simple(Tok::RParen, at));
+      } else if (c == '*') {
+        ++p_, out.push_back(simple(Tok::Star, at));
+      } else if (c == '+') {
+        ++p_, out.push_back(simple(Tok::Plus, at));
+      } else if (c == '?') {
+        ++p_, out.push_back(simple(Tok::Question, at));
+      } else if (c == '"') {
+        out.push_back(literal());
+      } else if (c == '[') {
+        out.push_back(byte_class());
+      } else if (isalpha(c) || c == '_') {
+        size_t q = p_ + 1;
+        while (q < n_ && (isalnum((unsigned char)s_[q]) || s_[q] == '_' || s_[q] == '-')) ++q;
+        Lexeme l = simple(Tok::Ident, at);
+        l.text.assign(s_ + p_, q - p_);
+        out.push_back(l);
+        p_ = q;
+      } else {
+        throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "unexpected byte at offset " + std::to_string(at)};
+      }
+    }
+    out.push_back(simple(Tok::End, n_));
+    return out;
+  }
+
+ private:
+  const char* s_;
+  size_t n_, p_ = 0;
+
+  static Lexeme simple(Tok k, size_t at) {
+    Lexeme l;
+    l.kind = k;
+    l.cls.fill(0);
+    l.pos = at;
+    return l;
+  }
+  void blank() {
+    while (p_ < n_) {
+      if (s_[p_] == '#') {
+        while (p_ < n_ && s_[p_] != '\n') ++p_;
+      } else if (s_[p_] == ' ' || s_[p_] == '\t' || s_[p_] == '\n' || s_[p_] == '\r') {
+        ++p_;
+      } else {
+        return;
+      }
+    }
+  }
+  static int hex(unsigned char c) {
+    if (c >= '0' && c <= '9') return c - '0';
+    c |= 0x20;
+    if (c >= 'a' && c <= 'f') return c - 'a' + 10;
+    return -1;
+  }
+  unsigned char escaped() {  // p_ is just past the backslash
+    if (p_ >= n_) throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "backslash at end of text"};
+    unsigned char c = (unsigned char)s_[p_++];
+    if (c == 'n') return 10;
+    if (c == 'r') return 13;
+    if (c == 't') return 9;
+    if (c == 'x') {
+      int a = p_ < n_ ? hex((unsigned char)s_[p_]) : -1, b = p_ + 1 < n_ ? hex((unsigned char)s_[p_ + 1]) : -1;
+      if (a < 0 || b < 0) throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "bad \\x escape at offset " + std::to_string(p_)};
+      p_ += 2;
+      return (unsigned char)(a * 16 + b);
+    }
+    return c;
+  }
+  Lexeme literal() {
+    Lexeme l = simple(Tok::Literal, p_);
+    ++p_;
+    while (true) {
+      if (p_ >= n_) throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "literal not closed (offset " + std::to_string(l.pos) + ")"};
+      unsigned char c = (unsigned char)s_[p_++];
+      if (c == '"') break;
+      l.text.push_back((char)(c == '\\' ? escaped() : c));
+    }
+    return l;
+  }
+  Lexeme byte_class() {
+    Lexeme l = simple(Tok::Class, p_);
+    ++p_;
+    bool invert = false;
+    if (p_ < n_ && s_[p_] == '^') invert = true, ++p_;
+    while (true) {
+      if (p_ >= n_) throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "class not closed (offset " + std::to_string(l.pos) + ")"};
+      unsigned char c = (unsigned char)s_[p_++];
+      if (c == ']') break;
+      unsigned lo = (c == '\\') ? escaped() : c, hi = lo;
+      if (p_ + 1 < n_ && s_[p_] == '-' && s_[p_ + 1] != ']') {
+        ++p_;
+        unsigned char e = (unsigned char)s_[p_++];
+        hi = (e == '\\') ? escaped() : e;
+        if (hi < lo) throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "range out of order (offset " + std::to_string(p_) + ")"};
+      }
+      for (unsigned b = lo; b <= hi; ++b) l.cls[b >> 5] |= 1u << (b & 31);
+    }
+    if (invert)
+      for (auto& w : l.cls) w = ~w;
+    bool any = false;
+    for (auto w : l.cls) any |= (w != 0);
+    if (!any) throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "empty byte class (offset " + std::to_string(l.pos) + ")"};
+    return l;
+  }
+};
+
+// ------------------------------------------------------------------------------------ parser
+
+// symbol: >= 0 non-terminal id, < 0 terminal class ~id
+struct Production {
+  int lhs;
+  std::vector<int> rhs;
+};
+
+class GrammarBuilder {
+ public:
+  std::vector<std::string> names;
+  std::vector<char> defined;
+  std::vector<Production> prods;
+  std::vector<Bits256> classes;
+
+  int nt(const std::string& name) {
+    auto it = ids_.find(name);
+    if (it != ids_.end()) return it->second;
+    int id = (int)names.size();
+    ids_[name] = id;
+    names.push_back(name);
+    defined.push_back(0);
+    return id;
+  }
+  int lookup(const std::string& name) const {
+    auto it = ids_.find(name);
+    return it == ids_.end() ? -1 : it->second;
+  }
+  int fresh(const std::string& hint) {
+    std::string nm = hint + "~" + std::to_string(++counter_);
+    int id = nt(nm);
+    defined[id] = 1;
+    return id;
+  }
+  int terminal(const Bits256& b) {
+    auto it = class_ids_.find(b);
+    if (it != class_ids_.end()) return ~it->second;
+    int id = (int)classes.size();
+    classes.push_back(b);
+    class_ids_[b] = id;
+    return ~id;
+  }
+
+ private:
+  std::map<std::string, int> ids_;
+  std::map<Bits256, int> class_ids_;
+  int counter_ = 0;
+};
+
+class Parser {
+ public:
+  Parser(std::vector<Lexeme> lx, GrammarBuilder& b) : lx_(std::move(lx)), b_(b) {}
+
+  void run() {
+    if (lx_[0].kind == Tok::End) throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "the grammar has no rules"};
+    while (lx_[i_].kind != Tok::End) {
+      if (!rule_starts_here())
+        throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "expected `name ::=` at offset " + std::to_string(lx_[i_].pos)};
+      int lhs = b_.nt(lx_[i_].text);
+      b_.defined[lhs] = 1;
+      ctx_ = lx_[i_].text;
+      i_ += 2;
+      alternatives(lhs);
+    }
+  }
+
+ private:
+  std::vector<Lexeme> lx_;
+  GrammarBuilder& b_;
+  size_t i_ = 0;
+  std::string ctx_;
+
+  bool rule_starts_here() const { return lx_[i_].kind == Tok::Ident && lx_[i_ + 1].kind == Tok::Define; }
+
+  void alternatives(int lhs) {
+    for (;;) {
+      std::vector<int> body = sequence();
+      b_.prods.push_back({lhs, body});
+      if (lx_[i_].kind == Tok::Bar) {
+        ++i_;
+        continue;
+      }
+      break;
+    }
+  }
+  std::vector<int> sequence() {
+    std::vector<int> out;
+    for (;;) {
+      Tok k = lx_[i_].kind;
+      if (k == Tok::End || k == Tok::Bar || k == Tok::RParen || rule_starts_here()) break;
+      std::vector<int> piece = postfixed();
+      out.insert(out.end(), piece.begin(), piece.end());
+    }
+    return out;
+  }
+  std::vector<int> postfixed() {
+    std::vector<int> unit = primary();
+    for (;;) {
+      Tok k = lx_[i_].kind;
+      if (k == Tok::Star) {  // X -> empty | X unit
+        int x = b_.fresh(ctx_);
+        std::vector<int> rec{x};
+        rec.insert(rec.end(), unit.begin(), unit.end());
+        b_.prods.push_back({x, {}});
+        b_.prods.push_back({x, rec});
+        unit = {x};
+      } else if (k == Tok::Plus) {  // X -> unit | X unit
+        int x = b_.fresh(ctx_);
+        std::vector<int> rec{x};
+        rec.insert(rec.end(), unit.begin(), unit.end());
+        b_.prods.push_back({x, unit});
+        b_.prods.push_back({x, rec});
+        unit = {x};
+      } else if (k == Tok::Question) {  // X -> empty | unit
+        int x = b_.fresh(ctx_);
+        b_.prods.push_back({x, {}});
+        b_.prods.push_back({x, unit});
+        unit = {x};
+      } else {
+        break;
+      }
+      ++i_;
+    }
+    return unit;
+  }
+  std::vector<int> primary() {
+    const Lexeme l = lx_[i_];
+    switch (l.kind) {
+      case Tok::Literal: {
+        ++i_;
+        std::vector<int> out;
+        for (unsigned char c : l.text) {
+          Bits256 one;
+          one.fill(0);
+          one[c >> 5] = 1u << (c & 31);
+          out.push_back(b_.terminal(one));
+        }
+        return out;
+      }
+      case Tok::Class:
+        ++i_;
+        return {b_.terminal(l.cls)};
+      case Tok::Ident:
+        ++i_;
+        return {b_.nt(l.text)};
+      case Tok::LParen: {
+        ++i_;
+        size_t first = b_.prods.size();
+        int x = b_.fresh(ctx_);
+        alternatives(x);
+        if (lx_[i_].kind != Tok::RParen)
+          throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "expected ) at offset " + std::to_string(lx_[i_].pos)};
+        ++i_;
+        // a group with one alternative is spliced in place
+        size_t count = 0, where = 0;
+        for (size_t p = first; p < b_.prods.size(); ++p)
+          if (b_.prods[p].lhs == x) ++count, where = p;
+        if (count == 1) {
+          std::vector<int> body = b_.prods[where].rhs;
+          b_.prods.erase(b_.prods.begin() + (long)where);
+          return body;
+        }
+        return {x};
+      }
+      default:
+        throw CompileError{FMT_ERR_GRAMMAR_SYNTAX, "unexpected token at offset " + std::to_string(l.pos)};
+    }
+  }
+};
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------ tables
+
+void compile_grammar(const char* text, size_t len, const std::string& start, HostTables& out) {
+  GrammarBuilder b;
+  int aug = b.nt("$");
+  b.defined[aug] = 1;
+  {
+    Lexer lx(text, len);
+    Parser ps(lx.run(), b);
+    ps.run();
+  }
+  for (size_t i = 0; i < b.names.size(); ++i)
+    if (!b.defined[i]) throw CompileError{FMT_ERR_UNDEFINED_SYMBOL, "undefined symbol '" + b.names[i] + "'"};
+  int start_id = b.lookup(start);
+  if (start_id < 0) throw CompileError{FMT_ERR_UNDEFINED_SYMBOL, "start rule '" + start + "' is not defined"};
+  b.prods.insert(b.prods.begin(), Production{aug, {start_id}});
+
+  const size_t n_all = b.names.size();
+  // productive non-terminals
+  std::vector<char> productive(n_all, 0);
+  for (bool again = true; again;) {
+    again = false;
+    for (auto& p : b.prods) {
+      if (productive[p.lhs]) continue;
+      bool ok = true;
+      for (int s : p.rhs) ok = ok && (s < 0 || productive[s]);
+      if (ok) productive[p.lhs] = 1, again = true;
+    }
+  }
+  if (!productive[aug]) throw CompileError{FMT_ERR_EMPTY_LANGUAGE, "the start rule derives no string"};
+  std::vector<Production> kept;
+  for (auto& p : b.prods) {
+    bool ok = productive[p.lhs];
+    for (int s : p.rhs) ok = ok && (s < 0 || productive[s]);
+    if (ok) kept.push_back(p);
+  }
+  // reachable from the augmented start
+  std::vector<char> reach(n_all, 0);
+  reach[aug] = 1;
+  for (bool again = true; again;) {
+    again = false;
+    for (auto& p : kept)
+      if (reach[p.lhs])
+        for (int s : p.rhs)
+          if (s >= 0 && !reach[s]) reach[s] = 1, again = true;
+  }
+  std::vector<Production> rules;
+  for (auto& p : kept)
+    if (reach[p.lhs]) rules.push_back(p);
+  // nullable
+  std::vector<char> nullable(n_all, 0);
+  for (bool again = true; again;) {
+    again = false;
+    for (auto& p : rules) {
+      if (nullable[p.lhs]) continue;
+      bool ok = true;
+      for (int s : p.rhs) ok = ok && (s >= 0 && nullable[s]);
+      if (ok) nullable[p.lhs] = 1, again = true;
+    }
+  }
+  // renumber non-terminals ($ = 0) and byte classes (only those still used)
+  std::vector<int> nt_new(n_all, -1);
+  int N = 0;
+  nt_new[aug] = N++;
+  for (auto& p : rules)
+    if (nt_new[p.lhs] < 0) nt_new[p.lhs] = N++;
+  std::vector<int> cls_new(b.classes.size(), -1);
+  int C = 0;
+  for (auto& p : rules)
+    for (int s : p.rhs)
+      if (s < 0 && cls_new[~s] < 0) cls_new[~s] = C++;
+  // empty productions are dropped: their effect lives in the nullable flags
+  std::vector<Production> solid;
+  for (auto& p : rules)
+    if (!p.rhs.empty()) solid.push_back(p);
+  size_t D = 0;
+  for (auto& p : solid) D += p.rhs.size() + 1;
+  if (D > 65535 || N > (int)MAX_NONTERMINALS || C > 65535)
+    throw CompileError{FMT_ERR_CAPACITY, "grammar too large: more than 65535 dotted rules or classes, or 4096 non-terminals"};
+
+  out.N = (uint32_t)N;
+  out.P = (uint32_t)solid.size();
+  out.D = (uint32_t)D;
+  out.C = (uint32_t)C;
+  out.Nw = ((uint32_t)N + 31) / 32;
+  out.nullable.assign(N, 0);
+  out.nt_names.assign(N, "");
+  out.n_nullable = 0;
+  for (size_t i = 0; i < n_all; ++i)
+    if (nt_new[i] >= 0) {
+      out.nullable[nt_new[i]] = (uint8_t)nullable[i];
+      out.nt_names[nt_new[i]] = b.names[i];
+      out.n_nullable += nullable[i] ? 1 : 0;
+    }
+  out.start_nullable = nullable[start_id] != 0;
+  out.class_bits.assign((size_t)std::max(C, 1) * 8, 0);
+  for (size_t c = 0; c < b.classes.size(); ++c)
+    if (cls_new[c] >= 0)
+      for (int w = 0; w < 8; ++w) out.class_bits[(size_t)cls_new[c] * 8 + w] = b.classes[c][w];
+
+  out.info.assign(D, 0);
+  out.lhs.assign(D, 0);
+  out.skip.assign(D, 0);
+  std::vector<std::vector<uint32_t>> first_item(N);  // start item of each rule, per non-terminal
+  uint32_t d = 0;
+  for (auto& p : solid) {  // solid[0] is $ -> start, so items 0 and 1 are the start and accept items
+    int L = nt_new[p.lhs];
+    first_item[L].push_back(d);
+    for (size_t k = 0; k <= p.rhs.size(); ++k, ++d) {
+      out.lhs[d] = (uint16_t)L;
+      if (k == p.rhs.size()) {
+        out.info[d] = (KIND_END << INFO_KIND_SHIFT) | (uint32_t)L;
+      } else if (p.rhs[k] < 0) {
+        out.info[d] = (KIND_TERM << INFO_KIND_SHIFT) | (uint32_t)cls_new[~p.rhs[k]];
+      } else {
+        uint32_t y = (uint32_t)nt_new[p.rhs[k]];
+        out.info[d] = (KIND_NT << INFO_KIND_SHIFT) | y | (out.nullable[y] ? INFO_NULLABLE : 0u);
+      }
+    }
+  }
+  for (uint32_t i = (uint32_t)D; i-- > 0;)
+    if ((out.info[i] >> INFO_KIND_SHIFT) == KIND_NT && (out.info[i] & INFO_NULLABLE))
+      out.skip[i] = (uint8_t)std::min<uint32_t>(255u, 1u + out.skip[i + 1]);
+  // direct items: the start item of every rule plus the items reached by moving the dot over
+  // leading nullable non-terminals; completed items are left out (their effect is the parent's skip)
+  out.direct_off.assign(N + 1, 0);
+  out.direct_items.clear();
+  for (int y = 0; y < N; ++y) {
+    out.direct_off[y] = (uint32_t)out.direct_items.size();
+    for (uint32_t s : first_item[y])
+      for (uint32_t j = 0; j <= out.skip[s]; ++j)
+        if ((out.info[s + j] >> INFO_KIND_SHIFT) != KIND_END) out.direct_items.push_back((uint16_t)(s + j));
+  }
+  out.direct_off[N] = (uint32_t)out.direct_items.size();
+  if (out.direct_items.empty()) out.direct_items.push_back(0);
+  // closure of "predicting Y also predicts Z"
+  out.nt_closure.assign((size_t)N * out.Nw, 0);
+  for (int y = 0; y < N; ++y) {
+    uint32_t* row = &out.nt_closure[(size_t)y * out.Nw];
+    std::vector<int> work{y};
+    row[y >> 5] |= 1u << (y & 31);
+    while (!work.empty()) {
+      int z = work.back();
+      work.pop_back();
+      for (uint32_t k = out.direct_off[z]; k < out.direct_off[z + 1]; ++k) {
+        uint32_t inf = out.info[out.direct_items[k]];
+        if ((inf >> INFO_KIND_SHIFT) == KIND_NT) {
+          uint32_t w = inf & INFO_ARG_MASK;
+          if (!((row[w >> 5] >> (w & 31)) & 1u)) row[w >> 5] |= 1u << (w & 31), work.push_back((int)w);
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------ trie
+
+void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t eos, uint32_t unit_max_nodes,
+                HostTables& out) {
+  out.V = V;
+  out.Wm = (V + 31) / 32;
+  out.eos = eos;
+  out.vocab_off.assign((size_t)V + 1, 0);
+  out.n_empty = 0;
+  for (uint32_t t = 0; t < V; ++t)
+    if (offs[t + 1] < offs[t]) throw CompileError{FMT_ERR_INVALID_ARG, "vocab_offsets must not decrease"};
+  uint64_t total = offs[V] - offs[0];
+  if (total > 0xFFFFFFF0ull) throw CompileError{FMT_ERR_CAPACITY, "vocabulary bytes exceed 4 GiB"};
+  out.vocab_bytes.assign(bytes + offs[0], bytes + offs[V]);
+  if (out.vocab_bytes.empty()) out.vocab_bytes.push_back(0);
+  std::vector<uint32_t> order;
+  order.reserve(V);
+  for (uint32_t t = 0; t < V; ++t) {
+    uint64_t l = offs[t + 1] - offs[t];
+    if (l > MAX_TOKEN_BYTES)
+      throw CompileError{FMT_ERR_CAPACITY, "token " + std::to_string(t) + " is longer than 32 bytes"};
+    out.vocab_off[t] = (uint32_t)(offs[t] - offs[0]);
+    if (l == 0) ++out.n_empty;
+    else order.push_back(t);
+  }
+  out.vocab_off[V] = (uint32_t)total;
+  const uint8_t* base = out.vocab_bytes.data();
+  auto tok_len = [&](uint32_t t) { return out.vocab_off[t + 1] - out.vocab_off[t]; };
+  auto tok_ptr = [&](uint32_t t) { return base + out.vocab_off[t]; };
+  std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+    uint32_t la = tok_len(a), lb = tok_len(b);
+    int c = memcmp(tok_ptr(a), tok_ptr(b), std::min(la, lb));
+    if (c != 0) return c < 0;
+    if (la != lb) return la < lb;
+    return a < b;
+  });
+  // breadth-first construction over ranges of the sorted token list
+  struct Range {
+    uint32_t lo, hi, depth;
+  };
+  out.child_off.clear();
+  out.node_byte.clear();
+  out.parent.clear();
+  out.node_depth.clear();
+  out.tok_off.clear();
+  out.tok_ids.clear();
+  std::vector<Range> nodes;
+  nodes.push_back({0, (uint32_t)order.size(), 0});
+  out.node_byte.push_back(0);
+  out.parent.push_back(0);
+  out.node_depth.push_back(0);
+  out.depth = 0;
+  for (size_t n = 0; n < nodes.size(); ++n) {
+    Range r = nodes[n];
+    out.child_off.push_back((uint32_t)nodes.size());
+    out.tok_off.push_back((uint32_t)out.tok_ids.size());
+    uint32_t i = r.lo;
+    while (i < r.hi && tok_len(order[i]) == r.depth) out.tok_ids.push_back(order[i++]);  // tokens ending here
+    while (i < r.hi) {
+      uint8_t c = tok_ptr(order[i])[r.depth];
+      uint32_t j = i;
+      while (j < r.hi && tok_ptr(order[j])[r.depth] == c) ++j;
+      nodes.push_back({i, j, r.depth + 1});
+      out.node_byte.push_back(c);
+      out.parent.push_back((uint32_t)n);
+      out.node_depth.push_back((uint8_t)(r.depth + 1));
+      out.depth = std::max(out.depth, r.depth + 1);
+      i = j;
+    }
+  }
+  out.T = (uint32_t)nodes.size();
+  out.child_off.push_back(out.T);
+  out.tok_off.push_back((uint32_t)out.tok_ids.size());
+  if (out.tok_ids.empty()) out.tok_ids.push_back(0);
+  // subtree sizes, then split large subtrees into work units
+  std::vector<uint32_t> size(out.T, 1);
+  for (uint32_t n = out.T; n-- > 1;) size[out.parent[n]] += size[n];
+  if (unit_max_nodes == 0) unit_max_nodes = 192;
+  std::vector<std::pair<uint32_t, uint32_t>> units;  // (size, node | kind << 31)
+  std::vector<uint32_t> stack;
+  for (uint32_t c = out.child_off[0]; c < out.child_off[1]; ++c) stack.push_back(c);
+  while (!stack.empty()) {
+    uint32_t n = stack.back();
+    stack.pop_back();
+    if (size[n] <= unit_max_nodes || out.node_depth[n] >= 4) {
+      units.push_back({size[n], n});
+    } else {
+      if (out.tok_off[n + 1] > out.tok_off[n]) units.push_back({1, n | 0x80000000u});
+      for (uint32_t c = out.child_off[n]; c < out.child_off[n + 1]; ++c) stack.push_back(c);
+    }
+  }
+  std::sort(units.begin(), units.end(), [](const std::pair<uint32_t, uint32_t>& a, const std::pair<uint32_t, uint32_t>& b) {
+    return a.first != b.first ? a.first > b.first : a.second < b.second;
+  });
+  out.unit_node.clear();
+  out.unit_kind.clear();
+  for (auto& u : units) {
+    out.unit_node.push_back(u.second & 0x7FFFFFFFu);
+    out.unit_kind.push_back((uint8_t)(u.second >> 31));
+  }
+}
+
+}  // namespace fmt

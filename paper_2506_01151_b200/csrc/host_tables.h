@@ -1,0 +1,62 @@
+// Host-side result of compiling a grammar and a vocabulary: flat integer tables that are
+// uploaded to the device as they are.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+namespace fmt {
+
+// item info word: bits 31..30 kind, bit 29 "post-dot non-terminal is nullable", bits 15..0 argument
+//   END : argument = left-hand side        (dot at the end of the rule)
+//   TERM: argument = byte-class id         (post-dot symbol is a terminal)
+//   NT  : argument = non-terminal id       (post-dot symbol is a non-terminal)
+enum : uint32_t { KIND_END = 0u, KIND_TERM = 1u, KIND_NT = 2u };
+constexpr uint32_t INFO_KIND_SHIFT = 30;
+constexpr uint32_t INFO_NULLABLE = 1u << 29;
+constexpr uint32_t INFO_ARG_MASK = 0xFFFFu;
+constexpr uint32_t ITEM_START = 0;   // $ -> . start
+constexpr uint32_t ITEM_ACCEPT = 1;  // $ -> start .
+constexpr uint32_t MAX_TOKEN_BYTES = 32;
+constexpr uint32_t MAX_NONTERMINALS = 4096;
+
+struct CompileError {
+  int code;
+  std::string msg;
+};
+
+struct HostTables {
+  // ---- grammar (Section 3.1; reduced as in Section 4.5)
+  uint32_t N = 0, P = 0, D = 0, C = 0, Nw = 0, n_nullable = 0;
+  bool start_nullable = false;
+  std::vector<uint32_t> info;          // [D]
+  std::vector<uint16_t> lhs;           // [D] left-hand side of the item's rule
+  std::vector<uint8_t> skip;           // [D] how many nullable non-terminals follow the dot in a row
+  std::vector<uint32_t> class_bits;    // [C][8] 256-bit byte classes
+  std::vector<uint32_t> nt_closure;    // [N][Nw] non-terminals predicted (transitively) with Y
+  std::vector<uint32_t> direct_off;    // [N+1]
+  std::vector<uint16_t> direct_items;  // start items of each non-terminal's rules, dots moved over
+                                       // leading nullable symbols, completed items left out
+  std::vector<uint8_t> nullable;       // [N]
+  std::vector<std::string> nt_names;   // [N]
+  // ---- vocabulary trie in CSR form, nodes in breadth-first order (root = 0)
+  uint32_t V = 0, Wm = 0, T = 0, depth = 0, n_empty = 0;
+  int32_t eos = -1;
+  std::vector<uint32_t> child_off;  // [T+1] children of node n are nodes child_off[n]..child_off[n+1]-1
+  std::vector<uint8_t> node_byte;   // [T]
+  std::vector<uint32_t> parent;     // [T]
+  std::vector<uint8_t> node_depth;  // [T]
+  std::vector<uint32_t> tok_off;    // [T+1] tokens whose bytes end at node n
+  std::vector<uint32_t> tok_ids;
+  std::vector<uint32_t> unit_node;  // work units of the mask kernel, largest first
+  std::vector<uint8_t> unit_kind;   // 0 whole subtree, 1 the node alone
+  std::vector<uint32_t> vocab_off;  // [V+1] byte offsets (32-bit) into vocab_bytes
+  std::vector<uint8_t> vocab_bytes;
+};
+
+// Both throw CompileError.
+void compile_grammar(const char* text, size_t len, const std::string& start, HostTables& out);
+void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t eos, uint32_t unit_max_nodes,
+                HostTables& out);
+
+}  // namespace fmt
