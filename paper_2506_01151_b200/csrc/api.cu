@@ -1,0 +1,394 @@
+// The C-ABI of include/fmt.h: handle management, uploads and kernel launches.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/fmt.h"
+#include "device_tables.h"
+#include "host_tables.h"
+#include "kernels.h"
+
+using namespace fmt;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+fmt_status fail(fmt_status code, const std::string& msg) {
+  g_last_error = msg;
+  return code;
+}
+fmt_status cuda_fail(cudaError_t e, const char* what) {
+  return fail(e == cudaErrorMemoryAllocation ? FMT_ERR_OOM : FMT_ERR_CUDA,
+              std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+struct DeviceBuffers {
+  std::vector<void*> ptrs;
+  ~DeviceBuffers() {
+    for (void* p : ptrs) cudaFree(p);
+  }
+  template <typename T>
+  cudaError_t upload(const std::vector<T>& v, const T** out) {
+    void* p = nullptr;
+    size_t bytes = std::max<size_t>(v.size() * sizeof(T), 16);
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) return e;
+    ptrs.push_back(p);
+    if (!v.empty()) {
+      e = cudaMemcpy(p, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice);
+      if (e != cudaSuccess) return e;
+    }
+    *out = static_cast<const T*>(p);
+    return cudaSuccess;
+  }
+  template <typename T>
+  cudaError_t alloc(size_t count, T** out, int fill_byte) {
+    void* p = nullptr;
+    size_t bytes = std::max<size_t>(count * sizeof(T), 16);
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) return e;
+    ptrs.push_back(p);
+    e = cudaMemset(p, fill_byte, bytes);
+    if (e != cudaSuccess) return e;
+    *out = static_cast<T*>(p);
+    return cudaSuccess;
+  }
+};
+
+}  // namespace
+
+struct fmt_grammar {
+  HostTables host;
+  GrammarDev dev{};
+  bool on_device = false;
+  int device = -1;
+  DeviceBuffers bufs;
+};
+
+struct fmt_state {
+  const fmt_grammar* g = nullptr;
+  StateDev dev{};
+  DeviceBuffers bufs;
+  int32_t* init_state_dev = nullptr;
+  int32_t* result_dev = nullptr;
+  uint8_t* query_dev = nullptr;  // scratch for fmt_state_query
+  int walk_grid = 1;
+};
+
+extern "C" {
+
+const char* fmt_last_error(void) { return g_last_error.c_str(); }
+
+fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule, const uint8_t* vocab_bytes,
+                       const uint64_t* vocab_offsets, uint32_t V, int32_t eos_token_id, const fmt_compile_options* opt,
+                       fmt_grammar** out) {
+  if (!out) return fail(FMT_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (!ebnf || !start_rule || !vocab_offsets || (!vocab_bytes && V > 0 && vocab_offsets[V] > vocab_offsets[0]))
+    return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  if (V == 0) return fail(FMT_ERR_INVALID_ARG, "the vocabulary is empty");
+  if (eos_token_id < -1 || eos_token_id >= (int64_t)V) return fail(FMT_ERR_INVALID_ARG, "eos_token_id out of range");
+  fmt_grammar* g = new (std::nothrow) fmt_grammar;
+  if (!g) return fail(FMT_ERR_OOM, "out of host memory");
+  try {
+    compile_grammar(ebnf, ebnf_len, start_rule, g->host);
+    static const uint8_t none = 0;
+    build_trie(vocab_bytes ? vocab_bytes : &none, vocab_offsets, V, eos_token_id, opt ? opt->unit_max_nodes : 0, g->host);
+    if (eos_token_id >= 0 && vocab_offsets[eos_token_id + 1] != vocab_offsets[eos_token_id])
+      throw CompileError{FMT_ERR_INVALID_ARG, "the EOS token must have no bytes"};
+  } catch (const CompileError& e) {
+    delete g;
+    return fail((fmt_status)e.code, e.msg);
+  } catch (const std::bad_alloc&) {
+    delete g;
+    return fail(FMT_ERR_OOM, "out of host memory");
+  }
+  if (!(opt && opt->host_only)) {
+    const HostTables& h = g->host;
+    GrammarDev& d = g->dev;
+    d.D = h.D, d.N = h.N, d.C = h.C, d.Nw = h.Nw;
+    d.V = h.V, d.Wm = h.Wm, d.T = h.T, d.U = (uint32_t)h.unit_node.size(), d.depth = h.depth;
+    d.eos = h.eos;
+    d.start_nullable = h.start_nullable ? 1u : 0u;
+    cudaError_t e = cudaGetDevice(&g->device);
+#define UP(field) if (e == cudaSuccess) e = g->bufs.upload(h.field, &d.field)
+    UP(info);
+    UP(lhs);
+    UP(skip);
+    UP(class_bits);
+    UP(nt_closure);
+    UP(direct_off);
+    UP(direct_items);
+    UP(child_off);
+    UP(node_byte);
+    UP(parent);
+    UP(node_depth);
+    UP(tok_off);
+    UP(tok_ids);
+    UP(unit_node);
+    UP(unit_kind);
+    UP(vocab_off);
+    UP(vocab_bytes);
+#undef UP
+    if (e != cudaSuccess) {
+      fmt_status st = cuda_fail(e, "uploading the grammar tables");
+      delete g;
+      return st;
+    }
+    g->on_device = true;
+  }
+  *out = g;
+  return FMT_OK;
+}
+
+void fmt_grammar_destroy(fmt_grammar* g) { delete g; }
+
+fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out) {
+  if (!g || !out) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  const HostTables& h = g->host;
+  out->n_nonterminals = h.N;
+  out->n_rules = h.P;
+  out->n_dotted = h.D;
+  out->n_classes = h.C;
+  out->n_nullable = h.n_nullable;
+  out->vocab_size = h.V;
+  out->mask_words = h.Wm;
+  out->trie_nodes = h.T;
+  out->trie_depth = h.depth;
+  out->n_units = (uint32_t)h.unit_node.size();
+  out->n_empty_tokens = h.n_empty;
+  out->start_nullable = h.start_nullable ? 1u : 0u;
+  return FMT_OK;
+}
+
+fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, size_t cap_bytes, size_t* size_bytes) {
+  if (!g || !size_bytes) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  const HostTables& h = g->host;
+  const void* src = nullptr;
+  size_t n = 0;
+  switch (which) {
+    case 0: src = h.child_off.data(), n = (size_t)(h.T + 1) * 4; break;
+    case 1: src = h.node_byte.data(), n = h.T; break;
+    case 2: src = h.parent.data(), n = (size_t)h.T * 4; break;
+    case 3: src = h.tok_off.data(), n = (size_t)(h.T + 1) * 4; break;
+    case 4: src = h.tok_ids.data(), n = (size_t)h.tok_off[h.T] * 4; break;
+    case 5: src = h.unit_node.data(), n = h.unit_node.size() * 4; break;
+    case 6: src = h.nullable.data(), n = h.N; break;
+    case 7: src = h.info.data(), n = (size_t)h.D * 4; break;
+    case 8: src = h.lhs.data(), n = (size_t)h.D * 2; break;
+    case 9: src = h.unit_kind.data(), n = h.unit_kind.size(); break;
+    default: return fail(FMT_ERR_INVALID_ARG, "unknown table");
+  }
+  *size_bytes = n;
+  if (out && cap_bytes) memcpy(out, src, std::min(n, cap_bytes));
+  return FMT_OK;
+}
+
+fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_state_options* opt, void* stream,
+                            fmt_state** out) {
+  if (!out) return fail(FMT_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (!g || batch == 0) return fail(FMT_ERR_INVALID_ARG, "NULL grammar or empty batch");
+  if (!g->on_device) return fail(FMT_ERR_INVALID_ARG, "the grammar was compiled host_only");
+  if (batch > 65535) return fail(FMT_ERR_INVALID_ARG, "batch above 65535");
+  cudaStream_t st = (cudaStream_t)stream;
+  fmt_state* s = new (std::nothrow) fmt_state;
+  if (!s) return fail(FMT_ERR_OOM, "out of host memory");
+  s->g = g;
+  StateDev& d = s->dev;
+  d.B = batch;
+  d.cache_on = (opt && opt->cache_disable) ? 0u : 1u;
+  d.chart_words = (opt && opt->chart_words) ? opt->chart_words : 65536u;
+  if (d.chart_words < 1024) d.chart_words = 1024;
+  d.max_states = (opt && opt->max_states) ? opt->max_states : 65536u;
+  d.max_mask_rows = (opt && opt->max_mask_rows) ? opt->max_mask_rows : 8192u;
+  d.pool_words = (opt && opt->pool_words) ? opt->pool_words : (64ull << 20);
+  if (!d.cache_on) {
+    d.max_states = 1;
+    d.max_mask_rows = 0;
+    d.pool_words = 32;
+  }
+  uint32_t ht = 1024;
+  while (ht < d.max_states * 2u) ht <<= 1;
+  d.ht_mask = ht - 1;
+  d.init_off = (uint64_t)batch * 3u * d.chart_words;
+  d.pool_base = d.init_off + d.chart_words;
+  d.big_arena_items = 1u << 16;
+  d.big_hset_slots = 1u << 13;
+
+  cudaError_t e = configure_kernels();
+  int per_sm = 0, sms = 0, dev = 0;
+  if (e == cudaSuccess) e = walk_blocks_per_sm(&per_sm);
+  if (e == cudaSuccess) e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess && per_sm < 1) {
+    delete s;
+    return fail(FMT_ERR_CUDA, "the walk kernel does not fit on this device");
+  }
+  s->walk_grid = std::max(1, per_sm * sms);
+  const size_t big_words = (size_t)s->walk_grid * walk_warps() * ((size_t)d.big_arena_items + d.big_hset_slots);
+#define AL(ptr, count, fill) if (e == cudaSuccess) e = s->bufs.alloc((size_t)(count), &(ptr), (fill))
+  AL(d.arena, d.pool_base + d.pool_words, 0);
+  AL(d.row_chart, batch, 0);
+  AL(d.row_buf, batch, 0xFF);
+  AL(d.row_state, batch, 0xFF);
+  AL(d.row_flags, batch, 0);
+  AL(d.row_mask, batch, 0xFF);
+  AL(d.ht, ht, 0);
+  AL(d.st_off, d.max_states, 0);
+  AL(d.st_mask, d.max_states, 0xFF);
+  AL(d.mask_rows, ((size_t)batch + d.max_mask_rows) * g->dev.Wm, 0);
+  AL(d.jobs, batch, 0);
+  AL(d.counters, CNT_TOTAL, 0);
+  AL(d.big_scratch, big_words, 0xFF);
+  AL(s->init_state_dev, 4, 0xFF);
+  AL(s->result_dev, 4, 0);
+  AL(s->query_dev, (size_t)batch * 16, 0);
+#undef AL
+  if (e != cudaSuccess) {
+    fmt_status stt = cuda_fail(e, "allocating the sequence state");
+    delete s;
+    return stt;
+  }
+  launch_init(g->dev, d, s->result_dev, st);
+  launch_intern_init(d, s->init_state_dev, st);
+  launch_reset(d, nullptr, batch, s->init_state_dev, st);
+  int32_t result = 0;
+  e = cudaMemcpyAsync(&result, s->result_dev, 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess) e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    fmt_status stt = cuda_fail(e, "building the start chart");
+    delete s;
+    return stt;
+  }
+  if (result != 1) {
+    delete s;
+    return fail(FMT_ERR_CAPACITY, "the start chart does not fit the configured capacities");
+  }
+  *out = s;
+  return FMT_OK;
+}
+
+void fmt_state_destroy(fmt_state* s) { delete s; }
+
+static fmt_status launched(const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, what);
+  return FMT_OK;
+}
+
+fmt_status fmt_state_reset(fmt_state* s, const uint32_t* rows_dev, uint32_t n, void* stream) {
+  if (!s) return fail(FMT_ERR_INVALID_ARG, "NULL state");
+  if (!rows_dev && n > s->dev.B) return fail(FMT_ERR_INVALID_ARG, "n exceeds the batch");
+  launch_reset(s->dev, rows_dev, n, s->init_state_dev, (cudaStream_t)stream);
+  return launched("fmt_state_reset");
+}
+
+fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t* status_dev, void* stream) {
+  if (!s || !token_ids_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  launch_advance(s->g->dev, s->dev, token_ids_dev, status_dev, (cudaStream_t)stream);
+  return launched("fmt_state_advance");
+}
+
+fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, void* stream) {
+  if (!s || !mask_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  if (stride_words < s->g->dev.Wm) return fail(FMT_ERR_INVALID_ARG, "stride_words is smaller than ceil(V/32)");
+  cudaStream_t st = (cudaStream_t)stream;
+  launch_fill(s->g->dev, s->dev, s->walk_grid, st);
+  launch_gather(s->g->dev, s->dev, mask_dev, stride_words, st);
+  launch_end_fill(s->dev, st);
+  return launched("fmt_fill_mask");
+}
+
+fmt_status fmt_apply_mask(const uint32_t* mask_dev, size_t stride_words, void* logits_dev, fmt_dtype dtype,
+                          uint32_t batch, uint32_t V, size_t row_stride_elems, void* stream) {
+  if (!mask_dev || !logits_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  if (dtype != FMT_BF16 && dtype != FMT_FP32) return fail(FMT_ERR_INVALID_ARG, "unknown dtype");
+  if (stride_words < (V + 31) / 32 || row_stride_elems < V) return fail(FMT_ERR_INVALID_ARG, "a stride is too small");
+  if (batch > 65535) return fail(FMT_ERR_INVALID_ARG, "batch above 65535");
+  launch_apply(mask_dev, stride_words, logits_dev, (int)dtype, batch, V, row_stride_elems, (cudaStream_t)stream);
+  return launched("fmt_apply_mask");
+}
+
+fmt_status fmt_fill_and_apply(fmt_state* s, uint32_t* mask_dev_or_null, size_t stride_words, void* logits_dev,
+                              fmt_dtype dtype, size_t row_stride_elems, void* stream) {
+  if (!s || !logits_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  if (dtype != FMT_BF16 && dtype != FMT_FP32) return fail(FMT_ERR_INVALID_ARG, "unknown dtype");
+  if (mask_dev_or_null && stride_words < s->g->dev.Wm)
+    return fail(FMT_ERR_INVALID_ARG, "stride_words is smaller than ceil(V/32)");
+  if (row_stride_elems < s->g->dev.V) return fail(FMT_ERR_INVALID_ARG, "row_stride_elems is smaller than V");
+  cudaStream_t st = (cudaStream_t)stream;
+  launch_fill(s->g->dev, s->dev, s->walk_grid, st);
+  launch_gather_apply(s->g->dev, s->dev, logits_dev, (int)dtype, row_stride_elems, mask_dev_or_null, stride_words, st);
+  launch_end_fill(s->dev, st);
+  return launched("fmt_fill_and_apply");
+}
+
+fmt_status fmt_state_cache_clear(fmt_state* s, void* stream) {
+  if (!s) return fail(FMT_ERR_INVALID_ARG, "NULL state");
+  if (!s->dev.cache_on) return FMT_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  StateDev& d = s->dev;
+  launch_evacuate(d, st);
+  cudaError_t e = cudaMemsetAsync(d.ht, 0, ((size_t)d.ht_mask + 1) * 4, st);
+  // counters: states, mask rows, jobs, work, error flag, pool top
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.counters, 0, 8 * 4, st);
+  if (e != cudaSuccess) return cuda_fail(e, "fmt_state_cache_clear");
+  launch_reintern(d, s->init_state_dev, st);
+  return launched("fmt_state_cache_clear");
+}
+
+fmt_status fmt_state_query(fmt_state* s, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets, uint32_t* n_items,
+                           int32_t* state_id, void* stream) {
+  if (!s) return fail(FMT_ERR_INVALID_ARG, "NULL state");
+  cudaStream_t st = (cudaStream_t)stream;
+  const uint32_t B = s->dev.B;
+  uint8_t* q = s->query_dev;
+  uint8_t* a = q;
+  uint8_t* f = q + B;
+  uint32_t* ns = reinterpret_cast<uint32_t*>(q + 4 * (size_t)B);
+  uint32_t* ni = ns + B;
+  int32_t* sid = reinterpret_cast<int32_t*>(ni + B);
+  launch_query(s->dev, a, f, ns, ni, sid, st);
+  std::vector<uint8_t> host((size_t)B * 16);
+  cudaError_t e = cudaMemcpyAsync(host.data(), q, host.size(), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e, "fmt_state_query");
+  if (accepting) memcpy(accepting, host.data(), B);
+  if (finished) memcpy(finished, host.data() + B, B);
+  if (n_sets) memcpy(n_sets, host.data() + 4 * (size_t)B, 4 * (size_t)B);
+  if (n_items) memcpy(n_items, host.data() + 8 * (size_t)B, 4 * (size_t)B);
+  if (state_id) memcpy(state_id, host.data() + 12 * (size_t)B, 4 * (size_t)B);
+  return FMT_OK;
+}
+
+fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
+  if (!s || !out) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  cudaStream_t st = (cudaStream_t)stream;
+  uint32_t c[CNT_TOTAL];
+  cudaError_t e = cudaMemcpyAsync(c, s->dev.counters, sizeof(c), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e, "fmt_get_stats");
+  auto u64 = [&](uint32_t slot) { return (uint64_t)c[slot] | ((uint64_t)c[slot + 1] << 32); };
+  out->steps_advanced = u64(CNT_STAT_ADV);
+  out->fills = u64(CNT_STAT_FILLS);
+  out->fills_computed = u64(CNT_STAT_COMPUTED);
+  out->fills_from_cache = u64(CNT_STAT_CACHED);
+  out->fills_shared = u64(CNT_STAT_SHARED);
+  out->states_cached = std::min<uint64_t>(c[CNT_N_STATES], s->dev.max_states);
+  out->mask_rows_cached = std::min<uint64_t>(c[CNT_N_MASK_ROWS], s->dev.max_mask_rows);
+  out->pool_words_used = std::min<uint64_t>(u64(CNT_POOL_LO), s->dev.pool_words);
+  out->chart_items_max = c[CNT_STAT_ITEMS_MAX];
+  out->chart_sets_max = c[CNT_STAT_SETS_MAX];
+  out->capacity_errors = u64(CNT_STAT_CAPERR);
+  out->big_mode_units = u64(CNT_STAT_BIG);
+  return FMT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,269 @@
+// One byte of input on a whole pruned chart, by one warp (used when a sequence advances):
+//   Scan -> Complete (fixpoint) -> Compact -> Predict     (phase order of Section 4.2.3)
+// and the state cache: the pruned chart, densely renumbered, is the cache key ("multiple
+// different input token sequences can correspond to the same pruned Earley states", Section 5.2).
+//
+// Compact keeps, besides the unfinished items of the new last set, exactly the items a later
+// Complete can still read: an item (Y -> mu . A nu, o') of an earlier set o stays iff a kept item
+// with left-hand side A and origin o exists (Figure 3: sets not on a reference chain of the last
+// set's items are removed; completed items go once their set is done).
+#pragma once
+#include "earley_device.cuh"
+
+namespace fmt {
+
+constexpr uint32_t ADV_CUR_CAP = 2048;     // items of one set (power of two)
+constexpr uint32_t ADV_HSET = 4096;        // hash slots (power of two)
+constexpr uint32_t ADV_MAX_ITEMS = 65536;  // items of a chart the live bitmap can describe
+constexpr uint32_t ADV_PAIRS = 1024;       // (set, non-terminal) needs of one Compact
+constexpr uint32_t ADV_MAX_SETS = 2048;
+constexpr uint32_t ADV_NT_WORDS = 256;     // 2 * Nw, Nw <= 128
+constexpr uint32_t ADV_WARP_WORDS =
+    ADV_CUR_CAP + ADV_HSET + ADV_MAX_ITEMS / 32 + ADV_PAIRS + ADV_MAX_SETS + ADV_NT_WORDS + W_CTRS;
+
+struct AdvScratch {
+  WarpCtx w;
+  uint32_t* live;   // [ADV_MAX_ITEMS/32] bitmap over the source chart's items
+  uint32_t* pairs;  // [ADV_PAIRS]
+  uint32_t* sets;   // [ADV_MAX_SETS] per-set live count, then new index
+};
+
+__device__ __forceinline__ AdvScratch adv_scratch(uint32_t* base) {
+  AdvScratch s;
+  s.w.cur = base;
+  s.w.cur_cap = ADV_CUR_CAP;
+  s.w.hset = base + ADV_CUR_CAP;
+  s.w.hset_mask = ADV_HSET - 1;
+  s.live = s.w.hset + ADV_HSET;
+  s.pairs = s.live + ADV_MAX_ITEMS / 32;
+  s.sets = s.pairs + ADV_PAIRS;
+  s.w.nt = s.sets + ADV_MAX_SETS;
+  s.w.ctr = s.w.nt + ADV_NT_WORDS;
+  return s;
+}
+
+struct ChartView {
+  const uint32_t* off;  // set_off
+  const uint32_t* items;
+  __device__ __forceinline__ void operator()(uint32_t o, const uint32_t*& p, uint32_t& n) const {
+    uint32_t a = off[o], b = off[o + 1];
+    p = items + a;
+    n = b - a;
+  }
+};
+
+__device__ __forceinline__ void clear_nt(const GrammarDev& G, const WarpCtx& w) {
+  __syncwarp();
+  for (uint32_t i = lane_id(); i < 2 * G.Nw; i += 32) w.nt[i] = 0u;
+  __syncwarp();
+}
+
+__device__ __forceinline__ void push_need(const AdvScratch& s, uint32_t o, uint32_t A) {
+  uint32_t key = (o << 16) | A;
+  int r = hset_insert(s.w.hset, s.w.hset_mask, key);
+  if (r == 0) return;  // already asked for
+  // r < 0 (hash full): ask again anyway, a repeated need only costs time
+  uint32_t idx = atomicAdd(&s.w.ctr[W_NPAIRS], 1u);
+  if (idx < ADV_PAIRS) s.pairs[idx] = key;
+  else s.w.ctr[W_OVERFLOW] = 1u;
+}
+
+// Hash of a finished chart (everything but the hash words themselves); two independent 32-bit sums.
+__device__ __forceinline__ void chart_hash(uint32_t* ch) {
+  const uint32_t lane = lane_id();
+  __syncwarp();
+  const uint32_t words = ch[CH_WORDS];
+  uint32_t h1 = 0, h2 = 0;
+  for (uint32_t i = lane; i < words; i += 32) {
+    if (i == CH_HASH_LO || i == CH_HASH_HI) continue;
+    uint32_t v = ch[i];
+    h1 += mix32(v ^ (i * 0x9E3779B1u));
+    h2 += mix32((v + 0x632BE5ABu) ^ (i * 0x85EBCA77u));
+  }
+  for (int d = 16; d > 0; d >>= 1) {
+    h1 += __shfl_xor_sync(FULL, h1, d);
+    h2 += __shfl_xor_sync(FULL, h2, d);
+  }
+  __syncwarp();
+  if (lane == 0) {
+    ch[CH_HASH_LO] = h1;
+    ch[CH_HASH_HI] = h2;
+  }
+  __syncwarp();
+}
+
+// Write the last set (cur[0..n), unsorted, completed items already removed) and finish the header.
+// dst already holds set_off[0..m_new) and the kept items of the earlier sets (`kept` of them).
+__device__ __forceinline__ int finish_chart(const AdvScratch& s, uint32_t* dst, uint32_t dst_cap, uint32_t m_new,
+                                            uint32_t kept, uint32_t n, bool accepting) {
+  const uint32_t lane = lane_id();
+  uint32_t words = CH_HDR + (m_new + 2) + kept + n;
+  if (words > dst_cap || kept + n >= ADV_MAX_ITEMS || n > ADV_CUR_CAP) return -1;
+  sort_items(s.w.cur, n, ADV_CUR_CAP);
+  uint32_t* items = dst + CH_HDR + (m_new + 2);
+  for (uint32_t i = lane; i < n; i += 32) items[kept + i] = s.w.cur[i];
+  if (lane == 0) {
+    dst[CH_SETS] = m_new + 1;
+    dst[CH_ITEMS] = kept + n;
+    dst[CH_FLAGS] = accepting ? CHART_ACCEPTING : 0u;
+    dst[CH_WORDS] = words;
+    dst[6] = 0;
+    dst[7] = 0;
+    dst[CH_HDR + m_new] = kept;          // first item of the last set
+    dst[CH_HDR + m_new + 1] = kept + n;  // end
+  }
+  __syncwarp();
+  chart_hash(dst);
+  return 1;
+}
+
+// The start chart: S[0] = closure of ($ -> . start, 0).
+__device__ int chart_init(const GrammarDev& G, const AdvScratch& s, uint32_t* dst, uint32_t dst_cap) {
+  const uint32_t lane = lane_id();
+  if (lane < W_CTRS) s.w.ctr[lane] = 0u;
+  clear_nt(G, s.w);
+  if (lane == 0) add_item(G, s.w, ITEM_START);
+  __syncwarp();
+  ChartView none{nullptr, nullptr};
+  complete_fixpoint(G, s.w, none, 0u, 0u);  // only collects post-dot non-terminals and the accept flag
+  uint32_t hashed = min(s.w.ctr[W_NCUR], s.w.cur_cap);
+  bool accepting = s.w.ctr[W_ACCEPT] != 0u;
+  hset_clear_items(s.w, hashed);
+  predict_into_cur(G, s.w, 0u);
+  if (s.w.ctr[W_OVERFLOW]) {
+    hset_clear_all(s.w.hset, s.w.hset_mask);
+    clear_nt(G, s.w);
+    return -1;
+  }
+  uint32_t n = drop_completed(G, s.w, min(s.w.ctr[W_NCUR], s.w.cur_cap));
+  return finish_chart(s, dst, dst_cap, 0u, 0u, n, accepting);
+}
+
+// One byte.  Returns 1 (dst holds the new chart), 0 (the byte cannot follow: dst is garbage) or
+// -1 (a capacity limit was hit).  src and dst must not overlap.
+__device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32_t* src, uint32_t byte,
+                          uint32_t* dst, uint32_t dst_cap) {
+  const uint32_t lane = lane_id();
+  const uint32_t m = src[CH_SETS];
+  const uint32_t n_items = src[CH_ITEMS];
+  const uint32_t* soff = src + CH_HDR;
+  const uint32_t* sitems = src + CH_HDR + m + 1;
+  if (m == 0 || m + 1 > ADV_MAX_SETS || n_items > ADV_MAX_ITEMS) return -1;
+  __syncwarp();
+  if (lane < W_CTRS) s.w.ctr[lane] = 0u;
+  __syncwarp();
+  // ---- Scan
+  uint32_t n = scan_into_cur(G, s.w, sitems + soff[m - 1], soff[m] - soff[m - 1], byte);
+  if (n == 0) return 0;
+  // ---- Complete
+  ChartView view{soff, sitems};
+  complete_fixpoint(G, s.w, view, m, 0u);
+  uint32_t hashed = min(s.w.ctr[W_NCUR], s.w.cur_cap);
+  if (s.w.ctr[W_OVERFLOW]) {
+    hset_clear_all(s.w.hset, s.w.hset_mask);
+    clear_nt(G, s.w);
+    return -1;
+  }
+  hset_clear_items(s.w, hashed);
+  bool accepting = s.w.ctr[W_ACCEPT] != 0u;
+  n = drop_completed(G, s.w, hashed);
+  // ---- Compact: which items of the earlier sets can a later Complete still read?
+  for (uint32_t i = lane; i < (n_items + 31) / 32; i += 32) s.live[i] = 0u;
+  __syncwarp();
+  for (uint32_t i = lane; i < n; i += 32) {
+    uint32_t it = s.w.cur[i];
+    if ((it >> 16) < m) push_need(s, it >> 16, __ldg(&G.lhs[it & 0xFFFFu]));
+  }
+  for (uint32_t head = 0;; ++head) {
+    __syncwarp();
+    uint32_t np = min(s.w.ctr[W_NPAIRS], ADV_PAIRS);
+    __syncwarp();
+    if (head >= np) break;
+    uint32_t key = s.pairs[head];
+    uint32_t o = key >> 16, A = key & 0xFFFFu;
+    uint32_t a = soff[o], b = soff[o + 1];
+    for (uint32_t k = a + lane; k < b; k += 32) {
+      uint32_t wi = sitems[k];
+      uint32_t inf = __ldg(&G.info[wi & 0xFFFFu]);
+      if ((inf >> INFO_KIND_SHIFT) == KIND_NT && (inf & INFO_ARG_MASK) == A) {
+        uint32_t bit = 1u << (k & 31u);
+        uint32_t old = atomicOr(&s.live[k >> 5], bit);
+        if (!(old & bit)) push_need(s, wi >> 16, __ldg(&G.lhs[wi & 0xFFFFu]));
+      }
+    }
+  }
+  hset_clear_all(s.w.hset, s.w.hset_mask);  // the hash held (set, non-terminal) pairs
+  if (s.w.ctr[W_OVERFLOW]) {
+    clear_nt(G, s.w);
+    return -1;
+  }
+  // ---- live items per set, new set numbers, new offsets
+  for (uint32_t k = lane; k < m; k += 32) {
+    uint32_t a = soff[k], b = soff[k + 1], c = 0;
+    for (uint32_t i = a; i < b; ++i) c += (s.live[i >> 5] >> (i & 31u)) & 1u;
+    s.sets[k] = c;
+  }
+  __syncwarp();
+  uint32_t m_new = 0, kept = 0;
+  for (uint32_t base = 0; base < m; base += 32) {
+    uint32_t k = base + lane;
+    uint32_t c = (k < m) ? s.sets[k] : 0u;
+    uint32_t keep = __ballot_sync(FULL, c > 0);
+    uint32_t my_new = m_new + __popc(keep & ((1u << lane) - 1u));
+    uint32_t incl = c;  // inclusive prefix sum of the counts within the wave
+    for (int d = 1; d < 32; d <<= 1) {
+      uint32_t t = __shfl_up_sync(FULL, incl, d);
+      if ((int)lane >= d) incl += t;
+    }
+    if (k < m) {
+      if (c > 0) {
+        if (CH_HDR + my_new < dst_cap) dst[CH_HDR + my_new] = kept + incl - c;
+        s.sets[k] = my_new;
+      } else {
+        s.sets[k] = 0xffffffffu;
+      }
+    }
+    kept += __shfl_sync(FULL, incl, 31);
+    m_new += __popc(keep);
+  }
+  __syncwarp();
+  uint32_t words_needed = CH_HDR + (m_new + 2) + kept;
+  if (words_needed + n + 64 > dst_cap) {
+    clear_nt(G, s.w);
+    return -1;
+  }
+  // ---- copy the live items, origins renumbered
+  uint32_t* ditems = dst + CH_HDR + (m_new + 2);
+  uint32_t bad = 0;
+  uint32_t out = 0;
+  for (uint32_t base = 0; base < n_items; base += 32) {
+    uint32_t i = base + lane;
+    bool lv = (i < n_items) && ((s.live[i >> 5] >> (i & 31u)) & 1u);
+    uint32_t bal = __ballot_sync(FULL, lv);
+    if (lv) {
+      uint32_t it = sitems[i];
+      uint32_t no = s.sets[it >> 16];
+      if (no == 0xffffffffu) bad = 1;
+      ditems[out + __popc(bal & ((1u << lane) - 1u))] = (no << 16) | (it & 0xFFFFu);
+    }
+    out += __popc(bal);
+  }
+  // ---- the new last set: renumber origins, then Predict with the new index
+  for (uint32_t i = lane; i < n; i += 32) {
+    uint32_t it = s.w.cur[i];
+    uint32_t o = it >> 16;
+    uint32_t no = (o < m) ? s.sets[o] : 0xffffffffu;  // origin m cannot occur yet: those items are predicted below
+    if (no == 0xffffffffu) bad = 1;
+    s.w.cur[i] = (no << 16) | (it & 0xFFFFu);
+  }
+  bad = __any_sync(FULL, bad);
+  __syncwarp();
+  if (lane == 0) s.w.ctr[W_NCUR] = n;
+  __syncwarp();
+  predict_into_cur(G, s.w, m_new);
+  if (bad || s.w.ctr[W_OVERFLOW]) return -1;
+  n = min(s.w.ctr[W_NCUR], s.w.cur_cap);
+  return finish_chart(s, dst, dst_cap, m_new, kept, n, accepting);
+}
+
+}  // namespace fmt

@@ -1,0 +1,89 @@
+// Device-side views of the compiled grammar / vocabulary and of a batch of sequences.
+#pragma once
+#include <cstdint>
+
+namespace fmt {
+
+struct GrammarDev {
+  uint32_t D, N, C, Nw;          // dotted rules, non-terminals, byte classes, words per non-terminal bitset
+  uint32_t V, Wm, T, U, depth;   // vocabulary, mask words, trie nodes, work units, longest token
+  int32_t eos;
+  uint32_t start_nullable;
+  const uint32_t* info;          // [D]
+  const uint16_t* lhs;           // [D]
+  const uint8_t* skip;           // [D]
+  const uint32_t* class_bits;    // [C][8]
+  const uint32_t* nt_closure;    // [N][Nw]
+  const uint32_t* direct_off;    // [N+1]
+  const uint16_t* direct_items;
+  const uint32_t* child_off;     // [T+1]
+  const uint8_t* node_byte;      // [T]
+  const uint32_t* parent;        // [T]
+  const uint8_t* node_depth;     // [T]
+  const uint32_t* tok_off;       // [T+1]
+  const uint32_t* tok_ids;
+  const uint32_t* unit_node;     // [U]
+  const uint8_t* unit_kind;      // [U]
+  const uint32_t* vocab_off;     // [V+1]
+  const uint8_t* vocab_bytes;
+};
+
+// A pruned chart in memory (uint32 words):
+//   [0] number of live Earley sets m      [1] total items          [2] flags (bit 0: accepting)
+//   [3] hash low   [4] hash high          [5] total words          [6],[7] unused
+//   [8 .. 8+m]     set_off[m+1]: first item of each set
+//   then the items, (origin << 16) | dotted-rule id, ascending within each set; origins index
+//   the live sets 0..m-1 (the dense renumbering that makes equal situations equal charts).
+constexpr uint32_t CH_SETS = 0, CH_ITEMS = 1, CH_FLAGS = 2, CH_HASH_LO = 3, CH_HASH_HI = 4, CH_WORDS = 5, CH_HDR = 8;
+constexpr uint32_t CHART_ACCEPTING = 1u;
+
+constexpr uint32_t ROW_FINISHED = 1u, ROW_BROKEN = 2u;
+
+// counters[] slots
+enum : uint32_t {
+  CNT_N_STATES = 0,
+  CNT_N_MASK_ROWS = 1,
+  CNT_N_JOBS = 2,
+  CNT_WORK = 3,
+  CNT_ERR = 4,          // sticky: some device routine hit a capacity limit
+  CNT_POOL_LO = 6,      // 64-bit pool top (words) lives in slots 6,7 (8-byte aligned)
+  CNT_STAT_ADV = 8,     // 64-bit statistics from here on, two slots each
+  CNT_STAT_FILLS = 10,
+  CNT_STAT_COMPUTED = 12,
+  CNT_STAT_CACHED = 14,
+  CNT_STAT_SHARED = 16,
+  CNT_STAT_ITEMS_MAX = 18,
+  CNT_STAT_SETS_MAX = 20,
+  CNT_STAT_CAPERR = 22,
+  CNT_STAT_BIG = 24,
+  CNT_TOTAL = 32
+};
+
+struct StateDev {
+  uint32_t B;
+  uint32_t chart_words;       // capacity of one private chart buffer
+  uint32_t cache_on;
+  uint32_t max_states, ht_mask, max_mask_rows;
+  uint64_t pool_base, pool_words;   // word offsets into arena / size of the pool
+  uint64_t init_off;                // word offset of the start chart
+  uint32_t* arena;            // [B*3 private buffers][start chart][pool]
+  uint64_t* row_chart;        // [B] word offset of the row's current chart
+  uint8_t* row_buf;           // [B] private buffer holding it (0..2) or 255 (pool / start chart)
+  int32_t* row_state;         // [B] cache id or -1
+  uint32_t* row_flags;        // [B]
+  int32_t* row_mask;          // [B] mask row holding the row's mask after a fill (or a special value)
+  uint32_t* ht;               // [ht_mask+1] id+1, 0 = empty
+  uint64_t* st_off;           // [max_states] word offset of the cached chart
+  int32_t* st_mask;           // [max_states] -1 none, >= 0 mask row, <= -2 claimed by row -(x+2)
+  uint32_t* mask_rows;        // [B + max_mask_rows][Wm]; rows 0..B-1 are per-row scratch
+  uint32_t* jobs;             // [B] rows whose mask must be computed
+  uint32_t* counters;         // [CNT_TOTAL]
+  uint32_t* big_scratch;      // per-warp large scratch areas of the trie walk
+  uint32_t big_arena_items, big_hset_slots;
+};
+
+constexpr int32_t MASK_ZERO = -1;       // row_mask: all-zero mask (broken row)
+constexpr int32_t MASK_EOS_ONLY = -2;   // row_mask: finished row
+constexpr int32_t MASK_ALIAS0 = -10;    // row_mask <= MASK_ALIAS0: same mask as row (MASK_ALIAS0 - x)
+
+}  // namespace fmt

@@ -1,0 +1,281 @@
+// Warp-cooperative Earley primitives (Section 3.2 of the paper: scan, complete, predict) on
+// sparse item lists.  One warp owns one set under construction; its lanes stride over items.
+//
+// An item is one uint32: (origin << 16) | dotted-rule id.  Moving the dot is "+1" on the id.
+// A set under construction lives in `cur` with a small open-addressing hash for uniqueness
+// ("each state set maintains only unique states").  Rules that derive the empty string never
+// appear as items: every item whose post-dot non-terminal is nullable is accompanied by the
+// item with the dot moved over it (table `skip`), and prediction uses precomputed closures.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "device_tables.h"
+#include "host_tables.h"
+
+namespace fmt {
+
+constexpr uint32_t FULL = 0xffffffffu;
+constexpr uint32_t EMPTY_SLOT = 0xffffffffu;
+
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31u; }
+
+__device__ __forceinline__ uint32_t mix32(uint32_t x) {
+  x ^= x >> 16;
+  x *= 0x7feb352du;
+  x ^= x >> 15;
+  x *= 0x846ca68bu;
+  x ^= x >> 16;
+  return x;
+}
+
+// per-warp counters kept in shared memory
+enum : uint32_t { W_NCUR = 0, W_OVERFLOW = 1, W_NPAIRS = 2, W_ACCEPT = 3, W_CTRS = 8 };
+
+struct WarpCtx {
+  uint32_t* cur;        // items of the set under construction (shared or global memory)
+  uint32_t cur_cap;
+  uint32_t* hset;       // uniqueness hash, all EMPTY_SLOT between uses
+  uint32_t hset_mask;   // slots - 1 (power of two)
+  uint32_t* nt;         // [2*Nw] shared: non-terminals after a dot, then their prediction closure
+  uint32_t* ctr;        // [W_CTRS] shared
+};
+
+// 1 inserted, 0 already there, -1 table full
+__device__ __forceinline__ int hset_insert(uint32_t* hset, uint32_t mask, uint32_t key) {
+  uint32_t h = mix32(key) & mask;
+  for (uint32_t probe = 0; probe <= mask; ++probe) {
+    uint32_t old = atomicCAS(&hset[h], EMPTY_SLOT, key);
+    if (old == EMPTY_SLOT) return 1;
+    if (old == key) return 0;
+    h = (h + 1) & mask;
+  }
+  return -1;
+}
+
+__device__ __forceinline__ void hset_clear_all(uint32_t* hset, uint32_t mask) {
+  __syncwarp();
+  for (uint32_t i = lane_id(); i <= mask; i += 32) hset[i] = EMPTY_SLOT;
+  __syncwarp();
+}
+
+// Remove the first `n` items of cur from the hash (they are exactly its contents).
+__device__ __forceinline__ void hset_clear_items(const WarpCtx& w, uint32_t n) {
+  __syncwarp();
+  if (n * 8u > w.hset_mask) {
+    hset_clear_all(w.hset, w.hset_mask);
+    return;
+  }
+  for (uint32_t i = lane_id(); i < n; i += 32) {
+    uint32_t key = w.cur[i];
+    uint32_t h = mix32(key) & w.hset_mask;
+    for (uint32_t probe = 0; probe <= w.hset_mask; ++probe) {
+      if (w.hset[h] == key) {
+        w.hset[h] = EMPTY_SLOT;
+        break;
+      }
+      h = (h + 1) & w.hset_mask;
+    }
+  }
+  __syncwarp();
+}
+
+// Add item `key` and the items reached by moving the dot over nullable non-terminals.
+// May be called by any subset of lanes.
+__device__ __forceinline__ void add_item(const GrammarDev& G, const WarpCtx& w, uint32_t key) {
+  uint32_t n = __ldg(&G.skip[key & 0xFFFFu]);
+  for (uint32_t j = 0; j <= n; ++j) {
+    int r = hset_insert(w.hset, w.hset_mask, key + j);
+    if (r == 1) {
+      uint32_t idx = atomicAdd(&w.ctr[W_NCUR], 1u);
+      if (idx < w.cur_cap) w.cur[idx] = key + j;
+      else w.ctr[W_OVERFLOW] = 1u;
+    } else if (r < 0) {
+      w.ctr[W_OVERFLOW] = 1u;
+    }
+  }
+}
+
+__device__ __forceinline__ bool class_has(const GrammarDev& G, uint32_t cls, uint32_t byte) {
+  return (__ldg(&G.class_bits[cls * 8u + (byte >> 5)]) >> (byte & 31u)) & 1u;
+}
+
+// Scan (Section 3.2): items of `set` whose post-dot terminal matches `byte`, dot advanced, go
+// into cur.  Returns the number of items in cur afterwards (uniform over the warp).
+__device__ __forceinline__ uint32_t scan_into_cur(const GrammarDev& G, const WarpCtx& w, const uint32_t* set,
+                                                  uint32_t len, uint32_t byte) {
+  for (uint32_t k = lane_id(); k < len; k += 32) {
+    uint32_t it = set[k];
+    uint32_t inf = __ldg(&G.info[it & 0xFFFFu]);
+    if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) add_item(G, w, it + 1u);
+  }
+  __syncwarp();
+  return min(w.ctr[W_NCUR], w.cur_cap);
+}
+
+// Complete (Section 3.2) to a fixpoint over cur, starting at item index `head`.  `view(o, ptr, len)`
+// yields the items of set o.  Completed items whose origin is the set itself are not processed:
+// they can only come from empty derivations, already covered by `skip`.  Non-terminals found
+// after a dot are collected in w.nt[0..Nw) for the prediction that follows; the accept item is
+// reported in ctr[W_ACCEPT].
+template <class View>
+__device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const WarpCtx& w, const View& view,
+                                                  uint32_t cur_index, uint32_t head) {
+  const uint32_t lane = lane_id();
+  for (;;) {
+    __syncwarp();
+    uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
+    uint32_t over = w.ctr[W_OVERFLOW];
+    __syncwarp();
+    if (head >= n || over) break;
+    uint32_t idx = head + lane;
+    bool have = idx < n;
+    uint32_t it = have ? w.cur[idx] : 0u;
+    uint32_t inf = have ? __ldg(&G.info[it & 0xFFFFu]) : 0u;
+    uint32_t kind = inf >> INFO_KIND_SHIFT;
+    if (have && kind == KIND_NT) {
+      uint32_t y = inf & INFO_ARG_MASK;
+      atomicOr(&w.nt[y >> 5], 1u << (y & 31u));
+    }
+    if (have && kind == KIND_END && (it & 0xFFFFu) == ITEM_ACCEPT) w.ctr[W_ACCEPT] = 1u;
+    bool done_item = have && kind == KIND_END && (it >> 16) != cur_index;
+    uint32_t bal = __ballot_sync(FULL, done_item);
+    while (bal) {
+      int src = __ffs(bal) - 1;
+      bal &= bal - 1;
+      uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, src);
+      uint32_t o = __shfl_sync(FULL, it >> 16, src);
+      const uint32_t* sp;
+      uint32_t sl;
+      view(o, sp, sl);
+      for (uint32_t k = lane; k < sl; k += 32) {
+        uint32_t wi = sp[k];
+        uint32_t winf = __ldg(&G.info[wi & 0xFFFFu]);
+        if ((winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X) add_item(G, w, wi + 1u);
+      }
+      __syncwarp();
+    }
+    head += 32;
+  }
+  __syncwarp();
+}
+
+// Predict (Section 3.2) for all non-terminals collected in w.nt[0..Nw): append the start items of
+// every rule of every non-terminal in their closure, origin = cur_index.  These items are all new
+// (nothing else in the set has this origin), so no uniqueness check is needed.
+__device__ __forceinline__ void predict_into_cur(const GrammarDev& G, const WarpCtx& w, uint32_t cur_index) {
+  const uint32_t lane = lane_id();
+  const uint32_t Nw = G.Nw;
+  uint32_t* ntmask = w.nt;
+  uint32_t* clos = w.nt + Nw;
+  __syncwarp();
+  for (uint32_t i = lane; i < Nw; i += 32) clos[i] = 0u;
+  __syncwarp();
+  for (uint32_t wi = 0; wi < Nw; ++wi) {
+    uint32_t bits = ntmask[wi];
+    while (bits) {
+      uint32_t y = wi * 32u + (uint32_t)(__ffs(bits) - 1);
+      bits &= bits - 1;
+      for (uint32_t i = lane; i < Nw; i += 32) clos[i] |= __ldg(&G.nt_closure[y * Nw + i]);
+    }
+  }
+  __syncwarp();
+  uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
+  bool over = false;
+  for (uint32_t wi = 0; wi < Nw && !over; ++wi) {
+    uint32_t bits = clos[wi];
+    while (bits) {
+      uint32_t z = wi * 32u + (uint32_t)(__ffs(bits) - 1);
+      bits &= bits - 1;
+      uint32_t lo = __ldg(&G.direct_off[z]), hi = __ldg(&G.direct_off[z + 1]);
+      if (n + (hi - lo) > w.cur_cap) {
+        over = true;
+        break;
+      }
+      for (uint32_t k = lo + lane; k < hi; k += 32)
+        w.cur[n + (k - lo)] = (cur_index << 16) | (uint32_t)__ldg(&G.direct_items[k]);
+      n += hi - lo;
+    }
+  }
+  __syncwarp();
+  if (lane == 0) {
+    w.ctr[W_NCUR] = n;
+    if (over) w.ctr[W_OVERFLOW] = 1u;
+  }
+  for (uint32_t i = lane; i < Nw; i += 32) ntmask[i] = 0u;
+  __syncwarp();
+}
+
+// Drop the items with the dot at the end from cur[0..n) in place; returns the new count.
+__device__ __forceinline__ uint32_t drop_completed(const GrammarDev& G, const WarpCtx& w, uint32_t n) {
+  const uint32_t lane = lane_id();
+  uint32_t out = 0;
+  __syncwarp();
+  for (uint32_t base = 0; base < n; base += 32) {
+    uint32_t idx = base + lane;
+    bool have = idx < n;
+    uint32_t it = have ? w.cur[idx] : 0u;
+    bool keep = have && (__ldg(&G.info[it & 0xFFFFu]) >> INFO_KIND_SHIFT) != KIND_END;
+    uint32_t bal = __ballot_sync(FULL, keep);
+    uint32_t pos = out + __popc(bal & ((1u << lane) - 1u));
+    __syncwarp();
+    if (keep) w.cur[pos] = it;
+    out += __popc(bal);
+    __syncwarp();
+  }
+  return out;
+}
+
+// OR of the byte classes of all post-dot terminals of a set: the bytes that can be scanned.
+__device__ __forceinline__ void scannable_bytes(const GrammarDev& G, const uint32_t* set, uint32_t len,
+                                                uint32_t* out8 /* shared */) {
+  uint32_t acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0u;
+  for (uint32_t k = lane_id(); k < len; k += 32) {
+    uint32_t inf = __ldg(&G.info[set[k] & 0xFFFFu]);
+    if ((inf >> INFO_KIND_SHIFT) == KIND_TERM) {
+      const uint4* p = reinterpret_cast<const uint4*>(G.class_bits + (inf & INFO_ARG_MASK) * 8u);
+      uint4 a = __ldg(p), b = __ldg(p + 1);
+      acc[0] |= a.x, acc[1] |= a.y, acc[2] |= a.z, acc[3] |= a.w;
+      acc[4] |= b.x, acc[5] |= b.y, acc[6] |= b.z, acc[7] |= b.w;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = __reduce_or_sync(FULL, acc[i]);
+  __syncwarp();
+  if (lane_id() == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) out8[i] = acc[i];
+  }
+  __syncwarp();
+}
+
+// Ascending bitonic sort of a[0..n); the array must have room for the next power of two >= max(n, 32),
+// which must not exceed cap_pow2.
+__device__ __forceinline__ void sort_items(uint32_t* a, uint32_t n, uint32_t cap_pow2) {
+  const uint32_t lane = lane_id();
+  uint32_t P = 32;
+  while (P < n) P <<= 1;
+  if (P > cap_pow2) P = cap_pow2;
+  __syncwarp();
+  for (uint32_t i = n + lane; i < P; i += 32) a[i] = 0xffffffffu;
+  __syncwarp();
+  for (uint32_t k = 2; k <= P; k <<= 1) {
+    for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+      for (uint32_t i = lane; i < P; i += 32) {
+        uint32_t l = i ^ j;
+        if (l > i) {
+          uint32_t x = a[i], y = a[l];
+          bool up = (i & k) == 0;
+          if ((x > y) == up) {
+            a[i] = y;
+            a[l] = x;
+          }
+        }
+      }
+      __syncwarp();
+    }
+  }
+}
+
+}  // namespace fmt

@@ -1,0 +1,29 @@
+// Host-callable launchers of the kernels in kernels.cu.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "device_tables.h"
+
+namespace fmt {
+
+cudaError_t configure_kernels();
+cudaError_t walk_blocks_per_sm(int* out);
+int walk_warps();
+
+void launch_init(const GrammarDev& G, const StateDev& S, int32_t* result_dev, cudaStream_t st);
+void launch_intern_init(const StateDev& S, int32_t* init_state_dev, cudaStream_t st);
+void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const int32_t* init_state_dev, cudaStream_t st);
+void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st);
+void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStream_t st);
+void launch_end_fill(const StateDev& S, cudaStream_t st);
+void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st);
+void launch_apply(const uint32_t* mask, size_t stride_words, void* logits, int dtype, uint32_t batch, uint32_t V,
+                  size_t row_stride, cudaStream_t st);
+void launch_gather_apply(const GrammarDev& G, const StateDev& S, void* logits, int dtype, size_t row_stride,
+                         uint32_t* mask_out, size_t stride_words, cudaStream_t st);
+void launch_evacuate(const StateDev& S, cudaStream_t st);
+void launch_reintern(const StateDev& S, int32_t* init_state_dev, cudaStream_t st);
+void launch_query(const StateDev& S, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets, uint32_t* n_items,
+                  int32_t* state_id, cudaStream_t st);
+
+}  // namespace fmt
