@@ -189,6 +189,13 @@ fmt_status fmt_state_cache_clear(fmt_state* s, void* stream);
 fmt_status fmt_state_query(fmt_state* s, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets,
                            uint32_t* n_items, int32_t* state_id, void* stream);
 
+/* Copy the pruned chart of one row to the host, for inspection and tests; synchronizes `stream`.
+ * Layout (uint32 words): [0] live sets m, [1] items, [2] flags (bit 0 accepting), [3],[4] hash,
+ * [5] total words, [6],[7] unused, then set_off[m+1], then the items (origin << 16 | dotted rule).
+ * Writes min(cap_words, total) words to `out` (may be NULL) and the total to *n_words. */
+fmt_status fmt_state_copy_chart(fmt_state* s, uint32_t row, uint32_t* out, size_t cap_words, size_t* n_words,
+                                void* stream);
+
 /* Counters since creation; synchronizes `stream`. */
 fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream);
 

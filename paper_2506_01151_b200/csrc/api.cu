@@ -368,6 +368,27 @@ fmt_status fmt_state_query(fmt_state* s, uint8_t* accepting, uint8_t* finished, 
   return FMT_OK;
 }
 
+fmt_status fmt_state_copy_chart(fmt_state* s, uint32_t row, uint32_t* out, size_t cap_words, size_t* n_words,
+                                void* stream) {
+  if (!s || !n_words || row >= s->dev.B) return fail(FMT_ERR_INVALID_ARG, "bad argument");
+  cudaStream_t st = (cudaStream_t)stream;
+  uint64_t off = 0;
+  cudaError_t e = cudaMemcpyAsync(&off, s->dev.row_chart + row, 8, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  uint32_t hdr[CH_HDR];
+  if (e == cudaSuccess) e = cudaMemcpyAsync(hdr, s->dev.arena + off, sizeof(hdr), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e, "fmt_state_copy_chart");
+  *n_words = hdr[CH_WORDS];
+  size_t n = std::min<size_t>(cap_words, hdr[CH_WORDS]);
+  if (out && n) {
+    e = cudaMemcpyAsync(out, s->dev.arena + off, n * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "fmt_state_copy_chart");
+  }
+  return FMT_OK;
+}
+
 fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   if (!s || !out) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
   cudaStream_t st = (cudaStream_t)stream;

@@ -154,7 +154,7 @@ __device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const War
       }
       __syncwarp();
     }
-    head += 32;
+    head = min(head + 32u, n);  // items appended during this wave start at index n
   }
   __syncwarp();
 }

@@ -1,0 +1,109 @@
+"""GPU parity: the CUDA library against the CPU oracle, bit for bit, through the C-ABI binding."""
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+from helpers import OracleBatch, describe_diff
+
+pytestmark = pytest.mark.gpu
+
+
+def run_workload(w, check_steps, rows=None, cache=True, fused_every=0, check_prefix_mask=True, **state_kw):
+    """Feed the workload through the library and the oracle; compare statuses every step and
+    masks (all rows in `rows`) at the steps in `check_steps`.  Returns the library's stats."""
+    import torch
+
+    import paper_2506_01151_b200 as fmt
+
+    dev = torch.device("cuda:0")
+    g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
+    st = fmt.State(g, w.batch, cache=cache, **state_kw)
+    ob = OracleBatch(w)
+    rows = list(range(w.batch)) if rows is None else rows
+    Wm = g.mask_words
+    mask = torch.zeros((w.batch, Wm), dtype=torch.int32, device=dev)
+    status = torch.zeros(w.batch, dtype=torch.int32, device=dev)
+
+    def advance(tokens):
+        tok = torch.from_numpy(np.ascontiguousarray(tokens, dtype=np.int32)).to(dev)
+        st.advance(tok, status)
+        got = status.cpu().numpy()
+        for b in range(w.batch):
+            want = ob.advance(b, int(tokens[b]))
+            assert got[b] == want, ("status", b, int(tokens[b]), w.vocab[int(tokens[b])] if tokens[b] >= 0 else None, got[b], want)
+
+    def compare(tag):
+        st.fill_mask(mask)
+        got = mask.cpu().numpy().view(np.uint32)
+        for b in rows:
+            want = ob.mask(b)
+            assert np.array_equal(got[b], want), (tag, b, describe_diff(w, got[b], want))
+
+    for p in range(w.prefix.shape[0]):
+        advance(w.prefix[p])
+    if check_prefix_mask:
+        compare("after prefix")
+    for i in range(w.steps):
+        r = np.nonzero(w.reset_before[i])[0]
+        if len(r):
+            st.reset(torch.from_numpy(r.astype(np.int32)).to(dev))
+            for b in r:
+                ob.reset(int(b))
+        advance(w.tokens[i])
+        if i in check_steps:
+            compare("step %d" % i)
+            if fused_every and (i % fused_every == 0):
+                logits = workloads.f32_to_bf16_bits(w.logits_f32(i))
+                lt = torch.from_numpy(logits.view(np.int16)).to(dev)
+                m2 = torch.zeros_like(mask)
+                st.fill_and_apply(lt, fmt.BF16, mask_dev=m2)
+                want_mask = np.stack([ob.mask(b) for b in range(w.batch)])
+                assert np.array_equal(m2.cpu().numpy().view(np.uint32), want_mask)
+                want = oracle.apply_mask(want_mask, logits, "bf16")
+                assert np.array_equal(lt.cpu().numpy().view(np.uint16), want)
+    q = st.query()
+    for b in range(w.batch):
+        assert bool(q["accepting"][b]) == ob.seqs[b].accepting, b
+        assert bool(q["finished"][b] == 1) == ob.finished[b], b
+    stats = st.stats()
+    assert stats["capacity_errors"] == 0
+    return stats, q
+
+
+def test_config1_every_step():
+    w = workloads.build(1)
+    stats, _ = run_workload(w, check_steps=set(range(w.steps)), fused_every=4)
+    assert stats["fills_computed"] > 0
+
+
+def test_config1_without_cache():
+    w = workloads.build(1)
+    stats, q = run_workload(w, check_steps=set(range(w.steps)), cache=False)
+    assert stats["fills_from_cache"] == 0 and (q["state_id"] == -1).all()
+
+
+def test_config2_small_vocab_every_step():
+    w = workloads.build(2, V=4000, batch=4, steps=96)
+    run_workload(w, check_steps=set(range(w.steps)), fused_every=16)
+
+
+def test_config2_full():
+    w = workloads.build(2)
+    stats, _ = run_workload(w, check_steps=set(range(0, w.steps, 8)) | {w.steps - 1}, fused_every=64)
+    assert stats["fills_from_cache"] + stats["fills_shared"] > 0  # pruned charts repeat (state cache)
+
+
+def test_config3_reduced():
+    w = workloads.build(3, V=20000, batch=8, steps=160)
+    run_workload(w, check_steps=set(range(0, 160, 8)), fused_every=40)
+
+
+def test_config4_reduced():
+    w = workloads.build(4, V=20000, batch=8, steps=128)
+    run_workload(w, check_steps=set(range(0, 128, 8)), fused_every=32)
+
+
+def test_config5_reduced():
+    w = workloads.build(5, V=20000, batch=8, steps=32, prefix_scale=0.25)
+    run_workload(w, check_steps=set(range(0, 32, 4)), fused_every=16)
