@@ -199,6 +199,18 @@ fmt_status fmt_state_copy_chart(fmt_state* s, uint32_t row, uint32_t* out, size_
 /* Counters since creation; synchronizes `stream`. */
 fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream);
 
+/* Kernel timing with CUDA events on the caller's stream (no counterpart in the paper: a
+ * measurement aid).  While enabled, every fmt_state_advance, the trie-walk kernel of every fill
+ * and every logits-masking kernel of this state is bracketed by a pair of events (up to 16384
+ * pairs per kind, later launches are not timed).  fmt_state_read_profile synchronizes those
+ * events, adds up the elapsed times and forgets them. */
+typedef struct {
+  double advance_ms, walk_ms, apply_ms;
+  uint64_t advance_launches, walk_launches, apply_launches;
+} fmt_profile;
+fmt_status fmt_state_set_profiling(fmt_state* s, int enable);
+fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
+
 const char* fmt_last_error(void);
 
 #ifdef __cplusplus

@@ -23,7 +23,7 @@ EXPORTS = [
     "fmt_compile", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table",
     "fmt_state_create", "fmt_state_destroy", "fmt_state_reset", "fmt_state_advance", "fmt_fill_mask",
     "fmt_apply_mask", "fmt_fill_and_apply", "fmt_state_cache_clear", "fmt_state_query", "fmt_state_copy_chart", "fmt_get_stats",
-    "fmt_last_error",
+    "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_last_error",
 ]
 
 
@@ -60,6 +60,11 @@ class Stats(C.Structure):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
 
 
+class Profile(C.Structure):
+    _fields_ = [("advance_ms", C.c_double), ("walk_ms", C.c_double), ("apply_ms", C.c_double),
+                ("advance_launches", C.c_uint64), ("walk_launches", C.c_uint64), ("apply_launches", C.c_uint64)]
+
+
 _lib = None
 
 
@@ -87,6 +92,8 @@ def lib():
         L.fmt_state_query.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.fmt_state_copy_chart.argtypes = [vp, u32, vp, sz, C.POINTER(sz), vp]
         L.fmt_get_stats.argtypes = [vp, C.POINTER(Stats), vp]
+        L.fmt_state_set_profiling.argtypes = [vp, C.c_int]
+        L.fmt_state_read_profile.argtypes = [vp, C.POINTER(Profile)]
         L.fmt_last_error.restype = C.c_char_p
         for name in EXPORTS:
             if name not in ("fmt_grammar_destroy", "fmt_state_destroy", "fmt_last_error"):
@@ -223,6 +230,14 @@ class State:
         items = buf[8 + m + 1 :]
         sets = [[(int(x & 0xFFFF), int(x >> 16)) for x in items[off[k] : off[k + 1]]] for k in range(m)]
         return {"sets": sets, "accepting": bool(buf[2] & 1), "words": int(buf[5])}
+
+    def set_profiling(self, on: bool):
+        _check(lib().fmt_state_set_profiling(self._h, 1 if on else 0))
+
+    def read_profile(self) -> dict:
+        out = Profile()
+        _check(lib().fmt_state_read_profile(self._h, C.byref(out)))
+        return {n: getattr(out, n) for n, _ in out._fields_}
 
     def stats(self, stream=None) -> dict:
         out = Stats()

@@ -70,7 +70,40 @@ struct fmt_grammar {
   DeviceBuffers bufs;
 };
 
+// CUDA-event pairs around the three kinds of kernels, filled while profiling is enabled.
+struct Profiler {
+  static constexpr size_t kMaxPairs = 16384;
+  bool on = false;
+  std::vector<cudaEvent_t> a[3], b[3];  // 0 advance, 1 walk, 2 logits masking
+  size_t used[3] = {0, 0, 0};
+  bool next(int kind, cudaEvent_t* before, cudaEvent_t* after) {
+    *before = *after = nullptr;
+    if (!on || used[kind] >= kMaxPairs) return false;
+    if (used[kind] == a[kind].size()) {
+      cudaEvent_t x, y;
+      if (cudaEventCreate(&x) != cudaSuccess) return false;
+      if (cudaEventCreate(&y) != cudaSuccess) {
+        cudaEventDestroy(x);
+        return false;
+      }
+      a[kind].push_back(x);
+      b[kind].push_back(y);
+    }
+    *before = a[kind][used[kind]];
+    *after = b[kind][used[kind]];
+    ++used[kind];
+    return true;
+  }
+  ~Profiler() {
+    for (int k = 0; k < 3; ++k) {
+      for (auto e : a[k]) cudaEventDestroy(e);
+      for (auto e : b[k]) cudaEventDestroy(e);
+    }
+  }
+};
+
 struct fmt_state {
+  Profiler prof;
   const fmt_grammar* g = nullptr;
   StateDev dev{};
   DeviceBuffers bufs;
@@ -292,7 +325,11 @@ fmt_status fmt_state_reset(fmt_state* s, const uint32_t* rows_dev, uint32_t n, v
 
 fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t* status_dev, void* stream) {
   if (!s || !token_ids_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  cudaEvent_t e0, e1;
+  s->prof.next(0, &e0, &e1);
+  if (e0) cudaEventRecord(e0, (cudaStream_t)stream);
   launch_advance(s->g->dev, s->dev, token_ids_dev, status_dev, (cudaStream_t)stream);
+  if (e1) cudaEventRecord(e1, (cudaStream_t)stream);
   return launched("fmt_state_advance");
 }
 
@@ -300,7 +337,9 @@ fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, 
   if (!s || !mask_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
   if (stride_words < s->g->dev.Wm) return fail(FMT_ERR_INVALID_ARG, "stride_words is smaller than ceil(V/32)");
   cudaStream_t st = (cudaStream_t)stream;
-  launch_fill(s->g->dev, s->dev, s->walk_grid, st);
+  cudaEvent_t w0, w1;
+  s->prof.next(1, &w0, &w1);
+  launch_fill(s->g->dev, s->dev, s->walk_grid, st, w0, w1);
   launch_gather(s->g->dev, s->dev, mask_dev, stride_words, st);
   launch_end_fill(s->dev, st);
   return launched("fmt_fill_mask");
@@ -324,8 +363,13 @@ fmt_status fmt_fill_and_apply(fmt_state* s, uint32_t* mask_dev_or_null, size_t s
     return fail(FMT_ERR_INVALID_ARG, "stride_words is smaller than ceil(V/32)");
   if (row_stride_elems < s->g->dev.V) return fail(FMT_ERR_INVALID_ARG, "row_stride_elems is smaller than V");
   cudaStream_t st = (cudaStream_t)stream;
-  launch_fill(s->g->dev, s->dev, s->walk_grid, st);
+  cudaEvent_t w0, w1, a0, a1;
+  s->prof.next(1, &w0, &w1);
+  s->prof.next(2, &a0, &a1);
+  launch_fill(s->g->dev, s->dev, s->walk_grid, st, w0, w1);
+  if (a0) cudaEventRecord(a0, st);
   launch_gather_apply(s->g->dev, s->dev, logits_dev, (int)dtype, row_stride_elems, mask_dev_or_null, stride_words, st);
+  if (a1) cudaEventRecord(a1, st);
   launch_end_fill(s->dev, st);
   return launched("fmt_fill_and_apply");
 }
@@ -386,6 +430,30 @@ fmt_status fmt_state_copy_chart(fmt_state* s, uint32_t row, uint32_t* out, size_
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e, "fmt_state_copy_chart");
   }
+  return FMT_OK;
+}
+
+fmt_status fmt_state_set_profiling(fmt_state* s, int enable) {
+  if (!s) return fail(FMT_ERR_INVALID_ARG, "NULL state");
+  s->prof.on = enable != 0;
+  return FMT_OK;
+}
+
+fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out) {
+  if (!s || !out) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  double ms[3] = {0, 0, 0};
+  for (int k = 0; k < 3; ++k) {
+    for (size_t i = 0; i < s->prof.used[k]; ++i) {
+      cudaError_t e = cudaEventSynchronize(s->prof.b[k][i]);
+      float t = 0.f;
+      if (e == cudaSuccess) e = cudaEventElapsedTime(&t, s->prof.a[k][i], s->prof.b[k][i]);
+      if (e != cudaSuccess) return cuda_fail(e, "fmt_state_read_profile");
+      ms[k] += t;
+    }
+  }
+  out->advance_ms = ms[0], out->walk_ms = ms[1], out->apply_ms = ms[2];
+  out->advance_launches = s->prof.used[0], out->walk_launches = s->prof.used[1], out->apply_launches = s->prof.used[2];
+  s->prof.used[0] = s->prof.used[1] = s->prof.used[2] = 0;
   return FMT_OK;
 }
 

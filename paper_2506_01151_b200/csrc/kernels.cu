@@ -768,10 +768,13 @@ void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const
 void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st) {
   advance_kernel<<<(S.B + ADV_WARPS - 1) / ADV_WARPS, ADV_WARPS * 32, adv_smem_bytes(), st>>>(G, S, tokens, status);
 }
-void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStream_t st) {
+void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStream_t st, cudaEvent_t before_walk,
+                 cudaEvent_t after_walk) {
   plan_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(G, S);
   prepare_rows_kernel<<<S.B, 256, 0, st>>>(G, S);
+  if (before_walk) cudaEventRecord(before_walk, st);
   walk_kernel<<<walk_grid, WALK_WARPS * 32, walk_smem_bytes(), st>>>(G, S);
+  if (after_walk) cudaEventRecord(after_walk, st);
   publish_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(S);
 }
 void launch_end_fill(const StateDev& S, cudaStream_t st) { end_fill_kernel<<<1, 1, 0, st>>>(S); }

@@ -14,7 +14,8 @@ void launch_init(const GrammarDev& G, const StateDev& S, int32_t* result_dev, cu
 void launch_intern_init(const StateDev& S, int32_t* init_state_dev, cudaStream_t st);
 void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const int32_t* init_state_dev, cudaStream_t st);
 void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st);
-void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStream_t st);
+void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStream_t st, cudaEvent_t before_walk = nullptr,
+                 cudaEvent_t after_walk = nullptr);
 void launch_end_fill(const StateDev& S, cudaStream_t st);
 void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st);
 void launch_apply(const uint32_t* mask, size_t stride_words, void* logits, int dtype, uint32_t batch, uint32_t V,
