@@ -211,6 +211,40 @@ typedef struct {
 fmt_status fmt_state_set_profiling(fmt_state* s, int enable);
 fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
 
+/*
+ * Masks for up to FMT_NOALLOC_MAX_CHARTS pruned charts without any memory allocation.
+ * (The paper has no counterpart; this is a convenience of this library.)
+ *
+ * Who needs it: code that must not call cudaMalloc / cudaFree while it runs - a serving loop
+ * whose device memory is entirely owned by a caching allocator or handed out up front, a
+ * real-time or library context where an allocation may synchronize the device or fail under
+ * memory pressure, a plugin that may only launch kernels.  fmt_fill_mask itself never allocates,
+ * but it needs an fmt_state, whose creation allocates hundreds of megabytes.  This call needs no
+ * fmt_state: it walks the vocabulary trie for charts the caller already holds in device memory
+ * (in the layout fmt_state_copy_chart documents) and uses a fixed scratch array that is part of
+ * the loaded library image (about 21 MB of device memory on every GPU that loads the library,
+ * held until the process exits).
+ *
+ *   g              a grammar compiled for the current device
+ *   charts_dev     device memory holding the charts
+ *   chart_offsets  HOST array of n+1 word offsets into charts_dev: chart r occupies words
+ *                  [chart_offsets[r], chart_offsets[r+1])
+ *   n              number of charts, at most FMT_NOALLOC_MAX_CHARTS (more: FMT_ERR_CAPACITY)
+ *   mask_dev       device output, n rows of exactly ceil(V/32) words (dense, no extra stride)
+ *   status_dev     device output or NULL, n int32: FMT_OK, FMT_ERR_INVALID_ARG (the chart's header
+ *                  does not fit its slot) or FMT_ERR_CAPACITY (an Earley set outgrew the fixed
+ *                  scratch; that row's mask is all-zero)
+ *
+ * The first call on each device looks up the scratch array's device address and raises the
+ * kernels' shared-memory limit; make that first call outside any stream capture.  Every call on
+ * a device uses the same scratch array: calls that may overlap on the GPU (different streams,
+ * different host threads) race and must be serialized by the caller.  The call enqueues work on
+ * `stream` and does not synchronize; it calls no cudaMalloc, cudaFree or other allocating routine.
+ */
+#define FMT_NOALLOC_MAX_CHARTS 64
+fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t* charts_dev, const uint64_t* chart_offsets,
+                                 uint32_t n, uint32_t* mask_dev, int32_t* status_dev, void* stream);
+
 const char* fmt_last_error(void);
 
 #ifdef __cplusplus

@@ -23,7 +23,7 @@ EXPORTS = [
     "fmt_compile", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table",
     "fmt_state_create", "fmt_state_destroy", "fmt_state_reset", "fmt_state_advance", "fmt_fill_mask",
     "fmt_apply_mask", "fmt_fill_and_apply", "fmt_state_cache_clear", "fmt_state_query", "fmt_state_copy_chart", "fmt_get_stats",
-    "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_last_error",
+    "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_fill_mask_noalloc", "fmt_last_error",
 ]
 
 
@@ -94,6 +94,7 @@ def lib():
         L.fmt_get_stats.argtypes = [vp, C.POINTER(Stats), vp]
         L.fmt_state_set_profiling.argtypes = [vp, C.c_int]
         L.fmt_state_read_profile.argtypes = [vp, C.POINTER(Profile)]
+        L.fmt_fill_mask_noalloc.argtypes = [vp, vp, vp, u32, vp, vp, vp]
         L.fmt_last_error.restype = C.c_char_p
         for name in EXPORTS:
             if name not in ("fmt_grammar_destroy", "fmt_state_destroy", "fmt_last_error"):
@@ -231,6 +232,14 @@ class State:
         sets = [[(int(x & 0xFFFF), int(x >> 16)) for x in items[off[k] : off[k + 1]]] for k in range(m)]
         return {"sets": sets, "accepting": bool(buf[2] & 1), "words": int(buf[5])}
 
+    def chart_words(self, row: int, stream=None) -> np.ndarray:
+        """The raw words of the row's pruned chart (the layout fmt_state_copy_chart documents)."""
+        n = C.c_size_t()
+        _check(lib().fmt_state_copy_chart(self._h, row, None, 0, C.byref(n), _ptr(stream)))
+        buf = np.zeros(n.value, dtype=np.uint32)
+        _check(lib().fmt_state_copy_chart(self._h, row, buf.ctypes.data, n.value, C.byref(n), _ptr(stream)))
+        return buf
+
     def set_profiling(self, on: bool):
         _check(lib().fmt_state_set_profiling(self._h, 1 if on else 0))
 
@@ -251,3 +260,16 @@ def apply_mask(mask_dev, logits_dev, dtype: int, batch: int, V: int, stride_word
     stride = (V + 31) // 32 if stride_words is None else stride_words
     rs = V if row_stride is None else row_stride
     _check(lib().fmt_apply_mask(_ptr(mask_dev), stride, _ptr(logits_dev), dtype, batch, V, rs, _ptr(stream)))
+
+
+NOALLOC_MAX_CHARTS = 64
+
+
+def fill_mask_noalloc(grammar: Grammar, charts_dev, chart_offsets: Sequence[int], mask_dev, status_dev=None, stream=None):
+    """fmt_fill_mask_noalloc: masks for charts already in device memory, using only the scratch
+    array built into the library (no allocation; see include/fmt.h for who needs that and why).
+    chart_offsets: n+1 word offsets into charts_dev; mask_dev: [n, ceil(V/32)] dense."""
+    offs = np.ascontiguousarray(chart_offsets, dtype=np.uint64)
+    n = len(offs) - 1
+    _check(lib().fmt_fill_mask_noalloc(grammar._h, _ptr(charts_dev), offs.ctypes.data, n, _ptr(mask_dev),
+                                       _ptr(status_dev), _ptr(stream)))

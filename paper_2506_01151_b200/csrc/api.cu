@@ -113,6 +113,15 @@ struct fmt_state {
   int walk_grid = 1;
 };
 
+namespace fmt {
+const GrammarDev* grammar_device_tables(const ::fmt_grammar* g, int* device) {
+  if (!g || !g->on_device) return nullptr;
+  if (device) *device = g->device;
+  return &g->dev;
+}
+void set_last_error(const char* msg) { g_last_error = msg; }
+}  // namespace fmt
+
 extern "C" {
 
 const char* fmt_last_error(void) { return g_last_error.c_str(); }

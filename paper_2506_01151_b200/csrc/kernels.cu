@@ -777,6 +777,9 @@ void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStre
   if (after_walk) cudaEventRecord(after_walk, st);
   publish_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(S);
 }
+void launch_walk(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) {
+  walk_kernel<<<grid, WALK_WARPS * 32, walk_smem_bytes(), st>>>(G, S);
+}
 void launch_end_fill(const StateDev& S, cudaStream_t st) { end_fill_kernel<<<1, 1, 0, st>>>(S); }
 void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st) {
   dim3 grid((unsigned)std::min<size_t>((stride_words + 255) / 256, 64), S.B);

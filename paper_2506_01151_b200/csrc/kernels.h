@@ -27,4 +27,14 @@ void launch_reintern(const StateDev& S, int32_t* init_state_dev, cudaStream_t st
 void launch_query(const StateDev& S, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets, uint32_t* n_items,
                   int32_t* state_id, cudaStream_t st);
 
+// the trie-walk kernel alone, on an arbitrary grid (used by the allocation-free entry point)
+void launch_walk(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st);
+
+}  // namespace fmt
+
+struct fmt_grammar;
+namespace fmt {
+// device tables of a compiled grammar, or nullptr for a host_only grammar; `device` gets its GPU
+const GrammarDev* grammar_device_tables(const ::fmt_grammar* g, int* device);
+void set_last_error(const char* msg);
 }  // namespace fmt
