@@ -107,3 +107,28 @@ def test_config4_reduced():
 def test_config5_reduced():
     w = workloads.build(5, V=20000, batch=8, steps=32, prefix_scale=0.25)
     run_workload(w, check_steps=set(range(0, 32, 4)), fused_every=16)
+
+
+# ---- full sizes, in the launch configuration the benchmark times; masks compared on sampled steps
+
+
+def _sampled(steps, every):
+    return set(range(0, steps, every)) | set(range(4)) | set(range(steps - 4, steps))
+
+
+def test_config3_full_size_sampled_steps():
+    w = workloads.build(3)
+    stats, _ = run_workload(w, check_steps=_sampled(w.steps, 16), fused_every=128, check_prefix_mask=False)
+    assert stats["fills_from_cache"] > stats["fills_computed"]  # the state cache carries most fills
+
+
+def test_config4_full_size_sampled_steps():
+    w = workloads.build(4)
+    run_workload(w, check_steps=_sampled(w.steps, 16), fused_every=128, check_prefix_mask=False)
+
+
+def test_config5_full_size_sampled_rows_and_steps():
+    w = workloads.build(5)
+    rows = list(range(0, w.batch, 16))
+    stats, q = run_workload(w, check_steps=set(range(0, w.steps, 4)), rows=rows, check_prefix_mask=False)
+    assert q["n_sets"].max() > 20  # deep nesting / ambiguous segments keep many sets alive
