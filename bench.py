@@ -259,7 +259,10 @@ def run_ours(args):
                   "shared": stats1["fills_shared"] - stats0["fills_shared"],
                   "hit_rate": 1.0 - jobs / max(1, fills), "states_cached": stats1["states_cached"],
                   "chart_items_max": stats1["chart_items_max"], "chart_sets_max": stats1["chart_sets_max"],
-                  "capacity_errors": stats1["capacity_errors"]},
+                  "capacity_errors": stats1["capacity_errors"],
+                  "walk_transitions": stats1["walk_transitions"] - stats0["walk_transitions"],
+                  "walk_states": stats1["walk_states"] - stats0["walk_states"],
+                  "big_mode": stats1["big_mode_units"] - stats0["big_mode_units"]},
         "cold": cold,
         "grammar": {"nonterminals": info.n_nonterminals, "rules": info.n_rules, "dotted": info.n_dotted,
                     "trie_nodes": info.trie_nodes, "units": info.n_units},

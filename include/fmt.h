@@ -61,7 +61,7 @@ typedef struct {
   uint32_t host_only;        /* 1: build the tables on the host only (no device needed; the
                                 grammar can be inspected but no state can be created) */
   uint32_t unit_max_nodes;   /* trie subtrees larger than this are split into several work
-                                units (default 192) */
+                                units (default 32) */
   uint32_t reserved[6];
 } fmt_compile_options;
 
@@ -72,7 +72,9 @@ typedef struct {
   uint32_t max_mask_rows;     /* cached mask rows (default 8192) */
   uint32_t chart_words;       /* capacity of one row's chart in uint32 words (default 65536) */
   uint64_t pool_words;        /* uint32 words of chart storage for the cache (default 64 Mi) */
-  uint32_t reserved[6];
+  uint32_t walk_states;       /* distinct Earley sets one mask computation may create while it
+                                 walks the vocabulary (default: 4 Mi / batch, within 2048..32768) */
+  uint32_t reserved[5];
 } fmt_state_options;
 
 typedef struct {
@@ -102,7 +104,9 @@ typedef struct {
   uint64_t chart_items_max;    /* largest pruned chart seen (items) */
   uint64_t chart_sets_max;     /* most live Earley sets seen in one chart */
   uint64_t capacity_errors;
-  uint64_t big_mode_units;     /* work units redone with the large scratch area */
+  uint64_t big_mode_units;     /* times the trie walk switched to its large scratch area */
+  uint64_t walk_transitions;   /* Earley steps (scan + complete + predict) done by the trie walk */
+  uint64_t walk_states;        /* distinct Earley sets created by the trie walk */
 } fmt_stats;
 
 /*
@@ -222,7 +226,7 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
  * but it needs an fmt_state, whose creation allocates hundreds of megabytes.  This call needs no
  * fmt_state: it walks the vocabulary trie for charts the caller already holds in device memory
  * (in the layout fmt_state_copy_chart documents) and uses a fixed scratch array that is part of
- * the loaded library image (about 21 MB of device memory on every GPU that loads the library,
+ * the loaded library image (about 36 MB of device memory on every GPU that loads the library,
  * held until the process exits).
  *
  *   g              a grammar compiled for the current device
@@ -232,8 +236,8 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
  *   n              number of charts, at most FMT_NOALLOC_MAX_CHARTS (more: FMT_ERR_CAPACITY)
  *   mask_dev       device output, n rows of exactly ceil(V/32) words (dense, no extra stride)
  *   status_dev     device output or NULL, n int32: FMT_OK, FMT_ERR_INVALID_ARG (the chart's header
- *                  does not fit its slot) or FMT_ERR_CAPACITY (an Earley set outgrew the fixed
- *                  scratch; that row's mask is all-zero)
+ *                  does not fit its slot) or FMT_ERR_CAPACITY (the Earley sets met while walking the
+ *                  vocabulary outgrew the fixed scratch; that row's mask is all-zero)
  *
  * The first call on each device looks up the scratch array's device address and raises the
  * kernels' shared-memory limit; make that first call outside any stream capture.  Every call on

@@ -163,6 +163,8 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
     UP(lhs);
     UP(skip);
     UP(class_bits);
+    UP(eq_of_byte);
+    d.n_eq = h.n_eq;
     UP(nt_closure);
     UP(direct_off);
     UP(direct_items);
@@ -261,7 +263,16 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   d.init_off = (uint64_t)batch * 3u * d.chart_words;
   d.pool_base = d.init_off + d.chart_words;
   d.big_arena_items = 1u << 16;
-  d.big_hset_slots = 1u << 13;
+  d.big_hset_slots = 1u << 14;
+  AutoDev& au = d.au;
+  au.cap = (opt && opt->walk_states) ? opt->walk_states : std::min(32768u, std::max(2048u, (4u << 20) / batch));
+  if (au.cap < 16) au.cap = 16;
+  if (au.cap > 60000) au.cap = 60000;
+  au.rec_words = (AR_TRANS + g->dev.n_eq + 31u) & ~31u;
+  uint32_t hs = 64;
+  while (hs < au.cap * 2u) hs <<= 1;
+  au.hash_mask = hs - 1;
+  au.items_cap = 128u << 20;
 
   cudaError_t e = configure_kernels();
   int per_sm = 0, sms = 0, dev = 0;
@@ -288,6 +299,10 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(d.jobs, batch, 0);
   AL(d.counters, CNT_TOTAL, 0);
   AL(d.big_scratch, big_words, 0xFF);
+  AL(au.recs, (size_t)batch * au.cap * au.rec_words, 0);
+  AL(au.hash, (size_t)batch * hs, 0);
+  AL(au.items, au.items_cap, 0);
+  AL(au.n_states, batch, 0);
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);
@@ -486,6 +501,8 @@ fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   out->chart_sets_max = c[CNT_STAT_SETS_MAX];
   out->capacity_errors = u64(CNT_STAT_CAPERR);
   out->big_mode_units = u64(CNT_STAT_BIG);
+  out->walk_transitions = u64(CNT_STAT_TRANS);
+  out->walk_states = u64(CNT_STAT_LOCAL);
   return FMT_OK;
 }
 

@@ -50,6 +50,7 @@ struct ChartView {
     p = items + a;
     n = b - a;
   }
+  __device__ __forceinline__ uint32_t fix(uint32_t item, uint32_t) const { return item; }
 };
 
 __device__ __forceinline__ void clear_nt(const GrammarDev& G, const WarpCtx& w) {

@@ -13,6 +13,8 @@ struct GrammarDev {
   const uint16_t* lhs;           // [D]
   const uint8_t* skip;           // [D]
   const uint32_t* class_bits;    // [C][8]
+  const uint8_t* eq_of_byte;     // [256] equivalence class of each byte (same membership in all byte classes)
+  uint32_t n_eq;
   const uint32_t* nt_closure;    // [N][Nw]
   const uint32_t* direct_off;    // [N+1]
   const uint16_t* direct_items;
@@ -46,6 +48,7 @@ enum : uint32_t {
   CNT_N_JOBS = 2,
   CNT_WORK = 3,
   CNT_ERR = 4,          // sticky: some device routine hit a capacity limit
+  CNT_AUTO_ITEMS = 5,   // top of the automaton's item pool (words), reset by every fill
   CNT_POOL_LO = 6,      // 64-bit pool top (words) lives in slots 6,7 (8-byte aligned)
   CNT_STAT_ADV = 8,     // 64-bit statistics from here on, two slots each
   CNT_STAT_FILLS = 10,
@@ -56,8 +59,33 @@ enum : uint32_t {
   CNT_STAT_SETS_MAX = 20,
   CNT_STAT_CAPERR = 22,
   CNT_STAT_BIG = 24,
+  CNT_STAT_TRANS = 26,  // transitions computed by the trie walk (Earley steps)
+  CNT_STAT_LOCAL = 28,  // local states created by the trie walk
   CNT_TOTAL = 32
 };
+
+// Per-job automaton of hash-consed Earley sets, built on demand by the trie walk.  A "local
+// state" is the Earley set reached from the job's base chart by some byte string; equal sets get
+// one id, so a transition (state, byte class) is computed once per job, whatever the number of
+// trie nodes that need it.  Items of a local state name their origin as: a set index of the base
+// chart (< m), m + k for local state k, or ORIGIN_SELF for the state itself.
+// Record of a state (rec_words uint32, a multiple of 32, so records never share a 128-byte line):
+//   [0] first item (word offset into items)  [1] item count  [2] hash  [4..11] scannable bytes
+//   [16 .. 16+n_eq) transition per byte class: T_UNKNOWN, T_PENDING (a warp is computing it),
+//                   T_DEAD or the next state's id
+struct AutoDev {
+  uint32_t cap;        // states per job, state 0 being the base chart's last set
+  uint32_t rec_words;
+  uint32_t hash_mask;  // hash slots per job - 1
+  uint32_t items_cap;  // words of the item pool shared by all jobs
+  uint32_t* recs;      // [jobs][cap][rec_words]
+  uint32_t* hash;      // [jobs][hash_mask + 1], id + 1 or 0
+  uint32_t* items;     // [items_cap]
+  uint32_t* n_states;  // [jobs]
+};
+constexpr uint32_t T_UNKNOWN = 0xffffffffu, T_DEAD = 0xfffffffeu, T_FAIL = 0xfffffffdu, T_PENDING = 0xfffffffcu;
+constexpr uint32_t ORIGIN_SELF = 0xFFFFu;
+constexpr uint32_t AR_ITEMS = 0, AR_N = 1, AR_HASH = 2, AR_SCAN = 4, AR_TRANS = 16;
 
 struct StateDev {
   uint32_t B;
@@ -80,6 +108,7 @@ struct StateDev {
   uint32_t* counters;         // [CNT_TOTAL]
   uint32_t* big_scratch;      // per-warp large scratch areas of the trie walk
   uint32_t big_arena_items, big_hset_slots;
+  AutoDev au;
 };
 
 constexpr int32_t MASK_ZERO = -1;       // row_mask: all-zero mask (broken row)

@@ -113,7 +113,8 @@ __device__ __forceinline__ uint32_t scan_into_cur(const GrammarDev& G, const War
 }
 
 // Complete (Section 3.2) to a fixpoint over cur, starting at item index `head`.  `view(o, ptr, len)`
-// yields the items of set o.  Completed items whose origin is the set itself are not processed:
+// yields the items of set o and `view.fix(item, o)` rewrites an item read from set o into the
+// naming used by the set under construction (identity for plain charts).  Completed items whose origin is the set itself are not processed:
 // they can only come from empty derivations, already covered by `skip`.  Non-terminals found
 // after a dot are collected in w.nt[0..Nw) for the prediction that follows; the accept item is
 // reported in ctr[W_ACCEPT].
@@ -150,7 +151,7 @@ __device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const War
       for (uint32_t k = lane; k < sl; k += 32) {
         uint32_t wi = sp[k];
         uint32_t winf = __ldg(&G.info[wi & 0xFFFFu]);
-        if ((winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X) add_item(G, w, wi + 1u);
+        if ((winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X) add_item(G, w, view.fix(wi, o) + 1u);
       }
       __syncwarp();
     }

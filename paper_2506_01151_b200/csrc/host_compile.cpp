@@ -427,6 +427,20 @@ void compile_grammar(const char* text, size_t len, const std::string& start, Hos
     if (cls_new[c] >= 0)
       for (int w = 0; w < 8; ++w) out.class_bits[(size_t)cls_new[c] * 8 + w] = b.classes[c][w];
 
+  // bytes are equivalent when every byte class contains both or neither: they scan the same items
+  {
+    std::map<std::vector<uint8_t>, uint32_t> seen;
+    out.eq_of_byte.assign(256, 0);
+    for (int byte = 0; byte < 256; ++byte) {
+      std::vector<uint8_t> member((size_t)C);
+      for (int c = 0; c < C; ++c) member[c] = (out.class_bits[(size_t)c * 8 + (byte >> 5)] >> (byte & 31)) & 1u;
+      auto it = seen.find(member);
+      if (it == seen.end()) it = seen.emplace(member, (uint32_t)seen.size()).first;
+      out.eq_of_byte[byte] = (uint8_t)it->second;
+    }
+    out.n_eq = (uint32_t)seen.size();
+  }
+
   out.info.assign(D, 0);
   out.lhs.assign(D, 0);
   out.skip.assign(D, 0);
@@ -559,20 +573,21 @@ void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t 
   // subtree sizes, then split large subtrees into work units
   std::vector<uint32_t> size(out.T, 1);
   for (uint32_t n = out.T; n-- > 1;) size[out.parent[n]] += size[n];
-  if (unit_max_nodes == 0) unit_max_nodes = 192;
+  if (unit_max_nodes == 0) unit_max_nodes = 32;
   std::vector<std::pair<uint32_t, uint32_t>> units;  // (size, node | kind << 31)
   std::vector<uint32_t> stack;
   for (uint32_t c = out.child_off[0]; c < out.child_off[1]; ++c) stack.push_back(c);
   while (!stack.empty()) {
     uint32_t n = stack.back();
     stack.pop_back();
-    if (size[n] <= unit_max_nodes || out.node_depth[n] >= 4) {
+    if (size[n] <= unit_max_nodes || out.node_depth[n] >= 8) {  // a unit's path from the root has at most 8 bytes
       units.push_back({size[n], n});
     } else {
       if (out.tok_off[n + 1] > out.tok_off[n]) units.push_back({1, n | 0x80000000u});
       for (uint32_t c = out.child_off[n]; c < out.child_off[n + 1]; ++c) stack.push_back(c);
     }
   }
+  // largest first: units that stay alive are then spread over many warps
   std::sort(units.begin(), units.end(), [](const std::pair<uint32_t, uint32_t>& a, const std::pair<uint32_t, uint32_t>& b) {
     return a.first != b.first ? a.first > b.first : a.second < b.second;
   });

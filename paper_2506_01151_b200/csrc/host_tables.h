@@ -37,6 +37,8 @@ struct HostTables {
   std::vector<uint32_t> direct_off;    // [N+1]
   std::vector<uint16_t> direct_items;  // start items of each non-terminal's rules, dots moved over
                                        // leading nullable symbols, completed items left out
+  std::vector<uint8_t> eq_of_byte;     // [256] bytes that belong to the same byte classes share a number
+  uint32_t n_eq = 0;                   // how many such equivalence classes of bytes there are
   std::vector<uint8_t> nullable;       // [N]
   std::vector<std::string> nt_names;   // [N]
   // ---- vocabulary trie in CSR form, nodes in breadth-first order (root = 0)

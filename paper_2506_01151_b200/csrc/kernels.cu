@@ -214,7 +214,10 @@ __global__ void __launch_bounds__(ADV_WARPS * 32) advance_kernel(GrammarDev G, S
 
 // One thread per row decides where the row's mask comes from.
 __global__ void plan_kernel(GrammarDev G, StateDev S) {
-  if (blockIdx.x == 0 && threadIdx.x == 0) S.counters[CNT_WORK] = 0u;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    S.counters[CNT_WORK] = 0u;
+    S.counters[CNT_AUTO_ITEMS] = 0u;
+  }
   const uint32_t row = blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= S.B) return;
   stat_add(S, CNT_STAT_FILLS, 1u);
@@ -270,290 +273,424 @@ __global__ void prepare_rows_kernel(GrammarDev G, StateDev S) {
 }
 
 // ===================================================================================== fill: walk
+//
+// The walk answers, for one job (a row whose mask must be computed) and every trie node, "is the
+// Earley set reached by this node's bytes non-empty?".  Sets are hash-consed per job (AutoDev):
+// a transition (state, byte class) is computed once, by whichever warp needs it first, with the
+// warp-cooperative scan / complete / predict of earley_device.cuh; everybody else finds it in the
+// state's record.  Nothing waits: two warps that miss the same transition at the same time both
+// compute it and meet in the same hash slot.  The trie is then walked with one LANE per work
+// unit (a subtree of at most a few hundred nodes), depth first, one table lookup per node.
 
 constexpr int WALK_WARPS = 8;
-constexpr uint32_t WALK_STAGE_WORDS = 4096;  // a base chart up to this size is staged in shared memory
-constexpr uint32_t WALK_ARENA = 1024;        // items of level sets per warp (fast mode)
-constexpr uint32_t WALK_HSET = 512;
-constexpr uint32_t WALK_NT_WORDS = 256;      // 2 * Nw
+constexpr uint32_t WALK_CUR = 1024;     // items of a set under construction per warp (fast mode, power of two)
+constexpr uint32_t WALK_HSET = 2048;    // uniqueness hash slots per warp (fast mode)
+constexpr uint32_t WALK_NT_WORDS = 256; // 2 * Nw
 constexpr uint32_t WALK_LEVELS = MAX_TOKEN_BYTES + 1;
-constexpr uint32_t UNITS_PER_CHUNK = 64;
+constexpr uint32_t WALK_WARP_WORDS = WALK_CUR + WALK_HSET + WALK_NT_WORDS + W_CTRS + 8;
 
-struct Frame {
-  uint32_t node, cursor, pending, batch, set_off, set_len;
-  uint32_t scan[8];
-};
-constexpr uint32_t FRAME_WORDS = sizeof(Frame) / 4;
-constexpr uint32_t WALK_PATH_WORDS = (MAX_TOKEN_BYTES + 4) / 4 + 1;
-constexpr uint32_t WALK_WARP_WORDS =
-    WALK_ARENA + WALK_HSET + WALK_LEVELS * FRAME_WORDS + WALK_NT_WORDS + W_CTRS + WALK_PATH_WORDS;
-constexpr uint32_t WALK_BLOCK_WORDS = WALK_STAGE_WORDS + 16;
-
-struct Walker {
-  const GrammarDev& G;
-  WarpCtx w;
-  uint32_t* arena;
-  uint32_t arena_cap;
-  Frame* frames;
-  uint8_t* path;
+struct JobCtx {
   const uint32_t* base_off;
   const uint32_t* base_items;
-  uint32_t m;  // live sets of the base chart
+  uint32_t m;         // live sets of the base chart
+  uint32_t* recs;     // this job's state records
+  uint32_t* hash;
+  uint32_t* n_states;
+  uint32_t cap;       // states this job may create (ids stay below ORIGIN_SELF - m)
   uint32_t* mask_row;
-  uint32_t top;  // items in use in the arena
+};
 
-  struct View {
-    const Walker& wk;
-    __device__ __forceinline__ void operator()(uint32_t o, const uint32_t*& p, uint32_t& n) const {
-      if (o < wk.m) {
-        uint32_t a = wk.base_off[o], b = wk.base_off[o + 1];
-        p = wk.base_items + a;
-        n = b - a;
-      } else {
-        const Frame& f = wk.frames[o - (wk.m - 1)];
-        p = wk.arena + f.set_off;
-        n = f.set_len;
-      }
-    }
-  };
-
-  __device__ __forceinline__ void emit_tokens(uint32_t node) const {
-    uint32_t a = __ldg(&G.tok_off[node]), b = __ldg(&G.tok_off[node + 1]);
-    for (uint32_t i = a; i < b; ++i) {
-      uint32_t t = __ldg(&G.tok_ids[i]);
-      atomicOr(&mask_row[t >> 5], 1u << (t & 31u));
+struct AutoView {
+  const JobCtx& J;
+  const AutoDev& A;
+  __device__ __forceinline__ void operator()(uint32_t o, const uint32_t*& p, uint32_t& n) const {
+    if (o < J.m) {
+      uint32_t a = J.base_off[o], b = J.base_off[o + 1];
+      p = J.base_items + a;
+      n = b - a;
+    } else {
+      const uint32_t* rec = J.recs + (size_t)(o - J.m) * A.rec_words;
+      p = A.items + rec[AR_ITEMS];
+      n = rec[AR_N];
     }
   }
+  // an item of local state o that names its own state as origin means "origin o"
+  __device__ __forceinline__ uint32_t fix(uint32_t item, uint32_t o) const {
+    return ((item >> 16) == ORIGIN_SELF) ? ((o << 16) | (item & 0xFFFFu)) : item;
+  }
+};
 
-  // The Earley set of trie depth `level`, reached from `parent` by `byte`:
-  // scan, complete, predict; no pruning inside a token.  1 ok, 0 empty, -1 overflow.
-  __device__ int step(const uint32_t* parent, uint32_t plen, uint32_t level, uint32_t byte) {
+struct WalkWarp {
+  const GrammarDev& G;
+  const StateDev& S;
+  WarpCtx w;
+  uint32_t cur_pow2;   // capacity of w.cur rounded down to a power of two (for the sort)
+  uint32_t* tmp8;      // shared
+
+  // Find or create the local state whose items are w.cur[0..n) (sorted).  Returns its id or T_FAIL.
+  __device__ uint32_t intern_set(const JobCtx& J, uint32_t n, uint32_t hash) {
     const uint32_t lane = lane_id();
-    if (top + 64 > arena_cap) return -1;
-    w.cur = arena + top;
-    w.cur_cap = arena_cap - top;
+    const AutoDev& A = S.au;
+    uint32_t slot = hash & A.hash_mask;
+    uint32_t my_id = T_FAIL;
+    for (uint32_t probe = 0; probe < 1024; ++probe) {
+      uint32_t v = 0;
+      if (lane == 0) v = ld_acquire(&J.hash[slot]);
+      v = __shfl_sync(FULL, v, 0);
+      if (v == 0) {
+        if (my_id == T_FAIL) {
+          uint32_t id = T_FAIL, ioff = 0;
+          if (lane == 0) {
+            if (ld_acquire(J.n_states) < J.cap) {
+              uint32_t got = atomicAdd(J.n_states, 1u);
+              uint32_t need = (max(n, 1u) + 31u) & ~31u;
+              if (got < J.cap && ld_acquire(&S.counters[CNT_AUTO_ITEMS]) + need <= A.items_cap) {
+                ioff = atomicAdd(&S.counters[CNT_AUTO_ITEMS], need);
+                if (ioff + need <= A.items_cap) id = got;
+              }
+            }
+          }
+          id = __shfl_sync(FULL, id, 0);
+          ioff = __shfl_sync(FULL, ioff, 0);
+          if (id == T_FAIL) return T_FAIL;
+          uint32_t* rec = J.recs + (size_t)id * A.rec_words;
+          uint32_t* items = A.items + ioff;
+          for (uint32_t i = lane; i < n; i += 32) items[i] = w.cur[i];
+          for (uint32_t i = lane; i < A.rec_words; i += 32) {
+            uint32_t v2 = 0u;
+            if (i == AR_ITEMS) v2 = ioff;
+            else if (i == AR_N) v2 = n;
+            else if (i == AR_HASH) v2 = hash;
+            else if (i >= AR_SCAN && i < AR_SCAN + 8) v2 = tmp8[i - AR_SCAN];
+            else if (i >= AR_TRANS) v2 = T_UNKNOWN;
+            rec[i] = v2;
+          }
+          __syncwarp();
+          __threadfence();
+          my_id = id;
+          if (lane == 0) stat_add(S, CNT_STAT_LOCAL, 1u);
+        }
+        uint32_t old = 0;
+        if (lane == 0) old = atomicCAS(&J.hash[slot], 0u, my_id + 1u);
+        old = __shfl_sync(FULL, old, 0);
+        if (old == 0) return my_id;
+        v = old;
+      }
+      const uint32_t sid = v - 1u;
+      const uint32_t* rec = J.recs + (size_t)sid * A.rec_words;
+      bool same = (__ldcg(rec + AR_HASH) == hash) && (__ldcg(rec + AR_N) == n);
+      if (same) {
+        const uint32_t* items = A.items + __ldcg(rec + AR_ITEMS);
+        for (uint32_t i = lane; i < n; i += 32)
+          if (__ldcg(items + i) != w.cur[i]) same = false;
+      }
+      same = __all_sync(FULL, same);
+      if (same) return sid;
+      slot = (slot + 1u) & A.hash_mask;
+    }
+    return T_FAIL;
+  }
+
+  // Compute, publish and return the transition of local state `ps` on `byte`: T_DEAD, a state
+  // id, or T_FAIL when a capacity was exceeded.  The first warp to ask claims the transition
+  // (T_PENDING); a warp that finds it claimed gets T_PENDING back and asks again later, unless
+  // `force` is set, in which case it computes the transition itself (both results are equal).
+  __device__ uint32_t compute(const JobCtx& J, uint32_t ps, uint32_t byte, bool force) {
+    const uint32_t lane = lane_id();
+    const AutoDev& A = S.au;
+    const uint32_t e = __ldg(&G.eq_of_byte[byte]);
+    uint32_t* slot = J.recs + (size_t)ps * A.rec_words + AR_TRANS + e;
+    uint32_t t = 0;
+    if (lane == 0) {
+      t = __ldcg(slot);
+      if (t == T_UNKNOWN) {
+        t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
+        if (t == T_UNKNOWN) t = T_FAIL;  // stands for "claimed by this warp" until the broadcast below
+      }
+    }
+    t = __shfl_sync(FULL, t, 0);
+    if (t == T_PENDING) {
+      if (!force) return T_PENDING;
+    } else if (t != T_FAIL) {
+      return t;  // published meanwhile
+    }
+    const uint32_t* pitems;
+    uint32_t plen;
+    AutoView view{J, A};
+    view(ps == 0 ? J.m - 1 : J.m + ps, pitems, plen);
     __syncwarp();
     if (lane < W_CTRS) w.ctr[lane] = 0u;
     __syncwarp();
-    uint32_t n = scan_into_cur(G, w, parent, plen, byte);
+    const uint32_t self_code = J.m + ps;
+    for (uint32_t k = lane; k < plen; k += 32) {
+      uint32_t it = pitems[k];
+      uint32_t inf = __ldg(&G.info[it & 0xFFFFu]);
+      if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) {
+        if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
+        add_item(G, w, it + 1u);
+      }
+    }
+    __syncwarp();
+    uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
     if (w.ctr[W_OVERFLOW]) {
       hset_clear_all(w.hset, w.hset_mask);
-      return -1;
+      return T_FAIL;
     }
-    if (n == 0) return 0;
-    const uint32_t cur_index = m - 1 + level;
-    complete_fixpoint(G, w, View{*this}, cur_index, 0u);
+    if (n == 0) {
+      if (lane == 0) atomicExch(slot, T_DEAD);
+      return T_DEAD;
+    }
+    complete_fixpoint(G, w, view, ORIGIN_SELF, 0u);
     uint32_t hashed = min(w.ctr[W_NCUR], w.cur_cap);
     if (w.ctr[W_OVERFLOW]) {
       hset_clear_all(w.hset, w.hset_mask);
       clear_nt(G, w);
-      return -1;
+      return T_FAIL;
     }
     hset_clear_items(w, hashed);
-    predict_into_cur(G, w, cur_index);
-    if (w.ctr[W_OVERFLOW]) return -1;
+    predict_into_cur(G, w, ORIGIN_SELF);
+    if (w.ctr[W_OVERFLOW]) return T_FAIL;
     n = drop_completed(G, w, min(w.ctr[W_NCUR], w.cur_cap));
+    sort_items(w.cur, n, cur_pow2);
+    uint32_t h = 0x9E3779B9u ^ n;
+    for (uint32_t i = lane; i < n; i += 32) h += mix32(w.cur[i] ^ (i * 0x85EBCA77u));
+    for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
+    scannable_bytes(G, w.cur, n, tmp8);
+    uint32_t id = intern_set(J, n, h);
+    if (id == T_FAIL) return T_FAIL;
     if (lane == 0) {
-      frames[level].set_off = top;
-      frames[level].set_len = n;
+      atomicExch(slot, id);
+      stat_add(S, CNT_STAT_TRANS, 1u);
     }
-    __syncwarp();
-    top += n;
-    return 1;
-  }
-
-  __device__ __forceinline__ void open_frame(uint32_t level, uint32_t node) {
-    Frame& f = frames[level];
-    __syncwarp();
-    if (lane_id() == 0) {
-      f.node = node;
-      f.cursor = __ldg(&G.child_off[node]);
-      f.pending = 0;
-      f.batch = 0;
-    }
-    __syncwarp();
-    scannable_bytes(G, arena + f.set_off, f.set_len, f.scan);
-  }
-
-  // One work unit.  1 done, -1 overflow.
-  __device__ int unit(uint32_t u, const uint32_t* base_scan) {
-    const uint32_t lane = lane_id();
-    const uint32_t root = __ldg(&G.unit_node[u]);
-    const uint32_t kind = __ldg(&G.unit_kind[u]);
-    const uint32_t dr = __ldg(&G.node_depth[root]);
-    if (dr == 0 || dr >= WALK_LEVELS) return 1;
-    __syncwarp();
-    if (lane == 0) {
-      uint32_t n = root;
-      for (uint32_t i = dr; i >= 1; --i) {
-        path[i] = __ldg(&G.node_byte[n]);
-        n = __ldg(&G.parent[n]);
-      }
-    }
-    __syncwarp();
-    const uint32_t first = path[1];
-    if (!((base_scan[first >> 5] >> (first & 31u)) & 1u)) return 1;  // the first byte cannot follow
-    top = 0;
-    const uint32_t* pset = base_items + base_off[m - 1];
-    uint32_t plen = base_off[m] - base_off[m - 1];
-    const uint32_t full_levels = kind ? dr - 1 : dr;
-    for (uint32_t L = 1; L <= full_levels; ++L) {
-      int r = step(pset, plen, L, path[L]);
-      if (r <= 0) return r == 0 ? 1 : -1;
-      pset = arena + frames[L].set_off;
-      plen = frames[L].set_len;
-    }
-    if (kind) {  // the node alone: does its last byte scan?
-      bool hit = false;
-      const uint32_t byte = path[dr];
-      for (uint32_t k = lane; k < plen; k += 32) {
-        uint32_t inf = __ldg(&G.info[pset[k] & 0xFFFFu]);
-        if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) hit = true;
-      }
-      if (__any_sync(FULL, hit) && lane == 0) emit_tokens(root);
-      return 1;
-    }
-    if (lane == 0) emit_tokens(root);
-    if (__ldg(&G.child_off[root + 1]) == __ldg(&G.child_off[root])) return 1;
-    open_frame(dr, root);
-    uint32_t depth = dr;
-    for (;;) {
-      Frame& f = frames[depth];
-      __syncwarp();
-      const uint32_t pending = f.pending;
-      if (pending == 0) {
-        const uint32_t c0 = f.cursor, cend = __ldg(&G.child_off[f.node + 1]);
-        if (c0 >= cend) {
-          top = f.set_off;
-          if (depth == dr) break;
-          --depth;
-          continue;
-        }
-        const uint32_t c = c0 + lane;
-        bool internal = false;
-        if (c < cend) {
-          const uint32_t b = __ldg(&G.node_byte[c]);
-          if ((f.scan[b >> 5] >> (b & 31u)) & 1u) {
-            emit_tokens(c);
-            internal = __ldg(&G.child_off[c + 1]) > __ldg(&G.child_off[c]);
-          }
-        }
-        const uint32_t bal = __ballot_sync(FULL, internal);
-        __syncwarp();
-        if (lane == 0) {
-          f.pending = bal;
-          f.batch = c0;
-          f.cursor = c0 + 32;
-        }
-      } else {
-        const uint32_t k = (uint32_t)__ffs(pending) - 1u;
-        const uint32_t c = f.batch + k;
-        const uint32_t poff = f.set_off, plen2 = f.set_len;
-        __syncwarp();
-        if (lane == 0) f.pending = pending & (pending - 1u);
-        __syncwarp();
-        if (depth + 1 >= WALK_LEVELS) continue;  // cannot happen: tokens are at most MAX_TOKEN_BYTES long
-        int r = step(arena + poff, plen2, depth + 1, __ldg(&G.node_byte[c]));
-        if (r < 0) return -1;
-        if (r > 0) {
-          ++depth;
-          open_frame(depth, c);
-        }
-      }
-    }
-    return 1;
+    return id;
   }
 };
 
-__global__ void __launch_bounds__(WALK_WARPS * 32) walk_kernel(GrammarDev G, StateDev S) {
+__device__ __forceinline__ void emit_tokens(const GrammarDev& G, uint32_t* mask_row, uint32_t node) {
+  uint32_t a = __ldg(&G.tok_off[node]), b = __ldg(&G.tok_off[node + 1]);
+  for (uint32_t i = a; i < b; ++i) {
+    uint32_t t = __ldg(&G.tok_ids[i]);
+    atomicOr(&mask_row[t >> 5], 1u << (t & 31u));
+  }
+}
+
+// Set up the automata of this call's jobs: empty hash, one state (the base chart's last set).
+__global__ void auto_init_kernel(GrammarDev G, StateDev S) {
+  const uint32_t j = blockIdx.x;
+  if (j >= S.counters[CNT_N_JOBS]) return;
+  const AutoDev& A = S.au;
+  uint32_t* hash = A.hash + (size_t)j * (A.hash_mask + 1);
+  for (uint32_t i = threadIdx.x; i <= A.hash_mask; i += blockDim.x) hash[i] = 0u;
+  uint32_t* rec0 = A.recs + (size_t)j * A.cap * A.rec_words;
+  for (uint32_t i = threadIdx.x; i < A.rec_words; i += blockDim.x)
+    if (i < AR_SCAN || i >= AR_SCAN + 8) rec0[i] = (i >= AR_TRANS) ? T_UNKNOWN : 0u;
+  if (threadIdx.x == 0) A.n_states[j] = 1u;
+  if (threadIdx.x < 32) {
+    const uint32_t row = S.jobs[j];
+    const uint32_t* ch = S.arena + S.row_chart[row];
+    const uint32_t m = ch[CH_SETS];
+    const uint32_t* off = ch + CH_HDR;
+    const uint32_t* items = ch + CH_HDR + m + 1;
+    __shared__ uint32_t sc[8];
+    scannable_bytes(G, items + off[m - 1], off[m] - off[m - 1], sc);
+    if (threadIdx.x < 8) rec0[AR_SCAN + threadIdx.x] = sc[threadIdx.x];
+  }
+}
+
+__global__ void __launch_bounds__(WALK_WARPS * 32, 2) walk_kernel(GrammarDev G, StateDev S) {
   extern __shared__ uint32_t smem[];
-  uint32_t* stage = smem;
-  uint32_t* base_scan = smem + WALK_STAGE_WORDS;  // [8]
-  uint32_t* blk = smem + WALK_STAGE_WORDS + 8;     // [8]
   const uint32_t warp = threadIdx.x >> 5, lane = lane_id();
-  uint32_t* mine = smem + WALK_BLOCK_WORDS + (size_t)warp * WALK_WARP_WORDS;
-  uint32_t* sm_arena = mine;
-  uint32_t* sm_hset = sm_arena + WALK_ARENA;
-  Frame* frames = reinterpret_cast<Frame*>(sm_hset + WALK_HSET);
-  uint32_t* nt = reinterpret_cast<uint32_t*>(frames) + WALK_LEVELS * FRAME_WORDS;
+  uint32_t* mine = smem + (size_t)warp * WALK_WARP_WORDS;
+  uint32_t* sm_cur = mine;
+  uint32_t* sm_hset = sm_cur + WALK_CUR;
+  uint32_t* nt = sm_hset + WALK_HSET;
   uint32_t* ctr = nt + WALK_NT_WORDS;
-  uint8_t* path = reinterpret_cast<uint8_t*>(ctr + W_CTRS);
+  uint32_t* tmp8 = ctr + W_CTRS;
   // the large scratch area of this warp (global memory)
   uint32_t* big = S.big_scratch + ((size_t)blockIdx.x * WALK_WARPS + warp) * ((size_t)S.big_arena_items + S.big_hset_slots);
+  const AutoDev& A = S.au;
 
   hset_clear_all(sm_hset, WALK_HSET - 1);
   for (uint32_t i = lane; i < WALK_NT_WORDS; i += 32) nt[i] = 0u;
   __syncwarp();
-  const uint32_t n_chunks = (G.U + UNITS_PER_CHUNK - 1) / UNITS_PER_CHUNK;
+  const uint32_t n_groups = (G.U + 31) / 32;
   const uint32_t n_jobs = S.counters[CNT_N_JOBS];
-  const uint32_t total = n_jobs * n_chunks;
+  const uint32_t total = n_jobs * n_groups;
+
+  WalkWarp ww{G, S};
+  ww.w.nt = nt;
+  ww.w.ctr = ctr;
+  ww.tmp8 = tmp8;
 
   for (;;) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      blk[0] = atomicAdd(&S.counters[CNT_WORK], 1u);
-      blk[1] = 0u;
-    }
-    __syncthreads();
-    const uint32_t item = blk[0];
-    if (item >= total) return;
-    const uint32_t job = item / n_chunks, chunk = item % n_chunks;
-    const uint32_t row = S.jobs[job];
+    uint32_t item = 0;
+    if (lane == 0) item = atomicAdd(&S.counters[CNT_WORK], 1u);
+    item = __shfl_sync(FULL, item, 0);
+    if (item >= total) break;
+    // consecutive items belong to different jobs, so that few warps explore one automaton at a time
+    const uint32_t j = item % n_jobs, grp = item / n_jobs;
+    const uint32_t row = S.jobs[j];
     const uint32_t* chart = S.arena + S.row_chart[row];
-    const uint32_t m = chart[CH_SETS], words = chart[CH_WORDS];
-    const uint32_t* base = chart;
-    if (words <= WALK_STAGE_WORDS) {
-      for (uint32_t i = threadIdx.x; i < words; i += blockDim.x) stage[i] = chart[i];
-      base = stage;
-    }
-    __syncthreads();
-    const uint32_t* base_off = base + CH_HDR;
-    const uint32_t* base_items = base + CH_HDR + m + 1;
-    if (warp == 0) scannable_bytes(G, base_items + base_off[m - 1], base_off[m] - base_off[m - 1], base_scan);
-    __syncthreads();
+    JobCtx J;
+    J.m = chart[CH_SETS];
+    J.base_off = chart + CH_HDR;
+    J.base_items = chart + CH_HDR + J.m + 1;
+    J.recs = A.recs + (size_t)j * A.cap * A.rec_words;
+    J.hash = A.hash + (size_t)j * (A.hash_mask + 1);
+    J.n_states = A.n_states + j;
+    J.cap = min(A.cap, (ORIGIN_SELF - 1u > J.m) ? ORIGIN_SELF - 1u - J.m : 0u);
+    J.mask_row = S.mask_rows + (size_t)S.row_mask[row] * G.Wm;
+    // fast mode: scratch in shared memory
+    ww.w.cur = sm_cur;
+    ww.w.cur_cap = WALK_CUR;
+    ww.cur_pow2 = WALK_CUR;
+    ww.w.hset = sm_hset;
+    ww.w.hset_mask = WALK_HSET - 1;
+    bool big_mode = false, broken = false, force = false;
+    uint32_t stalled = 0;
 
-    Walker wk{G};
-    wk.w.hset = sm_hset;
-    wk.w.hset_mask = WALK_HSET - 1;
-    wk.w.nt = nt;
-    wk.w.ctr = ctr;
-    wk.arena = sm_arena;
-    wk.arena_cap = WALK_ARENA;
-    wk.frames = frames;
-    wk.path = path;
-    wk.base_off = base_off;
-    wk.base_items = base_items;
-    wk.m = m;
-    wk.mask_row = S.mask_rows + (size_t)S.row_mask[row] * G.Wm;
-    wk.top = 0;
-    bool big_mode = false;
-    for (;;) {
-      uint32_t k = 0;
-      if (lane == 0) k = atomicAdd(&blk[1], 1u);
-      k = __shfl_sync(FULL, k, 0);
-      const uint32_t u = chunk + k * n_chunks;
-      if (u >= G.U) break;
-      int r = wk.unit(u, base_scan);
-      if (r < 0 && !big_mode) {  // redo the unit, and do the rest of this chunk, with the large scratch area
-        big_mode = true;
-        hset_clear_all(wk.w.hset, wk.w.hset_mask);
-        wk.arena = big;
-        wk.arena_cap = S.big_arena_items;
-        wk.w.hset = big + S.big_arena_items;
-        wk.w.hset_mask = S.big_hset_slots - 1;
-        clear_nt(G, wk.w);
-        if (lane == 0) stat_add(S, CNT_STAT_BIG, 1u);
-        r = wk.unit(u, base_scan);
-      }
-      if (r < 0) {  // even the large area is too small: the row's mask cannot be trusted
-        hset_clear_all(wk.w.hset, wk.w.hset_mask);
-        clear_nt(G, wk.w);
-        if (lane == 0) {
-          atomicOr(&S.row_flags[row], ROW_BROKEN);
-          atomicExch(&S.counters[CNT_ERR], 1u);
-          stat_add(S, CNT_STAT_CAPERR, 1u);
+    // ---- one work unit per lane
+    const uint32_t u = grp * 32 + lane;
+    uint32_t phase = 2;  // 0 following the unit's path from the root, 1 inside its subtree, 2 done
+    uint32_t root = 0, kind = 0, dr = 0, pk = 1, node = 0, depth = 0;
+    uint64_t path = 0;  // the bytes from the root to the unit's node, first byte lowest
+    uint16_t st[WALK_LEVELS];
+    st[0] = 0;
+    if (u < G.U) {
+      root = __ldg(&G.unit_node[u]);
+      kind = __ldg(&G.unit_kind[u]);
+      dr = __ldg(&G.node_depth[root]);
+      if (dr >= 1 && dr <= 8) {
+        uint32_t n = root;
+        for (uint32_t i = dr; i >= 1; --i) {
+          path |= (uint64_t)__ldg(&G.node_byte[n]) << (8 * (i - 1));
+          n = __ldg(&G.parent[n]);
         }
-        break;
+        phase = 0;
+      }
+    }
+    for (;;) {
+      uint32_t q_state = 0, q_byte = 0;
+      if (phase == 0) {
+        q_state = st[pk - 1];
+        q_byte = (uint32_t)(path >> (8 * (pk - 1))) & 0xFFu;
+      } else if (phase == 1) {
+        q_state = st[depth - 1];
+        q_byte = __ldg(&G.node_byte[node]);
+      }
+      const bool has_q = phase < 2;
+      if (__ballot_sync(FULL, has_q) == 0u) break;
+      uint32_t t = T_UNKNOWN, q_eq = 0;
+      if (has_q) {
+        q_eq = __ldg(&G.eq_of_byte[q_byte]);
+        const uint32_t* rec = J.recs + (size_t)q_state * A.rec_words;
+        // one 256-bit test rejects most bytes without touching the transition table
+        if (!((rec[AR_SCAN + (q_byte >> 5)] >> (q_byte & 31u)) & 1u)) t = T_DEAD;
+        else {
+          t = rec[AR_TRANS + q_eq];
+          if (t == T_UNKNOWN) t = __ldcg(rec + AR_TRANS + q_eq);
+        }
+      }
+      bool need = has_q && (t == T_UNKNOWN || t == T_PENDING);
+      bool waiting = false;  // the transition is being computed by another warp: ask again next round
+      uint32_t bal = __ballot_sync(FULL, need);
+      while (bal) {
+        const int src = __ffs(bal) - 1;
+        const uint32_t ps = __shfl_sync(FULL, q_state, src);
+        const uint32_t pb = __shfl_sync(FULL, q_byte, src);
+        const uint32_t pe = __shfl_sync(FULL, q_eq, src);
+        uint32_t r = ww.compute(J, ps, pb, force);
+        if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
+          big_mode = true;
+          hset_clear_all(ww.w.hset, ww.w.hset_mask);
+          clear_nt(G, ww.w);
+          ww.w.cur = big;
+          ww.w.cur_cap = S.big_arena_items;
+          ww.cur_pow2 = S.big_arena_items;
+          ww.w.hset = big + S.big_arena_items;
+          ww.w.hset_mask = S.big_hset_slots - 1;
+          if (lane == 0) stat_add(S, CNT_STAT_BIG, 1u);
+          r = ww.compute(J, ps, pb, true);
+        }
+        if (r == T_FAIL) {
+          broken = true;
+          break;
+        }
+        if (need && q_state == ps && q_eq == pe) {
+          need = false;
+          if (r == T_PENDING) waiting = true;
+          else t = r;
+        }
+        bal = __ballot_sync(FULL, need);
+      }
+      if (broken) break;
+      // If every lane that still has work waits for other warps, back off briefly; after many such
+      // rounds stop relying on them and compute the transitions here (bounded wait, no deadlock).
+      if (__ballot_sync(FULL, has_q && !waiting) == 0u) {
+        if (++stalled > 256u) force = true;
+        __nanosleep(stalled > 16u ? 400u : 50u);
+      } else {
+        stalled = 0;
+        force = false;
+      }
+      if (waiting) continue;
+      // ---- every lane moves on with its answer
+      if (phase == 0) {
+        if (t == T_DEAD) {
+          phase = 2;
+        } else {
+          st[pk] = (uint16_t)t;
+          if (pk == dr) {
+            emit_tokens(G, J.mask_row, root);
+            const uint32_t c0 = __ldg(&G.child_off[root]), c1 = __ldg(&G.child_off[root + 1]);
+            if (kind == 1 || c1 == c0) {
+              phase = 2;
+            } else {
+              node = c0;
+              depth = dr + 1;
+              phase = 1;
+            }
+          } else {
+            ++pk;
+          }
+        }
+      } else if (phase == 1) {
+        bool descend = false;
+        if (t != T_DEAD) {
+          emit_tokens(G, J.mask_row, node);
+          const uint32_t c0 = __ldg(&G.child_off[node]), c1 = __ldg(&G.child_off[node + 1]);
+          if (c1 > c0 && depth + 1 < WALK_LEVELS) {
+            st[depth] = (uint16_t)t;
+            node = c0;
+            ++depth;
+            descend = true;
+          }
+        }
+        if (!descend) {  // next sibling, or climb until there is one
+          for (;;) {
+            const uint32_t p = __ldg(&G.parent[node]);
+            if (node + 1 < __ldg(&G.child_off[p + 1])) {
+              ++node;
+              break;
+            }
+            node = p;
+            --depth;
+            if (node == root) {
+              phase = 2;
+              break;
+            }
+          }
+        }
+      }
+    }
+    if (big_mode) hset_clear_all(ww.w.hset, ww.w.hset_mask);
+    if (broken) {  // a capacity was exceeded: the row's mask cannot be trusted
+      hset_clear_all(ww.w.hset, ww.w.hset_mask);
+      clear_nt(G, ww.w);
+      if (lane == 0) {
+        atomicOr(&S.row_flags[row], ROW_BROKEN);
+        atomicExch(&S.counters[CNT_ERR], 1u);
+        stat_add(S, CNT_STAT_CAPERR, 1u);
       }
     }
   }
@@ -740,7 +877,7 @@ static inline cudaError_t opt_in_smem(const void* fn, size_t bytes) {
 
 static size_t adv_smem_bytes() { return (size_t)ADV_WARPS * ADV_WARP_WORDS * 4; }
 static size_t init_smem_bytes() { return (size_t)ADV_WARP_WORDS * 4; }
-static size_t walk_smem_bytes() { return ((size_t)WALK_BLOCK_WORDS + (size_t)WALK_WARPS * WALK_WARP_WORDS) * 4; }
+static size_t walk_smem_bytes() { return (size_t)WALK_WARPS * WALK_WARP_WORDS * 4; }
 int walk_warps() { return WALK_WARPS; }
 
 cudaError_t configure_kernels() {
@@ -772,12 +909,14 @@ void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStre
                  cudaEvent_t after_walk) {
   plan_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(G, S);
   prepare_rows_kernel<<<S.B, 256, 0, st>>>(G, S);
+  auto_init_kernel<<<S.B, 256, 0, st>>>(G, S);
   if (before_walk) cudaEventRecord(before_walk, st);
   walk_kernel<<<walk_grid, WALK_WARPS * 32, walk_smem_bytes(), st>>>(G, S);
   if (after_walk) cudaEventRecord(after_walk, st);
   publish_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(S);
 }
 void launch_walk(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) {
+  auto_init_kernel<<<S.B, 256, 0, st>>>(G, S);
   walk_kernel<<<grid, WALK_WARPS * 32, walk_smem_bytes(), st>>>(G, S);
 }
 void launch_end_fill(const StateDev& S, cudaStream_t st) { end_fill_kernel<<<1, 1, 0, st>>>(S); }

@@ -6,6 +6,7 @@
 // cudaGetSymbolAddress and passed as an ordinary pointer.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "../../include/fmt.h"
@@ -17,7 +18,7 @@ namespace {
 using namespace fmt;
 
 constexpr uint32_t NA_MAX = FMT_NOALLOC_MAX_CHARTS;
-constexpr uint32_t NA_GRID = 64;            // CTAs of the walk
+constexpr uint32_t NA_GRID = 32;            // CTAs of the walk
 constexpr uint32_t NA_ARENA_ITEMS = 8192;   // per-warp overflow area for Earley sets (items)
 constexpr uint32_t NA_HSET_SLOTS = 2048;    // per-warp overflow uniqueness hash
 // header: counters, then per-chart arrays
@@ -27,13 +28,24 @@ constexpr uint32_t NA_OFF_FLAGS = NA_OFF_JOBS + NA_MAX;          // [NA_MAX]
 constexpr uint32_t NA_OFF_MASKROW = NA_OFF_FLAGS + NA_MAX;       // [NA_MAX] int32
 constexpr uint32_t NA_OFF_CHART = NA_OFF_MASKROW + NA_MAX;       // [NA_MAX] uint64 (8-byte aligned)
 constexpr uint32_t NA_OFF_BAD = NA_OFF_CHART + 2 * NA_MAX;       // [NA_MAX] header check failed
+constexpr uint32_t NA_OFF_NSTATES = NA_OFF_BAD + NA_MAX;         // [NA_MAX] Earley sets created per chart
 constexpr uint32_t NA_HEADER_WORDS = 1024;
 constexpr size_t NA_WARPS = (size_t)NA_GRID * 8;
-constexpr size_t NA_WORDS = NA_HEADER_WORDS + NA_WARPS * (NA_ARENA_ITEMS + NA_HSET_SLOTS);
-static_assert(NA_OFF_BAD + NA_MAX <= NA_HEADER_WORDS, "header too small");
+constexpr size_t NA_BIG_WORDS = NA_WARPS * (NA_ARENA_ITEMS + NA_HSET_SLOTS);
+// the walk's tables of Earley sets: per chart 64 Ki words of records and 2048 hash slots, and one
+// pool of 2 Mi item words for all charts of a call
+constexpr uint32_t NA_REC_WORDS_PER_CHART = 65536;
+constexpr uint32_t NA_HASH_SLOTS = 2048;
+constexpr uint32_t NA_ITEM_WORDS = 2u << 20;
+constexpr size_t NA_OFF_BIG = NA_HEADER_WORDS;
+constexpr size_t NA_OFF_RECS = NA_OFF_BIG + NA_BIG_WORDS;
+constexpr size_t NA_OFF_HASH = NA_OFF_RECS + (size_t)NA_MAX * NA_REC_WORDS_PER_CHART;
+constexpr size_t NA_OFF_ITEMS = NA_OFF_HASH + (size_t)NA_MAX * NA_HASH_SLOTS;
+constexpr size_t NA_WORDS = NA_OFF_ITEMS + NA_ITEM_WORDS;
+static_assert(NA_OFF_NSTATES + NA_MAX <= NA_HEADER_WORDS, "header too small");
 static_assert((NA_OFF_CHART % 2) == 0, "64-bit offsets must be 8-byte aligned");
 
-// ~21 MB, held by every GPU that loads the library until the process exits
+// ~36 MB, held by every GPU that loads the library until the process exits
 static __device__ __align__(256) uint32_t g_noalloc_scratch[NA_WORDS];
 
 struct Offsets {
@@ -63,6 +75,7 @@ __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scrat
     S.row_flags[r] = 0u;
   }
   for (size_t i = tid; i < (size_t)n * G.Wm; i += nth) mask[i] = 0u;
+  if (tid == 0) S.counters[CNT_AUTO_ITEMS] = 0u;
   uint32_t* big = S.big_scratch;
   const size_t per_warp = (size_t)NA_ARENA_ITEMS + NA_HSET_SLOTS;
   for (size_t i = tid; i < NA_WARPS * NA_HSET_SLOTS; i += nth)
@@ -154,9 +167,17 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   S.row_mask = reinterpret_cast<int32_t*>(scratch + NA_OFF_MASKROW);
   S.row_chart = reinterpret_cast<uint64_t*>(scratch + NA_OFF_CHART);
   S.mask_rows = mask_dev;
-  S.big_scratch = scratch + NA_HEADER_WORDS;
+  S.big_scratch = scratch + NA_OFF_BIG;
   S.big_arena_items = NA_ARENA_ITEMS;
   S.big_hset_slots = NA_HSET_SLOTS;
+  S.au.rec_words = (AR_TRANS + G->n_eq + 31u) & ~31u;
+  S.au.cap = std::min<uint32_t>(1024u, NA_REC_WORDS_PER_CHART / S.au.rec_words);
+  S.au.hash_mask = NA_HASH_SLOTS - 1;
+  S.au.items_cap = NA_ITEM_WORDS;
+  S.au.recs = scratch + NA_OFF_RECS;
+  S.au.hash = scratch + NA_OFF_HASH;
+  S.au.items = scratch + NA_OFF_ITEMS;
+  S.au.n_states = scratch + NA_OFF_NSTATES;
   cudaStream_t st = (cudaStream_t)stream;
   noalloc_prepare_kernel<<<256, 256, 0, st>>>(*G, S, scratch, charts_dev, off, n, mask_dev);
   noalloc_jobs_kernel<<<1, 32, 0, st>>>(*G, S, scratch, charts_dev, n, mask_dev);
