@@ -265,7 +265,7 @@ def run_ours(args):
                   "big_mode": stats1["big_mode_units"] - stats0["big_mode_units"]},
         "cold": cold,
         "grammar": {"nonterminals": info.n_nonterminals, "rules": info.n_rules, "dotted": info.n_dotted,
-                    "trie_nodes": info.trie_nodes, "units": info.n_units},
+                    "trie_nodes": info.trie_nodes, "byte_classes": info.n_byte_classes},
     }
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, W, budget_s=args.cpu_seconds)

@@ -60,9 +60,7 @@ typedef struct fmt_state fmt_state;
 typedef struct {
   uint32_t host_only;        /* 1: build the tables on the host only (no device needed; the
                                 grammar can be inspected but no state can be created) */
-  uint32_t unit_max_nodes;   /* trie subtrees larger than this are split into several work
-                                units (default 32) */
-  uint32_t reserved[6];
+  uint32_t reserved[7];
 } fmt_compile_options;
 
 /* Options of fmt_state_create.  Zero-initialise; 0 means "default". */
@@ -87,7 +85,7 @@ typedef struct {
   uint32_t mask_words;       /* ceil(V/32) */
   uint32_t trie_nodes;       /* T, including the root */
   uint32_t trie_depth;       /* longest token in bytes */
-  uint32_t n_units;          /* work units of the mask kernel */
+  uint32_t n_byte_classes;   /* bytes fall into this many classes that no grammar terminal tells apart */
   uint32_t n_empty_tokens;   /* tokens with no bytes (EOS included) */
   uint32_t start_nullable;   /* 1 if the empty string is a sentence */
 } fmt_grammar_info;
@@ -104,7 +102,7 @@ typedef struct {
   uint64_t chart_items_max;    /* largest pruned chart seen (items) */
   uint64_t chart_sets_max;     /* most live Earley sets seen in one chart */
   uint64_t capacity_errors;
-  uint64_t big_mode_units;     /* times the trie walk switched to its large scratch area */
+  uint64_t big_mode_units;     /* times a warp of the trie sweep switched to its large scratch area */
   uint64_t walk_transitions;   /* Earley steps (scan + complete + predict) done by the trie walk */
   uint64_t walk_states;        /* distinct Earley sets created by the trie walk */
 } fmt_stats;
@@ -135,9 +133,10 @@ fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out);
 /*
  * Copy one host-side table of the compiled grammar, for inspection and tests.
  *   which: 0 trie child_off [T+1] u32   1 trie node_byte [T] u8    2 trie parent [T] u32
- *          3 trie tok_off [T+1] u32     4 trie tok_ids u32         5 unit_node [U] u32
+ *          3 trie tok_off [T+1] u32     4 trie tok_ids u32         5 level offsets [depth+2] u32
  *          6 nullable flags [N] u8      7 item info [D] u32        8 item lhs [D] u16
- *          9 unit_kind [U] u8 (0 = whole subtree, 1 = the node alone)
+ *          9 tok_node [V] u32 (node where a token ends, 0xFFFFFFFF if it has no bytes)
+ *         10 byte class of each byte [256] u8
  * Writes min(cap_bytes, size) bytes to `out` (may be NULL) and the full size to *size_bytes.
  */
 fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, size_t cap_bytes, size_t* size_bytes);
@@ -226,14 +225,15 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
  * but it needs an fmt_state, whose creation allocates hundreds of megabytes.  This call needs no
  * fmt_state: it walks the vocabulary trie for charts the caller already holds in device memory
  * (in the layout fmt_state_copy_chart documents) and uses a fixed scratch array that is part of
- * the loaded library image (about 36 MB of device memory on every GPU that loads the library,
+ * the loaded library image (about 52 MB of device memory on every GPU that loads the library,
  * held until the process exits).
  *
  *   g              a grammar compiled for the current device
  *   charts_dev     device memory holding the charts
  *   chart_offsets  HOST array of n+1 word offsets into charts_dev: chart r occupies words
  *                  [chart_offsets[r], chart_offsets[r+1])
- *   n              number of charts, at most FMT_NOALLOC_MAX_CHARTS (more: FMT_ERR_CAPACITY)
+ *   n              number of charts, at most FMT_NOALLOC_MAX_CHARTS, and n x (trie nodes of the
+ *                  vocabulary) at most 8 Mi (beyond either limit: FMT_ERR_CAPACITY)
  *   mask_dev       device output, n rows of exactly ceil(V/32) words (dense, no extra stride)
  *   status_dev     device output or NULL, n int32: FMT_OK, FMT_ERR_INVALID_ARG (the chart's header
  *                  does not fit its slot) or FMT_ERR_CAPACITY (the Earley sets met while walking the

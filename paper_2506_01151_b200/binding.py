@@ -34,7 +34,7 @@ class FmtError(RuntimeError):
 
 
 class CompileOptions(C.Structure):
-    _fields_ = [("host_only", C.c_uint32), ("unit_max_nodes", C.c_uint32), ("reserved", C.c_uint32 * 6)]
+    _fields_ = [("host_only", C.c_uint32), ("reserved", C.c_uint32 * 7)]
 
 
 class StateOptions(C.Structure):
@@ -48,7 +48,7 @@ class StateOptions(C.Structure):
 class GrammarInfo(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in (
         "n_nonterminals", "n_rules", "n_dotted", "n_classes", "n_nullable", "vocab_size", "mask_words",
-        "trie_nodes", "trie_depth", "n_units", "n_empty_tokens", "start_nullable")]
+        "trie_nodes", "trie_depth", "n_byte_classes", "n_empty_tokens", "start_nullable")]
 
 
 class Stats(C.Structure):
@@ -119,21 +119,19 @@ def _ptr(x) -> Optional[int]:
 
 
 _TABLE_DTYPES = {0: np.uint32, 1: np.uint8, 2: np.uint32, 3: np.uint32, 4: np.uint32, 5: np.uint32, 6: np.uint8,
-                 7: np.uint32, 8: np.uint16, 9: np.uint8}
+                 7: np.uint32, 8: np.uint16, 9: np.uint32, 10: np.uint8}
 
 
 class Grammar:
     """fmt_compile: grammar text + vocabulary -> device tables and byte trie."""
 
-    def __init__(self, ebnf, start: str, vocab: Sequence[bytes], eos: int = -1, host_only: bool = False,
-                 unit_max_nodes: int = 0):
+    def __init__(self, ebnf, start: str, vocab: Sequence[bytes], eos: int = -1, host_only: bool = False):
         src = ebnf.encode("latin-1") if isinstance(ebnf, str) else bytes(ebnf)
         offs = np.zeros(len(vocab) + 1, dtype=np.uint64)
         offs[1:] = np.cumsum([len(t) for t in vocab], dtype=np.uint64)
         blob = np.frombuffer(b"".join(vocab) + b"\0", dtype=np.uint8).copy()
         opt = CompileOptions()
         opt.host_only = 1 if host_only else 0
-        opt.unit_max_nodes = unit_max_nodes
         h = C.c_void_p()
         _check(lib().fmt_compile(src, len(src), start.encode(), blob.ctypes.data, offs.ctypes.data, len(vocab), eos,
                                  C.byref(opt), C.byref(h)))

@@ -140,7 +140,7 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
   try {
     compile_grammar(ebnf, ebnf_len, start_rule, g->host);
     static const uint8_t none = 0;
-    build_trie(vocab_bytes ? vocab_bytes : &none, vocab_offsets, V, eos_token_id, opt ? opt->unit_max_nodes : 0, g->host);
+    build_trie(vocab_bytes ? vocab_bytes : &none, vocab_offsets, V, eos_token_id, g->host);
     if (eos_token_id >= 0 && vocab_offsets[eos_token_id + 1] != vocab_offsets[eos_token_id])
       throw CompileError{FMT_ERR_INVALID_ARG, "the EOS token must have no bytes"};
   } catch (const CompileError& e) {
@@ -154,14 +154,13 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
     const HostTables& h = g->host;
     GrammarDev& d = g->dev;
     d.D = h.D, d.N = h.N, d.C = h.C, d.Nw = h.Nw;
-    d.V = h.V, d.Wm = h.Wm, d.T = h.T, d.U = (uint32_t)h.unit_node.size(), d.depth = h.depth;
+    d.V = h.V, d.Wm = h.Wm, d.T = h.T, d.depth = h.depth;
     d.eos = h.eos;
     d.start_nullable = h.start_nullable ? 1u : 0u;
     cudaError_t e = cudaGetDevice(&g->device);
 #define UP(field) if (e == cudaSuccess) e = g->bufs.upload(h.field, &d.field)
     UP(info);
     UP(lhs);
-    UP(skip);
     UP(class_bits);
     UP(eq_of_byte);
     d.n_eq = h.n_eq;
@@ -174,8 +173,8 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
     UP(node_depth);
     UP(tok_off);
     UP(tok_ids);
-    UP(unit_node);
-    UP(unit_kind);
+    UP(lvl_off);
+    UP(tok_node);
     UP(vocab_off);
     UP(vocab_bytes);
 #undef UP
@@ -204,7 +203,7 @@ fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out) {
   out->mask_words = h.Wm;
   out->trie_nodes = h.T;
   out->trie_depth = h.depth;
-  out->n_units = (uint32_t)h.unit_node.size();
+  out->n_byte_classes = h.n_eq;
   out->n_empty_tokens = h.n_empty;
   out->start_nullable = h.start_nullable ? 1u : 0u;
   return FMT_OK;
@@ -221,11 +220,12 @@ fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, si
     case 2: src = h.parent.data(), n = (size_t)h.T * 4; break;
     case 3: src = h.tok_off.data(), n = (size_t)(h.T + 1) * 4; break;
     case 4: src = h.tok_ids.data(), n = (size_t)h.tok_off[h.T] * 4; break;
-    case 5: src = h.unit_node.data(), n = h.unit_node.size() * 4; break;
+    case 5: src = h.lvl_off.data(), n = h.lvl_off.size() * 4; break;
     case 6: src = h.nullable.data(), n = h.N; break;
     case 7: src = h.info.data(), n = (size_t)h.D * 4; break;
     case 8: src = h.lhs.data(), n = (size_t)h.D * 2; break;
-    case 9: src = h.unit_kind.data(), n = h.unit_kind.size(); break;
+    case 9: src = h.tok_node.data(), n = h.tok_node.size() * 4; break;
+    case 10: src = h.eq_of_byte.data(), n = 256; break;
     default: return fail(FMT_ERR_INVALID_ARG, "unknown table");
   }
   *size_bytes = n;
@@ -274,9 +274,10 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   au.hash_mask = hs - 1;
   au.items_cap = 128u << 20;
 
+  sweep_layout(g->dev, &au.smem_bytes, &au.tables_in_smem);
   cudaError_t e = configure_kernels();
   int per_sm = 0, sms = 0, dev = 0;
-  if (e == cudaSuccess) e = walk_blocks_per_sm(&per_sm);
+  if (e == cudaSuccess) e = walk_blocks_per_sm(&per_sm, au.smem_bytes);
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e == cudaSuccess && per_sm < 1) {
@@ -303,6 +304,10 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(au.hash, (size_t)batch * hs, 0);
   AL(au.items, au.items_cap, 0);
   AL(au.n_states, batch, 0);
+  au.st_stride = (g->dev.T + 63u) & ~63u;
+  AL(au.st, (size_t)batch * au.st_stride, 0xFF);
+  au.req_cap = 1u << 20;
+  AL(au.req, au.req_cap, 0);
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);

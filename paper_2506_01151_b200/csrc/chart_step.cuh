@@ -185,7 +185,7 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     uint32_t a = soff[o], b = soff[o + 1];
     for (uint32_t k = a + lane; k < b; k += 32) {
       uint32_t wi = sitems[k];
-      uint32_t inf = __ldg(&G.info[wi & 0xFFFFu]);
+      uint32_t inf = G.info[wi & 0xFFFFu];
       if ((inf >> INFO_KIND_SHIFT) == KIND_NT && (inf & INFO_ARG_MASK) == A) {
         uint32_t bit = 1u << (k & 31u);
         uint32_t old = atomicOr(&s.live[k >> 5], bit);

@@ -6,12 +6,11 @@ namespace fmt {
 
 struct GrammarDev {
   uint32_t D, N, C, Nw;          // dotted rules, non-terminals, byte classes, words per non-terminal bitset
-  uint32_t V, Wm, T, U, depth;   // vocabulary, mask words, trie nodes, work units, longest token
+  uint32_t V, Wm, T, depth;      // vocabulary, mask words, trie nodes, longest token
   int32_t eos;
   uint32_t start_nullable;
   const uint32_t* info;          // [D]
   const uint16_t* lhs;           // [D]
-  const uint8_t* skip;           // [D]
   const uint32_t* class_bits;    // [C][8]
   const uint8_t* eq_of_byte;     // [256] equivalence class of each byte (same membership in all byte classes)
   uint32_t n_eq;
@@ -24,8 +23,8 @@ struct GrammarDev {
   const uint8_t* node_depth;     // [T]
   const uint32_t* tok_off;       // [T+1]
   const uint32_t* tok_ids;
-  const uint32_t* unit_node;     // [U]
-  const uint8_t* unit_kind;      // [U]
+  const uint32_t* lvl_off;       // [depth+2]
+  const uint32_t* tok_node;      // [V]
   const uint32_t* vocab_off;     // [V+1]
   const uint8_t* vocab_bytes;
 };
@@ -61,7 +60,11 @@ enum : uint32_t {
   CNT_STAT_BIG = 24,
   CNT_STAT_TRANS = 26,  // transitions computed by the trie walk (Earley steps)
   CNT_STAT_LOCAL = 28,  // local states created by the trie walk
-  CNT_TOTAL = 32
+  CNT_BAR = 30,         // grid barrier of the trie sweep: arrivals
+  CNT_BAR_ERR = 31,     // a block gave up waiting at the barrier
+  CNT_LEVEL_ALIVE = 32, // [MAX_TOKEN_BYTES + 2] per trie depth: some node of some job was alive
+  CNT_LEVEL_REQ = 68,   // [MAX_TOKEN_BYTES + 2] per trie depth: transitions queued for computation
+  CNT_TOTAL = 104
 };
 
 // Per-job automaton of hash-consed Earley sets, built on demand by the trie walk.  A "local
@@ -82,7 +85,14 @@ struct AutoDev {
   uint32_t* hash;      // [jobs][hash_mask + 1], id + 1 or 0
   uint32_t* items;     // [items_cap]
   uint32_t* n_states;  // [jobs]
+  uint16_t* st;        // [jobs][st_stride] local state reached at every trie node (ST_DEAD if none)
+  uint32_t st_stride;
+  unsigned long long* req;  // [req_cap] transitions to compute at the current depth: job << 32 | state << 8 | byte
+  uint32_t req_cap;
+  uint32_t smem_bytes;      // dynamic shared memory of the sweep kernel
+  uint32_t tables_in_smem;  // 1: item info, byte classes and byte class numbers are staged in shared memory
 };
+constexpr uint16_t ST_DEAD = 0xFFFFu, ST_PENDING = 0xFFFEu;
 constexpr uint32_t T_UNKNOWN = 0xffffffffu, T_DEAD = 0xfffffffeu, T_FAIL = 0xfffffffdu, T_PENDING = 0xfffffffcu;
 constexpr uint32_t ORIGIN_SELF = 0xFFFFu;
 constexpr uint32_t AR_ITEMS = 0, AR_N = 1, AR_HASH = 2, AR_SCAN = 4, AR_TRANS = 16;

@@ -82,7 +82,7 @@ __device__ __forceinline__ void hset_clear_items(const WarpCtx& w, uint32_t n) {
 // Add item `key` and the items reached by moving the dot over nullable non-terminals.
 // May be called by any subset of lanes.
 __device__ __forceinline__ void add_item(const GrammarDev& G, const WarpCtx& w, uint32_t key) {
-  uint32_t n = __ldg(&G.skip[key & 0xFFFFu]);
+  uint32_t n = (G.info[key & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK;
   for (uint32_t j = 0; j <= n; ++j) {
     int r = hset_insert(w.hset, w.hset_mask, key + j);
     if (r == 1) {
@@ -96,7 +96,7 @@ __device__ __forceinline__ void add_item(const GrammarDev& G, const WarpCtx& w, 
 }
 
 __device__ __forceinline__ bool class_has(const GrammarDev& G, uint32_t cls, uint32_t byte) {
-  return (__ldg(&G.class_bits[cls * 8u + (byte >> 5)]) >> (byte & 31u)) & 1u;
+  return (G.class_bits[cls * 8u + (byte >> 5)] >> (byte & 31u)) & 1u;
 }
 
 // Scan (Section 3.2): items of `set` whose post-dot terminal matches `byte`, dot advanced, go
@@ -105,7 +105,7 @@ __device__ __forceinline__ uint32_t scan_into_cur(const GrammarDev& G, const War
                                                   uint32_t len, uint32_t byte) {
   for (uint32_t k = lane_id(); k < len; k += 32) {
     uint32_t it = set[k];
-    uint32_t inf = __ldg(&G.info[it & 0xFFFFu]);
+    uint32_t inf = G.info[it & 0xFFFFu];
     if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) add_item(G, w, it + 1u);
   }
   __syncwarp();
@@ -131,7 +131,7 @@ __device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const War
     uint32_t idx = head + lane;
     bool have = idx < n;
     uint32_t it = have ? w.cur[idx] : 0u;
-    uint32_t inf = have ? __ldg(&G.info[it & 0xFFFFu]) : 0u;
+    uint32_t inf = have ? G.info[it & 0xFFFFu] : 0u;
     uint32_t kind = inf >> INFO_KIND_SHIFT;
     if (have && kind == KIND_NT) {
       uint32_t y = inf & INFO_ARG_MASK;
@@ -150,7 +150,7 @@ __device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const War
       view(o, sp, sl);
       for (uint32_t k = lane; k < sl; k += 32) {
         uint32_t wi = sp[k];
-        uint32_t winf = __ldg(&G.info[wi & 0xFFFFu]);
+        uint32_t winf = G.info[wi & 0xFFFFu];
         if ((winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X) add_item(G, w, view.fix(wi, o) + 1u);
       }
       __syncwarp();
@@ -215,7 +215,7 @@ __device__ __forceinline__ uint32_t drop_completed(const GrammarDev& G, const Wa
     uint32_t idx = base + lane;
     bool have = idx < n;
     uint32_t it = have ? w.cur[idx] : 0u;
-    bool keep = have && (__ldg(&G.info[it & 0xFFFFu]) >> INFO_KIND_SHIFT) != KIND_END;
+    bool keep = have && (G.info[it & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
     uint32_t bal = __ballot_sync(FULL, keep);
     uint32_t pos = out + __popc(bal & ((1u << lane) - 1u));
     __syncwarp();
@@ -233,10 +233,10 @@ __device__ __forceinline__ void scannable_bytes(const GrammarDev& G, const uint3
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0u;
   for (uint32_t k = lane_id(); k < len; k += 32) {
-    uint32_t inf = __ldg(&G.info[set[k] & 0xFFFFu]);
+    uint32_t inf = G.info[set[k] & 0xFFFFu];
     if ((inf >> INFO_KIND_SHIFT) == KIND_TERM) {
       const uint4* p = reinterpret_cast<const uint4*>(G.class_bits + (inf & INFO_ARG_MASK) * 8u);
-      uint4 a = __ldg(p), b = __ldg(p + 1);
+      uint4 a = p[0], b = p[1];
       acc[0] |= a.x, acc[1] |= a.y, acc[2] |= a.z, acc[3] |= a.w;
       acc[4] |= b.x, acc[5] |= b.y, acc[6] |= b.z, acc[7] |= b.w;
     }

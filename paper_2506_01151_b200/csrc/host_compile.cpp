@@ -1,4 +1,4 @@
-// Grammar text -> reduced grammar -> flat tables; vocabulary -> CSR byte trie and work units.
+// Grammar text -> reduced grammar -> flat tables; vocabulary -> CSR byte trie in level order.
 //
 // Follows the paper's Section 3.1 (rules A -> alpha), Section 4.5 (remove useless rules; handle
 // rules deriving the empty string once, at compile time) and Section 4.1 (the whole vocabulary
@@ -464,6 +464,7 @@ void compile_grammar(const char* text, size_t len, const std::string& start, Hos
   for (uint32_t i = (uint32_t)D; i-- > 0;)
     if ((out.info[i] >> INFO_KIND_SHIFT) == KIND_NT && (out.info[i] & INFO_NULLABLE))
       out.skip[i] = (uint8_t)std::min<uint32_t>(255u, 1u + out.skip[i + 1]);
+  for (uint32_t i = 0; i < (uint32_t)D; ++i) out.info[i] |= (uint32_t)out.skip[i] << INFO_SKIP_SHIFT;
   // direct items: the start item of every rule plus the items reached by moving the dot over
   // leading nullable non-terminals; completed items are left out (their effect is the parent's skip)
   out.direct_off.assign(N + 1, 0);
@@ -498,8 +499,7 @@ void compile_grammar(const char* text, size_t len, const std::string& start, Hos
 
 // ------------------------------------------------------------------------------------ trie
 
-void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t eos, uint32_t unit_max_nodes,
-                HostTables& out) {
+void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t eos, HostTables& out) {
   out.V = V;
   out.Wm = (V + 31) / 32;
   out.eos = eos;
@@ -570,33 +570,16 @@ void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t 
   out.child_off.push_back(out.T);
   out.tok_off.push_back((uint32_t)out.tok_ids.size());
   if (out.tok_ids.empty()) out.tok_ids.push_back(0);
-  // subtree sizes, then split large subtrees into work units
-  std::vector<uint32_t> size(out.T, 1);
-  for (uint32_t n = out.T; n-- > 1;) size[out.parent[n]] += size[n];
-  if (unit_max_nodes == 0) unit_max_nodes = 32;
-  std::vector<std::pair<uint32_t, uint32_t>> units;  // (size, node | kind << 31)
-  std::vector<uint32_t> stack;
-  for (uint32_t c = out.child_off[0]; c < out.child_off[1]; ++c) stack.push_back(c);
-  while (!stack.empty()) {
-    uint32_t n = stack.back();
-    stack.pop_back();
-    if (size[n] <= unit_max_nodes || out.node_depth[n] >= 8) {  // a unit's path from the root has at most 8 bytes
-      units.push_back({size[n], n});
-    } else {
-      if (out.tok_off[n + 1] > out.tok_off[n]) units.push_back({1, n | 0x80000000u});
-      for (uint32_t c = out.child_off[n]; c < out.child_off[n + 1]; ++c) stack.push_back(c);
-    }
-  }
-  // largest first: units that stay alive are then spread over many warps
-  std::sort(units.begin(), units.end(), [](const std::pair<uint32_t, uint32_t>& a, const std::pair<uint32_t, uint32_t>& b) {
-    return a.first != b.first ? a.first > b.first : a.second < b.second;
-  });
-  out.unit_node.clear();
-  out.unit_kind.clear();
-  for (auto& u : units) {
-    out.unit_node.push_back(u.second & 0x7FFFFFFFu);
-    out.unit_kind.push_back((uint8_t)(u.second >> 31));
-  }
+  // breadth-first numbering makes every depth a contiguous range of nodes
+  out.lvl_off.assign(out.depth + 2, out.T);
+  out.lvl_off[0] = 0;
+  for (uint32_t n = out.T; n-- > 0;) out.lvl_off[out.node_depth[n]] = n;
+  out.lvl_off[out.depth + 1] = out.T;
+  for (uint32_t L = out.depth; L >= 1; --L)
+    if (out.lvl_off[L] > out.lvl_off[L + 1]) out.lvl_off[L] = out.lvl_off[L + 1];
+  out.tok_node.assign(V, 0xFFFFFFFFu);
+  for (uint32_t n = 0; n < out.T; ++n)
+    for (uint32_t i = out.tok_off[n]; i < out.tok_off[n + 1] && i < (uint32_t)order.size(); ++i) out.tok_node[out.tok_ids[i]] = n;
 }
 
 }  // namespace fmt

@@ -7,7 +7,8 @@
 
 namespace fmt {
 
-// item info word: bits 31..30 kind, bit 29 "post-dot non-terminal is nullable", bits 15..0 argument
+// item info word: bits 31..30 kind, bit 29 "post-dot non-terminal is nullable", bits 23..16 how many
+// nullable non-terminals follow the dot in a row (the dot may move over them), bits 15..0 argument
 //   END : argument = left-hand side        (dot at the end of the rule)
 //   TERM: argument = byte-class id         (post-dot symbol is a terminal)
 //   NT  : argument = non-terminal id       (post-dot symbol is a non-terminal)
@@ -15,6 +16,7 @@ enum : uint32_t { KIND_END = 0u, KIND_TERM = 1u, KIND_NT = 2u };
 constexpr uint32_t INFO_KIND_SHIFT = 30;
 constexpr uint32_t INFO_NULLABLE = 1u << 29;
 constexpr uint32_t INFO_ARG_MASK = 0xFFFFu;
+constexpr uint32_t INFO_SKIP_SHIFT = 16, INFO_SKIP_MASK = 0xFFu;
 constexpr uint32_t ITEM_START = 0;   // $ -> . start
 constexpr uint32_t ITEM_ACCEPT = 1;  // $ -> start .
 constexpr uint32_t MAX_TOKEN_BYTES = 32;
@@ -50,15 +52,14 @@ struct HostTables {
   std::vector<uint8_t> node_depth;  // [T]
   std::vector<uint32_t> tok_off;    // [T+1] tokens whose bytes end at node n
   std::vector<uint32_t> tok_ids;
-  std::vector<uint32_t> unit_node;  // work units of the mask kernel, largest first
-  std::vector<uint8_t> unit_kind;   // 0 whole subtree, 1 the node alone
+  std::vector<uint32_t> lvl_off;    // [depth+2] nodes of depth L are lvl_off[L]..lvl_off[L+1]-1
+  std::vector<uint32_t> tok_node;   // [V] node where the token's bytes end, 0xFFFFFFFF for empty tokens
   std::vector<uint32_t> vocab_off;  // [V+1] byte offsets (32-bit) into vocab_bytes
   std::vector<uint8_t> vocab_bytes;
 };
 
 // Both throw CompileError.
 void compile_grammar(const char* text, size_t len, const std::string& start, HostTables& out);
-void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t eos, uint32_t unit_max_nodes,
-                HostTables& out);
+void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t eos, HostTables& out);
 
 }  // namespace fmt

@@ -212,82 +212,72 @@ __global__ void __launch_bounds__(ADV_WARPS * 32) advance_kernel(GrammarDev G, S
 
 // ===================================================================================== fill: plan
 
-// One thread per row decides where the row's mask comes from.
-__global__ void plan_kernel(GrammarDev G, StateDev S) {
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
+// One block decides, row by row, where each mask comes from: the state cache, another row of
+// this call with the same chart, or a fresh computation (a "job").
+__global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
+  if (threadIdx.x < CNT_TOTAL - CNT_BAR) S.counters[CNT_BAR + threadIdx.x] = 0u;  // barrier and level counters
+  if (threadIdx.x == 0) {
+    S.counters[CNT_N_JOBS] = 0u;
     S.counters[CNT_WORK] = 0u;
     S.counters[CNT_AUTO_ITEMS] = 0u;
   }
-  const uint32_t row = blockIdx.x * blockDim.x + threadIdx.x;
-  if (row >= S.B) return;
-  stat_add(S, CNT_STAT_FILLS, 1u);
-  const uint32_t flags = S.row_flags[row];
-  if (flags & ROW_BROKEN) {
-    S.row_mask[row] = MASK_ZERO;
-    return;
-  }
-  if (flags & ROW_FINISHED) {
-    S.row_mask[row] = MASK_EOS_ONLY;
-    return;
-  }
-  const int32_t sid = S.row_state[row];
-  if (sid >= 0) {
-    int32_t old = atomicCAS(&S.st_mask[sid], -1, -2 - (int32_t)row);
-    if (old >= 0) {  // cached
-      S.row_mask[row] = old;
-      stat_add(S, CNT_STAT_CACHED, 1u);
-      return;
-    }
-    if (old <= -2) {  // another row of this call computes it
-      S.row_mask[row] = MASK_ALIAS0 - (-2 - old);
-      stat_add(S, CNT_STAT_SHARED, 1u);
-      return;
-    }
-    // this row computes it, into a cache row if one is left
-    int32_t mrow = (int32_t)row;
-    if (ld_acquire(&S.counters[CNT_N_MASK_ROWS]) < S.max_mask_rows) {
-      uint32_t got = atomicAdd(&S.counters[CNT_N_MASK_ROWS], 1u);
-      if (got < S.max_mask_rows) mrow = (int32_t)(S.B + got);
-    }
-    S.row_mask[row] = mrow;
-  } else {
-    S.row_mask[row] = (int32_t)row;
-  }
-  stat_add(S, CNT_STAT_COMPUTED, 1u);
-  uint32_t j = atomicAdd(&S.counters[CNT_N_JOBS], 1u);
-  S.jobs[j] = row;
-}
-
-// Zero the mask rows about to be computed and set their EOS bit.
-__global__ void prepare_rows_kernel(GrammarDev G, StateDev S) {
-  const uint32_t j = blockIdx.x;
-  if (j >= S.counters[CNT_N_JOBS]) return;
-  const uint32_t row = S.jobs[j];
-  uint32_t* m = S.mask_rows + (size_t)S.row_mask[row] * G.Wm;
-  for (uint32_t i = threadIdx.x; i < G.Wm; i += blockDim.x) m[i] = 0u;
   __syncthreads();
-  if (threadIdx.x == 0 && G.eos >= 0) {
-    const uint32_t* ch = S.arena + S.row_chart[row];
-    if (ch[CH_FLAGS] & CHART_ACCEPTING) m[(uint32_t)G.eos >> 5] |= 1u << ((uint32_t)G.eos & 31u);
+  for (uint32_t row = threadIdx.x; row < S.B; row += blockDim.x) {
+    stat_add(S, CNT_STAT_FILLS, 1u);
+    const uint32_t flags = S.row_flags[row];
+    if (flags & ROW_BROKEN) {
+      S.row_mask[row] = MASK_ZERO;
+      continue;
+    }
+    if (flags & ROW_FINISHED) {
+      S.row_mask[row] = MASK_EOS_ONLY;
+      continue;
+    }
+    const int32_t sid = S.row_state[row];
+    if (sid >= 0) {
+      int32_t old = atomicCAS(&S.st_mask[sid], -1, -2 - (int32_t)row);
+      if (old >= 0) {  // cached
+        S.row_mask[row] = old;
+        stat_add(S, CNT_STAT_CACHED, 1u);
+        continue;
+      }
+      if (old <= -2) {  // another row of this call computes it
+        S.row_mask[row] = MASK_ALIAS0 - (-2 - old);
+        stat_add(S, CNT_STAT_SHARED, 1u);
+        continue;
+      }
+      // this row computes it, into a cache row if one is left
+      int32_t mrow = (int32_t)row;
+      if (ld_acquire(&S.counters[CNT_N_MASK_ROWS]) < S.max_mask_rows) {
+        uint32_t got = atomicAdd(&S.counters[CNT_N_MASK_ROWS], 1u);
+        if (got < S.max_mask_rows) mrow = (int32_t)(S.B + got);
+      }
+      S.row_mask[row] = mrow;
+    } else {
+      S.row_mask[row] = (int32_t)row;
+    }
+    stat_add(S, CNT_STAT_COMPUTED, 1u);
+    uint32_t j = atomicAdd(&S.counters[CNT_N_JOBS], 1u);
+    S.jobs[j] = row;
   }
 }
 
-// ===================================================================================== fill: walk
+// ===================================================================================== fill: sweep
 //
-// The walk answers, for one job (a row whose mask must be computed) and every trie node, "is the
-// Earley set reached by this node's bytes non-empty?".  Sets are hash-consed per job (AutoDev):
-// a transition (state, byte class) is computed once, by whichever warp needs it first, with the
-// warp-cooperative scan / complete / predict of earley_device.cuh; everybody else finds it in the
-// state's record.  Nothing waits: two warps that miss the same transition at the same time both
-// compute it and meet in the same hash slot.  The trie is then walked with one LANE per work
-// unit (a subtree of at most a few hundred nodes), depth first, one table lookup per node.
+// For every job (a row whose mask must be computed) and every trie node the sweep answers "is the
+// Earley set reached by this node's bytes non-empty?".  Sets are hash-consed per job (AutoDev): a
+// transition (set, byte class) is computed once, by whichever warp needs it first, with the
+// warp-cooperative scan / complete / predict of earley_device.cuh; everybody else reads it from
+// the set's record.  The trie is processed one depth at a time by the whole grid, one THREAD per
+// (job, node): st[node] = transition(st[parent], byte).  Reads of parent, byte and writes of st
+// are coalesced because nodes are numbered breadth first.  A grid barrier separates the depths;
+// the kernel is launched cooperatively so that all CTAs are resident, and the barrier gives up
+// (and flags an error) after a bounded number of polls instead of hanging.
 
-constexpr int WALK_WARPS = 8;
-constexpr uint32_t WALK_CUR = 1024;     // items of a set under construction per warp (fast mode, power of two)
-constexpr uint32_t WALK_HSET = 2048;    // uniqueness hash slots per warp (fast mode)
-constexpr uint32_t WALK_NT_WORDS = 256; // 2 * Nw
-constexpr uint32_t WALK_LEVELS = MAX_TOKEN_BYTES + 1;
-constexpr uint32_t WALK_WARP_WORDS = WALK_CUR + WALK_HSET + WALK_NT_WORDS + W_CTRS + 8;
+constexpr int SWEEP_WARPS = 8;
+constexpr uint32_t SWEEP_CUR = 512;     // items of a set under construction per warp (fast mode, power of two)
+constexpr uint32_t SWEEP_HSET = 1024;   // uniqueness hash slots per warp (fast mode)
+constexpr uint32_t SWEEP_TABLE_BYTES = 24 * 1024;  // budget for grammar tables staged in shared memory
 
 struct JobCtx {
   const uint32_t* base_off;
@@ -297,8 +287,27 @@ struct JobCtx {
   uint32_t* hash;
   uint32_t* n_states;
   uint32_t cap;       // states this job may create (ids stay below ORIGIN_SELF - m)
-  uint32_t* mask_row;
+  uint16_t* st;
+  uint32_t row;
+  bool accepting;
 };
+
+__device__ __forceinline__ JobCtx job_ctx(const StateDev& S, uint32_t j) {
+  const AutoDev& A = S.au;
+  JobCtx J;
+  J.row = S.jobs[j];
+  const uint32_t* chart = S.arena + S.row_chart[J.row];
+  J.m = chart[CH_SETS];
+  J.accepting = (chart[CH_FLAGS] & CHART_ACCEPTING) != 0u;
+  J.base_off = chart + CH_HDR;
+  J.base_items = chart + CH_HDR + J.m + 1;
+  J.recs = A.recs + (size_t)j * A.cap * A.rec_words;
+  J.hash = A.hash + (size_t)j * (A.hash_mask + 1);
+  J.n_states = A.n_states + j;
+  J.cap = min(A.cap, (ORIGIN_SELF - 1u > J.m) ? ORIGIN_SELF - 1u - J.m : 0u);
+  J.st = A.st + (size_t)j * A.st_stride;
+  return J;
+}
 
 struct AutoView {
   const JobCtx& J;
@@ -320,12 +329,13 @@ struct AutoView {
   }
 };
 
-struct WalkWarp {
+struct SweepWarp {
   const GrammarDev& G;
   const StateDev& S;
   WarpCtx w;
-  uint32_t cur_pow2;   // capacity of w.cur rounded down to a power of two (for the sort)
-  uint32_t* tmp8;      // shared
+  uint32_t cur_pow2;  // capacity of w.cur (a power of two, for the sort)
+  uint32_t* tmp8;     // shared
+  uint32_t n_computed = 0, n_created = 0;  // statistics, flushed once at the end of the kernel
 
   // Find or create the local state whose items are w.cur[0..n) (sorted).  Returns its id or T_FAIL.
   __device__ uint32_t intern_set(const JobCtx& J, uint32_t n, uint32_t hash) {
@@ -341,13 +351,11 @@ struct WalkWarp {
         if (my_id == T_FAIL) {
           uint32_t id = T_FAIL, ioff = 0;
           if (lane == 0) {
-            if (ld_acquire(J.n_states) < J.cap) {
-              uint32_t got = atomicAdd(J.n_states, 1u);
-              uint32_t need = (max(n, 1u) + 31u) & ~31u;
-              if (got < J.cap && ld_acquire(&S.counters[CNT_AUTO_ITEMS]) + need <= A.items_cap) {
-                ioff = atomicAdd(&S.counters[CNT_AUTO_ITEMS], need);
-                if (ioff + need <= A.items_cap) id = got;
-              }
+            const uint32_t got = atomicAdd(J.n_states, 1u);
+            const uint32_t need = (max(n, 1u) + 31u) & ~31u;
+            if (got < J.cap) {
+              ioff = atomicAdd(&S.counters[CNT_AUTO_ITEMS], need);
+              if (ioff <= A.items_cap && need <= A.items_cap - ioff) id = got;
             }
           }
           id = __shfl_sync(FULL, id, 0);
@@ -368,7 +376,7 @@ struct WalkWarp {
           __syncwarp();
           __threadfence();
           my_id = id;
-          if (lane == 0) stat_add(S, CNT_STAT_LOCAL, 1u);
+          ++n_created;
         }
         uint32_t old = 0;
         if (lane == 0) old = atomicCAS(&J.hash[slot], 0u, my_id + 1u);
@@ -398,7 +406,7 @@ struct WalkWarp {
   __device__ uint32_t compute(const JobCtx& J, uint32_t ps, uint32_t byte, bool force) {
     const uint32_t lane = lane_id();
     const AutoDev& A = S.au;
-    const uint32_t e = __ldg(&G.eq_of_byte[byte]);
+    const uint32_t e = G.eq_of_byte[byte];
     uint32_t* slot = J.recs + (size_t)ps * A.rec_words + AR_TRANS + e;
     uint32_t t = 0;
     if (lane == 0) {
@@ -424,7 +432,7 @@ struct WalkWarp {
     const uint32_t self_code = J.m + ps;
     for (uint32_t k = lane; k < plen; k += 32) {
       uint32_t it = pitems[k];
-      uint32_t inf = __ldg(&G.info[it & 0xFFFFu]);
+      uint32_t inf = G.info[it & 0xFFFFu];
       if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) {
         if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
         add_item(G, w, it + 1u);
@@ -458,251 +466,252 @@ struct WalkWarp {
     scannable_bytes(G, w.cur, n, tmp8);
     uint32_t id = intern_set(J, n, h);
     if (id == T_FAIL) return T_FAIL;
-    if (lane == 0) {
-      atomicExch(slot, id);
-      stat_add(S, CNT_STAT_TRANS, 1u);
-    }
+    if (lane == 0) atomicExch(slot, id);
+    ++n_computed;
     return id;
   }
 };
 
-__device__ __forceinline__ void emit_tokens(const GrammarDev& G, uint32_t* mask_row, uint32_t node) {
-  uint32_t a = __ldg(&G.tok_off[node]), b = __ldg(&G.tok_off[node + 1]);
-  for (uint32_t i = a; i < b; ++i) {
-    uint32_t t = __ldg(&G.tok_ids[i]);
-    atomicOr(&mask_row[t >> 5], 1u << (t & 31u));
+// All CTAs of the (cooperatively launched) grid meet here.  Returns false if the sweep must be
+// abandoned: some CTA waited longer than the limit, which only a fault elsewhere can cause.
+__device__ __forceinline__ bool grid_barrier(const StateDev& S, uint32_t& phase) {
+  __shared__ uint32_t ok_s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    ++phase;
+    __threadfence();
+    atomicAdd(&S.counters[CNT_BAR], 1u);
+    const uint32_t target = phase * gridDim.x;
+    uint32_t ok = 1u;
+    for (uint32_t polls = 0;; ++polls) {
+      if (ld_acquire(&S.counters[CNT_BAR]) >= target) break;
+      if (polls > (1u << 24) || ld_acquire(&S.counters[CNT_BAR_ERR])) {
+        atomicExch(&S.counters[CNT_BAR_ERR], 1u);
+        ok = 0u;
+        break;
+      }
+      __nanosleep(40);
+    }
+    __threadfence();
+    ok_s = ok;
   }
+  __syncthreads();
+  const bool ok = ok_s != 0u;
+  __syncthreads();
+  return ok;
 }
 
-// Set up the automata of this call's jobs: empty hash, one state (the base chart's last set).
-__global__ void auto_init_kernel(GrammarDev G, StateDev S) {
-  const uint32_t j = blockIdx.x;
-  if (j >= S.counters[CNT_N_JOBS]) return;
-  const AutoDev& A = S.au;
-  uint32_t* hash = A.hash + (size_t)j * (A.hash_mask + 1);
-  for (uint32_t i = threadIdx.x; i <= A.hash_mask; i += blockDim.x) hash[i] = 0u;
-  uint32_t* rec0 = A.recs + (size_t)j * A.cap * A.rec_words;
-  for (uint32_t i = threadIdx.x; i < A.rec_words; i += blockDim.x)
-    if (i < AR_SCAN || i >= AR_SCAN + 8) rec0[i] = (i >= AR_TRANS) ? T_UNKNOWN : 0u;
-  if (threadIdx.x == 0) A.n_states[j] = 1u;
-  if (threadIdx.x < 32) {
-    const uint32_t row = S.jobs[j];
-    const uint32_t* ch = S.arena + S.row_chart[row];
-    const uint32_t m = ch[CH_SETS];
-    const uint32_t* off = ch + CH_HDR;
-    const uint32_t* items = ch + CH_HDR + m + 1;
-    __shared__ uint32_t sc[8];
-    scannable_bytes(G, items + off[m - 1], off[m] - off[m - 1], sc);
-    if (threadIdx.x < 8) rec0[AR_SCAN + threadIdx.x] = sc[threadIdx.x];
-  }
+// What the Earley set at `node` is, given that its mark says "pending": the transition it waited
+// for has been computed meanwhile.  `parent_state` is the (final) state of its parent.
+__device__ __forceinline__ uint32_t settled(const GrammarDev& G, const AutoDev& A, const JobCtx& J, uint32_t parent_state,
+                                            uint32_t byte) {
+  const uint32_t* slot = J.recs + (size_t)parent_state * A.rec_words + AR_TRANS + G.eq_of_byte[byte];
+  return __ldcg(slot);
 }
 
-__global__ void __launch_bounds__(WALK_WARPS * 32, 2) walk_kernel(GrammarDev G, StateDev S) {
-  extern __shared__ uint32_t smem[];
-  const uint32_t warp = threadIdx.x >> 5, lane = lane_id();
-  uint32_t* mine = smem + (size_t)warp * WALK_WARP_WORDS;
-  uint32_t* sm_cur = mine;
-  uint32_t* sm_hset = sm_cur + WALK_CUR;
-  uint32_t* nt = sm_hset + WALK_HSET;
-  uint32_t* ctr = nt + WALK_NT_WORDS;
-  uint32_t* tmp8 = ctr + W_CTRS;
-  // the large scratch area of this warp (global memory)
-  uint32_t* big = S.big_scratch + ((size_t)blockIdx.x * WALK_WARPS + warp) * ((size_t)S.big_arena_items + S.big_hset_slots);
-  const AutoDev& A = S.au;
+constexpr uint32_t SWEEP_PER_LANE = 4;  // trie nodes per lane and pass iteration (independent loads in flight)
 
-  hset_clear_all(sm_hset, WALK_HSET - 1);
-  for (uint32_t i = lane; i < WALK_NT_WORDS; i += 32) nt[i] = 0u;
-  __syncwarp();
-  const uint32_t n_groups = (G.U + 31) / 32;
+__global__ void __launch_bounds__(SWEEP_WARPS * 32, 3) sweep_kernel(GrammarDev Gg, StateDev S) {
   const uint32_t n_jobs = S.counters[CNT_N_JOBS];
-  const uint32_t total = n_jobs * n_groups;
+  if (n_jobs == 0) return;  // every CTA sees the same count: nobody is left at a barrier
+  extern __shared__ __align__(16) uint32_t smem[];
+  const uint32_t warp = threadIdx.x >> 5, lane = lane_id();
+  const AutoDev& A = S.au;
+  const uint32_t ntw = (2u * Gg.Nw + 7u) & ~7u;
+  const uint32_t warp_words = SWEEP_CUR + SWEEP_HSET + ntw + W_CTRS + 8;
+  uint32_t* mine = smem + (size_t)warp * warp_words;
+  uint32_t* sm_cur = mine;
+  uint32_t* sm_hset = sm_cur + SWEEP_CUR;
+  uint32_t* nt = sm_hset + SWEEP_HSET;
+  uint32_t* ctr = nt + ntw;
+  uint32_t* tmp8 = ctr + W_CTRS;
+  // ---- the small grammar tables every Earley step reads go to shared memory when they fit
+  GrammarDev G = Gg;
+  if (A.tables_in_smem) {
+    uint32_t* tab = smem + (size_t)SWEEP_WARPS * warp_words;
+    const uint32_t d4 = (Gg.D + 3u) & ~3u;
+    for (uint32_t i = threadIdx.x; i < Gg.D; i += blockDim.x) tab[i] = Gg.info[i];
+    for (uint32_t i = threadIdx.x; i < Gg.C * 8u; i += blockDim.x) tab[d4 + i] = Gg.class_bits[i];
+    uint8_t* eq = reinterpret_cast<uint8_t*>(tab + d4 + Gg.C * 8u);
+    for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x) eq[i] = Gg.eq_of_byte[i];
+    G.info = tab;
+    G.class_bits = tab + d4;
+    G.eq_of_byte = eq;
+  }
+  uint32_t* big = S.big_scratch + ((size_t)blockIdx.x * SWEEP_WARPS + warp) * ((size_t)S.big_arena_items + S.big_hset_slots);
+  const uint32_t gw = blockIdx.x * SWEEP_WARPS + warp, GW = gridDim.x * SWEEP_WARPS;
+  uint32_t bar_phase = 0;
 
-  WalkWarp ww{G, S};
-  ww.w.nt = nt;
-  ww.w.ctr = ctr;
-  ww.tmp8 = tmp8;
+  hset_clear_all(sm_hset, SWEEP_HSET - 1);
+  for (uint32_t i = lane; i < ntw; i += 32) nt[i] = 0u;
+  __syncthreads();
 
-  for (;;) {
-    uint32_t item = 0;
-    if (lane == 0) item = atomicAdd(&S.counters[CNT_WORK], 1u);
-    item = __shfl_sync(FULL, item, 0);
-    if (item >= total) break;
-    // consecutive items belong to different jobs, so that few warps explore one automaton at a time
-    const uint32_t j = item % n_jobs, grp = item / n_jobs;
-    const uint32_t row = S.jobs[j];
-    const uint32_t* chart = S.arena + S.row_chart[row];
-    JobCtx J;
-    J.m = chart[CH_SETS];
-    J.base_off = chart + CH_HDR;
-    J.base_items = chart + CH_HDR + J.m + 1;
-    J.recs = A.recs + (size_t)j * A.cap * A.rec_words;
-    J.hash = A.hash + (size_t)j * (A.hash_mask + 1);
-    J.n_states = A.n_states + j;
-    J.cap = min(A.cap, (ORIGIN_SELF - 1u > J.m) ? ORIGIN_SELF - 1u - J.m : 0u);
-    J.mask_row = S.mask_rows + (size_t)S.row_mask[row] * G.Wm;
-    // fast mode: scratch in shared memory
-    ww.w.cur = sm_cur;
-    ww.w.cur_cap = WALK_CUR;
-    ww.cur_pow2 = WALK_CUR;
-    ww.w.hset = sm_hset;
-    ww.w.hset_mask = WALK_HSET - 1;
-    bool big_mode = false, broken = false, force = false;
-    uint32_t stalled = 0;
-
-    // ---- one work unit per lane
-    const uint32_t u = grp * 32 + lane;
-    uint32_t phase = 2;  // 0 following the unit's path from the root, 1 inside its subtree, 2 done
-    uint32_t root = 0, kind = 0, dr = 0, pk = 1, node = 0, depth = 0;
-    uint64_t path = 0;  // the bytes from the root to the unit's node, first byte lowest
-    uint16_t st[WALK_LEVELS];
-    st[0] = 0;
-    if (u < G.U) {
-      root = __ldg(&G.unit_node[u]);
-      kind = __ldg(&G.unit_kind[u]);
-      dr = __ldg(&G.node_depth[root]);
-      if (dr >= 1 && dr <= 8) {
-        uint32_t n = root;
-        for (uint32_t i = dr; i >= 1; --i) {
-          path |= (uint64_t)__ldg(&G.node_byte[n]) << (8 * (i - 1));
-          n = __ldg(&G.parent[n]);
-        }
-        phase = 0;
-      }
-    }
-    for (;;) {
-      uint32_t q_state = 0, q_byte = 0;
-      if (phase == 0) {
-        q_state = st[pk - 1];
-        q_byte = (uint32_t)(path >> (8 * (pk - 1))) & 0xFFu;
-      } else if (phase == 1) {
-        q_state = st[depth - 1];
-        q_byte = __ldg(&G.node_byte[node]);
-      }
-      const bool has_q = phase < 2;
-      if (__ballot_sync(FULL, has_q) == 0u) break;
-      uint32_t t = T_UNKNOWN, q_eq = 0;
-      if (has_q) {
-        q_eq = __ldg(&G.eq_of_byte[q_byte]);
-        const uint32_t* rec = J.recs + (size_t)q_state * A.rec_words;
-        // one 256-bit test rejects most bytes without touching the transition table
-        if (!((rec[AR_SCAN + (q_byte >> 5)] >> (q_byte & 31u)) & 1u)) t = T_DEAD;
-        else {
-          t = rec[AR_TRANS + q_eq];
-          if (t == T_UNKNOWN) t = __ldcg(rec + AR_TRANS + q_eq);
-        }
-      }
-      bool need = has_q && (t == T_UNKNOWN || t == T_PENDING);
-      bool waiting = false;  // the transition is being computed by another warp: ask again next round
-      uint32_t bal = __ballot_sync(FULL, need);
-      while (bal) {
-        const int src = __ffs(bal) - 1;
-        const uint32_t ps = __shfl_sync(FULL, q_state, src);
-        const uint32_t pb = __shfl_sync(FULL, q_byte, src);
-        const uint32_t pe = __shfl_sync(FULL, q_eq, src);
-        uint32_t r = ww.compute(J, ps, pb, force);
-        if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
-          big_mode = true;
-          hset_clear_all(ww.w.hset, ww.w.hset_mask);
-          clear_nt(G, ww.w);
-          ww.w.cur = big;
-          ww.w.cur_cap = S.big_arena_items;
-          ww.cur_pow2 = S.big_arena_items;
-          ww.w.hset = big + S.big_arena_items;
-          ww.w.hset_mask = S.big_hset_slots - 1;
-          if (lane == 0) stat_add(S, CNT_STAT_BIG, 1u);
-          r = ww.compute(J, ps, pb, true);
-        }
-        if (r == T_FAIL) {
-          broken = true;
-          break;
-        }
-        if (need && q_state == ps && q_eq == pe) {
-          need = false;
-          if (r == T_PENDING) waiting = true;
-          else t = r;
-        }
-        bal = __ballot_sync(FULL, need);
-      }
-      if (broken) break;
-      // If every lane that still has work waits for other warps, back off briefly; after many such
-      // rounds stop relying on them and compute the transitions here (bounded wait, no deadlock).
-      if (__ballot_sync(FULL, has_q && !waiting) == 0u) {
-        if (++stalled > 256u) force = true;
-        __nanosleep(stalled > 16u ? 400u : 50u);
-      } else {
-        stalled = 0;
-        force = false;
-      }
-      if (waiting) continue;
-      // ---- every lane moves on with its answer
-      if (phase == 0) {
-        if (t == T_DEAD) {
-          phase = 2;
-        } else {
-          st[pk] = (uint16_t)t;
-          if (pk == dr) {
-            emit_tokens(G, J.mask_row, root);
-            const uint32_t c0 = __ldg(&G.child_off[root]), c1 = __ldg(&G.child_off[root + 1]);
-            if (kind == 1 || c1 == c0) {
-              phase = 2;
-            } else {
-              node = c0;
-              depth = dr + 1;
-              phase = 1;
-            }
-          } else {
-            ++pk;
-          }
-        }
-      } else if (phase == 1) {
-        bool descend = false;
-        if (t != T_DEAD) {
-          emit_tokens(G, J.mask_row, node);
-          const uint32_t c0 = __ldg(&G.child_off[node]), c1 = __ldg(&G.child_off[node + 1]);
-          if (c1 > c0 && depth + 1 < WALK_LEVELS) {
-            st[depth] = (uint16_t)t;
-            node = c0;
-            ++depth;
-            descend = true;
-          }
-        }
-        if (!descend) {  // next sibling, or climb until there is one
-          for (;;) {
-            const uint32_t p = __ldg(&G.parent[node]);
-            if (node + 1 < __ldg(&G.child_off[p + 1])) {
-              ++node;
-              break;
-            }
-            node = p;
-            --depth;
-            if (node == root) {
-              phase = 2;
-              break;
-            }
-          }
-        }
-      }
-    }
-    if (big_mode) hset_clear_all(ww.w.hset, ww.w.hset_mask);
-    if (broken) {  // a capacity was exceeded: the row's mask cannot be trusted
-      hset_clear_all(ww.w.hset, ww.w.hset_mask);
-      clear_nt(G, ww.w);
-      if (lane == 0) {
-        atomicOr(&S.row_flags[row], ROW_BROKEN);
-        atomicExch(&S.counters[CNT_ERR], 1u);
-        stat_add(S, CNT_STAT_CAPERR, 1u);
-      }
+  // ---- the automata start with one state each: the base chart's last set
+  for (uint32_t j = blockIdx.x; j < n_jobs; j += gridDim.x) {
+    uint32_t* hash = A.hash + (size_t)j * (A.hash_mask + 1);
+    for (uint32_t i = threadIdx.x; i <= A.hash_mask; i += blockDim.x) hash[i] = 0u;
+    uint32_t* rec0 = A.recs + (size_t)j * A.cap * A.rec_words;
+    for (uint32_t i = threadIdx.x; i < A.rec_words; i += blockDim.x)
+      if (i < AR_SCAN || i >= AR_SCAN + 8) rec0[i] = (i >= AR_TRANS) ? T_UNKNOWN : 0u;
+    if (threadIdx.x == 0) A.n_states[j] = 1u;
+    if (warp == 0) {
+      JobCtx J = job_ctx(S, j);
+      scannable_bytes(G, J.base_items + J.base_off[J.m - 1], J.base_off[J.m] - J.base_off[J.m - 1], tmp8);
+      if (lane < 8) rec0[AR_SCAN + lane] = tmp8[lane];
     }
   }
-}
+  if (!grid_barrier(S, bar_phase)) return;
 
-// ===================================================================================== fill: publish / gather / apply
+  SweepWarp sw{G, S};
+  sw.w.nt = nt;
+  sw.w.ctr = ctr;
+  sw.tmp8 = tmp8;
+  sw.w.cur = sm_cur;
+  sw.w.cur_cap = SWEEP_CUR;
+  sw.cur_pow2 = SWEEP_CUR;
+  sw.w.hset = sm_hset;
+  sw.w.hset_mask = SWEEP_HSET - 1;
+  bool big_mode = false;
 
-__device__ __forceinline__ int32_t resolve_mask_row(const StateDev& S, uint32_t row) {
-  int32_t r = S.row_mask[row];
-  if (r <= MASK_ALIAS0) r = S.row_mask[(uint32_t)(MASK_ALIAS0 - r)];
-  if (S.row_flags[row] & ROW_BROKEN) r = MASK_ZERO;
-  return r;
+  uint32_t last_level = 0;
+  for (uint32_t L = 1; L <= G.depth; ++L) {
+    const uint32_t lo = __ldg(&G.lvl_off[L]), hi = __ldg(&G.lvl_off[L + 1]);
+    constexpr uint32_t CH = 32 * SWEEP_PER_LANE;
+    const uint32_t nL = hi - lo, cpj = (nL + CH - 1) / CH;
+    const uint32_t chunks = n_jobs * cpj;
+    // ---- the pass: one thread per (job, node).  Known transitions are final; an unknown one is
+    // claimed by the first thread that meets it, which queues it for the compute phase below, and
+    // the node is marked pending.  A pending PARENT (marked at the previous depth, computed since)
+    // is settled on the way; pending leaves are settled when the mask words are formed.
+    bool any_alive = false;
+    for (uint32_t c = gw; c < chunks; c += GW) {
+      const uint32_t j = c / cpj;
+      const uint32_t first = lo + (c % cpj) * CH + lane;
+      const JobCtx J = job_ctx(S, j);
+      uint32_t node[SWEEP_PER_LANE], byte[SWEEP_PER_LANE], par[SWEEP_PER_LANE], ps[SWEEP_PER_LANE];
+#pragma unroll
+      for (uint32_t u = 0; u < SWEEP_PER_LANE; ++u) {
+        node[u] = first + 32u * u;
+        const bool v = node[u] < hi;
+        byte[u] = v ? __ldg(&G.node_byte[node[u]]) : 0u;
+        par[u] = (v && L > 1) ? __ldg(&G.parent[node[u]]) : 0u;
+      }
+#pragma unroll
+      for (uint32_t u = 0; u < SWEEP_PER_LANE; ++u)
+        ps[u] = (node[u] < hi) ? ((L == 1) ? 0u : (uint32_t)__ldcg(J.st + par[u])) : (uint32_t)ST_DEAD;  // written by other SMs: bypass L1
+#pragma unroll
+      for (uint32_t u = 0; u < SWEEP_PER_LANE; ++u) {
+        if (node[u] >= hi) continue;
+        uint32_t p_state = ps[u];
+        if (p_state == ST_PENDING) {  // settle the parent first
+          const uint32_t gp_state = (L == 2) ? 0u : (uint32_t)__ldcg(J.st + __ldg(&G.parent[par[u]]));
+          const uint32_t t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
+          if (t2 == T_UNKNOWN || t2 == T_PENDING) {  // only if the queue overflowed: give the row up rather than guess
+            atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+            atomicExch(&S.counters[CNT_ERR], 1u);
+            p_state = ST_DEAD;
+          } else {
+            p_state = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+          }
+          J.st[par[u]] = (uint16_t)p_state;
+        }
+        uint32_t t = T_DEAD;
+        if (p_state != ST_DEAD) {
+          const uint32_t* rec = J.recs + (size_t)p_state * A.rec_words;
+          // one 256-bit test rejects most bytes without touching the transition table
+          if ((rec[AR_SCAN + (byte[u] >> 5)] >> (byte[u] & 31u)) & 1u) {
+            uint32_t* slot = J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[byte[u]];
+            t = *slot;
+            if (t == T_UNKNOWN || t == T_PENDING) t = __ldcg(slot);
+            if (t == T_UNKNOWN) {
+              t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
+              if (t == T_UNKNOWN) {  // ours to queue
+                const uint32_t at = atomicAdd(&S.counters[CNT_LEVEL_REQ + L], 1u);
+                if (at < A.req_cap) A.req[at] = ((unsigned long long)j << 32) | ((unsigned long long)p_state << 8) | byte[u];
+                t = T_PENDING;
+              }
+            }
+          }
+        }
+        J.st[node[u]] = (t == T_PENDING) ? ST_PENDING : (t == T_DEAD) ? ST_DEAD : (uint16_t)t;
+        any_alive |= (t != T_DEAD);
+      }
+    }
+    __syncwarp();
+    if (__any_sync(FULL, any_alive) && lane == 0) atomicOr(&S.counters[CNT_LEVEL_ALIVE + L], 1u);
+    if (!grid_barrier(S, bar_phase)) return;
+    last_level = L;
+    if (ld_acquire(&S.counters[CNT_LEVEL_ALIVE + L]) == 0u) break;  // nothing survives this depth in any job
+    const uint32_t n_req = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), A.req_cap);
+    if (n_req == 0) continue;  // nothing was unknown at this depth
+    // ---- compute phase: one queued transition per warp at a time, all warps of the grid in parallel
+    for (uint32_t i = gw; i < n_req; i += GW) {
+      const unsigned long long rq = __ldcg(A.req + i);
+      const uint32_t j = (uint32_t)(rq >> 32), p_state = (uint32_t)(rq >> 8) & 0xFFFFu, pb = (uint32_t)rq & 0xFFu;
+      const JobCtx J = job_ctx(S, j);
+      uint32_t r = sw.compute(J, p_state, pb, true);
+      if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
+        big_mode = true;
+        hset_clear_all(sw.w.hset, sw.w.hset_mask);
+        clear_nt(G, sw.w);
+        sw.w.cur = big;
+        sw.w.cur_cap = S.big_arena_items;
+        sw.cur_pow2 = S.big_arena_items;
+        sw.w.hset = big + S.big_arena_items;
+        sw.w.hset_mask = S.big_hset_slots - 1;
+        if (lane == 0) stat_add(S, CNT_STAT_BIG, 1u);
+        r = sw.compute(J, p_state, pb, true);
+      }
+      if (r == T_FAIL) {  // a capacity was exceeded: the row's mask cannot be trusted
+        hset_clear_all(sw.w.hset, sw.w.hset_mask);
+        clear_nt(G, sw.w);
+        if (lane == 0) {
+          atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+          atomicExch(&S.counters[CNT_ERR], 1u);
+          stat_add(S, CNT_STAT_CAPERR, 1u);
+          atomicExch(J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[pb], T_DEAD);  // lets the sweep go on
+        }
+      }
+    }
+    if (!grid_barrier(S, bar_phase)) return;
+  }
+  if (big_mode) hset_clear_all(sw.w.hset, sw.w.hset_mask);
+  if (lane == 0 && (sw.n_computed | sw.n_created)) {
+    stat_add(S, CNT_STAT_TRANS, sw.n_computed);
+    stat_add(S, CNT_STAT_LOCAL, sw.n_created);
+  }
+
+  // ---- mask words: 32 tokens per warp pass, one ballot per word (token t is valid iff the node
+  // where its bytes end was reached alive; EOS iff the chart is accepting)
+  const uint32_t Wm = G.Wm;
+  for (uint32_t c = gw; c < n_jobs * Wm; c += GW) {
+    const uint32_t j = c / Wm, wd = c % Wm;
+    const JobCtx J = job_ctx(S, j);
+    const uint32_t tok = wd * 32 + lane;
+    bool ok = false;
+    if (tok < G.V) {
+      const uint32_t node = __ldg(&G.tok_node[tok]);
+      if (node == 0xFFFFFFFFu) {
+        ok = ((int32_t)tok == G.eos) && J.accepting;
+      } else if (__ldg(&G.node_depth[node]) <= last_level) {
+        uint32_t s = __ldcg(J.st + node);
+        if (s == ST_PENDING) {  // a leaf that waited for a transition: its parent is final by now
+          const uint32_t p = __ldg(&G.parent[node]);
+          const uint32_t p_state = (p == 0) ? 0u : (uint32_t)__ldcg(J.st + p);
+          const uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node]));
+          if (t2 == T_UNKNOWN || t2 == T_PENDING || p_state == ST_PENDING) {
+            atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+            s = ST_DEAD;
+          } else {
+            s = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+          }
+        }
+        ok = s != ST_DEAD;
+      }
+    }
+    const uint32_t word = __ballot_sync(FULL, ok);
+    if (lane == 0) S.mask_rows[(size_t)S.row_mask[J.row] * Wm + wd] = word;
+  }
 }
 
 // Publish the masks computed in this call to the cache (or release the claim when the row had
@@ -713,14 +722,21 @@ __global__ void publish_kernel(StateDev S) {
   if (j < n_jobs) {
     const uint32_t row = S.jobs[j];
     const int32_t sid = S.row_state[row];
-    const bool broken = S.row_flags[row] & ROW_BROKEN;
+    const bool broken = (S.row_flags[row] & ROW_BROKEN) || S.counters[CNT_BAR_ERR];
+    if (S.counters[CNT_BAR_ERR]) atomicOr(&S.row_flags[row], ROW_BROKEN);
     if (sid >= 0) {
       const int32_t mrow = S.row_mask[row];
       S.st_mask[sid] = (!broken && mrow >= (int32_t)S.B) ? mrow : -1;
     }
   }
 }
-__global__ void end_fill_kernel(StateDev S) { S.counters[CNT_N_JOBS] = 0u; }
+
+__device__ __forceinline__ int32_t resolve_mask_row(const StateDev& S, uint32_t row) {
+  int32_t r = S.row_mask[row];
+  if (r <= MASK_ALIAS0) r = S.row_mask[(uint32_t)(MASK_ALIAS0 - r)];
+  if (S.row_flags[row] & ROW_BROKEN) r = MASK_ZERO;
+  return r;
+}
 
 // mask_out[row][w] for every row
 __global__ void gather_kernel(GrammarDev G, StateDev S, uint32_t* out, size_t stride_words) {
@@ -877,19 +893,29 @@ static inline cudaError_t opt_in_smem(const void* fn, size_t bytes) {
 
 static size_t adv_smem_bytes() { return (size_t)ADV_WARPS * ADV_WARP_WORDS * 4; }
 static size_t init_smem_bytes() { return (size_t)ADV_WARP_WORDS * 4; }
-static size_t walk_smem_bytes() { return (size_t)WALK_WARPS * WALK_WARP_WORDS * 4; }
-int walk_warps() { return WALK_WARPS; }
+// Dynamic shared memory of the sweep for a grammar: per-warp scratch plus, if they fit the
+// budget, the item-info / byte-class / byte-class-number tables.
+void sweep_layout(const GrammarDev& G, uint32_t* smem_bytes, uint32_t* tables_in_smem) {
+  const uint32_t ntw = (2u * G.Nw + 7u) & ~7u;
+  const uint32_t warp_words = SWEEP_CUR + SWEEP_HSET + ntw + W_CTRS + 8;
+  uint32_t bytes = SWEEP_WARPS * warp_words * 4u;
+  const uint32_t tab = (((G.D + 3u) & ~3u) + G.C * 8u + 64u) * 4u;
+  *tables_in_smem = tab <= SWEEP_TABLE_BYTES ? 1u : 0u;
+  if (*tables_in_smem) bytes += tab;
+  *smem_bytes = bytes;
+}
+int walk_warps() { return SWEEP_WARPS; }
 
 cudaError_t configure_kernels() {
   cudaError_t e;
   if ((e = opt_in_smem((const void*)init_kernel, init_smem_bytes())) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)advance_kernel, adv_smem_bytes())) != cudaSuccess) return e;
-  if ((e = opt_in_smem((const void*)walk_kernel, walk_smem_bytes())) != cudaSuccess) return e;
+  if ((e = opt_in_smem((const void*)sweep_kernel, 160 * 1024)) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
-cudaError_t walk_blocks_per_sm(int* out) {
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, walk_kernel, WALK_WARPS * 32, walk_smem_bytes());
+cudaError_t walk_blocks_per_sm(int* out, uint32_t smem_bytes) {
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, sweep_kernel, SWEEP_WARPS * 32, smem_bytes);
 }
 
 void launch_init(const GrammarDev& G, const StateDev& S, int32_t* result_dev, cudaStream_t st) {
@@ -905,21 +931,24 @@ void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const
 void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st) {
   advance_kernel<<<(S.B + ADV_WARPS - 1) / ADV_WARPS, ADV_WARPS * 32, adv_smem_bytes(), st>>>(G, S, tokens, status);
 }
+static void launch_sweep_coop(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) {
+  GrammarDev g = G;
+  StateDev s = S;
+  void* args[] = {&g, &s};
+  cudaLaunchCooperativeKernel((const void*)sweep_kernel, dim3((unsigned)grid), dim3(SWEEP_WARPS * 32), args,
+                              S.au.smem_bytes, st);
+}
 void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStream_t st, cudaEvent_t before_walk,
                  cudaEvent_t after_walk) {
-  plan_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(G, S);
-  prepare_rows_kernel<<<S.B, 256, 0, st>>>(G, S);
-  auto_init_kernel<<<S.B, 256, 0, st>>>(G, S);
+  plan_kernel<<<1, 1024, 0, st>>>(G, S);
   if (before_walk) cudaEventRecord(before_walk, st);
-  walk_kernel<<<walk_grid, WALK_WARPS * 32, walk_smem_bytes(), st>>>(G, S);
+  launch_sweep_coop(G, S, walk_grid, st);
   if (after_walk) cudaEventRecord(after_walk, st);
   publish_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(S);
 }
-void launch_walk(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) {
-  auto_init_kernel<<<S.B, 256, 0, st>>>(G, S);
-  walk_kernel<<<grid, WALK_WARPS * 32, walk_smem_bytes(), st>>>(G, S);
-}
-void launch_end_fill(const StateDev& S, cudaStream_t st) { end_fill_kernel<<<1, 1, 0, st>>>(S); }
+// the sweep alone, for jobs the caller has already listed (used by the allocation-free entry point)
+void launch_walk(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) { launch_sweep_coop(G, S, grid, st); }
+void launch_end_fill(const StateDev& S, cudaStream_t st) { (void)S; (void)st; }
 void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st) {
   dim3 grid((unsigned)std::min<size_t>((stride_words + 255) / 256, 64), S.B);
   gather_kernel<<<grid, 256, 0, st>>>(G, S, out, stride_words);

@@ -7,7 +7,8 @@
 namespace fmt {
 
 cudaError_t configure_kernels();
-cudaError_t walk_blocks_per_sm(int* out);
+cudaError_t walk_blocks_per_sm(int* out, uint32_t smem_bytes);
+void sweep_layout(const GrammarDev& G, uint32_t* smem_bytes, uint32_t* tables_in_smem);
 int walk_warps();
 
 void launch_init(const GrammarDev& G, const StateDev& S, int32_t* result_dev, cudaStream_t st);

@@ -23,7 +23,8 @@ constexpr uint32_t NA_ARENA_ITEMS = 8192;   // per-warp overflow area for Earley
 constexpr uint32_t NA_HSET_SLOTS = 2048;    // per-warp overflow uniqueness hash
 // header: counters, then per-chart arrays
 constexpr uint32_t NA_OFF_COUNTERS = 0;                          // [CNT_TOTAL]
-constexpr uint32_t NA_OFF_JOBS = 64;                             // [NA_MAX]
+constexpr uint32_t NA_OFF_JOBS = 128;                            // [NA_MAX]
+constexpr uint32_t NA_REQ_CAP = 1u << 16;                        // transitions queued per trie depth
 constexpr uint32_t NA_OFF_FLAGS = NA_OFF_JOBS + NA_MAX;          // [NA_MAX]
 constexpr uint32_t NA_OFF_MASKROW = NA_OFF_FLAGS + NA_MAX;       // [NA_MAX] int32
 constexpr uint32_t NA_OFF_CHART = NA_OFF_MASKROW + NA_MAX;       // [NA_MAX] uint64 (8-byte aligned)
@@ -41,11 +42,16 @@ constexpr size_t NA_OFF_BIG = NA_HEADER_WORDS;
 constexpr size_t NA_OFF_RECS = NA_OFF_BIG + NA_BIG_WORDS;
 constexpr size_t NA_OFF_HASH = NA_OFF_RECS + (size_t)NA_MAX * NA_REC_WORDS_PER_CHART;
 constexpr size_t NA_OFF_ITEMS = NA_OFF_HASH + (size_t)NA_MAX * NA_HASH_SLOTS;
-constexpr size_t NA_WORDS = NA_OFF_ITEMS + NA_ITEM_WORDS;
+// per (chart, trie node) one uint16: which Earley set the node's bytes lead to
+constexpr size_t NA_ST_ENTRIES = 8u << 20;
+constexpr size_t NA_OFF_ST = NA_OFF_ITEMS + NA_ITEM_WORDS;
+constexpr size_t NA_OFF_REQ = NA_OFF_ST + NA_ST_ENTRIES / 2;       // 8-byte aligned: all sizes above are even
+constexpr size_t NA_WORDS = NA_OFF_REQ + 2 * (size_t)NA_REQ_CAP;
+static_assert(CNT_TOTAL <= NA_OFF_JOBS, "the counters overlap the job list");
 static_assert(NA_OFF_NSTATES + NA_MAX <= NA_HEADER_WORDS, "header too small");
 static_assert((NA_OFF_CHART % 2) == 0, "64-bit offsets must be 8-byte aligned");
 
-// ~36 MB, held by every GPU that loads the library until the process exits
+// ~52 MB, held by every GPU that loads the library until the process exits
 static __device__ __align__(256) uint32_t g_noalloc_scratch[NA_WORDS];
 
 struct Offsets {
@@ -82,21 +88,13 @@ __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scrat
     big[(i / NA_HSET_SLOTS) * per_warp + NA_ARENA_ITEMS + (i % NA_HSET_SLOTS)] = 0xffffffffu;
 }
 
-// One thread: the job list holds the charts whose header was accepted; accepting charts get
-// their EOS bit.  (Runs after the prepare kernel, so the masks are already zero.)
-__global__ void noalloc_jobs_kernel(GrammarDev G, StateDev S, const uint32_t* scratch, const uint32_t* charts,
-                                    uint32_t n, uint32_t* mask) {
+// One thread: the job list holds the charts whose header was accepted.
+__global__ void noalloc_jobs_kernel(StateDev S, const uint32_t* scratch, uint32_t n) {
   if (blockIdx.x != 0 || threadIdx.x != 0) return;
   uint32_t j = 0;
-  for (uint32_t r = 0; r < n; ++r) {
-    if (scratch[NA_OFF_BAD + r]) continue;
-    S.jobs[j++] = r;
-    const uint32_t* ch = charts + S.row_chart[r];
-    if (G.eos >= 0 && (ch[CH_FLAGS] & CHART_ACCEPTING))
-      mask[(size_t)r * G.Wm + ((uint32_t)G.eos >> 5)] |= 1u << ((uint32_t)G.eos & 31u);
-  }
+  for (uint32_t r = 0; r < n; ++r)
+    if (!scratch[NA_OFF_BAD + r]) S.jobs[j++] = r;
   S.counters[CNT_N_JOBS] = j;
-  S.counters[CNT_WORK] = 0u;
 }
 
 __global__ void noalloc_finish_kernel(GrammarDev G, StateDev S, const uint32_t* scratch, uint32_t n, uint32_t* mask,
@@ -147,6 +145,10 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   if (!G) return fail(FMT_ERR_INVALID_ARG, "the grammar was compiled host_only");
   if (cudaGetDevice(&dev) != cudaSuccess || dev != gdev || dev < 0 || dev >= kMaxDevices)
     return fail(FMT_ERR_INVALID_ARG, "the grammar belongs to another device than the current one");
+  const size_t st_stride = ((size_t)G->T + 63u) & ~(size_t)63u;
+  if ((size_t)n * st_stride > NA_ST_ENTRIES)
+    return fail(FMT_ERR_CAPACITY,
+                "fmt_fill_mask_noalloc: charts x trie nodes exceeds the built-in scratch (8 Mi entries); pass fewer charts per call");
   Offsets off;
   for (uint32_t r = 0; r <= n; ++r) {
     off.v[r] = chart_offsets[r];
@@ -178,9 +180,14 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   S.au.hash = scratch + NA_OFF_HASH;
   S.au.items = scratch + NA_OFF_ITEMS;
   S.au.n_states = scratch + NA_OFF_NSTATES;
+  S.au.st = reinterpret_cast<uint16_t*>(scratch + NA_OFF_ST);
+  S.au.st_stride = (uint32_t)st_stride;
+  S.au.req = reinterpret_cast<unsigned long long*>(scratch + NA_OFF_REQ);
+  S.au.req_cap = NA_REQ_CAP;
+  sweep_layout(*G, &S.au.smem_bytes, &S.au.tables_in_smem);
   cudaStream_t st = (cudaStream_t)stream;
   noalloc_prepare_kernel<<<256, 256, 0, st>>>(*G, S, scratch, charts_dev, off, n, mask_dev);
-  noalloc_jobs_kernel<<<1, 32, 0, st>>>(*G, S, scratch, charts_dev, n, mask_dev);
+  noalloc_jobs_kernel<<<1, 32, 0, st>>>(S, scratch, n);
   launch_walk(*G, S, (int)NA_GRID, st);
   noalloc_finish_kernel<<<n, 128, 0, st>>>(*G, S, scratch, n, mask_dev, status_dev);
   e = cudaGetLastError();

@@ -65,23 +65,26 @@ def test_trie_is_a_valid_csr_trie(config, kw):
     n = walk(child_off, node_byte, vocab[300])
     assert {299, 300} <= set(tok_ids[tok_off[n]:tok_off[n + 1]].tolist())
     assert info.trie_depth == max(len(t) for t in vocab)
-    # work units: every node below the root is covered exactly once
-    unit_node, unit_kind = g.table(5), g.table(9)
-    covered = np.zeros(T, dtype=np.int32)
-    size = np.ones(T, dtype=np.int64)
-    for n in range(T - 1, 0, -1):
-        size[parent[n]] += size[n]
-    sub = np.zeros(T, dtype=bool)
-    sub[unit_node[unit_kind == 0]] = True
-    for n in unit_node[unit_kind == 1]:
-        covered[n] += 1
-    inside = np.zeros(T, dtype=np.int32)
-    for n in range(1, T):  # parents come before children in breadth-first order
-        inside[n] = inside[parent[n]] + (1 if sub[n] else 0)
-    covered += inside
-    has_tok = np.diff(tok_off.astype(np.int64)) > 0
-    assert (covered[1:][has_tok[1:]] == 1).all()
-    assert (covered[1:] <= 1).all()
+    # breadth-first numbering: every depth is one contiguous range, parents come before children
+    lvl = g.table(5)
+    assert len(lvl) == info.trie_depth + 2 and lvl[0] == 0 and lvl[1] == 1 and lvl[-1] == T
+    depth = np.zeros(T, dtype=np.int64)
+    for n in range(1, T):
+        assert parent[n] < n
+        depth[n] = depth[parent[n]] + 1
+    for L in range(info.trie_depth + 1):
+        assert (depth[lvl[L]:lvl[L + 1]] == L).all() and lvl[L] < lvl[L + 1]
+    # token -> node is the inverse of the per-node token lists
+    tok_node = g.table(9)
+    assert len(tok_node) == len(vocab)
+    for t in range(0, len(vocab), 23):
+        if vocab[t]:
+            assert tok_node[t] == walk(child_off, node_byte, vocab[t])
+        else:
+            assert tok_node[t] == 0xFFFFFFFF
+    # bytes in one class behave alike: for this grammar digits must share a class, '(' and ')' must not
+    eq = g.table(10)
+    assert info.n_byte_classes == len(set(eq.tolist()))
 
 
 def test_grammar_reduction_and_nullability():
