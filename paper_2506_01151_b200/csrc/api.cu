@@ -159,14 +159,31 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
     d.start_nullable = h.start_nullable ? 1u : 0u;
     cudaError_t e = cudaGetDevice(&g->device);
 #define UP(field) if (e == cudaSuccess) e = g->bufs.upload(h.field, &d.field)
-    UP(info);
     UP(lhs);
-    UP(class_bits);
-    UP(eq_of_byte);
     d.n_eq = h.n_eq;
-    UP(nt_closure);
-    UP(direct_off);
-    UP(direct_items);
+    {  // info | class_bits | eq_of_byte | nt_closure | direct_off | direct_items, each 16-byte aligned
+      std::vector<uint32_t> blob;
+      auto put = [&](const void* src, size_t bytes) {
+        size_t at = blob.size();
+        blob.resize(at + ((bytes + 15) / 16) * 4, 0u);
+        memcpy(blob.data() + at, src, bytes);
+        return at;
+      };
+      const size_t o_info = put(h.info.data(), h.info.size() * 4);
+      const size_t o_cls = put(h.class_bits.data(), h.class_bits.size() * 4);
+      const size_t o_eq = put(h.eq_of_byte.data(), 256);
+      const size_t o_clo = put(h.nt_closure.data(), h.nt_closure.size() * 4);
+      const size_t o_doff = put(h.direct_off.data(), h.direct_off.size() * 4);
+      const size_t o_dit = put(h.direct_items.data(), h.direct_items.size() * 2);
+      if (e == cudaSuccess) e = g->bufs.upload(blob, &d.hot_block);
+      d.hot_words = (uint32_t)blob.size();
+      d.info = d.hot_block + o_info;
+      d.class_bits = d.hot_block + o_cls;
+      d.eq_of_byte = reinterpret_cast<const uint8_t*>(d.hot_block + o_eq);
+      d.nt_closure = d.hot_block + o_clo;
+      d.direct_off = d.hot_block + o_doff;
+      d.direct_items = reinterpret_cast<const uint16_t*>(d.hot_block + o_dit);
+    }
     UP(child_off);
     UP(node_byte);
     UP(parent);
@@ -308,6 +325,7 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(au.st, (size_t)batch * au.st_stride, 0xFF);
   au.req_cap = 1u << 20;
   AL(au.req, au.req_cap, 0);
+  AL(au.job_info, batch, 0);
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);

@@ -12,20 +12,22 @@
 
 namespace fmt {
 
-constexpr uint32_t ADV_CUR_CAP = 2048;     // items of one set (power of two)
-constexpr uint32_t ADV_HSET = 4096;        // hash slots (power of two)
+constexpr uint32_t ADV_CUR_CAP = 1024;     // items of one set (power of two)
+constexpr uint32_t ADV_HSET = 2048;        // hash slots (power of two)
 constexpr uint32_t ADV_MAX_ITEMS = 65536;  // items of a chart the live bitmap can describe
 constexpr uint32_t ADV_PAIRS = 1024;       // (set, non-terminal) needs of one Compact
 constexpr uint32_t ADV_MAX_SETS = 2048;
 constexpr uint32_t ADV_NT_WORDS = 256;     // 2 * Nw, Nw <= 128
+constexpr uint32_t ADV_STAGE = 2048;       // a source chart up to this many words is read from shared memory
 constexpr uint32_t ADV_WARP_WORDS =
-    ADV_CUR_CAP + ADV_HSET + ADV_MAX_ITEMS / 32 + ADV_PAIRS + ADV_MAX_SETS + ADV_NT_WORDS + W_CTRS;
+    ADV_CUR_CAP + ADV_HSET + ADV_MAX_ITEMS / 32 + ADV_PAIRS + ADV_MAX_SETS + ADV_NT_WORDS + W_CTRS + ADV_STAGE;
 
 struct AdvScratch {
   WarpCtx w;
   uint32_t* live;   // [ADV_MAX_ITEMS/32] bitmap over the source chart's items
   uint32_t* pairs;  // [ADV_PAIRS]
   uint32_t* sets;   // [ADV_MAX_SETS] per-set live count, then new index
+  uint32_t* stage;  // [ADV_STAGE]
 };
 
 __device__ __forceinline__ AdvScratch adv_scratch(uint32_t* base) {
@@ -39,6 +41,7 @@ __device__ __forceinline__ AdvScratch adv_scratch(uint32_t* base) {
   s.sets = s.pairs + ADV_PAIRS;
   s.w.nt = s.sets + ADV_MAX_SETS;
   s.w.ctr = s.w.nt + ADV_NT_WORDS;
+  s.stage = s.w.ctr + W_CTRS;
   return s;
 }
 
@@ -69,52 +72,50 @@ __device__ __forceinline__ void push_need(const AdvScratch& s, uint32_t o, uint3
   else s.w.ctr[W_OVERFLOW] = 1u;
 }
 
-// Hash of a finished chart (everything but the hash words themselves); two independent 32-bit sums.
-__device__ __forceinline__ void chart_hash(uint32_t* ch) {
-  const uint32_t lane = lane_id();
-  __syncwarp();
-  const uint32_t words = ch[CH_WORDS];
+// The chart hash is a sum over (word index, value) pairs, so it can be accumulated while the
+// words are written, in any order and by any lane.  Two independent 32-bit sums.
+struct HashAcc {
   uint32_t h1 = 0, h2 = 0;
-  for (uint32_t i = lane; i < words; i += 32) {
-    if (i == CH_HASH_LO || i == CH_HASH_HI) continue;
-    uint32_t v = ch[i];
+  __device__ __forceinline__ void add(uint32_t i, uint32_t v) {
     h1 += mix32(v ^ (i * 0x9E3779B1u));
     h2 += mix32((v + 0x632BE5ABu) ^ (i * 0x85EBCA77u));
   }
-  for (int d = 16; d > 0; d >>= 1) {
-    h1 += __shfl_xor_sync(FULL, h1, d);
-    h2 += __shfl_xor_sync(FULL, h2, d);
-  }
-  __syncwarp();
-  if (lane == 0) {
-    ch[CH_HASH_LO] = h1;
-    ch[CH_HASH_HI] = h2;
-  }
-  __syncwarp();
+};
+__device__ __forceinline__ void put(uint32_t* ch, HashAcc& h, uint32_t i, uint32_t v) {
+  ch[i] = v;
+  h.add(i, v);
 }
 
 // Write the last set (cur[0..n), unsorted, completed items already removed) and finish the header.
-// dst already holds set_off[0..m_new) and the kept items of the earlier sets (`kept` of them).
+// dst already holds set_off[0..m_new) and the kept items of the earlier sets (`kept` of them), all
+// accounted for in `h`.
 __device__ __forceinline__ int finish_chart(const AdvScratch& s, uint32_t* dst, uint32_t dst_cap, uint32_t m_new,
-                                            uint32_t kept, uint32_t n, bool accepting) {
+                                            uint32_t kept, uint32_t n, bool accepting, HashAcc h) {
   const uint32_t lane = lane_id();
   uint32_t words = CH_HDR + (m_new + 2) + kept + n;
   if (words > dst_cap || kept + n >= ADV_MAX_ITEMS || n > ADV_CUR_CAP) return -1;
   sort_items(s.w.cur, n, ADV_CUR_CAP);
-  uint32_t* items = dst + CH_HDR + (m_new + 2);
-  for (uint32_t i = lane; i < n; i += 32) items[kept + i] = s.w.cur[i];
+  const uint32_t items_at = CH_HDR + (m_new + 2);
+  for (uint32_t i = lane; i < n; i += 32) put(dst, h, items_at + kept + i, s.w.cur[i]);
   if (lane == 0) {
-    dst[CH_SETS] = m_new + 1;
-    dst[CH_ITEMS] = kept + n;
-    dst[CH_FLAGS] = accepting ? CHART_ACCEPTING : 0u;
-    dst[CH_WORDS] = words;
-    dst[6] = 0;
-    dst[7] = 0;
-    dst[CH_HDR + m_new] = kept;          // first item of the last set
-    dst[CH_HDR + m_new + 1] = kept + n;  // end
+    put(dst, h, CH_SETS, m_new + 1);
+    put(dst, h, CH_ITEMS, kept + n);
+    put(dst, h, CH_FLAGS, accepting ? CHART_ACCEPTING : 0u);
+    put(dst, h, CH_WORDS, words);
+    put(dst, h, 6, 0u);
+    put(dst, h, 7, 0u);
+    put(dst, h, CH_HDR + m_new, kept);          // first item of the last set
+    put(dst, h, CH_HDR + m_new + 1, kept + n);  // end
+  }
+  for (int d = 16; d > 0; d >>= 1) {
+    h.h1 += __shfl_xor_sync(FULL, h.h1, d);
+    h.h2 += __shfl_xor_sync(FULL, h.h2, d);
+  }
+  if (lane == 0) {
+    dst[CH_HASH_LO] = h.h1;
+    dst[CH_HASH_HI] = h.h2;
   }
   __syncwarp();
-  chart_hash(dst);
   return 1;
 }
 
@@ -137,7 +138,7 @@ __device__ int chart_init(const GrammarDev& G, const AdvScratch& s, uint32_t* ds
     return -1;
   }
   uint32_t n = drop_completed(G, s.w, min(s.w.ctr[W_NCUR], s.w.cur_cap));
-  return finish_chart(s, dst, dst_cap, 0u, 0u, n, accepting);
+  return finish_chart(s, dst, dst_cap, 0u, 0u, n, accepting, HashAcc{});
 }
 
 // One byte.  Returns 1 (dst holds the new chart), 0 (the byte cannot follow: dst is garbage) or
@@ -147,10 +148,16 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
   const uint32_t lane = lane_id();
   const uint32_t m = src[CH_SETS];
   const uint32_t n_items = src[CH_ITEMS];
+  if (m == 0 || m + 1 > ADV_MAX_SETS || n_items > ADV_MAX_ITEMS) return -1;
+  // small charts are read from shared memory from here on
+  const uint32_t src_words = src[CH_WORDS];
+  __syncwarp();
+  if (src_words <= ADV_STAGE) {
+    for (uint32_t i = lane; i < src_words; i += 32) s.stage[i] = src[i];
+    src = s.stage;
+  }
   const uint32_t* soff = src + CH_HDR;
   const uint32_t* sitems = src + CH_HDR + m + 1;
-  if (m == 0 || m + 1 > ADV_MAX_SETS || n_items > ADV_MAX_ITEMS) return -1;
-  __syncwarp();
   if (lane < W_CTRS) s.w.ctr[lane] = 0u;
   __syncwarp();
   // ---- Scan
@@ -175,26 +182,49 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     uint32_t it = s.w.cur[i];
     if ((it >> 16) < m) push_need(s, it >> 16, __ldg(&G.lhs[it & 0xFFFFu]));
   }
-  for (uint32_t head = 0;; ++head) {
+  // needs are served a wave at a time, one lane per (set, non-terminal) need
+  for (uint32_t head = 0;;) {
     __syncwarp();
-    uint32_t np = min(s.w.ctr[W_NPAIRS], ADV_PAIRS);
+    const uint32_t np = min(s.w.ctr[W_NPAIRS], ADV_PAIRS);
     __syncwarp();
     if (head >= np) break;
-    uint32_t key = s.pairs[head];
-    uint32_t o = key >> 16, A = key & 0xFFFFu;
-    uint32_t a = soff[o], b = soff[o + 1];
-    for (uint32_t k = a + lane; k < b; k += 32) {
-      uint32_t wi = sitems[k];
-      uint32_t inf = G.info[wi & 0xFFFFu];
-      if ((inf >> INFO_KIND_SHIFT) == KIND_NT && (inf & INFO_ARG_MASK) == A) {
-        uint32_t bit = 1u << (k & 31u);
-        uint32_t old = atomicOr(&s.live[k >> 5], bit);
-        if (!(old & bit)) push_need(s, wi >> 16, __ldg(&G.lhs[wi & 0xFFFFu]));
+    const uint32_t mine = head + lane;
+    if (mine < np) {
+      const uint32_t key = s.pairs[mine];
+      const uint32_t o = key >> 16, A = key & 0xFFFFu;
+      const uint32_t a = soff[o], b = soff[o + 1];
+      for (uint32_t k = a; k < b; ++k) {
+        const uint32_t wi = sitems[k];
+        const uint32_t inf = G.info[wi & 0xFFFFu];
+        if ((inf >> INFO_KIND_SHIFT) == KIND_NT && (inf & INFO_ARG_MASK) == A) {
+          const uint32_t bit = 1u << (k & 31u);
+          const uint32_t old = atomicOr(&s.live[k >> 5], bit);
+          if (!(old & bit)) push_need(s, wi >> 16, __ldg(&G.lhs[wi & 0xFFFFu]));
+        }
       }
     }
+    head = min(head + 32u, np);
   }
-  hset_clear_all(s.w.hset, s.w.hset_mask);  // the hash held (set, non-terminal) pairs
+  const uint32_t n_pairs = min(s.w.ctr[W_NPAIRS], ADV_PAIRS);
+  __syncwarp();
+  if (n_pairs * 8u > s.w.hset_mask) {
+    hset_clear_all(s.w.hset, s.w.hset_mask);  // the hash held (set, non-terminal) pairs
+  } else {
+    for (uint32_t i = lane; i < n_pairs; i += 32) {
+      const uint32_t key = s.pairs[i];
+      uint32_t hh = mix32(key) & s.w.hset_mask;
+      for (uint32_t probe = 0; probe <= s.w.hset_mask; ++probe) {
+        if (s.w.hset[hh] == key) {
+          s.w.hset[hh] = EMPTY_SLOT;
+          break;
+        }
+        hh = (hh + 1) & s.w.hset_mask;
+      }
+    }
+    __syncwarp();
+  }
   if (s.w.ctr[W_OVERFLOW]) {
+    hset_clear_all(s.w.hset, s.w.hset_mask);
     clear_nt(G, s.w);
     return -1;
   }
@@ -205,6 +235,7 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     s.sets[k] = c;
   }
   __syncwarp();
+  HashAcc h;
   uint32_t m_new = 0, kept = 0;
   for (uint32_t base = 0; base < m; base += 32) {
     uint32_t k = base + lane;
@@ -218,7 +249,7 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     }
     if (k < m) {
       if (c > 0) {
-        if (CH_HDR + my_new < dst_cap) dst[CH_HDR + my_new] = kept + incl - c;
+        if (CH_HDR + my_new < dst_cap) put(dst, h, CH_HDR + my_new, kept + incl - c);
         s.sets[k] = my_new;
       } else {
         s.sets[k] = 0xffffffffu;
@@ -234,7 +265,7 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     return -1;
   }
   // ---- copy the live items, origins renumbered
-  uint32_t* ditems = dst + CH_HDR + (m_new + 2);
+  const uint32_t items_at = CH_HDR + (m_new + 2);
   uint32_t bad = 0;
   uint32_t out = 0;
   for (uint32_t base = 0; base < n_items; base += 32) {
@@ -245,7 +276,7 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
       uint32_t it = sitems[i];
       uint32_t no = s.sets[it >> 16];
       if (no == 0xffffffffu) bad = 1;
-      ditems[out + __popc(bal & ((1u << lane) - 1u))] = (no << 16) | (it & 0xFFFFu);
+      put(dst, h, items_at + out + __popc(bal & ((1u << lane) - 1u)), (no << 16) | (it & 0xFFFFu));
     }
     out += __popc(bal);
   }
@@ -264,7 +295,7 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
   predict_into_cur(G, s.w, m_new);
   if (bad || s.w.ctr[W_OVERFLOW]) return -1;
   n = min(s.w.ctr[W_NCUR], s.w.cur_cap);
-  return finish_chart(s, dst, dst_cap, m_new, kept, n, accepting);
+  return finish_chart(s, dst, dst_cap, m_new, kept, n, accepting, h);
 }
 
 }  // namespace fmt

@@ -23,6 +23,11 @@ struct GrammarDev {
   const uint8_t* node_depth;     // [T]
   const uint32_t* tok_off;       // [T+1]
   const uint32_t* tok_ids;
+  // The tables above that every Earley step reads (info, class_bits, eq_of_byte, nt_closure,
+  // direct_off, direct_items) sit in one contiguous block so that a kernel can copy them into
+  // shared memory at once and shift the six pointers.
+  const uint32_t* hot_block;
+  uint32_t hot_words;
   const uint32_t* lvl_off;       // [depth+2]
   const uint32_t* tok_node;      // [V]
   const uint32_t* vocab_off;     // [V+1]
@@ -90,7 +95,8 @@ struct AutoDev {
   unsigned long long* req;  // [req_cap] transitions to compute at the current depth: job << 32 | state << 8 | byte
   uint32_t req_cap;
   uint32_t smem_bytes;      // dynamic shared memory of the sweep kernel
-  uint32_t tables_in_smem;  // 1: item info, byte classes and byte class numbers are staged in shared memory
+  uint32_t tables_in_smem;  // 1: the grammar's hot tables are staged in shared memory
+  uint4* job_info;          // [jobs] x: chart offset low, y: chart offset high, z: live sets m, w: row | accepting << 31
 };
 constexpr uint16_t ST_DEAD = 0xFFFFu, ST_PENDING = 0xFFFEu;
 constexpr uint32_t T_UNKNOWN = 0xffffffffu, T_DEAD = 0xfffffffeu, T_FAIL = 0xfffffffdu, T_PENDING = 0xfffffffcu;

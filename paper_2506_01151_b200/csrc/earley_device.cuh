@@ -162,7 +162,8 @@ __device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const War
 
 // Predict (Section 3.2) for all non-terminals collected in w.nt[0..Nw): append the start items of
 // every rule of every non-terminal in their closure, origin = cur_index.  These items are all new
-// (nothing else in the set has this origin), so no uniqueness check is needed.
+// (nothing else in the set has this origin), so no uniqueness check is needed.  Each lane expands
+// one non-terminal of the closure at a time; a warp scan gives every lane its place in cur.
 __device__ __forceinline__ void predict_into_cur(const GrammarDev& G, const WarpCtx& w, uint32_t cur_index) {
   const uint32_t lane = lane_id();
   const uint32_t Nw = G.Nw;
@@ -176,25 +177,36 @@ __device__ __forceinline__ void predict_into_cur(const GrammarDev& G, const Warp
     while (bits) {
       uint32_t y = wi * 32u + (uint32_t)(__ffs(bits) - 1);
       bits &= bits - 1;
-      for (uint32_t i = lane; i < Nw; i += 32) clos[i] |= __ldg(&G.nt_closure[y * Nw + i]);
+      for (uint32_t i = lane; i < Nw; i += 32) clos[i] |= G.nt_closure[y * Nw + i];
     }
   }
   __syncwarp();
   uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
   bool over = false;
   for (uint32_t wi = 0; wi < Nw && !over; ++wi) {
-    uint32_t bits = clos[wi];
-    while (bits) {
-      uint32_t z = wi * 32u + (uint32_t)(__ffs(bits) - 1);
-      bits &= bits - 1;
-      uint32_t lo = __ldg(&G.direct_off[z]), hi = __ldg(&G.direct_off[z + 1]);
-      if (n + (hi - lo) > w.cur_cap) {
+    const uint32_t bits = clos[wi];
+    const uint32_t cnt = __popc(bits);
+    for (uint32_t base = 0; base < cnt && !over; base += 32) {
+      const uint32_t k = base + lane;
+      uint32_t lo = 0, len = 0;
+      if (k < cnt) {
+        const uint32_t z = wi * 32u + __fns(bits, 0, k + 1);
+        lo = G.direct_off[z];
+        len = G.direct_off[z + 1] - lo;
+      }
+      uint32_t incl = len;
+      for (int d = 1; d < 32; d <<= 1) {
+        uint32_t t = __shfl_up_sync(FULL, incl, d);
+        if ((int)lane >= d) incl += t;
+      }
+      const uint32_t total = __shfl_sync(FULL, incl, 31);
+      if (n + total > w.cur_cap) {
         over = true;
         break;
       }
-      for (uint32_t k = lo + lane; k < hi; k += 32)
-        w.cur[n + (k - lo)] = (cur_index << 16) | (uint32_t)__ldg(&G.direct_items[k]);
-      n += hi - lo;
+      uint32_t at = n + incl - len;
+      for (uint32_t i = 0; i < len; ++i) w.cur[at + i] = (cur_index << 16) | (uint32_t)G.direct_items[lo + i];
+      n += total;
     }
   }
   __syncwarp();
@@ -204,6 +216,21 @@ __device__ __forceinline__ void predict_into_cur(const GrammarDev& G, const Warp
   }
   for (uint32_t i = lane; i < Nw; i += 32) ntmask[i] = 0u;
   __syncwarp();
+}
+
+// Copy the grammar's hot tables into shared memory (all threads of the block take part, the
+// caller synchronizes) and return a view of the grammar that reads them from there.
+__device__ __forceinline__ GrammarDev stage_hot_tables(const GrammarDev& Gg, uint32_t* dst) {
+  for (uint32_t i = threadIdx.x; i < Gg.hot_words; i += blockDim.x) dst[i] = Gg.hot_block[i];
+  GrammarDev G = Gg;
+  G.info = dst + (Gg.info - Gg.hot_block);
+  G.class_bits = dst + (Gg.class_bits - Gg.hot_block);
+  G.eq_of_byte = reinterpret_cast<const uint8_t*>(dst + (reinterpret_cast<const uint32_t*>(Gg.eq_of_byte) - Gg.hot_block));
+  G.nt_closure = dst + (Gg.nt_closure - Gg.hot_block);
+  G.direct_off = dst + (Gg.direct_off - Gg.hot_block);
+  G.direct_items = reinterpret_cast<const uint16_t*>(dst + (reinterpret_cast<const uint32_t*>(Gg.direct_items) - Gg.hot_block));
+  G.hot_block = dst;
+  return G;
 }
 
 // Drop the items with the dot at the end from cur[0..n) in place; returns the new count.
@@ -255,6 +282,22 @@ __device__ __forceinline__ void scannable_bytes(const GrammarDev& G, const uint3
 // which must not exceed cap_pow2.
 __device__ __forceinline__ void sort_items(uint32_t* a, uint32_t n, uint32_t cap_pow2) {
   const uint32_t lane = lane_id();
+  if (n <= 32) {  // one item per lane, compare-exchange through shuffles
+    __syncwarp();
+    uint32_t v = (lane < n) ? a[lane] : 0xffffffffu;
+#pragma unroll
+    for (uint32_t k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+      for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+        const uint32_t other = __shfl_xor_sync(FULL, v, j);
+        const bool up = (lane & k) == 0, lower = (lane & j) == 0;
+        v = (lower == up) ? min(v, other) : max(v, other);
+      }
+    }
+    if (lane < n) a[lane] = v;
+    __syncwarp();
+    return;
+  }
   uint32_t P = 32;
   while (P < n) P <<= 1;
   if (P > cap_pow2) P = cap_pow2;

@@ -136,11 +136,18 @@ __global__ void reset_kernel(StateDev S, const uint32_t* rows, uint32_t n, const
 
 constexpr int ADV_WARPS = 4;
 
-__global__ void __launch_bounds__(ADV_WARPS * 32) advance_kernel(GrammarDev G, StateDev S, const int32_t* tokens,
+constexpr uint32_t HOT_TABLE_BYTES = 24 * 1024;  // grammar tables up to this size are staged in shared memory
+
+__global__ void __launch_bounds__(ADV_WARPS * 32) advance_kernel(GrammarDev Gg, StateDev S, const int32_t* tokens,
                                                                   int32_t* status) {
-  extern __shared__ uint32_t smem[];
+  extern __shared__ __align__(16) uint32_t smem[];
   const uint32_t warp = threadIdx.x >> 5, lane = lane_id();
   const uint32_t row = blockIdx.x * ADV_WARPS + warp;
+  GrammarDev G = Gg;
+  if (Gg.hot_words * 4u <= HOT_TABLE_BYTES) {
+    G = stage_hot_tables(Gg, smem + (size_t)ADV_WARPS * ADV_WARP_WORDS);
+    __syncthreads();
+  }
   if (row >= S.B) return;
   AdvScratch s = adv_scratch(smem + (size_t)warp * ADV_WARP_WORDS);
   auto finish = [&](int32_t st) {
@@ -277,7 +284,6 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
 constexpr int SWEEP_WARPS = 8;
 constexpr uint32_t SWEEP_CUR = 512;     // items of a set under construction per warp (fast mode, power of two)
 constexpr uint32_t SWEEP_HSET = 1024;   // uniqueness hash slots per warp (fast mode)
-constexpr uint32_t SWEEP_TABLE_BYTES = 24 * 1024;  // budget for grammar tables staged in shared memory
 
 struct JobCtx {
   const uint32_t* base_off;
@@ -292,13 +298,23 @@ struct JobCtx {
   bool accepting;
 };
 
+// (phase 0 of the sweep) what later phases need to know about job j, in one 16-byte record
+__device__ __forceinline__ void make_job_info(const StateDev& S, uint32_t j) {
+  const uint32_t row = S.jobs[j];
+  const uint64_t off = S.row_chart[row];
+  const uint32_t* chart = S.arena + off;
+  const uint32_t acc = (chart[CH_FLAGS] & CHART_ACCEPTING) ? 0x80000000u : 0u;
+  S.au.job_info[j] = make_uint4((uint32_t)off, (uint32_t)(off >> 32), chart[CH_SETS], row | acc);
+}
+
 __device__ __forceinline__ JobCtx job_ctx(const StateDev& S, uint32_t j) {
   const AutoDev& A = S.au;
+  const uint4 ji = __ldcg(A.job_info + j);
   JobCtx J;
-  J.row = S.jobs[j];
-  const uint32_t* chart = S.arena + S.row_chart[J.row];
-  J.m = chart[CH_SETS];
-  J.accepting = (chart[CH_FLAGS] & CHART_ACCEPTING) != 0u;
+  J.row = ji.w & 0x7FFFFFFFu;
+  J.accepting = (ji.w >> 31) != 0u;
+  const uint32_t* chart = S.arena + (((uint64_t)ji.y << 32) | ji.x);
+  J.m = ji.z;
   J.base_off = chart + CH_HDR;
   J.base_items = chart + CH_HDR + J.m + 1;
   J.recs = A.recs + (size_t)j * A.cap * A.rec_words;
@@ -466,7 +482,7 @@ struct SweepWarp {
     scannable_bytes(G, w.cur, n, tmp8);
     uint32_t id = intern_set(J, n, h);
     if (id == T_FAIL) return T_FAIL;
-    if (lane == 0) atomicExch(slot, id);
+    if (lane == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(slot), "r"(id) : "memory");
     ++n_computed;
     return id;
   }
@@ -527,17 +543,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 3) sweep_kernel(GrammarDev G
   uint32_t* tmp8 = ctr + W_CTRS;
   // ---- the small grammar tables every Earley step reads go to shared memory when they fit
   GrammarDev G = Gg;
-  if (A.tables_in_smem) {
-    uint32_t* tab = smem + (size_t)SWEEP_WARPS * warp_words;
-    const uint32_t d4 = (Gg.D + 3u) & ~3u;
-    for (uint32_t i = threadIdx.x; i < Gg.D; i += blockDim.x) tab[i] = Gg.info[i];
-    for (uint32_t i = threadIdx.x; i < Gg.C * 8u; i += blockDim.x) tab[d4 + i] = Gg.class_bits[i];
-    uint8_t* eq = reinterpret_cast<uint8_t*>(tab + d4 + Gg.C * 8u);
-    for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x) eq[i] = Gg.eq_of_byte[i];
-    G.info = tab;
-    G.class_bits = tab + d4;
-    G.eq_of_byte = eq;
-  }
+  if (A.tables_in_smem) G = stage_hot_tables(Gg, smem + (size_t)SWEEP_WARPS * warp_words);
   uint32_t* big = S.big_scratch + ((size_t)blockIdx.x * SWEEP_WARPS + warp) * ((size_t)S.big_arena_items + S.big_hset_slots);
   const uint32_t gw = blockIdx.x * SWEEP_WARPS + warp, GW = gridDim.x * SWEEP_WARPS;
   uint32_t bar_phase = 0;
@@ -555,6 +561,9 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 3) sweep_kernel(GrammarDev G
       if (i < AR_SCAN || i >= AR_SCAN + 8) rec0[i] = (i >= AR_TRANS) ? T_UNKNOWN : 0u;
     if (threadIdx.x == 0) A.n_states[j] = 1u;
     if (warp == 0) {
+      if (lane == 0) make_job_info(S, j);
+      __syncwarp();
+      __threadfence_block();
       JobCtx J = job_ctx(S, j);
       scannable_bytes(G, J.base_items + J.base_off[J.m - 1], J.base_off[J.m] - J.base_off[J.m - 1], tmp8);
       if (lane < 8) rec0[AR_SCAN + lane] = tmp8[lane];
@@ -891,7 +900,9 @@ static inline cudaError_t opt_in_smem(const void* fn, size_t bytes) {
   return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
-static size_t adv_smem_bytes() { return (size_t)ADV_WARPS * ADV_WARP_WORDS * 4; }
+static size_t adv_smem_bytes(const GrammarDev& G) {
+  return (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + (G.hot_words * 4u <= HOT_TABLE_BYTES ? G.hot_words * 4u : 0u);
+}
 static size_t init_smem_bytes() { return (size_t)ADV_WARP_WORDS * 4; }
 // Dynamic shared memory of the sweep for a grammar: per-warp scratch plus, if they fit the
 // budget, the item-info / byte-class / byte-class-number tables.
@@ -899,8 +910,8 @@ void sweep_layout(const GrammarDev& G, uint32_t* smem_bytes, uint32_t* tables_in
   const uint32_t ntw = (2u * G.Nw + 7u) & ~7u;
   const uint32_t warp_words = SWEEP_CUR + SWEEP_HSET + ntw + W_CTRS + 8;
   uint32_t bytes = SWEEP_WARPS * warp_words * 4u;
-  const uint32_t tab = (((G.D + 3u) & ~3u) + G.C * 8u + 64u) * 4u;
-  *tables_in_smem = tab <= SWEEP_TABLE_BYTES ? 1u : 0u;
+  const uint32_t tab = G.hot_words * 4u;
+  *tables_in_smem = tab <= HOT_TABLE_BYTES ? 1u : 0u;
   if (*tables_in_smem) bytes += tab;
   *smem_bytes = bytes;
 }
@@ -909,7 +920,7 @@ int walk_warps() { return SWEEP_WARPS; }
 cudaError_t configure_kernels() {
   cudaError_t e;
   if ((e = opt_in_smem((const void*)init_kernel, init_smem_bytes())) != cudaSuccess) return e;
-  if ((e = opt_in_smem((const void*)advance_kernel, adv_smem_bytes())) != cudaSuccess) return e;
+  if ((e = opt_in_smem((const void*)advance_kernel, (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + HOT_TABLE_BYTES)) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)sweep_kernel, 160 * 1024)) != cudaSuccess) return e;
   return cudaSuccess;
 }
@@ -929,7 +940,7 @@ void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const
   reset_kernel<<<(n + 127) / 128, 128, 0, st>>>(S, rows_dev, n, init_state_dev);
 }
 void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st) {
-  advance_kernel<<<(S.B + ADV_WARPS - 1) / ADV_WARPS, ADV_WARPS * 32, adv_smem_bytes(), st>>>(G, S, tokens, status);
+  advance_kernel<<<(S.B + ADV_WARPS - 1) / ADV_WARPS, ADV_WARPS * 32, adv_smem_bytes(G), st>>>(G, S, tokens, status);
 }
 static void launch_sweep_coop(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) {
   GrammarDev g = G;

@@ -30,6 +30,7 @@ constexpr uint32_t NA_OFF_MASKROW = NA_OFF_FLAGS + NA_MAX;       // [NA_MAX] int
 constexpr uint32_t NA_OFF_CHART = NA_OFF_MASKROW + NA_MAX;       // [NA_MAX] uint64 (8-byte aligned)
 constexpr uint32_t NA_OFF_BAD = NA_OFF_CHART + 2 * NA_MAX;       // [NA_MAX] header check failed
 constexpr uint32_t NA_OFF_NSTATES = NA_OFF_BAD + NA_MAX;         // [NA_MAX] Earley sets created per chart
+constexpr uint32_t NA_OFF_JOBINFO = NA_OFF_NSTATES + NA_MAX;     // [NA_MAX] uint4 (16-byte aligned)
 constexpr uint32_t NA_HEADER_WORDS = 1024;
 constexpr size_t NA_WARPS = (size_t)NA_GRID * 8;
 constexpr size_t NA_BIG_WORDS = NA_WARPS * (NA_ARENA_ITEMS + NA_HSET_SLOTS);
@@ -48,7 +49,8 @@ constexpr size_t NA_OFF_ST = NA_OFF_ITEMS + NA_ITEM_WORDS;
 constexpr size_t NA_OFF_REQ = NA_OFF_ST + NA_ST_ENTRIES / 2;       // 8-byte aligned: all sizes above are even
 constexpr size_t NA_WORDS = NA_OFF_REQ + 2 * (size_t)NA_REQ_CAP;
 static_assert(CNT_TOTAL <= NA_OFF_JOBS, "the counters overlap the job list");
-static_assert(NA_OFF_NSTATES + NA_MAX <= NA_HEADER_WORDS, "header too small");
+static_assert(NA_OFF_JOBINFO + 4 * NA_MAX <= NA_HEADER_WORDS, "header too small");
+static_assert((NA_OFF_JOBINFO % 4) == 0, "job records must be 16-byte aligned");
 static_assert((NA_OFF_CHART % 2) == 0, "64-bit offsets must be 8-byte aligned");
 
 // ~52 MB, held by every GPU that loads the library until the process exits
@@ -184,6 +186,7 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   S.au.st_stride = (uint32_t)st_stride;
   S.au.req = reinterpret_cast<unsigned long long*>(scratch + NA_OFF_REQ);
   S.au.req_cap = NA_REQ_CAP;
+  S.au.job_info = reinterpret_cast<uint4*>(scratch + NA_OFF_JOBINFO);
   sweep_layout(*G, &S.au.smem_bytes, &S.au.tables_in_smem);
   cudaStream_t st = (cudaStream_t)stream;
   noalloc_prepare_kernel<<<256, 256, 0, st>>>(*G, S, scratch, charts_dev, off, n, mask_dev);
