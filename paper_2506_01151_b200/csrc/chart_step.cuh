@@ -1,5 +1,7 @@
-// One byte of input on a whole pruned chart, by one warp (used when a sequence advances):
-//   Scan -> Complete (fixpoint) -> Compact -> Predict     (phase order of Section 4.2.3)
+// One token on a whole pruned chart, by one warp (used when a sequence advances).  Per byte:
+//   Scan -> Complete (fixpoint) -> Predict; after the token's last byte: Compact (Section 4.2.3),
+// which leaves exactly the chart that compacting after every byte would leave (an item needed at
+// the end was needed at every step before), at a fraction of the work,
 // and the state cache: the pruned chart, densely renumbered, is the cache key ("multiple
 // different input token sequences can correspond to the same pruned Earley states", Section 5.2).
 //
@@ -12,7 +14,7 @@
 
 namespace fmt {
 
-constexpr uint32_t ADV_CUR_CAP = 1024;     // items of one set (power of two)
+constexpr uint32_t ADV_CUR_CAP = 2048;     // items of the sets a token adds to a chart (shared-memory arena)
 constexpr uint32_t ADV_HSET = 2048;        // hash slots (power of two)
 constexpr uint32_t ADV_MAX_ITEMS = 65536;  // items of a chart the live bitmap can describe
 constexpr uint32_t ADV_PAIRS = 1024;       // (set, non-terminal) needs of one Compact
@@ -93,8 +95,8 @@ __device__ __forceinline__ int finish_chart(const AdvScratch& s, uint32_t* dst, 
                                             uint32_t kept, uint32_t n, bool accepting, HashAcc h) {
   const uint32_t lane = lane_id();
   uint32_t words = CH_HDR + (m_new + 2) + kept + n;
-  if (words > dst_cap || kept + n >= ADV_MAX_ITEMS || n > ADV_CUR_CAP) return -1;
-  sort_items(s.w.cur, n, ADV_CUR_CAP);
+  if (words > dst_cap || kept + n >= ADV_MAX_ITEMS) return -1;
+  sort_items(s.w.cur, n, 1u << 30);
   const uint32_t items_at = CH_HDR + (m_new + 2);
   for (uint32_t i = lane; i < n; i += 32) put(dst, h, items_at + kept + i, s.w.cur[i]);
   if (lane == 0) {
@@ -141,14 +143,42 @@ __device__ int chart_init(const GrammarDev& G, const AdvScratch& s, uint32_t* ds
   return finish_chart(s, dst, dst_cap, 0u, 0u, n, accepting, HashAcc{});
 }
 
-// One byte.  Returns 1 (dst holds the new chart), 0 (the byte cannot follow: dst is garbage) or
-// -1 (a capacity limit was hit).  src and dst must not overlap.
-__device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32_t* src, uint32_t byte,
-                          uint32_t* dst, uint32_t dst_cap) {
+// Where set o of "source chart + the token's sets so far" lives.  Sets 0..m-1 are the source
+// chart's, set m-1+L is the token's L-th.
+struct TokenView {
+  const uint32_t* soff;
+  const uint32_t* sitems;
+  uint32_t m;
+  const uint32_t* arena;
+  const uint32_t* lvl_off;  // [MAX_TOKEN_BYTES + 2] first item of each level in the arena
+  __device__ __forceinline__ void operator()(uint32_t o, const uint32_t*& p, uint32_t& n) const {
+    if (o < m) {
+      uint32_t a = soff[o], b = soff[o + 1];
+      p = sitems + a;
+      n = b - a;
+    } else {
+      const uint32_t L = o - (m - 1);
+      p = arena + lvl_off[L];
+      n = lvl_off[L + 1] - lvl_off[L];
+    }
+  }
+  __device__ __forceinline__ uint32_t fix(uint32_t item, uint32_t) const { return item; }
+  // position of item k of set o in the live bitmap (source items first, then the arena)
+  __device__ __forceinline__ uint32_t bit_base(uint32_t o, uint32_t n_items) const {
+    return (o < m) ? soff[o] : n_items + lvl_off[o - (m - 1)];
+  }
+};
+
+// All bytes of one token.  Returns 1 (dst holds the new chart), 0 (some byte cannot follow: dst
+// is garbage), -1 (a capacity limit was hit) or -2 (the arena for the token's sets is too small:
+// the caller may retry with a larger one).  src and dst must not overlap.  `arena` (arena_cap
+// items, a power of two if the last set is to be sorted in place) holds the token's sets.
+__device__ int token_step(const GrammarDev& G, AdvScratch& s, const uint32_t* src, const uint8_t* bytes, uint32_t len,
+                          uint32_t* dst, uint32_t dst_cap, uint32_t* arena, uint32_t arena_cap) {
   const uint32_t lane = lane_id();
   const uint32_t m = src[CH_SETS];
   const uint32_t n_items = src[CH_ITEMS];
-  if (m == 0 || m + 1 > ADV_MAX_SETS || n_items > ADV_MAX_ITEMS) return -1;
+  if (m == 0 || m + len + MAX_TOKEN_BYTES + 4 > ADV_MAX_SETS || n_items > ADV_MAX_ITEMS || len > MAX_TOKEN_BYTES) return -1;
   // small charts are read from shared memory from here on
   const uint32_t src_words = src[CH_WORDS];
   __syncwarp();
@@ -156,34 +186,62 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     for (uint32_t i = lane; i < src_words; i += 32) s.stage[i] = src[i];
     src = s.stage;
   }
-  const uint32_t* soff = src + CH_HDR;
-  const uint32_t* sitems = src + CH_HDR + m + 1;
-  if (lane < W_CTRS) s.w.ctr[lane] = 0u;
+  uint32_t* lvl_off = s.sets + ADV_MAX_SETS - (MAX_TOKEN_BYTES + 2);  // the tail of `sets` is free until Compact ends
+  TokenView view{src + CH_HDR, src + CH_HDR + m + 1, m, arena, lvl_off};
+  const uint32_t* soff = view.soff;
+  const uint32_t* sitems = view.sitems;
+  if (lane == 0) lvl_off[0] = 0, lvl_off[1] = 0;
   __syncwarp();
-  // ---- Scan
-  uint32_t n = scan_into_cur(G, s.w, sitems + soff[m - 1], soff[m] - soff[m - 1], byte);
-  if (n == 0) return 0;
-  // ---- Complete
-  ChartView view{soff, sitems};
-  complete_fixpoint(G, s.w, view, m, 0u);
-  uint32_t hashed = min(s.w.ctr[W_NCUR], s.w.cur_cap);
-  if (s.w.ctr[W_OVERFLOW]) {
-    hset_clear_all(s.w.hset, s.w.hset_mask);
-    clear_nt(G, s.w);
-    return -1;
+  // ---- per byte: Scan, Complete, Predict; the new set is appended to the arena
+  uint32_t top = 0;
+  bool accepting = false;
+  const uint32_t* prev = sitems + soff[m - 1];
+  uint32_t prev_len = soff[m] - soff[m - 1];
+  for (uint32_t L = 1; L <= len; ++L) {
+    if (top + 64 > arena_cap) return -2;
+    s.w.cur = arena + top;
+    s.w.cur_cap = arena_cap - top;
+    __syncwarp();
+    if (lane < W_CTRS) s.w.ctr[lane] = 0u;
+    __syncwarp();
+    uint32_t n = scan_into_cur(G, s.w, prev, prev_len, __ldg(&bytes[L - 1]));
+    if (s.w.ctr[W_OVERFLOW]) {
+      hset_clear_all(s.w.hset, s.w.hset_mask);
+      return -2;
+    }
+    if (n == 0) return 0;
+    const uint32_t index = m - 1 + L;
+    complete_fixpoint(G, s.w, view, index, 0u);
+    uint32_t hashed = min(s.w.ctr[W_NCUR], s.w.cur_cap);
+    if (s.w.ctr[W_OVERFLOW]) {
+      hset_clear_all(s.w.hset, s.w.hset_mask);
+      clear_nt(G, s.w);
+      return -2;
+    }
+    hset_clear_items(s.w, hashed);
+    accepting = s.w.ctr[W_ACCEPT] != 0u;
+    predict_into_cur(G, s.w, index);
+    if (s.w.ctr[W_OVERFLOW]) return -2;
+    n = drop_completed(G, s.w, min(s.w.ctr[W_NCUR], s.w.cur_cap));
+    prev = arena + top;
+    prev_len = n;
+    top += n;
+    if (lane == 0) lvl_off[L + 1] = top;
+    __syncwarp();
   }
-  hset_clear_items(s.w, hashed);
-  bool accepting = s.w.ctr[W_ACCEPT] != 0u;
-  n = drop_completed(G, s.w, hashed);
-  // ---- Compact: which items of the earlier sets can a later Complete still read?
-  for (uint32_t i = lane; i < (n_items + 31) / 32; i += 32) s.live[i] = 0u;
+  // ---- Compact once: which items of the earlier sets can a later Complete still read?
+  const uint32_t last = m - 1 + len;           // index of the last set
+  const uint32_t last_at = lvl_off[len];       // its first item in the arena
+  const uint32_t n_last = top - last_at;
+  const uint32_t n_bits = n_items + last_at;   // source items, then the token's earlier sets
+  if (n_bits > ADV_MAX_ITEMS) return -1;
+  for (uint32_t i = lane; i < (n_bits + 31) / 32; i += 32) s.live[i] = 0u;
   __syncwarp();
-  for (uint32_t i = lane; i < n; i += 32) {
-    uint32_t it = s.w.cur[i];
-    if ((it >> 16) < m) push_need(s, it >> 16, __ldg(&G.lhs[it & 0xFFFFu]));
+  for (uint32_t i = lane; i < n_last; i += 32) {
+    uint32_t it = arena[last_at + i];
+    if ((it >> 16) < last) push_need(s, it >> 16, __ldg(&G.lhs[it & 0xFFFFu]));
   }
-  // needs are served a wave at a time, one lane per (set, non-terminal) need
-  for (uint32_t head = 0;;) {
+  for (uint32_t head = 0;;) {  // needs are served a wave at a time, one lane per (set, non-terminal) need
     __syncwarp();
     const uint32_t np = min(s.w.ctr[W_NPAIRS], ADV_PAIRS);
     __syncwarp();
@@ -192,13 +250,17 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     if (mine < np) {
       const uint32_t key = s.pairs[mine];
       const uint32_t o = key >> 16, A = key & 0xFFFFu;
-      const uint32_t a = soff[o], b = soff[o + 1];
-      for (uint32_t k = a; k < b; ++k) {
-        const uint32_t wi = sitems[k];
+      const uint32_t* sp;
+      uint32_t sl;
+      view(o, sp, sl);
+      const uint32_t base = view.bit_base(o, n_items);
+      for (uint32_t k = 0; k < sl; ++k) {
+        const uint32_t wi = sp[k];
         const uint32_t inf = G.info[wi & 0xFFFFu];
         if ((inf >> INFO_KIND_SHIFT) == KIND_NT && (inf & INFO_ARG_MASK) == A) {
-          const uint32_t bit = 1u << (k & 31u);
-          const uint32_t old = atomicOr(&s.live[k >> 5], bit);
+          const uint32_t pos = base + k;
+          const uint32_t bit = 1u << (pos & 31u);
+          const uint32_t old = atomicOr(&s.live[pos >> 5], bit);
           if (!(old & bit)) push_need(s, wi >> 16, __ldg(&G.lhs[wi & 0xFFFFu]));
         }
       }
@@ -228,18 +290,23 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     clear_nt(G, s.w);
     return -1;
   }
-  // ---- live items per set, new set numbers, new offsets
-  for (uint32_t k = lane; k < m; k += 32) {
-    uint32_t a = soff[k], b = soff[k + 1], c = 0;
-    for (uint32_t i = a; i < b; ++i) c += (s.live[i >> 5] >> (i & 31u)) & 1u;
+  // ---- live items per earlier set, new set numbers, new offsets
+  const uint32_t M = last;  // earlier sets: 0..last-1
+  for (uint32_t k = lane; k < M; k += 32) {
+    const uint32_t* sp;
+    uint32_t sl;
+    view(k, sp, sl);
+    const uint32_t base = view.bit_base(k, n_items);
+    uint32_t c = 0;
+    for (uint32_t i = 0; i < sl; ++i) c += (s.live[(base + i) >> 5] >> ((base + i) & 31u)) & 1u;
     s.sets[k] = c;
   }
   __syncwarp();
   HashAcc h;
   uint32_t m_new = 0, kept = 0;
-  for (uint32_t base = 0; base < m; base += 32) {
+  for (uint32_t base = 0; base < M; base += 32) {
     uint32_t k = base + lane;
-    uint32_t c = (k < m) ? s.sets[k] : 0u;
+    uint32_t c = (k < M) ? s.sets[k] : 0u;
     uint32_t keep = __ballot_sync(FULL, c > 0);
     uint32_t my_new = m_new + __popc(keep & ((1u << lane) - 1u));
     uint32_t incl = c;  // inclusive prefix sum of the counts within the wave
@@ -247,7 +314,8 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
       uint32_t t = __shfl_up_sync(FULL, incl, d);
       if ((int)lane >= d) incl += t;
     }
-    if (k < m) {
+    __syncwarp();
+    if (k < M) {
       if (c > 0) {
         if (CH_HDR + my_new < dst_cap) put(dst, h, CH_HDR + my_new, kept + incl - c);
         s.sets[k] = my_new;
@@ -259,43 +327,40 @@ __device__ int chart_step(const GrammarDev& G, const AdvScratch& s, const uint32
     m_new += __popc(keep);
   }
   __syncwarp();
-  uint32_t words_needed = CH_HDR + (m_new + 2) + kept;
-  if (words_needed + n + 64 > dst_cap) {
-    clear_nt(G, s.w);
-    return -1;
-  }
-  // ---- copy the live items, origins renumbered
+  if (CH_HDR + (m_new + 2) + kept + n_last + 64 > dst_cap) return -1;
+  // ---- copy the live items (source chart first, then the token's earlier sets), origins renumbered
   const uint32_t items_at = CH_HDR + (m_new + 2);
   uint32_t bad = 0;
   uint32_t out = 0;
-  for (uint32_t base = 0; base < n_items; base += 32) {
+  for (uint32_t base = 0; base < n_bits; base += 32) {
     uint32_t i = base + lane;
-    bool lv = (i < n_items) && ((s.live[i >> 5] >> (i & 31u)) & 1u);
+    bool lv = (i < n_bits) && ((s.live[i >> 5] >> (i & 31u)) & 1u);
     uint32_t bal = __ballot_sync(FULL, lv);
     if (lv) {
-      uint32_t it = sitems[i];
+      uint32_t it = (i < n_items) ? sitems[i] : arena[i - n_items];
       uint32_t no = s.sets[it >> 16];
       if (no == 0xffffffffu) bad = 1;
       put(dst, h, items_at + out + __popc(bal & ((1u << lane) - 1u)), (no << 16) | (it & 0xFFFFu));
     }
     out += __popc(bal);
   }
-  // ---- the new last set: renumber origins, then Predict with the new index
-  for (uint32_t i = lane; i < n; i += 32) {
-    uint32_t it = s.w.cur[i];
+  // ---- the last set: renumber origins (its own index becomes m_new), move it to the front of the
+  // arena region it occupies so that it can be sorted in place
+  for (uint32_t i = lane; i < n_last; i += 32) {
+    uint32_t it = arena[last_at + i];
     uint32_t o = it >> 16;
-    uint32_t no = (o < m) ? s.sets[o] : 0xffffffffu;  // origin m cannot occur yet: those items are predicted below
+    uint32_t no = (o == last) ? m_new : s.sets[o];
     if (no == 0xffffffffu) bad = 1;
-    s.w.cur[i] = (no << 16) | (it & 0xFFFFu);
+    arena[last_at + i] = (no << 16) | (it & 0xFFFFu);
   }
   bad = __any_sync(FULL, bad);
   __syncwarp();
-  if (lane == 0) s.w.ctr[W_NCUR] = n;
-  __syncwarp();
-  predict_into_cur(G, s.w, m_new);
-  if (bad || s.w.ctr[W_OVERFLOW]) return -1;
-  n = min(s.w.ctr[W_NCUR], s.w.cur_cap);
-  return finish_chart(s, dst, dst_cap, m_new, kept, n, accepting, h);
+  if (bad) return -1;
+  uint32_t P = 32;
+  while (P < n_last) P <<= 1;
+  if (last_at + P > arena_cap) return -2;  // the sort pads the set to a power of two
+  s.w.cur = arena + last_at;
+  return finish_chart(s, dst, dst_cap, m_new, kept, n_last, accepting, h);
 }
 
 }  // namespace fmt

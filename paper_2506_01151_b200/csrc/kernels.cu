@@ -173,30 +173,30 @@ __global__ void __launch_bounds__(ADV_WARPS * 32) advance_kernel(GrammarDev Gg, 
   hset_clear_all(s.w.hset, s.w.hset_mask);
   for (uint32_t i = lane; i < ADV_NT_WORDS; i += 32) s.w.nt[i] = 0u;
   __syncwarp();
-  // two private buffers that do not hold the current chart
+  // a private buffer that does not hold the current chart
   const uint32_t held = S.row_buf[row];
-  const uint32_t t0 = (held == 0) ? 1u : 0u;
-  const uint32_t t1 = (held == 2 || held == 255) ? (t0 == 0 ? 1u : 2u) : 2u;
-  uint32_t which = t0;
-  const uint32_t* src = cur;
-  uint32_t* dst = nullptr;
-  for (uint32_t i = b0; i < b1; ++i) {
-    dst = private_buf(S, row, which);
-    int r = chart_step(G, s, src, __ldg(&G.vocab_bytes[i]), dst, S.chart_words);
-    if (r == 0) return finish(FMT_ERR_TOKEN_REJECTED);
-    if (r < 0) {
-      if (lane == 0) {
-        S.row_flags[row] = flags | ROW_BROKEN;
-        atomicExch(&S.counters[CNT_ERR], 1u);
-        stat_add(S, CNT_STAT_CAPERR, 1u);
-      }
-      return finish(FMT_ERR_CAPACITY);
-    }
-    src = dst;
-    which = (which == t0) ? t1 : t0;
+  const uint32_t final_buf = (held == 0) ? 1u : 0u;
+  uint32_t* dst = private_buf(S, row, final_buf);
+  uint32_t* const sm_arena = s.w.cur;
+  int r = token_step(G, s, cur, G.vocab_bytes + b0, b1 - b0, dst, S.chart_words, sm_arena, ADV_CUR_CAP);
+  if (r == -2) {  // the token's sets outgrew shared memory: use the row's third private buffer as the arena
+    uint32_t* big = private_buf(S, row, 2);
+    uint32_t cap = 32;
+    while (cap * 2u <= S.chart_words) cap *= 2u;
+    hset_clear_all(s.w.hset, s.w.hset_mask);
+    for (uint32_t i = lane; i < ADV_NT_WORDS; i += 32) s.w.nt[i] = 0u;
     __syncwarp();
+    r = (held == 2) ? -1 : token_step(G, s, cur, G.vocab_bytes + b0, b1 - b0, dst, S.chart_words, big, cap);
   }
-  const uint32_t final_buf = (which == t0) ? t1 : t0;
+  if (r == 0) return finish(FMT_ERR_TOKEN_REJECTED);
+  if (r < 0) {
+    if (lane == 0) {
+      S.row_flags[row] = flags | ROW_BROKEN;
+      atomicExch(&S.counters[CNT_ERR], 1u);
+      stat_add(S, CNT_STAT_CAPERR, 1u);
+    }
+    return finish(FMT_ERR_CAPACITY);
+  }
   if (lane == 0) {
     stat_add(S, CNT_STAT_ADV, 1u);
     stat_max(S, CNT_STAT_ITEMS_MAX, dst[CH_ITEMS]);
