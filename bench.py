@@ -156,7 +156,7 @@ class Driver:
         self.state.advance(self.tokens[i], self.status, stream=s)
         lg = self.ring[i % self.n_ring] if logits is None else logits
         self.state.fill_and_apply(lg, self.fmt.BF16, stream=s)
-        self.launches += 7  # advance; plan, prepare, walk, publish, mask+apply, end
+        self.launches += 5  # advance; plan, sweep, publish, mask+apply
 
 
 def run_ours(args):
@@ -223,12 +223,12 @@ def run_ours(args):
     peak, peak_kind = measured_peaks()
     B, V, Wm = w.batch, w.V, info.mask_words
     # algorithmic bytes per launch of each kernel kind ("Roofline")
-    trie_bytes = info.trie_nodes * (4 + 1 + 4 + 4) + 4 * V
+    trie_bytes = info.trie_nodes * (1 + 4 + 1) + 4 * V  # node byte, parent, depth; token -> node
     jobs = stats1["fills_computed"] - stats0["fills_computed"]
     walk_bytes_per_launch = trie_bytes + (jobs / max(1, K)) * (4 * Wm + 2048)
     apply_bytes_per_launch = B * (4 * Wm + 2 * V)
     kinds = {
-        "walk_kernel": (prof["walk_ms"], prof["walk_launches"], walk_bytes_per_launch),
+        "sweep_kernel": (prof["walk_ms"], prof["walk_launches"], walk_bytes_per_launch),
         "gather_apply_kernel": (prof["apply_ms"], prof["apply_launches"], apply_bytes_per_launch),
         "advance_kernel": (prof["advance_ms"], prof["advance_launches"], B * 2 * 4 * 256),
     }
