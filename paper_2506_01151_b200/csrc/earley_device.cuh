@@ -185,6 +185,7 @@ __device__ __forceinline__ void predict_into_cur(const GrammarDev& G, const Warp
   bool over = false;
   for (uint32_t wi = 0; wi < Nw && !over; ++wi) {
     const uint32_t bits = clos[wi];
+    if (bits == 0u) continue;  // (uniform) most words of the closure are empty
     const uint32_t cnt = __popc(bits);
     for (uint32_t base = 0; base < cnt && !over; base += 32) {
       const uint32_t k = base + lane;

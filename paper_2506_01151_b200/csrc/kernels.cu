@@ -352,6 +352,7 @@ struct SweepWarp {
   uint32_t cur_pow2;  // capacity of w.cur (a power of two, for the sort)
   uint32_t* tmp8;     // shared
   uint32_t n_computed = 0, n_created = 0;  // statistics, flushed once at the end of the kernel
+  uint32_t chunk_at = 0, chunk_left = 0;   // this warp's private piece of the item pool (lane 0's copy counts)
 
   // Find or create the local state whose items are w.cur[0..n) (sorted).  Returns its id or T_FAIL.
   __device__ uint32_t intern_set(const JobCtx& J, uint32_t n, uint32_t hash) {
@@ -370,8 +371,17 @@ struct SweepWarp {
             const uint32_t got = atomicAdd(J.n_states, 1u);
             const uint32_t need = (max(n, 1u) + 31u) & ~31u;
             if (got < J.cap) {
-              ioff = atomicAdd(&S.counters[CNT_AUTO_ITEMS], need);
-              if (ioff <= A.items_cap && need <= A.items_cap - ioff) id = got;
+              if (need > chunk_left) {  // take a new piece of the pool: one atomic per ~4 Ki item words
+                const uint32_t take = max(need, 4096u);
+                chunk_at = atomicAdd(&S.counters[CNT_AUTO_ITEMS], take);
+                chunk_left = (chunk_at <= A.items_cap && take <= A.items_cap - chunk_at) ? take : 0u;
+              }
+              if (need <= chunk_left) {
+                ioff = chunk_at;
+                chunk_at += need;
+                chunk_left -= need;
+                id = got;
+              }
             }
           }
           id = __shfl_sync(FULL, id, 0);
