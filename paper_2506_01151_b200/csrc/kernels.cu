@@ -773,57 +773,66 @@ __global__ void gather_kernel(GrammarDev G, StateDev S, uint32_t* out, size_t st
   }
 }
 
-// logits[t] = -inf where bit t is 0, for one row.  Each thread handles 8 consecutive tokens
-// (16 bytes of bf16, 32 bytes of fp32) when the row is 16-byte aligned, else one token at a time.
-// Groups whose 8 tokens are all valid are not touched; groups whose 8 tokens are all invalid are
-// stored without being read.
+// logits[t] = -inf where bit t is 0, for one row.  Each thread takes one mask word (32 tokens:
+// 64 bytes of bf16, 128 bytes of fp32) at a time and handles it in groups of 8 tokens with 16-byte
+// accesses when the row is 16-byte aligned, else token by token.  Groups whose 8 tokens are all
+// valid are not touched; groups whose 8 tokens are all invalid are stored without being read.
+template <typename T>
+__device__ __forceinline__ void apply_group(T* p, uint32_t bits) {  // 8 tokens at p, 16-byte aligned
+  if (sizeof(T) == 2) {
+    uint4* q = reinterpret_cast<uint4*>(p);
+    uint4 v = (bits == 0) ? make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u) : *q;
+    if (bits != 0) {
+      uint32_t* e = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        uint32_t x = e[i];
+        if (!((bits >> (2 * i)) & 1u)) x = (x & 0xFFFF0000u) | 0xFF80u;
+        if (!((bits >> (2 * i + 1)) & 1u)) x = (x & 0x0000FFFFu) | 0xFF800000u;
+        e[i] = x;
+      }
+    }
+    *q = v;
+  } else {
+    uint4* q = reinterpret_cast<uint4*>(p);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t hb = (bits >> (4 * h)) & 0xFu;
+      if (hb == 0xFu) continue;
+      uint4 v = (hb == 0) ? make_uint4(0, 0, 0, 0) : q[h];
+      if (!(hb & 1u)) v.x = 0xFF800000u;
+      if (!(hb & 2u)) v.y = 0xFF800000u;
+      if (!(hb & 4u)) v.z = 0xFF800000u;
+      if (!(hb & 8u)) v.w = 0xFF800000u;
+      q[h] = v;
+    }
+  }
+}
+
 template <typename T>
 __device__ __forceinline__ void apply_row(const uint32_t* mask_row, int32_t special, int32_t eos, T* logits, uint32_t V,
                                           uint32_t* mask_out) {
   const uint32_t nthreads = gridDim.x * blockDim.x;
   const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
   const bool aligned = (reinterpret_cast<uintptr_t>(logits) & 15u) == 0;
-  const uint32_t groups = (V + 7) / 8;
+  const uint32_t words = (V + 31) / 32;
   const T neg = sizeof(T) == 2 ? (T)0xFF80u : (T)0xFF800000u;
-  for (uint32_t g = tid; g < groups; g += nthreads) {
-    const uint32_t t0 = g * 8;
+  for (uint32_t wd = tid; wd < words; wd += nthreads) {
     uint32_t word = 0;
-    if (mask_row) word = __ldg(&mask_row[t0 >> 5]);
-    else if (special == MASK_EOS_ONLY && eos >= 0 && (t0 >> 5) == ((uint32_t)eos >> 5)) word = 1u << ((uint32_t)eos & 31u);
-    if (mask_out && (t0 & 31u) == 0) mask_out[t0 >> 5] = word;
-    const uint32_t bits = (word >> (t0 & 31u)) & 0xFFu;
-    if (bits == 0xFFu) continue;
-    if (aligned && t0 + 8 <= V) {
-      if (sizeof(T) == 2) {
-        uint4* p = reinterpret_cast<uint4*>(logits + t0);
-        uint4 v = (bits == 0) ? make_uint4(0, 0, 0, 0) : *p;
-        uint32_t* e = reinterpret_cast<uint32_t*>(&v);
+    if (mask_row) word = __ldg(&mask_row[wd]);
+    else if (special == MASK_EOS_ONLY && eos >= 0 && wd == ((uint32_t)eos >> 5)) word = 1u << ((uint32_t)eos & 31u);
+    if (mask_out) mask_out[wd] = word;
+    if (word == 0xFFFFFFFFu) continue;
+    const uint32_t t0 = wd * 32;
+    if (aligned && t0 + 32 <= V) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint32_t lo = (bits >> (2 * i)) & 1u, hi = (bits >> (2 * i + 1)) & 1u;
-          uint32_t x = e[i];
-          if (!lo) x = (x & 0xFFFF0000u) | 0xFF80u;
-          if (!hi) x = (x & 0x0000FFFFu) | 0xFF800000u;
-          e[i] = x;
-        }
-        *p = v;
-      } else {
-        uint4* p = reinterpret_cast<uint4*>(logits + t0);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          uint32_t hb = (bits >> (4 * h)) & 0xFu;
-          if (hb == 0xFu) continue;
-          uint4 v = (hb == 0) ? make_uint4(0, 0, 0, 0) : p[h];
-          if (!(hb & 1u)) v.x = 0xFF800000u;
-          if (!(hb & 2u)) v.y = 0xFF800000u;
-          if (!(hb & 4u)) v.z = 0xFF800000u;
-          if (!(hb & 8u)) v.w = 0xFF800000u;
-          p[h] = v;
-        }
+      for (uint32_t gq = 0; gq < 4; ++gq) {
+        const uint32_t bits = (word >> (8 * gq)) & 0xFFu;
+        if (bits != 0xFFu) apply_group<T>(logits + t0 + 8 * gq, bits);
       }
     } else {
-      for (uint32_t i = 0; i < 8 && t0 + i < V; ++i)
-        if (!((bits >> i) & 1u)) logits[t0 + i] = neg;
+      for (uint32_t i = 0; i < 32 && t0 + i < V; ++i)
+        if (!((word >> i) & 1u)) logits[t0 + i] = neg;
     }
   }
 }
@@ -977,13 +986,13 @@ void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t
 void launch_apply(const uint32_t* mask, size_t stride_words, void* logits, int dtype, uint32_t batch, uint32_t V,
                   size_t row_stride, cudaStream_t st) {
   if (batch == 0 || V == 0) return;
-  dim3 grid((unsigned)std::min<uint32_t>(((V + 7) / 8 + 255) / 256, 64), batch);
+  dim3 grid((unsigned)std::min<uint32_t>(((V + 31) / 32 + 255) / 256, 64), batch);
   if (dtype == FMT_BF16) apply_kernel<uint16_t><<<grid, 256, 0, st>>>(mask, stride_words, (uint16_t*)logits, V, row_stride);
   else apply_kernel<uint32_t><<<grid, 256, 0, st>>>(mask, stride_words, (uint32_t*)logits, V, row_stride);
 }
 void launch_gather_apply(const GrammarDev& G, const StateDev& S, void* logits, int dtype, size_t row_stride,
                          uint32_t* mask_out, size_t stride_words, cudaStream_t st) {
-  dim3 grid((unsigned)std::min<uint32_t>(((G.V + 7) / 8 + 255) / 256, 64), S.B);
+  dim3 grid((unsigned)std::min<uint32_t>(((G.V + 31) / 32 + 255) / 256, 64), S.B);
   if (dtype == FMT_BF16)
     gather_apply_kernel<uint16_t><<<grid, 256, 0, st>>>(G, S, (uint16_t*)logits, row_stride, mask_out, stride_words);
   else
