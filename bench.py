@@ -33,6 +33,9 @@ METRIC = "vocab-mask token-checks/s"
 UNIT = "token-checks/s"
 DEFAULT_CONFIG = 3
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (config 3 only; taken on the kernels as committed with those summaries)
+NCU_TRAFFIC_BYTES = {3: {"sweep_kernel": 4.02e6, "gather_apply_kernel": 7.9e6, "advance_kernel": 1.4e5}}
 
 
 # --------------------------------------------------------------------------- small helpers
@@ -274,7 +277,7 @@ def run_ours(args):
     achieved = d_bytes / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else 0.0
     roofline = {
         "bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "traffic": None, "peak_source": peak_kind + " copy bandwidth", "avg_launch_us": avg_ms * 1e3,
+        "traffic": NCU_TRAFFIC_BYTES.get(args.config, {}).get(dom), "peak_source": peak_kind + " copy bandwidth", "avg_launch_us": avg_ms * 1e3,
         "bytes_per_launch": d_bytes,
         "per_kernel_ms": {k: v[0] for k, v in kinds.items()},
         "hbm_floor_us_per_step": (apply_bytes_per_launch + trie_bytes) / (peak * 1e9) * 1e6,
