@@ -212,7 +212,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
     K, W = args.steps, args.warmup
-    w = workloads.build(args.config, steps=K + W)
+    w = workloads.build(args.config, steps=K + W, batch=args.batch)
     drv = Driver(w, device)
     drv.feed_prefix()
     for i in range(W):
@@ -261,13 +261,13 @@ def run_ours(args):
     info = drv.grammar.info()
     peak, peak_kind = measured_peaks()
     B, V, Wm = w.batch, w.V, info.mask_words
-    # algorithmic bytes per launch of each kernel kind ("Roofline")
+    # algorithmic bytes per launch of each kernel kind: what the method itself must move through HBM
     trie_bytes = info.trie_nodes * (1 + 4 + 1) + 4 * V  # node byte, parent, depth; token -> node
     jobs = stats1["fills_computed"] - stats0["fills_computed"]
     walk_bytes_per_launch = trie_bytes + (jobs / max(1, K)) * (4 * Wm + 2048)
     apply_bytes_per_launch = B * (4 * Wm + 2 * V)
     kinds = {
-        "sweep_kernel": (prof["walk_ms"], prof["walk_launches"], walk_bytes_per_launch),
+        "sweep_kernel": (prof["sweep_ms"], prof["sweep_launches"], walk_bytes_per_launch),
         "gather_apply_kernel": (prof["apply_ms"], prof["apply_launches"], apply_bytes_per_launch),
         "advance_kernel": (prof["advance_ms"], prof["advance_launches"], B * 2 * 4 * 256),
     }
@@ -299,8 +299,8 @@ def run_ours(args):
                   "hit_rate": 1.0 - jobs / max(1, fills), "states_cached": stats1["states_cached"],
                   "chart_items_max": stats1["chart_items_max"], "chart_sets_max": stats1["chart_sets_max"],
                   "capacity_errors": stats1["capacity_errors"],
-                  "walk_transitions": stats1["walk_transitions"] - stats0["walk_transitions"],
-                  "walk_states": stats1["walk_states"] - stats0["walk_states"],
+                  "sweep_transitions": stats1["sweep_transitions"] - stats0["sweep_transitions"],
+                  "sweep_states": stats1["sweep_states"] - stats0["sweep_states"],
                   "big_mode": stats1["big_mode_units"] - stats0["big_mode_units"]},
         "cold": cold,
         "grammar": {"nonterminals": info.n_nonterminals, "rules": info.n_rules, "dotted": info.n_dotted,
@@ -333,7 +333,7 @@ def measure_cold(drv: "Driver", w, start: int, n: int):
         total += e0.elapsed_time(e1)
     prof = drv.state.read_profile()
     drv.state.set_profiling(False)
-    return {"fills": n, "ms_per_fill": total / n, "walk_ms_per_fill": prof["walk_ms"] / max(1, prof["walk_launches"]),
+    return {"fills": n, "ms_per_fill": total / n, "sweep_ms_per_fill": prof["sweep_ms"] / max(1, prof["sweep_launches"]),
             "token_checks_per_s": w.batch * w.V / (total / n * 1e-3),
             "what": "fmt_fill_mask with the state cache emptied before each call: every distinct row state walks the trie"}
 
@@ -430,7 +430,7 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     K, W = args.steps, args.warmup
-    w = workloads.build(args.config, steps=K + W)
+    w = workloads.build(args.config, steps=K + W, batch=args.batch)
     rows = min(w.batch, 4)
     g, vocab, seqs, advance = oracle_sample(w, 0, rows)
     for i in range(W):
@@ -465,6 +465,7 @@ def main():
     ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--config", type=int, default=DEFAULT_CONFIG)
+    ap.add_argument("--batch", type=int, default=None, help="override the config's batch size (not the headline workload)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

@@ -70,8 +70,8 @@ typedef struct {
   uint32_t max_mask_rows;     /* cached mask rows (default 8192) */
   uint32_t chart_words;       /* capacity of one row's chart in uint32 words (default 65536) */
   uint64_t pool_words;        /* uint32 words of chart storage for the cache (default 64 Mi) */
-  uint32_t walk_states;       /* distinct Earley sets one mask computation may create while it
-                                 walks the vocabulary (default: 4 Mi / batch, within 2048..32768) */
+  uint32_t sweep_states;       /* distinct Earley sets one mask computation may create while it
+                                 sweeps the vocabulary (default: 4 Mi / batch, within 2048..32768) */
   uint32_t reserved[5];
 } fmt_state_options;
 
@@ -93,7 +93,7 @@ typedef struct {
 typedef struct {
   uint64_t steps_advanced;     /* row-advances that changed a chart */
   uint64_t fills;              /* rows asked for a mask */
-  uint64_t fills_computed;     /* rows whose mask was computed by the trie walk */
+  uint64_t fills_computed;     /* rows whose mask was computed by the trie sweep */
   uint64_t fills_from_cache;   /* rows served from a cached mask */
   uint64_t fills_shared;       /* rows that shared another row's mask computed in the same call */
   uint64_t states_cached;      /* distinct pruned charts held by the cache */
@@ -103,8 +103,8 @@ typedef struct {
   uint64_t chart_sets_max;     /* most live Earley sets seen in one chart */
   uint64_t capacity_errors;
   uint64_t big_mode_units;     /* times a warp of the trie sweep switched to its large scratch area */
-  uint64_t walk_transitions;   /* Earley steps (scan + complete + predict) done by the trie walk */
-  uint64_t walk_states;        /* distinct Earley sets created by the trie walk */
+  uint64_t sweep_transitions;   /* Earley steps (scan + complete + predict) done by the trie sweep */
+  uint64_t sweep_states;        /* distinct Earley sets created by the trie sweep */
 } fmt_stats;
 
 /*
@@ -167,7 +167,7 @@ fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t
 /*
  * Write the mask of every row (Sections 3.3, 4.1): mask_dev[row * stride_words + w].
  * stride_words >= ceil(V/32).  Rows whose pruned chart is in the state cache copy the cached
- * mask; the others walk the vocabulary trie.
+ * mask; the others sweep the vocabulary trie.
  */
 fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, void* stream);
 
@@ -203,13 +203,13 @@ fmt_status fmt_state_copy_chart(fmt_state* s, uint32_t row, uint32_t* out, size_
 fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream);
 
 /* Kernel timing with CUDA events on the caller's stream (no counterpart in the paper: a
- * measurement aid).  While enabled, every fmt_state_advance, the trie-walk kernel of every fill
+ * measurement aid).  While enabled, every fmt_state_advance, the trie-sweep kernel of every fill
  * and every logits-masking kernel of this state is bracketed by a pair of events (up to 16384
  * pairs per kind, later launches are not timed).  fmt_state_read_profile synchronizes those
  * events, adds up the elapsed times and forgets them. */
 typedef struct {
-  double advance_ms, walk_ms, apply_ms;
-  uint64_t advance_launches, walk_launches, apply_launches;
+  double advance_ms, sweep_ms, apply_ms;
+  uint64_t advance_launches, sweep_launches, apply_launches;
 } fmt_profile;
 fmt_status fmt_state_set_profiling(fmt_state* s, int enable);
 fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
@@ -223,7 +223,7 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
  * real-time or library context where an allocation may synchronize the device or fail under
  * memory pressure, a plugin that may only launch kernels.  fmt_fill_mask itself never allocates,
  * but it needs an fmt_state, whose creation allocates hundreds of megabytes.  This call needs no
- * fmt_state: it walks the vocabulary trie for charts the caller already holds in device memory
+ * fmt_state: it sweeps the vocabulary trie for charts the caller already holds in device memory
  * (in the layout fmt_state_copy_chart documents) and uses a fixed scratch array that is part of
  * the loaded library image (about 52 MB of device memory on every GPU that loads the library,
  * held until the process exits).
@@ -236,7 +236,7 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
  *                  vocabulary) at most 8 Mi (beyond either limit: FMT_ERR_CAPACITY)
  *   mask_dev       device output, n rows of exactly ceil(V/32) words (dense, no extra stride)
  *   status_dev     device output or NULL, n int32: FMT_OK, FMT_ERR_INVALID_ARG (the chart's header
- *                  does not fit its slot) or FMT_ERR_CAPACITY (the Earley sets met while walking the
+ *                  does not fit its slot) or FMT_ERR_CAPACITY (the Earley sets met while sweeping the
  *                  vocabulary outgrew the fixed scratch; that row's mask is all-zero)
  *
  * The first call on each device looks up the scratch array's device address and raises the

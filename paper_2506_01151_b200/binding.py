@@ -40,7 +40,7 @@ class CompileOptions(C.Structure):
 class StateOptions(C.Structure):
     _fields_ = [
         ("cache_disable", C.c_uint32), ("max_states", C.c_uint32), ("max_mask_rows", C.c_uint32),
-        ("chart_words", C.c_uint32), ("pool_words", C.c_uint64), ("walk_states", C.c_uint32),
+        ("chart_words", C.c_uint32), ("pool_words", C.c_uint64), ("sweep_states", C.c_uint32),
         ("reserved", C.c_uint32 * 5),
     ]
 
@@ -55,15 +55,15 @@ class Stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "steps_advanced", "fills", "fills_computed", "fills_from_cache", "fills_shared", "states_cached",
         "mask_rows_cached", "pool_words_used", "chart_items_max", "chart_sets_max", "capacity_errors",
-        "big_mode_units", "walk_transitions", "walk_states")]
+        "big_mode_units", "sweep_transitions", "sweep_states")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
 
 
 class Profile(C.Structure):
-    _fields_ = [("advance_ms", C.c_double), ("walk_ms", C.c_double), ("apply_ms", C.c_double),
-                ("advance_launches", C.c_uint64), ("walk_launches", C.c_uint64), ("apply_launches", C.c_uint64)]
+    _fields_ = [("advance_ms", C.c_double), ("sweep_ms", C.c_double), ("apply_ms", C.c_double),
+                ("advance_launches", C.c_uint64), ("sweep_launches", C.c_uint64), ("apply_launches", C.c_uint64)]
 
 
 _lib = None
@@ -164,7 +164,7 @@ class State:
     """fmt_state_*: a batch of sequences on the device."""
 
     def __init__(self, grammar: Grammar, batch: int, stream=None, cache: bool = True, max_states: int = 0,
-                 max_mask_rows: int = 0, pool_words: int = 0, chart_words: int = 0, walk_states: int = 0):
+                 max_mask_rows: int = 0, pool_words: int = 0, chart_words: int = 0, sweep_states: int = 0):
         self.grammar = grammar
         self.batch = batch
         opt = StateOptions()
@@ -173,7 +173,7 @@ class State:
         opt.max_mask_rows = max_mask_rows
         opt.pool_words = pool_words
         opt.chart_words = chart_words
-        opt.walk_states = walk_states
+        opt.sweep_states = sweep_states
         h = C.c_void_p()
         _check(lib().fmt_state_create(grammar._h, batch, C.byref(opt), _ptr(stream), C.byref(h)))
         self._h = h

@@ -74,7 +74,7 @@ struct fmt_grammar {
 struct Profiler {
   static constexpr size_t kMaxPairs = 16384;
   bool on = false;
-  std::vector<cudaEvent_t> a[3], b[3];  // 0 advance, 1 walk, 2 logits masking
+  std::vector<cudaEvent_t> a[3], b[3];  // 0 advance, 1 trie sweep, 2 logits masking
   size_t used[3] = {0, 0, 0};
   bool next(int kind, cudaEvent_t* before, cudaEvent_t* after) {
     *before = *after = nullptr;
@@ -110,7 +110,7 @@ struct fmt_state {
   int32_t* init_state_dev = nullptr;
   int32_t* result_dev = nullptr;
   uint8_t* query_dev = nullptr;  // scratch for fmt_state_query
-  int walk_grid = 1;
+  int sweep_grid = 1;
 };
 
 namespace fmt {
@@ -184,12 +184,9 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
       d.direct_off = d.hot_block + o_doff;
       d.direct_items = reinterpret_cast<const uint16_t*>(d.hot_block + o_dit);
     }
-    UP(child_off);
     UP(node_byte);
     UP(parent);
     UP(node_depth);
-    UP(tok_off);
-    UP(tok_ids);
     UP(lvl_off);
     UP(tok_node);
     UP(vocab_off);
@@ -282,7 +279,7 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   d.big_arena_items = 1u << 16;
   d.big_hset_slots = 1u << 14;
   AutoDev& au = d.au;
-  au.cap = (opt && opt->walk_states) ? opt->walk_states : std::min(32768u, std::max(2048u, (4u << 20) / batch));
+  au.cap = (opt && opt->sweep_states) ? opt->sweep_states : std::min(32768u, std::max(2048u, (4u << 20) / batch));
   if (au.cap < 16) au.cap = 16;
   if (au.cap > 60000) au.cap = 60000;
   au.rec_words = (AR_TRANS + g->dev.n_eq + 31u) & ~31u;
@@ -294,15 +291,15 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   sweep_layout(g->dev, &au.smem_bytes, &au.tables_in_smem);
   cudaError_t e = configure_kernels();
   int per_sm = 0, sms = 0, dev = 0;
-  if (e == cudaSuccess) e = walk_blocks_per_sm(&per_sm, au.smem_bytes);
+  if (e == cudaSuccess) e = sweep_blocks_per_sm(&per_sm, au.smem_bytes);
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e == cudaSuccess && per_sm < 1) {
     delete s;
-    return fail(FMT_ERR_CUDA, "the walk kernel does not fit on this device");
+    return fail(FMT_ERR_CUDA, "the sweep kernel does not fit on this device");
   }
-  s->walk_grid = std::max(1, per_sm * sms);
-  const size_t big_words = (size_t)s->walk_grid * walk_warps() * ((size_t)d.big_arena_items + d.big_hset_slots);
+  s->sweep_grid = std::max(1, per_sm * sms);
+  const size_t big_words = (size_t)s->sweep_grid * sweep_warps() * ((size_t)d.big_arena_items + d.big_hset_slots);
 #define AL(ptr, count, fill) if (e == cudaSuccess) e = s->bufs.alloc((size_t)(count), &(ptr), (fill))
   AL(d.arena, d.pool_base + d.pool_words, 0);
   AL(d.row_chart, batch, 0);
@@ -386,9 +383,8 @@ fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, 
   cudaStream_t st = (cudaStream_t)stream;
   cudaEvent_t w0, w1;
   s->prof.next(1, &w0, &w1);
-  launch_fill(s->g->dev, s->dev, s->walk_grid, st, w0, w1);
+  launch_fill(s->g->dev, s->dev, s->sweep_grid, st, w0, w1);
   launch_gather(s->g->dev, s->dev, mask_dev, stride_words, st);
-  launch_end_fill(s->dev, st);
   return launched("fmt_fill_mask");
 }
 
@@ -413,11 +409,10 @@ fmt_status fmt_fill_and_apply(fmt_state* s, uint32_t* mask_dev_or_null, size_t s
   cudaEvent_t w0, w1, a0, a1;
   s->prof.next(1, &w0, &w1);
   s->prof.next(2, &a0, &a1);
-  launch_fill(s->g->dev, s->dev, s->walk_grid, st, w0, w1);
+  launch_fill(s->g->dev, s->dev, s->sweep_grid, st, w0, w1);
   if (a0) cudaEventRecord(a0, st);
   launch_gather_apply(s->g->dev, s->dev, logits_dev, (int)dtype, row_stride_elems, mask_dev_or_null, stride_words, st);
   if (a1) cudaEventRecord(a1, st);
-  launch_end_fill(s->dev, st);
   return launched("fmt_fill_and_apply");
 }
 
@@ -498,8 +493,8 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out) {
       ms[k] += t;
     }
   }
-  out->advance_ms = ms[0], out->walk_ms = ms[1], out->apply_ms = ms[2];
-  out->advance_launches = s->prof.used[0], out->walk_launches = s->prof.used[1], out->apply_launches = s->prof.used[2];
+  out->advance_ms = ms[0], out->sweep_ms = ms[1], out->apply_ms = ms[2];
+  out->advance_launches = s->prof.used[0], out->sweep_launches = s->prof.used[1], out->apply_launches = s->prof.used[2];
   s->prof.used[0] = s->prof.used[1] = s->prof.used[2] = 0;
   return FMT_OK;
 }
@@ -524,8 +519,8 @@ fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   out->chart_sets_max = c[CNT_STAT_SETS_MAX];
   out->capacity_errors = u64(CNT_STAT_CAPERR);
   out->big_mode_units = u64(CNT_STAT_BIG);
-  out->walk_transitions = u64(CNT_STAT_TRANS);
-  out->walk_states = u64(CNT_STAT_LOCAL);
+  out->sweep_transitions = u64(CNT_STAT_TRANS);
+  out->sweep_states = u64(CNT_STAT_LOCAL);
   return FMT_OK;
 }
 

@@ -17,12 +17,9 @@ struct GrammarDev {
   const uint32_t* nt_closure;    // [N][Nw]
   const uint32_t* direct_off;    // [N+1]
   const uint16_t* direct_items;
-  const uint32_t* child_off;     // [T+1]
   const uint8_t* node_byte;      // [T]
   const uint32_t* parent;        // [T]
   const uint8_t* node_depth;     // [T]
-  const uint32_t* tok_off;       // [T+1]
-  const uint32_t* tok_ids;
   // The tables above that every Earley step reads (info, class_bits, eq_of_byte, nt_closure,
   // direct_off, direct_items) sit in one contiguous block so that a kernel can copy them into
   // shared memory at once and shift the six pointers.
@@ -50,7 +47,6 @@ enum : uint32_t {
   CNT_N_STATES = 0,
   CNT_N_MASK_ROWS = 1,
   CNT_N_JOBS = 2,
-  CNT_WORK = 3,
   CNT_ERR = 4,          // sticky: some device routine hit a capacity limit
   CNT_AUTO_ITEMS = 5,   // top of the automaton's item pool (words), reset by every fill
   CNT_POOL_LO = 6,      // 64-bit pool top (words) lives in slots 6,7 (8-byte aligned)
@@ -63,8 +59,8 @@ enum : uint32_t {
   CNT_STAT_SETS_MAX = 20,
   CNT_STAT_CAPERR = 22,
   CNT_STAT_BIG = 24,
-  CNT_STAT_TRANS = 26,  // transitions computed by the trie walk (Earley steps)
-  CNT_STAT_LOCAL = 28,  // local states created by the trie walk
+  CNT_STAT_TRANS = 26,  // transitions computed by the trie sweep (Earley steps)
+  CNT_STAT_LOCAL = 28,  // local states created by the trie sweep
   CNT_BAR = 30,         // grid barrier of the trie sweep: arrivals
   CNT_BAR_ERR = 31,     // a block gave up waiting at the barrier
   CNT_LEVEL_ALIVE = 32, // [MAX_TOKEN_BYTES + 2] per trie depth: some node of some job was alive

@@ -1,4 +1,4 @@
-// CUDA kernels of the mask path (sm_100a): advance, plan / walk / publish of the mask fill, gather
+// CUDA kernels of the mask path (sm_100a): advance, plan / sweep / publish of the mask fill, gather
 // and the logits masking.  Integer work only: no tensor cores are involved anywhere.
 #include <cuda_runtime.h>
 
@@ -225,7 +225,6 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
   if (threadIdx.x < CNT_TOTAL - CNT_BAR) S.counters[CNT_BAR + threadIdx.x] = 0u;  // barrier and level counters
   if (threadIdx.x == 0) {
     S.counters[CNT_N_JOBS] = 0u;
-    S.counters[CNT_WORK] = 0u;
     S.counters[CNT_AUTO_ITEMS] = 0u;
   }
   __syncthreads();
@@ -934,7 +933,7 @@ void sweep_layout(const GrammarDev& G, uint32_t* smem_bytes, uint32_t* tables_in
   if (*tables_in_smem) bytes += tab;
   *smem_bytes = bytes;
 }
-int walk_warps() { return SWEEP_WARPS; }
+int sweep_warps() { return SWEEP_WARPS; }
 
 cudaError_t configure_kernels() {
   cudaError_t e;
@@ -944,7 +943,7 @@ cudaError_t configure_kernels() {
   return cudaSuccess;
 }
 
-cudaError_t walk_blocks_per_sm(int* out, uint32_t smem_bytes) {
+cudaError_t sweep_blocks_per_sm(int* out, uint32_t smem_bytes) {
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, sweep_kernel, SWEEP_WARPS * 32, smem_bytes);
 }
 
@@ -968,17 +967,16 @@ static void launch_sweep_coop(const GrammarDev& G, const StateDev& S, int grid, 
   cudaLaunchCooperativeKernel((const void*)sweep_kernel, dim3((unsigned)grid), dim3(SWEEP_WARPS * 32), args,
                               S.au.smem_bytes, st);
 }
-void launch_fill(const GrammarDev& G, const StateDev& S, int walk_grid, cudaStream_t st, cudaEvent_t before_walk,
-                 cudaEvent_t after_walk) {
+void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_sweep,
+                 cudaEvent_t after_sweep) {
   plan_kernel<<<1, 1024, 0, st>>>(G, S);
-  if (before_walk) cudaEventRecord(before_walk, st);
-  launch_sweep_coop(G, S, walk_grid, st);
-  if (after_walk) cudaEventRecord(after_walk, st);
+  if (before_sweep) cudaEventRecord(before_sweep, st);
+  launch_sweep_coop(G, S, sweep_grid, st);
+  if (after_sweep) cudaEventRecord(after_sweep, st);
   publish_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(S);
 }
 // the sweep alone, for jobs the caller has already listed (used by the allocation-free entry point)
-void launch_walk(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) { launch_sweep_coop(G, S, grid, st); }
-void launch_end_fill(const StateDev& S, cudaStream_t st) { (void)S; (void)st; }
+void launch_sweep(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) { launch_sweep_coop(G, S, grid, st); }
 void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st) {
   dim3 grid((unsigned)std::min<size_t>((stride_words + 255) / 256, 64), S.B);
   gather_kernel<<<grid, 256, 0, st>>>(G, S, out, stride_words);

@@ -1,6 +1,6 @@
-// fmt_fill_mask_noalloc: the trie walk for callers that may not allocate device memory.
+// fmt_fill_mask_noalloc: the trie sweep for callers that may not allocate device memory.
 //
-// All scratch the walk needs lives in one file-scope __device__ array that is part of the
+// All scratch the sweep needs lives in one file-scope __device__ array that is part of the
 // library image.  Host code must not pass the array's name to a kernel (on the host it is only
 // a stand-in symbol): the device address is looked up once per device with
 // cudaGetSymbolAddress and passed as an ordinary pointer.
@@ -18,7 +18,7 @@ namespace {
 using namespace fmt;
 
 constexpr uint32_t NA_MAX = FMT_NOALLOC_MAX_CHARTS;
-constexpr uint32_t NA_GRID = 32;            // CTAs of the walk
+constexpr uint32_t NA_GRID = 32;            // CTAs of the sweep
 constexpr uint32_t NA_ARENA_ITEMS = 8192;   // per-warp overflow area for Earley sets (items)
 constexpr uint32_t NA_HSET_SLOTS = 2048;    // per-warp overflow uniqueness hash
 // header: counters, then per-chart arrays
@@ -34,7 +34,7 @@ constexpr uint32_t NA_OFF_JOBINFO = NA_OFF_NSTATES + NA_MAX;     // [NA_MAX] uin
 constexpr uint32_t NA_HEADER_WORDS = 1024;
 constexpr size_t NA_WARPS = (size_t)NA_GRID * 8;
 constexpr size_t NA_BIG_WORDS = NA_WARPS * (NA_ARENA_ITEMS + NA_HSET_SLOTS);
-// the walk's tables of Earley sets: per chart 64 Ki words of records and 2048 hash slots, and one
+// the sweep's tables of Earley sets: per chart 64 Ki words of records and 2048 hash slots, and one
 // pool of 2 Mi item words for all charts of a call
 constexpr uint32_t NA_REC_WORDS_PER_CHART = 65536;
 constexpr uint32_t NA_HASH_SLOTS = 2048;
@@ -62,7 +62,7 @@ struct Offsets {
 
 // Fill the header for this call, check each chart's header against its slot, zero the output
 // masks (setting the EOS bit of accepting charts) and clear the overflow hashes, which must be
-// all-empty before the walk and may hold anything after an earlier call that broke off.
+// all-empty before the sweep and may hold anything after an earlier call that broke off.
 __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scratch, const uint32_t* charts, Offsets off,
                                        uint32_t n, uint32_t* mask) {
   const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -121,7 +121,7 @@ cudaError_t scratch_for_current_device(int dev, uint32_t** out) {
     uint32_t* p = nullptr;
     cudaError_t e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);
     if (e != cudaSuccess) return e;
-    e = configure_kernels();  // raises the dynamic shared-memory limit of the walk kernel on this device
+    e = configure_kernels();  // raises the dynamic shared-memory limit of the sweep kernel on this device
     if (e != cudaSuccess) return e;
     g_scratch_addr[dev] = p;
   }
@@ -164,7 +164,7 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   StateDev S{};
   S.B = n;
   S.cache_on = 0;
-  S.arena = const_cast<uint32_t*>(charts_dev);  // the walk only reads charts
+  S.arena = const_cast<uint32_t*>(charts_dev);  // the sweep only reads charts
   S.counters = scratch + NA_OFF_COUNTERS;
   S.jobs = scratch + NA_OFF_JOBS;
   S.row_flags = scratch + NA_OFF_FLAGS;
@@ -191,7 +191,7 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   cudaStream_t st = (cudaStream_t)stream;
   noalloc_prepare_kernel<<<256, 256, 0, st>>>(*G, S, scratch, charts_dev, off, n, mask_dev);
   noalloc_jobs_kernel<<<1, 32, 0, st>>>(S, scratch, n);
-  launch_walk(*G, S, (int)NA_GRID, st);
+  launch_sweep(*G, S, (int)NA_GRID, st);
   noalloc_finish_kernel<<<n, 128, 0, st>>>(*G, S, scratch, n, mask_dev, status_dev);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(FMT_ERR_CUDA, cudaGetErrorString(e));

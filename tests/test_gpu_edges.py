@@ -255,7 +255,7 @@ def test_capacity_overflow_is_reported_not_guessed():
     assert st.query()["finished"].tolist() == [2, 2]
     assert st.stats()["capacity_errors"] >= 2
     # a state with too few walk states reports the capacity problem through the mask (all-zero) as well
-    st2 = fmt.State(g, 1, walk_states=16)
+    st2 = fmt.State(g, 1, sweep_states=16)
     assert _advance(st2, [ord("[")]) == [0]
     for c in names[0].encode():
         assert _advance(st2, [c]) == [0]
