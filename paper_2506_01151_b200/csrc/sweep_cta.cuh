@@ -1,0 +1,581 @@
+// The trie sweep of the mask fill: one CTA per job (a row whose mask must be computed).
+//
+// For its job the CTA answers, for every trie node, "is the Earley set reached by this node's bytes
+// non-empty?" (Sections 3.3 and 4.1: a token is valid iff every Earley set along its bytes stays
+// non-empty).  Sets are hash-consed per job (AutoDev): a transition (set, byte class) is computed
+// once, with the warp-cooperative scan / complete / predict of earley_device.cuh, and every other
+// node that needs it reads it from the set's record.  The automaton (records, items, hash), the
+// job's base chart, the grammar's hot tables and the mask row under construction live in the CTA's
+// shared memory; only automata that outgrow it spill into the CTA's slice of global memory.
+//
+// The trie is processed one depth at a time, one THREAD per node: st[node] =
+// transition(st[parent], byte).  Nodes are numbered breadth first, so a depth is a contiguous
+// range, the children of consecutive parents are consecutive, and whole chunks of TRIE_CHUNK nodes
+// whose parents are all dead are skipped after one look at a bitmap ("some node of this group of
+// 32 is alive").  A transition nobody has computed yet is claimed by the first thread that meets
+// it and queued; after the pass the warps take the queued transitions, one each, then the nodes
+// that waited are settled.  Only __syncthreads() separates the phases: nothing waits on another
+// CTA, and jobs are handed out through an atomic ticket.
+#pragma once
+#include "chart_step.cuh"
+
+namespace fmt {
+
+constexpr int SW_WARPS = 16;
+constexpr int SW_THREADS = SW_WARPS * 32;
+constexpr uint32_t SW_CUR = 256;        // items of a set under construction per warp (fast mode, power of two)
+constexpr uint32_t SW_HSET = 512;       // uniqueness hash slots per warp (fast mode)
+constexpr uint32_t SW_QUEUE = 512;      // transitions queued per round
+constexpr uint32_t SW_HASH = 4096;      // slots of the shared-memory hash of Earley sets
+constexpr uint32_t SW_HASH_MAX = 2560;  // sets it may hold; later ones go to the CTA's overflow hash
+constexpr uint32_t SW_CHUNKS = SW_THREADS;  // chunks tested per round, one per thread
+constexpr uint32_t SW_SMEM_BUDGET = 227u * 1024u;
+constexpr uint32_t SW_CHART_SM = 4096;  // words of a base chart staged in shared memory
+constexpr uint32_t SW_PER_LANE = TRIE_CHUNK / 32;
+
+// control words in shared memory
+enum : uint32_t {
+  SC_N_STATES = 0,   // Earley sets of the job so far
+  SC_ITEMS_TOP,      // top of the shared-memory item pool
+  SC_Q_N,            // queued transitions
+  SC_PEND_N,         // waiting nodes of the current depth
+  SC_CH_N0,          // alive chunks of the round (two counters, used alternately)
+  SC_CH_N1,
+  SC_ALIVE,          // some node of the current depth is alive
+  SC_FAIL,           // a capacity was exceeded: the row's mask cannot be trusted
+  SC_GL_HASH,        // the overflow hash is in use
+  SC_N_SMHASH,       // sets entered into the shared-memory hash
+  SC_TRANS,          // transitions computed (statistics)
+  SC_JOB,            // the job in hand
+  SC_BIG,            // warps that switched to their large scratch (statistics)
+  SC_TOTAL = 16
+};
+
+// word offsets into the dynamic shared memory
+struct SweepSmem {
+  uint32_t tables, mask, warps, warp_words, chart, hash, queue, chunks, bits, ctl, recs, items, total;
+};
+
+__host__ __device__ inline uint32_t sw_pad4(uint32_t words) { return (words + 3u) & ~3u; }
+
+__host__ __device__ inline SweepSmem sweep_smem(const GrammarDev& G, const AutoDev& A) {
+  SweepSmem L;
+  uint32_t at = 0;
+  L.tables = at, at += sw_pad4(A.tables_in_smem ? G.hot_words : 0u);
+  L.mask = at, at += sw_pad4(A.mask_in_smem ? G.Wm : 0u);
+  L.warp_words = SW_CUR + SW_HSET + ((2u * G.Nw + 7u) & ~7u) + W_CTRS + 8u;
+  L.warps = at, at += SW_WARPS * L.warp_words;
+  L.chart = at, at += sw_pad4(A.chart_sm_words);
+  L.hash = at, at += SW_HASH;
+  L.queue = at, at += SW_QUEUE;
+  L.chunks = at, at += SW_CHUNKS;
+  L.bits = at, at += sw_pad4(2u * A.bit_words);
+  L.ctl = at, at += SC_TOTAL;
+  L.recs = at, at += sw_pad4(A.sm_states * A.rec_words);
+  L.items = at, at += sw_pad4(A.sm_items);
+  L.total = at;
+  return L;
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_cta(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.cta.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_volatile(const uint32_t* p) { return *reinterpret_cast<const volatile uint32_t*>(p); }
+
+// What the CTA knows about its job and where the job's automaton lives.
+struct CtaAuto {
+  uint32_t rec_words, sm_states, sm_items, cap;
+  uint32_t* ctl;       // shared
+  uint32_t* sm_recs;   // shared
+  uint32_t* sm_itm;    // shared
+  uint32_t* sm_hash;   // shared
+  uint32_t* gl_recs;   // this CTA's slice
+  uint32_t* gl_hash;   // this CTA's slice
+  uint32_t gl_hash_mask;
+  uint32_t* gl_items;  // pool shared by all CTAs
+  const uint32_t* base_off;
+  const uint32_t* base_items;
+  uint32_t m;          // live sets of the base chart
+
+  __device__ __forceinline__ uint32_t* rec(uint32_t id) const {
+    return id < sm_states ? sm_recs + id * rec_words : gl_recs + (size_t)(id - sm_states) * rec_words;
+  }
+  __device__ __forceinline__ uint32_t* items_at(uint32_t off) const {
+    return off < sm_items ? sm_itm + off : gl_items + (off - sm_items);
+  }
+  __device__ __forceinline__ uint16_t* trans(uint32_t id) const { return reinterpret_cast<uint16_t*>(rec(id) + AR_TRANS); }
+};
+
+struct CtaView {
+  const CtaAuto& a;
+  __device__ __forceinline__ void operator()(uint32_t o, const uint32_t*& p, uint32_t& n) const {
+    if (o < a.m) {
+      const uint32_t x = a.base_off[o], y = a.base_off[o + 1];
+      p = a.base_items + x;
+      n = y - x;
+    } else {
+      const uint32_t* r = a.rec(o - a.m);
+      p = a.items_at(r[AR_ITEMS]);
+      n = r[AR_N];
+    }
+  }
+  // an item of local state o that names its own state as origin means "origin o"
+  __device__ __forceinline__ uint32_t fix(uint32_t item, uint32_t o) const {
+    return ((item >> 16) == ORIGIN_SELF) ? ((o << 16) | (item & 0xFFFFu)) : item;
+  }
+};
+
+// The Earley step of one warp.
+struct SweepWarp {
+  const GrammarDev& G;
+  const StateDev& S;
+  const CtaAuto& a;
+  WarpCtx w;
+  uint32_t cur_pow2;  // capacity of w.cur (a power of two, for the sort)
+  uint32_t* tmp8;     // shared
+  uint32_t chunk_at = 0, chunk_left = 0;  // this warp's piece of the global item pool (lane 0's copy counts)
+
+  // A new set with the items w.cur[0..n): returns its id or T_FAIL.
+  __device__ uint32_t create_set(uint32_t n, uint32_t hash) {
+    const uint32_t lane = lane_id();
+    uint32_t id = T_FAIL, ioff = 0;
+    if (lane == 0) {
+      const uint32_t got = atomicAdd(&a.ctl[SC_N_STATES], 1u);
+      const uint32_t need = max(n, 1u);
+      if (got < a.cap) {
+        const uint32_t at = (ld_volatile(&a.ctl[SC_ITEMS_TOP]) < a.sm_items) ? atomicAdd(&a.ctl[SC_ITEMS_TOP], need) : a.sm_items;
+        if (at < a.sm_items && need <= a.sm_items - at) {
+          ioff = at;
+          id = got;
+        } else {
+          if (need > chunk_left) {  // a new piece of the global pool: one atomic per ~4 Ki item words
+            const uint32_t take = max(need, 4096u);
+            chunk_at = atomicAdd(&S.counters[CNT_AUTO_ITEMS], take);
+            chunk_left = (chunk_at <= S.au.items_cap && take <= S.au.items_cap - chunk_at) ? take : 0u;
+          }
+          if (need <= chunk_left) {
+            ioff = a.sm_items + chunk_at;
+            chunk_at += need;
+            chunk_left -= need;
+            id = got;
+          }
+        }
+      }
+    }
+    id = __shfl_sync(FULL, id, 0);
+    ioff = __shfl_sync(FULL, ioff, 0);
+    if (id == T_FAIL) return T_FAIL;
+    uint32_t* rec = a.rec(id);
+    uint32_t* items = a.items_at(ioff);
+    for (uint32_t i = lane; i < n; i += 32) items[i] = w.cur[i];
+    for (uint32_t i = lane; i < a.rec_words; i += 32) {
+      uint32_t v = 0u;
+      if (i == AR_ITEMS) v = ioff;
+      else if (i == AR_N) v = n;
+      else if (i == AR_HASH) v = hash;
+      else if (i >= AR_SCAN && i < AR_SCAN + 8) v = tmp8[i - AR_SCAN];
+      else if (i >= AR_TRANS) v = 0xFFFFFFFFu;  // two T16_UNKNOWN
+      rec[i] = v;
+    }
+    __syncwarp();
+    __threadfence_block();
+    return id;
+  }
+
+  // Find or create the set whose items are w.cur[0..n) (sorted).  Returns its id or T_FAIL.  Sets
+  // entered by two warps at the same moment may, rarely, get two ids; the automaton stays correct.
+  __device__ uint32_t intern_set(uint32_t n, uint32_t hash) {
+    const uint32_t lane = lane_id();
+    uint32_t* table = a.sm_hash;
+    uint32_t mask = SW_HASH - 1u;
+    uint32_t slot = hash & mask;
+    bool in_gl = false, room = false;
+    uint32_t my_id = T_FAIL;
+    for (uint32_t probe = 0; probe < 8192u; ++probe) {
+      uint32_t v = 0;
+      if (lane == 0) v = ld_acquire_cta(&table[slot]);
+      v = __shfl_sync(FULL, v, 0);
+      if (v == 0) {
+        if (!in_gl) {  // not in the shared-memory table: look in the overflow table, or reserve a place here
+          uint32_t go_gl = 0;
+          if (lane == 0) {
+            go_gl = ld_volatile(&a.ctl[SC_GL_HASH]);
+            if (!go_gl && !room) {
+              if (atomicAdd(&a.ctl[SC_N_SMHASH], 1u) >= SW_HASH_MAX) {
+                atomicExch(&a.ctl[SC_GL_HASH], 1u);
+                go_gl = 1u;
+              }
+            }
+          }
+          go_gl = __shfl_sync(FULL, go_gl, 0);
+          if (go_gl) {
+            in_gl = true;
+            table = a.gl_hash;
+            mask = a.gl_hash_mask;
+            slot = hash & mask;
+            continue;
+          }
+          room = true;
+        }
+        if (my_id == T_FAIL) {
+          my_id = create_set(n, hash);
+          if (my_id == T_FAIL) return T_FAIL;
+        }
+        uint32_t old = 0;
+        if (lane == 0) old = atomicCAS(&table[slot], 0u, my_id + 1u);
+        old = __shfl_sync(FULL, old, 0);
+        if (old == 0) return my_id;
+        v = old;
+      }
+      const uint32_t sid = v - 1u;
+      const uint32_t* rec = a.rec(sid);
+      bool same = (ld_volatile(rec + AR_HASH) == hash) && (ld_volatile(rec + AR_N) == n);
+      if (same) {
+        const uint32_t* items = a.items_at(ld_volatile(rec + AR_ITEMS));
+        for (uint32_t i = lane; i < n; i += 32)
+          if (ld_volatile(items + i) != w.cur[i]) same = false;
+      }
+      same = __all_sync(FULL, same);
+      if (same) return sid;
+      slot = (slot + 1u) & mask;
+    }
+    return T_FAIL;
+  }
+
+  // The transition of set `ps` on `byte`: T_DEAD, a set id, or T_FAIL when a capacity was exceeded.
+  __device__ uint32_t compute(uint32_t ps, uint32_t byte) {
+    const uint32_t lane = lane_id();
+    const uint32_t* pitems;
+    uint32_t plen;
+    CtaView view{a};
+    view(ps == 0 ? a.m - 1 : a.m + ps, pitems, plen);
+    __syncwarp();
+    if (lane < W_CTRS) w.ctr[lane] = 0u;
+    __syncwarp();
+    const uint32_t self_code = a.m + ps;
+    for (uint32_t k = lane; k < plen; k += 32) {
+      uint32_t it = pitems[k];
+      uint32_t inf = G.info[it & 0xFFFFu];
+      if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) {
+        if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
+        add_item(G, w, it + 1u);
+      }
+    }
+    __syncwarp();
+    uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
+    if (w.ctr[W_OVERFLOW]) {
+      hset_clear_all(w.hset, w.hset_mask);
+      return T_FAIL;
+    }
+    if (n == 0) return T_DEAD;
+    complete_fixpoint(G, w, view, ORIGIN_SELF, 0u);
+    const uint32_t hashed = min(w.ctr[W_NCUR], w.cur_cap);
+    if (w.ctr[W_OVERFLOW]) {
+      hset_clear_all(w.hset, w.hset_mask);
+      clear_nt(G, w);
+      return T_FAIL;
+    }
+    hset_clear_items(w, hashed);
+    predict_into_cur(G, w, ORIGIN_SELF);
+    if (w.ctr[W_OVERFLOW]) return T_FAIL;
+    n = drop_completed(G, w, min(w.ctr[W_NCUR], w.cur_cap));
+    sort_items(w.cur, n, cur_pow2);
+    uint32_t h = 0x9E3779B9u ^ n;
+    for (uint32_t i = lane; i < n; i += 32) h += mix32(w.cur[i] ^ (i * 0x85EBCA77u));
+    for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
+    scannable_bytes(G, w.cur, n, tmp8);
+    return intern_set(n, h);
+  }
+};
+
+// The state a node reaches from parent state `ps` on `byte`: ST_DEAD, ST_PENDING (the transition
+// is not known yet: it has been queued, by this thread if nobody did before) or the state's id.
+__device__ __forceinline__ uint32_t step_node(const GrammarDev& G, const CtaAuto& a, uint32_t* queue, uint32_t ps,
+                                              uint32_t byte) {
+  const uint32_t* rec = a.rec(ps);
+  // one 256-bit test rejects most bytes without touching the transition table
+  if (!((rec[AR_SCAN + (byte >> 5)] >> (byte & 31u)) & 1u)) return ST_DEAD;
+  uint16_t* tr = a.trans(ps) + G.eq_of_byte[byte];
+  uint32_t t = *reinterpret_cast<volatile uint16_t*>(tr);
+  if (t == T16_UNKNOWN) {
+    t = atomicCAS(tr, (unsigned short)T16_UNKNOWN, (unsigned short)T16_PENDING);
+    if (t == T16_UNKNOWN) {  // ours to queue
+      const uint32_t at = atomicAdd(&a.ctl[SC_Q_N], 1u);
+      if (at < SW_QUEUE) queue[at] = (ps << 8) | byte;
+      else *reinterpret_cast<volatile uint16_t*>(tr) = T16_UNKNOWN;  // no room in this round: somebody claims it again in the next
+      return ST_PENDING;
+    }
+  }
+  if (t == T16_PENDING || t == T16_UNKNOWN) return ST_PENDING;
+  return (t == T16_DEAD) ? (uint32_t)ST_DEAD : t;
+}
+
+__device__ __forceinline__ void set_tokens(const GrammarDev& G, uint32_t* mask, uint32_t node) {
+  const uint32_t tok = __ldg(&G.node_tok[node]);
+  if (tok == NODE_TOK_NONE) return;
+  if (tok != NODE_TOK_MANY) {
+    atomicOr(&mask[tok >> 5], 1u << (tok & 31u));
+    return;
+  }
+  for (uint32_t i = __ldg(&G.tok_off[node]), e = __ldg(&G.tok_off[node + 1]); i < e; ++i) {
+    const uint32_t t = __ldg(&G.tok_ids[i]);
+    atomicOr(&mask[t >> 5], 1u << (t & 31u));
+  }
+}
+
+__global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, StateDev S) {
+  const uint32_t n_jobs = S.counters[CNT_N_JOBS];
+  if (blockIdx.x >= n_jobs) return;  // more CTAs than jobs
+  extern __shared__ __align__(16) uint32_t smem[];
+  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = lane_id();
+  const AutoDev& A = S.au;
+  const SweepSmem L = sweep_smem(Gg, A);
+  GrammarDev G = Gg;
+  if (A.tables_in_smem) G = stage_hot_tables(Gg, smem + L.tables);
+  uint32_t* const ctl = smem + L.ctl;
+  uint32_t* const queue = smem + L.queue;
+  uint32_t* const chunks = smem + L.chunks;
+  uint32_t* const bits = smem + L.bits;
+  uint32_t* const chart_sm = smem + L.chart;
+  uint32_t* const mask_sm = smem + L.mask;
+
+  CtaAuto a;
+  a.rec_words = A.rec_words, a.sm_states = A.sm_states, a.sm_items = A.sm_items;
+  a.ctl = ctl;
+  a.sm_recs = smem + L.recs;
+  a.sm_itm = smem + L.items;
+  a.sm_hash = smem + L.hash;
+  a.gl_recs = A.recs + (size_t)blockIdx.x * (A.cap - A.sm_states) * A.rec_words;
+  a.gl_hash = A.hash + (size_t)blockIdx.x * (A.gl_hash_mask + 1u);
+  a.gl_hash_mask = A.gl_hash_mask;
+  a.gl_items = A.items;
+  uint16_t* const st_base = A.st + (size_t)blockIdx.x * 2u * A.level_pad;
+  uint32_t* const pend = A.pend + (size_t)blockIdx.x * A.level_pad;
+
+  uint32_t* mine = smem + L.warps + (size_t)warp * L.warp_words;
+  SweepWarp sw{G, S, a};
+  sw.w.cur = mine;
+  sw.w.cur_cap = SW_CUR;
+  sw.cur_pow2 = SW_CUR;
+  sw.w.hset = mine + SW_CUR;
+  sw.w.hset_mask = SW_HSET - 1;
+  sw.w.nt = sw.w.hset + SW_HSET;
+  const uint32_t ntw = (2u * G.Nw + 7u) & ~7u;
+  sw.w.ctr = sw.w.nt + ntw;
+  sw.tmp8 = sw.w.ctr + W_CTRS;
+  uint32_t* const big = S.big_scratch + ((size_t)blockIdx.x * SW_WARPS + warp) * ((size_t)S.big_arena_items + S.big_hset_slots);
+  bool big_mode = false;
+  hset_clear_all(sw.w.hset, SW_HSET - 1);
+  for (uint32_t i = lane; i < ntw; i += 32) sw.w.nt[i] = 0u;
+  if (tid < SC_TOTAL) ctl[tid] = 0u;
+  uint32_t stat_trans = 0, stat_states = 0;  // thread 0's copies count
+
+  for (;;) {
+    __syncthreads();
+    const bool gl_hash_dirty = ctl[SC_GL_HASH] != 0u;  // left by the job before
+    __syncthreads();
+    if (tid == 0) ctl[SC_JOB] = atomicAdd(&S.counters[CNT_JOB_NEXT], 1u);
+    __syncthreads();
+    const uint32_t j = ctl[SC_JOB];
+    if (j >= n_jobs) {  // leave the overflow hash all zero for the next launch
+      if (gl_hash_dirty)
+        for (uint32_t i = tid; i <= a.gl_hash_mask; i += SW_THREADS) a.gl_hash[i] = 0u;
+      break;
+    }
+
+    // ---- the job: its chart, an automaton with one state (the chart's last set), an empty mask
+    const uint32_t row = S.jobs[j];
+    const uint32_t* chart = S.arena + S.row_chart[row];
+    const uint32_t m = chart[CH_SETS];
+    const uint32_t chart_words = chart[CH_WORDS];
+    const bool accepting = (chart[CH_FLAGS] & CHART_ACCEPTING) != 0u;
+    uint32_t* const mask = A.mask_in_smem ? mask_sm : S.mask_rows + (size_t)S.row_mask[row] * G.Wm;
+    if (chart_words <= A.chart_sm_words) {
+      for (uint32_t i = tid; i < chart_words; i += SW_THREADS) chart_sm[i] = chart[i];
+      chart = chart_sm;
+    }
+    a.base_off = chart + CH_HDR;
+    a.base_items = chart + CH_HDR + m + 1;
+    a.m = m;
+    a.cap = min(min(A.cap, AUTO_MAX_STATES), (ORIGIN_SELF - 1u > m) ? ORIGIN_SELF - 1u - m : 0u);
+    for (uint32_t i = tid; i < SW_HASH; i += SW_THREADS) a.sm_hash[i] = 0u;
+    if (gl_hash_dirty)
+      for (uint32_t i = tid; i <= a.gl_hash_mask; i += SW_THREADS) a.gl_hash[i] = 0u;
+    for (uint32_t i = tid; i < G.Wm; i += SW_THREADS) mask[i] = 0u;
+    for (uint32_t i = tid; i < 2u * A.bit_words; i += SW_THREADS) bits[i] = 0u;
+    if (tid < SC_TOTAL && tid != SC_JOB) ctl[tid] = 0u;
+    uint32_t* rec0 = a.rec(0);
+    for (uint32_t i = tid; i < a.rec_words; i += SW_THREADS)
+      if (i < AR_SCAN || i >= AR_SCAN + 8) rec0[i] = (i >= AR_TRANS) ? 0xFFFFFFFFu : 0u;
+    __syncthreads();
+    if (warp == 0) {
+      scannable_bytes(G, a.base_items + a.base_off[m - 1], a.base_off[m] - a.base_off[m - 1], sw.tmp8);
+      if (lane < 8) rec0[AR_SCAN + lane] = sw.tmp8[lane];
+      if (lane == 0) {
+        ctl[SC_N_STATES] = 1u;
+        bits[0] = 1u;    // depth 0 is the root alone, alive,
+        st_base[0] = 0;  // in state 0
+        if (accepting && G.eos >= 0) mask[(uint32_t)G.eos >> 5] = 1u << ((uint32_t)G.eos & 31u);
+      }
+    }
+    __syncthreads();
+
+    uint32_t round = 0;
+    for (uint32_t Lv = 1; Lv <= G.depth; ++Lv) {
+      const uint32_t lo_prev = __ldg(&G.lvl_off[Lv - 1]), lo = __ldg(&G.lvl_off[Lv]), hi = __ldg(&G.lvl_off[Lv + 1]);
+      if (hi == lo) break;
+      const uint32_t coff = __ldg(&G.lvl_chunk_off[Lv]), nch = __ldg(&G.lvl_chunk_off[Lv + 1]) - coff;
+      const uint16_t* st_prev = st_base + (size_t)((Lv - 1) & 1u) * A.level_pad;
+      uint16_t* st_cur = st_base + (size_t)(Lv & 1u) * A.level_pad;
+      const uint32_t* bits_prev = bits + ((Lv - 1) & 1u) * A.bit_words;
+      uint32_t* bits_cur = bits + (Lv & 1u) * A.bit_words;
+      for (uint32_t i = tid; i < A.bit_words; i += SW_THREADS) bits_cur[i] = 0u;
+      if (tid == 0) ctl[SC_ALIVE] = 0u, ctl[SC_PEND_N] = 0u, ctl[SC_Q_N] = 0u;
+      __syncthreads();
+
+      // ---- the pass over this depth
+      for (uint32_t base = 0; base < nch; base += SW_CHUNKS, ++round) {
+        uint32_t* const n_alive_ctr = &ctl[SC_CH_N0 + (round & 1u)];
+        if (tid == 0) ctl[SC_CH_N0 + ((round + 1u) & 1u)] = 0u;  // the other counter, for the next round
+        const uint32_t c = base + tid;
+        bool visit = false;
+        if (c < nch) {  // is any parent of this chunk's nodes alive?
+          const uint2 pr = __ldg(&G.chunk_par[coff + c]);
+          const uint32_t g0 = (pr.x - lo_prev) >> 5, g1 = (pr.y - lo_prev) >> 5;
+          for (uint32_t wd = g0 >> 5; wd <= (g1 >> 5) && !visit; ++wd) {
+            uint32_t b = bits_prev[wd];
+            if (wd == (g0 >> 5)) b &= 0xFFFFFFFFu << (g0 & 31u);
+            if (wd == (g1 >> 5)) b &= 0xFFFFFFFFu >> (31u - (g1 & 31u));
+            visit = b != 0u;
+          }
+        }
+        const uint32_t bal = __ballot_sync(FULL, visit);
+        uint32_t at = 0;
+        if (lane == 0 && bal) at = atomicAdd(n_alive_ctr, (uint32_t)__popc(bal));
+        at = __shfl_sync(FULL, at, 0);
+        if (visit) chunks[at + __popc(bal & ((1u << lane) - 1u))] = c;
+        __syncthreads();
+        const uint32_t n_alive = *n_alive_ctr;
+        for (uint32_t k = warp; k < n_alive; k += SW_WARPS) {
+          const uint32_t first = lo + chunks[k] * TRIE_CHUNK + lane;
+          uint32_t byte[SW_PER_LANE], par[SW_PER_LANE], ps[SW_PER_LANE];
+#pragma unroll
+          for (uint32_t u = 0; u < SW_PER_LANE; ++u) {
+            const uint32_t node = first + 32u * u;
+            const bool v = node < hi;
+            byte[u] = v ? __ldg(&G.node_byte[node]) : 0u;
+            par[u] = v ? __ldg(&G.parent[node]) - lo_prev : 0xFFFFFFFFu;
+          }
+#pragma unroll
+          for (uint32_t u = 0; u < SW_PER_LANE; ++u) {
+            ps[u] = ST_DEAD;
+            if (par[u] != 0xFFFFFFFFu && ((bits_prev[par[u] >> 10] >> ((par[u] >> 5) & 31u)) & 1u)) ps[u] = st_prev[par[u]];
+          }
+#pragma unroll
+          for (uint32_t u = 0; u < SW_PER_LANE; ++u) {
+            const uint32_t node = first + 32u * u;
+            const bool v = node < hi;
+            uint32_t t = ST_DEAD;
+            if (ps[u] != ST_DEAD) t = step_node(G, a, queue, ps[u], byte[u]);
+            if (v) st_cur[node - lo] = (uint16_t)t;
+            const bool alive = t != ST_DEAD, waits = t == ST_PENDING;
+            if (alive && !waits) set_tokens(G, mask, node);
+            const uint32_t wb = __ballot_sync(FULL, waits);
+            if (wb) {
+              uint32_t pa = 0;
+              if (lane == 0) pa = atomicAdd(&ctl[SC_PEND_N], (uint32_t)__popc(wb));
+              pa = __shfl_sync(FULL, pa, 0);
+              if (waits) pend[pa + __popc(wb & ((1u << lane) - 1u))] = node;
+            }
+            if (__ballot_sync(FULL, alive) && lane == 0) {
+              const uint32_t g = (node - lo) >> 5;
+              atomicOr(&bits_cur[g >> 5], 1u << (g & 31u));
+              ctl[SC_ALIVE] = 1u;
+            }
+          }
+        }
+        __syncthreads();
+      }
+
+      // ---- compute the queued transitions, settle the nodes that waited; again while some still wait
+      for (uint32_t rounds = 0;; ++rounds) {
+        const uint32_t nq = min(ctl[SC_Q_N], SW_QUEUE), np = ctl[SC_PEND_N];
+        if (nq == 0) break;
+        if (rounds > (1u << 16)) {  // cannot happen (every round settles at least one transition); never spin
+          if (tid == 0) ctl[SC_FAIL] = 1u;
+          break;
+        }
+        for (uint32_t i = warp; i < nq; i += SW_WARPS) {
+          const uint32_t ps = queue[i] >> 8, pb = queue[i] & 0xFFu;
+          uint32_t r = sw.compute(ps, pb);
+          if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
+            big_mode = true;
+            hset_clear_all(sw.w.hset, sw.w.hset_mask);
+            clear_nt(G, sw.w);
+            sw.w.cur = big;
+            sw.w.cur_cap = S.big_arena_items;
+            sw.cur_pow2 = S.big_arena_items;
+            sw.w.hset = big + S.big_arena_items;
+            sw.w.hset_mask = S.big_hset_slots - 1;
+            if (lane == 0) atomicAdd(&ctl[SC_BIG], 1u);
+            r = sw.compute(ps, pb);
+          }
+          if (r == T_FAIL) {  // a capacity was exceeded: the row's mask cannot be trusted
+            hset_clear_all(sw.w.hset, sw.w.hset_mask);
+            clear_nt(G, sw.w);
+            if (lane == 0) ctl[SC_FAIL] = 1u;
+            r = T_DEAD;  // lets the sweep go on
+          }
+          if (lane == 0) {
+            *reinterpret_cast<volatile uint16_t*>(a.trans(ps) + G.eq_of_byte[pb]) = (r == T_DEAD) ? T16_DEAD : (uint16_t)r;
+            atomicAdd(&ctl[SC_TRANS], 1u);
+          }
+        }
+        __syncthreads();
+        if (tid == 0) ctl[SC_Q_N] = 0u;
+        __syncthreads();
+        for (uint32_t i = tid; i < np; i += SW_THREADS) {
+          const uint32_t node = pend[i];
+          if (node == 0xFFFFFFFFu) continue;  // settled in an earlier round
+          const uint32_t ps = st_prev[__ldg(&G.parent[node]) - lo_prev];
+          const uint32_t t = step_node(G, a, queue, ps, __ldg(&G.node_byte[node]));
+          if (t == ST_PENDING) continue;
+          st_cur[node - lo] = (uint16_t)t;
+          if (t != ST_DEAD) set_tokens(G, mask, node);
+          pend[i] = 0xFFFFFFFFu;
+        }
+        __syncthreads();
+      }
+      const bool any_alive = ctl[SC_ALIVE] != 0u;
+      __syncthreads();  // everybody has read the flag before the next depth resets it
+      if (!any_alive) break;  // nothing survives this depth
+    }
+
+    // ---- the job's result
+    __syncthreads();
+    const bool failed = ctl[SC_FAIL] != 0u;
+    if (A.mask_in_smem) {
+      uint32_t* out = S.mask_rows + (size_t)S.row_mask[row] * G.Wm;
+      for (uint32_t i = tid; i < G.Wm; i += SW_THREADS) out[i] = mask_sm[i];
+    }
+    if (tid == 0) {
+      if (failed) {
+        atomicOr(&S.row_flags[row], ROW_BROKEN);
+        atomicExch(&S.counters[CNT_ERR], 1u);
+        stat_add(S, CNT_STAT_CAPERR, 1u);
+      }
+      stat_trans += ctl[SC_TRANS];
+      stat_states += min(ctl[SC_N_STATES], a.cap) - 1u;
+      if (ctl[SC_BIG]) stat_add(S, CNT_STAT_BIG, ctl[SC_BIG]);
+    }
+  }
+  if (big_mode) hset_clear_all(sw.w.hset, sw.w.hset_mask);
+  if (tid == 0) {
+    stat_add(S, CNT_STAT_TRANS, stat_trans);
+    stat_add(S, CNT_STAT_LOCAL, stat_states);
+  }
+}
+
+}  // namespace fmt
