@@ -81,7 +81,7 @@ enum : uint32_t {
 // below, so small automata (the common case) never leave the SM.
 // Record of a state (rec_words uint32):
 //   [0] first item (word offset: < sm_items shared memory, else sm_items + offset into `items`)
-//   [1] item count  [2] hash  [4..11] scannable bytes
+//   [1] item count  [2] hash of the kernel  [3] items of the kernel (they come first)  [4..11] scannable bytes
 //   [12 ..) one uint16 per byte class: T16_UNKNOWN, T16_PENDING (queued for computation),
 //           T16_DEAD or the next state's id
 struct AutoDev {
@@ -109,7 +109,7 @@ constexpr uint16_t T16_UNKNOWN = 0xFFFFu, T16_DEAD = 0xFFFEu, T16_PENDING = 0xFF
 constexpr uint32_t T_DEAD = 0xfffffffeu, T_FAIL = 0xfffffffdu;
 constexpr uint32_t ORIGIN_SELF = 0xFFFFu;
 constexpr uint32_t AUTO_MAX_STATES = 0xFF00u;  // ids stay below the uint16 marks above and, plus m, below ORIGIN_SELF
-constexpr uint32_t AR_ITEMS = 0, AR_N = 1, AR_HASH = 2, AR_SCAN = 4, AR_TRANS = 12;
+constexpr uint32_t AR_ITEMS = 0, AR_N = 1, AR_HASH = 2, AR_NK = 3, AR_SCAN = 4, AR_TRANS = 12;
 
 struct StateDev {
   uint32_t B;

@@ -162,53 +162,61 @@ __device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const War
 
 // Predict (Section 3.2) for all non-terminals collected in w.nt[0..Nw): append the start items of
 // every rule of every non-terminal in their closure, origin = cur_index.  These items are all new
-// (nothing else in the set has this origin), so no uniqueness check is needed.  Each lane expands
-// one non-terminal of the closure at a time; a warp scan gives every lane its place in cur.
+// (nothing else in the set has this origin), so no uniqueness check is needed.  One closure word
+// (32 non-terminals) per pass: a warp scan gives every lane the place of its non-terminal's items;
+// short lists are copied by their lane, long ones (alternations of many literals) by the whole warp.
 __device__ __forceinline__ void predict_into_cur(const GrammarDev& G, const WarpCtx& w, uint32_t cur_index) {
   const uint32_t lane = lane_id();
   const uint32_t Nw = G.Nw;
   uint32_t* ntmask = w.nt;
   uint32_t* clos = w.nt + Nw;
   __syncwarp();
-  for (uint32_t i = lane; i < Nw; i += 32) clos[i] = 0u;
-  __syncwarp();
-  for (uint32_t wi = 0; wi < Nw; ++wi) {
-    uint32_t bits = ntmask[wi];
-    while (bits) {
-      uint32_t y = wi * 32u + (uint32_t)(__ffs(bits) - 1);
-      bits &= bits - 1;
-      for (uint32_t i = lane; i < Nw; i += 32) clos[i] |= G.nt_closure[y * Nw + i];
+  for (uint32_t i = lane; i < Nw; i += 32) {  // each lane owns some words of the closure
+    uint32_t acc = 0u;
+    for (uint32_t wi = 0; wi < Nw; ++wi) {
+      uint32_t bits = ntmask[wi];
+      while (bits) {
+        const uint32_t y = wi * 32u + (uint32_t)(__ffs(bits) - 1);
+        bits &= bits - 1;
+        acc |= G.nt_closure[y * Nw + i];
+      }
     }
+    clos[i] = acc;
   }
   __syncwarp();
   uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
   bool over = false;
-  for (uint32_t wi = 0; wi < Nw && !over; ++wi) {
+  for (uint32_t wi = 0; wi < Nw; ++wi) {
     const uint32_t bits = clos[wi];
     if (bits == 0u) continue;  // (uniform) most words of the closure are empty
-    const uint32_t cnt = __popc(bits);
-    for (uint32_t base = 0; base < cnt && !over; base += 32) {
-      const uint32_t k = base + lane;
-      uint32_t lo = 0, len = 0;
-      if (k < cnt) {
-        const uint32_t z = wi * 32u + __fns(bits, 0, k + 1);
-        lo = G.direct_off[z];
-        len = G.direct_off[z + 1] - lo;
-      }
-      uint32_t incl = len;
-      for (int d = 1; d < 32; d <<= 1) {
-        uint32_t t = __shfl_up_sync(FULL, incl, d);
-        if ((int)lane >= d) incl += t;
-      }
-      const uint32_t total = __shfl_sync(FULL, incl, 31);
-      if (n + total > w.cur_cap) {
-        over = true;
-        break;
-      }
-      uint32_t at = n + incl - len;
-      for (uint32_t i = 0; i < len; ++i) w.cur[at + i] = (cur_index << 16) | (uint32_t)G.direct_items[lo + i];
-      n += total;
+    uint32_t lo = 0, len = 0;
+    if ((bits >> lane) & 1u) {
+      const uint32_t z = wi * 32u + lane;
+      lo = G.direct_off[z];
+      len = G.direct_off[z + 1] - lo;
     }
+    uint32_t incl = len;
+    for (int d = 1; d < 32; d <<= 1) {
+      uint32_t t = __shfl_up_sync(FULL, incl, d);
+      if ((int)lane >= d) incl += t;
+    }
+    const uint32_t total = __shfl_sync(FULL, incl, 31);
+    if (n + total > w.cur_cap) {
+      over = true;
+      break;
+    }
+    const uint32_t at = n + incl - len;
+    const bool is_long = len > 8u;
+    if (!is_long)
+      for (uint32_t i = 0; i < len; ++i) w.cur[at + i] = (cur_index << 16) | (uint32_t)G.direct_items[lo + i];
+    uint32_t longs = __ballot_sync(FULL, is_long);
+    while (longs) {
+      const int src = __ffs(longs) - 1;
+      longs &= longs - 1;
+      const uint32_t slo = __shfl_sync(FULL, lo, src), slen = __shfl_sync(FULL, len, src), sat = __shfl_sync(FULL, at, src);
+      for (uint32_t i = lane; i < slen; i += 32) w.cur[sat + i] = (cur_index << 16) | (uint32_t)G.direct_items[slo + i];
+    }
+    n += total;
   }
   __syncwarp();
   if (lane == 0) {
@@ -217,6 +225,18 @@ __device__ __forceinline__ void predict_into_cur(const GrammarDev& G, const Warp
   }
   for (uint32_t i = lane; i < Nw; i += 32) ntmask[i] = 0u;
   __syncwarp();
+}
+
+// Is `key` in the uniqueness hash?
+__device__ __forceinline__ bool hset_contains(const uint32_t* hset, uint32_t mask, uint32_t key) {
+  uint32_t h = mix32(key) & mask;
+  for (uint32_t probe = 0; probe <= mask; ++probe) {
+    const uint32_t v = hset[h];
+    if (v == key) return true;
+    if (v == EMPTY_SLOT) return false;
+    h = (h + 1) & mask;
+  }
+  return false;
 }
 
 // Copy the grammar's hot tables into shared memory (all threads of the block take part, the

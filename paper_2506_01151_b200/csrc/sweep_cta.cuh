@@ -127,18 +127,25 @@ struct CtaView {
   }
 };
 
-// The Earley step of one warp.
+// The Earley step of one warp.  Two forms of the same step (Section 3.2: scan, complete to a
+// fixpoint, predict): while the scanned and completed items ("kernel") number at most 32 they sit
+// one per lane and uniqueness is a matter of shuffles and ballots; larger sets go through the
+// hash-based primitives of earley_device.cuh.  Either way the predicted items are a function of
+// the kernel, so a set is looked up by its kernel alone (an order-independent hash, then an exact
+// comparison as sets) BEFORE anything is predicted, and a set already known costs no prediction.
+// A set's items are stored kernel first; nothing is sorted.
+constexpr uint32_t T_RETRY = 0xfffffffbu;  // the lane-resident form does not apply: take the general one
+
 struct SweepWarp {
   const GrammarDev& G;
   const StateDev& S;
   const CtaAuto& a;
   WarpCtx w;
-  uint32_t cur_pow2;  // capacity of w.cur (a power of two, for the sort)
   uint32_t* tmp8;     // shared
   uint32_t chunk_at = 0, chunk_left = 0;  // this warp's piece of the global item pool (lane 0's copy counts)
 
-  // A new set with the items w.cur[0..n): returns its id or T_FAIL.
-  __device__ uint32_t create_set(uint32_t n, uint32_t hash) {
+  // A new set with the items w.cur[0..n), the first nk of them its kernel: returns its id or T_FAIL.
+  __device__ uint32_t create_set(uint32_t n, uint32_t nk, uint32_t hash) {
     const uint32_t lane = lane_id();
     uint32_t id = T_FAIL, ioff = 0;
     if (lane == 0) {
@@ -175,6 +182,7 @@ struct SweepWarp {
       if (i == AR_ITEMS) v = ioff;
       else if (i == AR_N) v = n;
       else if (i == AR_HASH) v = hash;
+      else if (i == AR_NK) v = nk;
       else if (i >= AR_SCAN && i < AR_SCAN + 8) v = tmp8[i - AR_SCAN];
       else if (i >= AR_TRANS) v = 0xFFFFFFFFu;  // two T16_UNKNOWN
       rec[i] = v;
@@ -184,68 +192,196 @@ struct SweepWarp {
     return id;
   }
 
-  // Find or create the set whose items are w.cur[0..n) (sorted).  Returns its id or T_FAIL.  Sets
-  // entered by two warps at the same moment may, rarely, get two ids; the automaton stays correct.
-  __device__ uint32_t intern_set(uint32_t n, uint32_t hash) {
+  // The set whose kernel has nk items and this hash and consists of items for which `member`
+  // holds: its id, or T_FAIL if there is none.  member(x, valid) is called by all lanes.
+  template <class Member>
+  __device__ uint32_t lookup_set(uint32_t nk, uint32_t hash, Member member) {
     const uint32_t lane = lane_id();
-    uint32_t* table = a.sm_hash;
-    uint32_t mask = SW_HASH - 1u;
+    for (int t = 0; t < 2; ++t) {
+      if (t == 1 && !ld_volatile(&a.ctl[SC_GL_HASH])) break;
+      const uint32_t* table = t ? a.gl_hash : a.sm_hash;
+      const uint32_t mask = t ? a.gl_hash_mask : SW_HASH - 1u;
+      uint32_t slot = hash & mask;
+      for (uint32_t probe = 0; probe <= mask; ++probe) {
+        uint32_t v = 0;
+        if (lane == 0) v = ld_acquire_cta(&table[slot]);
+        v = __shfl_sync(FULL, v, 0);
+        if (v == 0) break;
+        if (same_set(v - 1u, nk, hash, member)) return v - 1u;
+        slot = (slot + 1u) & mask;
+      }
+    }
+    return T_FAIL;
+  }
+
+  // Is the set `sid` the one with this hash and a kernel of nk items for which `member` holds?
+  template <class Member>
+  __device__ __forceinline__ bool same_set(uint32_t sid, uint32_t nk, uint32_t hash, Member member) {
+    const uint32_t lane = lane_id();
+    const uint32_t* rec = a.rec(sid);
+    if (ld_volatile(rec + AR_HASH) != hash || ld_volatile(rec + AR_NK) != nk) return false;
+    const uint32_t* items = a.items_at(ld_volatile(rec + AR_ITEMS));
+    bool ok = true;
+    for (uint32_t base = 0; base < nk; base += 32) {
+      const bool valid = base + lane < nk;
+      const uint32_t x = valid ? ld_volatile(items + base + lane) : 0u;
+      ok = member(x, valid) && ok;
+    }
+    return __all_sync(FULL, ok);
+  }
+
+  // Enter the freshly created set `id` into the hash, unless an equal set got there first (several
+  // warps often reach the same new set at the same moment): returns the id to use.
+  template <class Member>
+  __device__ uint32_t insert_set(uint32_t id, uint32_t nk, uint32_t hash, Member member) {
+    const uint32_t lane = lane_id();
+    uint32_t use_gl = 0;
+    if (lane == 0) {
+      use_gl = ld_volatile(&a.ctl[SC_GL_HASH]);
+      if (!use_gl && atomicAdd(&a.ctl[SC_N_SMHASH], 1u) >= SW_HASH_MAX) {
+        atomicExch(&a.ctl[SC_GL_HASH], 1u);
+        use_gl = 1u;
+      }
+    }
+    use_gl = __shfl_sync(FULL, use_gl, 0);
+    uint32_t* table = use_gl ? a.gl_hash : a.sm_hash;
+    const uint32_t mask = use_gl ? a.gl_hash_mask : SW_HASH - 1u;
     uint32_t slot = hash & mask;
-    bool in_gl = false, room = false;
-    uint32_t my_id = T_FAIL;
-    for (uint32_t probe = 0; probe < 8192u; ++probe) {
-      uint32_t v = 0;
-      if (lane == 0) v = ld_acquire_cta(&table[slot]);
-      v = __shfl_sync(FULL, v, 0);
-      if (v == 0) {
-        if (!in_gl) {  // not in the shared-memory table: look in the overflow table, or reserve a place here
-          uint32_t go_gl = 0;
-          if (lane == 0) {
-            go_gl = ld_volatile(&a.ctl[SC_GL_HASH]);
-            if (!go_gl && !room) {
-              if (atomicAdd(&a.ctl[SC_N_SMHASH], 1u) >= SW_HASH_MAX) {
-                atomicExch(&a.ctl[SC_GL_HASH], 1u);
-                go_gl = 1u;
-              }
-            }
-          }
-          go_gl = __shfl_sync(FULL, go_gl, 0);
-          if (go_gl) {
-            in_gl = true;
-            table = a.gl_hash;
-            mask = a.gl_hash_mask;
-            slot = hash & mask;
-            continue;
-          }
-          room = true;
-        }
-        if (my_id == T_FAIL) {
-          my_id = create_set(n, hash);
-          if (my_id == T_FAIL) return T_FAIL;
-        }
-        uint32_t old = 0;
-        if (lane == 0) old = atomicCAS(&table[slot], 0u, my_id + 1u);
-        old = __shfl_sync(FULL, old, 0);
-        if (old == 0) return my_id;
-        v = old;
-      }
-      const uint32_t sid = v - 1u;
-      const uint32_t* rec = a.rec(sid);
-      bool same = (ld_volatile(rec + AR_HASH) == hash) && (ld_volatile(rec + AR_N) == n);
-      if (same) {
-        const uint32_t* items = a.items_at(ld_volatile(rec + AR_ITEMS));
-        for (uint32_t i = lane; i < n; i += 32)
-          if (ld_volatile(items + i) != w.cur[i]) same = false;
-      }
-      same = __all_sync(FULL, same);
-      if (same) return sid;
+    for (uint32_t probe = 0; probe <= mask; ++probe) {
+      uint32_t old = 0;
+      if (lane == 0) old = atomicCAS(&table[slot], 0u, id + 1u);
+      old = __shfl_sync(FULL, old, 0);
+      if (old == 0u) return id;
+      __threadfence_block();
+      if (same_set(old - 1u, nk, hash, member)) return old - 1u;
       slot = (slot + 1u) & mask;
     }
     return T_FAIL;
   }
 
-  // The transition of set `ps` on `byte`: T_DEAD, a set id, or T_FAIL when a capacity was exceeded.
-  __device__ uint32_t compute(uint32_t ps, uint32_t byte) {
+  // The kernel w.cur[0..nk) is new: predict, describe, store and enter the set.
+  template <class Member>
+  __device__ uint32_t finish_new(uint32_t nk, uint32_t hash, Member member) {
+    const uint32_t lane = lane_id();
+    __syncwarp();
+    if (lane == 0) w.ctr[W_NCUR] = nk, w.ctr[W_OVERFLOW] = 0u;
+    predict_into_cur(G, w, ORIGIN_SELF);
+    if (w.ctr[W_OVERFLOW]) return T_RETRY;
+    const uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
+    scannable_bytes(G, w.cur, n, tmp8);
+    const uint32_t id = create_set(n, nk, hash);
+    return id == T_FAIL ? T_FAIL : insert_set(id, nk, hash, member);
+  }
+
+  // (lane-resident form) The candidates c .. c + skip of the lanes with `v` set join cur[0..n)
+  // unless already there.  `mine` is cur[lane].  Returns the new count, above 32 when they do not fit.
+  __device__ __forceinline__ uint32_t append_small(uint32_t c, bool v, uint32_t skip, uint32_t n, uint32_t& mine) {
+    const uint32_t lane = lane_id();
+    const uint32_t maxskip = __reduce_max_sync(FULL, v ? skip : 0u);
+    for (uint32_t j = 0; j <= maxskip; ++j) {
+      const bool vj = v && j <= skip;
+      const uint32_t cj = c + j;
+      const uint32_t vm = __ballot_sync(FULL, vj);
+      if (!vm) continue;
+      bool keep = vj;
+      if (vj) keep = (uint32_t)(__ffs(__match_any_sync(vm, cj)) - 1) == lane;  // one of equal candidates
+      for (uint32_t i = 0; i < n; ++i)
+        if (__shfl_sync(FULL, mine, i) == cj) keep = false;
+      const uint32_t kb = __ballot_sync(FULL, keep);
+      const uint32_t nn = n + __popc(kb);
+      if (nn > 32u) return nn;
+      if (keep) w.cur[n + __popc(kb & ((1u << lane) - 1u))] = cj;
+      __syncwarp();
+      n = nn;
+      mine = lane < n ? w.cur[lane] : 0u;
+    }
+    return n;
+  }
+
+  __device__ uint32_t compute_small(uint32_t ps, uint32_t byte) {
+    const uint32_t lane = lane_id();
+    const uint32_t* pitems;
+    uint32_t plen;
+    CtaView view{a};
+    view(ps == 0 ? a.m - 1 : a.m + ps, pitems, plen);
+    const uint32_t self_code = a.m + ps;
+    uint32_t n = 0, mine = 0;
+    __syncwarp();
+    // ---- scan
+    for (uint32_t base = 0; base < plen; base += 32) {
+      const uint32_t k = base + lane;
+      uint32_t it = k < plen ? pitems[k] : 0u;
+      const uint32_t inf = k < plen ? G.info[it & 0xFFFFu] : 0u;
+      const bool hit = (inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte);
+      if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
+      const uint32_t skip = hit ? (G.info[(it + 1u) & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
+      if (__any_sync(FULL, hit)) n = append_small(it + 1u, hit, skip, n, mine);
+      if (n > 32u) return T_RETRY;
+    }
+    if (n == 0) return T_DEAD;
+    // ---- complete to a fixpoint: lanes [head, n) hold the items not looked at yet
+    uint32_t head = 0;
+    while (head < n) {
+      const bool have = lane >= head && lane < n;
+      const uint32_t inf = have ? G.info[mine & 0xFFFFu] : 0u;
+      const uint32_t kind = inf >> INFO_KIND_SHIFT;
+      if (have && kind == KIND_NT) {
+        const uint32_t y = inf & INFO_ARG_MASK;
+        atomicOr(&w.nt[y >> 5], 1u << (y & 31u));
+      }
+      uint32_t bal = __ballot_sync(FULL, have && kind == KIND_END && (mine >> 16) != ORIGIN_SELF);
+      const uint32_t it = mine;
+      head = n;
+      while (bal) {
+        const int src = __ffs(bal) - 1;
+        bal &= bal - 1;
+        const uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, src);
+        const uint32_t o = __shfl_sync(FULL, it >> 16, src);
+        const uint32_t* sp;
+        uint32_t sl;
+        view(o, sp, sl);
+        for (uint32_t base = 0; base < sl; base += 32) {
+          const uint32_t k = base + lane;
+          const uint32_t wi = k < sl ? sp[k] : 0u;
+          const uint32_t winf = k < sl ? G.info[wi & 0xFFFFu] : 0u;
+          const bool match = (winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X;
+          const uint32_t cand = view.fix(wi, o) + 1u;
+          const uint32_t skip = match ? (G.info[cand & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
+          if (__any_sync(FULL, match)) n = append_small(cand, match, skip, n, mine);
+          if (n > 32u) {
+            clear_nt(G, w);
+            return T_RETRY;
+          }
+        }
+      }
+    }
+    // ---- the kernel: what is left when the completed items go
+    const bool keep = lane < n && (G.info[mine & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
+    const uint32_t kb = __ballot_sync(FULL, keep);
+    const uint32_t nk = __popc(kb);
+    uint32_t h = keep ? mix32(mine) : 0u;
+    for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
+    h = mix32(h + nk * 0x9E3779B9u);
+    __syncwarp();
+    if (keep) w.cur[__popc(kb & ((1u << lane) - 1u))] = mine;
+    __syncwarp();
+    mine = lane < nk ? w.cur[lane] : 0u;
+    auto member = [&](uint32_t x, bool valid) {  // the kernel sits one item per lane
+      bool found = false;
+      for (uint32_t i = 0; i < nk; ++i)
+        if (__shfl_sync(FULL, mine, i) == x) found = true;
+      return found || !valid;
+    };
+    const uint32_t id = lookup_set(nk, h, member);
+    if (id != T_FAIL) {
+      clear_nt(G, w);
+      return id;
+    }
+    return finish_new(nk, h, member);
+  }
+
+  // The general form, for sets of any size (w.cur may be the warp's large area).
+  __device__ uint32_t compute_general(uint32_t ps, uint32_t byte) {
     const uint32_t lane = lane_id();
     const uint32_t* pitems;
     uint32_t plen;
@@ -264,12 +400,11 @@ struct SweepWarp {
       }
     }
     __syncwarp();
-    uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
     if (w.ctr[W_OVERFLOW]) {
       hset_clear_all(w.hset, w.hset_mask);
       return T_FAIL;
     }
-    if (n == 0) return T_DEAD;
+    if (w.ctr[W_NCUR] == 0u) return T_DEAD;
     complete_fixpoint(G, w, view, ORIGIN_SELF, 0u);
     const uint32_t hashed = min(w.ctr[W_NCUR], w.cur_cap);
     if (w.ctr[W_OVERFLOW]) {
@@ -277,16 +412,31 @@ struct SweepWarp {
       clear_nt(G, w);
       return T_FAIL;
     }
-    hset_clear_items(w, hashed);
-    predict_into_cur(G, w, ORIGIN_SELF);
-    if (w.ctr[W_OVERFLOW]) return T_FAIL;
-    n = drop_completed(G, w, min(w.ctr[W_NCUR], w.cur_cap));
-    sort_items(w.cur, n, cur_pow2);
-    uint32_t h = 0x9E3779B9u ^ n;
-    for (uint32_t i = lane; i < n; i += 32) h += mix32(w.cur[i] ^ (i * 0x85EBCA77u));
+    // the kernel: the items that are not completed; all of cur[0..hashed) are in the uniqueness hash
+    uint32_t nk = 0, h = 0;
+    for (uint32_t base = 0; base < hashed; base += 32) {
+      const uint32_t i = base + lane;
+      const uint32_t it = i < hashed ? w.cur[i] : 0u;
+      const bool keep = i < hashed && (G.info[it & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
+      if (keep) h += mix32(it);
+      nk += __popc(__ballot_sync(FULL, keep));
+    }
     for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
-    scannable_bytes(G, w.cur, n, tmp8);
-    return intern_set(n, h);
+    h = mix32(h + nk * 0x9E3779B9u);
+    const uint32_t id = lookup_set(nk, h, [&](uint32_t x, bool valid) { return !valid || hset_contains(w.hset, w.hset_mask, x); });
+    hset_clear_items(w, hashed);
+    if (id != T_FAIL) {
+      clear_nt(G, w);
+      return id;
+    }
+    drop_completed(G, w, hashed);
+    // the kernel is cur[0..nk) now and no longer in the hash: a set met while entering this one is compared item by item
+    const uint32_t r = finish_new(nk, h, [&](uint32_t x, bool valid) {
+      bool found = !valid;
+      for (uint32_t i = 0; i < nk && !found; ++i) found = w.cur[i] == x;
+      return found;
+    });
+    return r == T_RETRY ? T_FAIL : r;
   }
 };
 
@@ -358,7 +508,6 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
   SweepWarp sw{G, S, a};
   sw.w.cur = mine;
   sw.w.cur_cap = SW_CUR;
-  sw.cur_pow2 = SW_CUR;
   sw.w.hset = mine + SW_CUR;
   sw.w.hset_mask = SW_HSET - 1;
   sw.w.nt = sw.w.hset + SW_HSET;
@@ -509,18 +658,18 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
         }
         for (uint32_t i = warp; i < nq; i += SW_WARPS) {
           const uint32_t ps = queue[i] >> 8, pb = queue[i] & 0xFFu;
-          uint32_t r = sw.compute(ps, pb);
+          uint32_t r = big_mode ? T_RETRY : sw.compute_small(ps, pb);
+          if (r == T_RETRY) r = sw.compute_general(ps, pb);
           if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
             big_mode = true;
             hset_clear_all(sw.w.hset, sw.w.hset_mask);
             clear_nt(G, sw.w);
             sw.w.cur = big;
             sw.w.cur_cap = S.big_arena_items;
-            sw.cur_pow2 = S.big_arena_items;
             sw.w.hset = big + S.big_arena_items;
             sw.w.hset_mask = S.big_hset_slots - 1;
             if (lane == 0) atomicAdd(&ctl[SC_BIG], 1u);
-            r = sw.compute(ps, pb);
+            r = sw.compute_general(ps, pb);
           }
           if (r == T_FAIL) {  // a capacity was exceeded: the row's mask cannot be trusted
             hset_clear_all(sw.w.hset, sw.w.hset_mask);
