@@ -48,6 +48,7 @@ enum : uint32_t {
   SC_TRANS,          // transitions computed (statistics)
   SC_JOB,            // the job in hand
   SC_BIG,            // warps that switched to their large scratch (statistics)
+  SC_AGAIN,          // some node still waits after this round
   SC_TOTAL = 16
 };
 
@@ -440,10 +441,130 @@ struct SweepWarp {
   }
 };
 
+// ---- the Earley step of one THREAD, for the commonest transition there is: along the bytes of a
+// literal, where a set of a few items, each with a terminal after the dot, scans into a set of the
+// same kind.  Nothing completes and nothing is predicted, so the new set is just the scanned
+// items; the thread that claimed the transition computes it on the spot and its node needs no
+// second visit.  Anything else (more than TS_MAX items, an item that ends or meets a non-terminal)
+// is left to the warps.  Sets are entered with the same hash and the same compare-on-conflict
+// protocol as the warps use, so both kinds of step find each other's sets.
+constexpr uint32_t TS_MAX = 6;
+constexpr uint32_t TS_WARP = 0xfffffffau;  // not a case for a single thread
+
+__device__ __forceinline__ bool ts_same(const CtaAuto& a, uint32_t sid, const uint32_t (&out)[TS_MAX], uint32_t cnt, uint32_t h) {
+  const uint32_t* rec = a.rec(sid);
+  if (ld_volatile(rec + AR_HASH) != h || ld_volatile(rec + AR_NK) != cnt) return false;
+  const uint32_t* items = a.items_at(ld_volatile(rec + AR_ITEMS));
+  bool same = true;
+#pragma unroll
+  for (uint32_t i = 0; i < TS_MAX; ++i) {
+    if (i < cnt) {
+      const uint32_t x = ld_volatile(items + i);
+      bool found = false;
+#pragma unroll
+      for (uint32_t k = 0; k < TS_MAX; ++k) found |= (k < cnt && out[k] == x);
+      same &= found;
+    }
+  }
+  return same;
+}
+
+__device__ uint32_t thread_step(const GrammarDev& G, const StateDev& S, const CtaAuto& a, uint32_t ps, uint32_t byte) {
+  const uint32_t* pitems;
+  uint32_t plen;
+  CtaView view{a};
+  view(ps == 0 ? a.m - 1 : a.m + ps, pitems, plen);
+  if (plen > TS_MAX) return TS_WARP;
+  const uint32_t self_code = a.m + ps;
+  uint32_t out[TS_MAX];
+  uint32_t scan[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) scan[i] = 0u;
+  uint32_t cnt = 0, hsum = 0;
+#pragma unroll
+  for (uint32_t k = 0; k < TS_MAX; ++k) {
+    out[k] = 0u;
+    if (k < plen) {
+      uint32_t it = pitems[k];
+      const uint32_t inf = G.info[it & 0xFFFFu];
+      if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) {
+        if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
+        const uint32_t c = it + 1u;
+        const uint32_t cinf = G.info[c & 0xFFFFu];
+        if ((cinf >> INFO_KIND_SHIFT) != KIND_TERM) return TS_WARP;
+        const uint4* cb = reinterpret_cast<const uint4*>(G.class_bits + (cinf & INFO_ARG_MASK) * 8u);
+        const uint4 x = cb[0], y = cb[1];
+        scan[0] |= x.x, scan[1] |= x.y, scan[2] |= x.z, scan[3] |= x.w;
+        scan[4] |= y.x, scan[5] |= y.y, scan[6] |= y.z, scan[7] |= y.w;
+#pragma unroll
+        for (uint32_t q = 0; q < TS_MAX; ++q)
+          if (q == cnt) out[q] = c;
+        ++cnt;
+        hsum += mix32(c);
+      }
+    }
+  }
+  if (cnt == 0) return T_DEAD;
+  const uint32_t h = mix32(hsum + cnt * 0x9E3779B9u);
+  // ---- known already?
+  for (int t = 0; t < 2; ++t) {
+    if (t == 1 && !ld_volatile(&a.ctl[SC_GL_HASH])) break;
+    const uint32_t* table = t ? a.gl_hash : a.sm_hash;
+    const uint32_t mask = t ? a.gl_hash_mask : SW_HASH - 1u;
+    uint32_t slot = h & mask;
+    for (uint32_t probe = 0; probe <= mask; ++probe) {
+      const uint32_t v = ld_acquire_cta(&table[slot]);
+      if (v == 0) break;
+      if (ts_same(a, v - 1u, out, cnt, h)) return v - 1u;
+      slot = (slot + 1u) & mask;
+    }
+  }
+  // ---- a new set
+  const uint32_t id = atomicAdd(&a.ctl[SC_N_STATES], 1u);
+  if (id >= a.cap) return T_FAIL;
+  uint32_t ioff;
+  {
+    const uint32_t at = (ld_volatile(&a.ctl[SC_ITEMS_TOP]) < a.sm_items) ? atomicAdd(&a.ctl[SC_ITEMS_TOP], cnt) : a.sm_items;
+    if (at < a.sm_items && cnt <= a.sm_items - at) {
+      ioff = at;
+    } else {
+      const uint32_t g = atomicAdd(&S.counters[CNT_AUTO_ITEMS], cnt);
+      if (g > S.au.items_cap || cnt > S.au.items_cap - g) return T_FAIL;
+      ioff = a.sm_items + g;
+    }
+  }
+  uint32_t* items = a.items_at(ioff);
+#pragma unroll
+  for (uint32_t i = 0; i < TS_MAX; ++i)
+    if (i < cnt) items[i] = out[i];
+  uint32_t* rec = a.rec(id);
+  rec[AR_ITEMS] = ioff, rec[AR_N] = cnt, rec[AR_HASH] = h, rec[AR_NK] = cnt;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) rec[AR_SCAN + i] = scan[i];
+  for (uint32_t i = AR_TRANS; i < a.rec_words; ++i) rec[i] = 0xFFFFFFFFu;
+  __threadfence_block();
+  uint32_t use_gl = ld_volatile(&a.ctl[SC_GL_HASH]);
+  if (!use_gl && atomicAdd(&a.ctl[SC_N_SMHASH], 1u) >= SW_HASH_MAX) {
+    atomicExch(&a.ctl[SC_GL_HASH], 1u);
+    use_gl = 1u;
+  }
+  uint32_t* table = use_gl ? a.gl_hash : a.sm_hash;
+  const uint32_t mask = use_gl ? a.gl_hash_mask : SW_HASH - 1u;
+  uint32_t slot = h & mask;
+  for (uint32_t probe = 0; probe <= mask; ++probe) {
+    const uint32_t old = atomicCAS(&table[slot], 0u, id + 1u);
+    if (old == 0u) return id;
+    __threadfence_block();
+    if (ts_same(a, old - 1u, out, cnt, h)) return old - 1u;
+    slot = (slot + 1u) & mask;
+  }
+  return T_FAIL;
+}
+
 // The state a node reaches from parent state `ps` on `byte`: ST_DEAD, ST_PENDING (the transition
 // is not known yet: it has been queued, by this thread if nobody did before) or the state's id.
-__device__ __forceinline__ uint32_t step_node(const GrammarDev& G, const CtaAuto& a, uint32_t* queue, uint32_t ps,
-                                              uint32_t byte) {
+__device__ __forceinline__ uint32_t step_node(const GrammarDev& G, const StateDev& S, const CtaAuto& a, uint32_t* queue,
+                                              uint32_t ps, uint32_t byte) {
   const uint32_t* rec = a.rec(ps);
   // one 256-bit test rejects most bytes without touching the transition table
   if (!((rec[AR_SCAN + (byte >> 5)] >> (byte & 31u)) & 1u)) return ST_DEAD;
@@ -451,7 +572,14 @@ __device__ __forceinline__ uint32_t step_node(const GrammarDev& G, const CtaAuto
   uint32_t t = *reinterpret_cast<volatile uint16_t*>(tr);
   if (t == T16_UNKNOWN) {
     t = atomicCAS(tr, (unsigned short)T16_UNKNOWN, (unsigned short)T16_PENDING);
-    if (t == T16_UNKNOWN) {  // ours to queue
+    if (t == T16_UNKNOWN) {  // ours: compute it here if it is a step along a literal, else queue it for a warp
+      uint32_t r = thread_step(G, S, a, ps, byte);
+      if (r != TS_WARP) {
+        if (r == T_FAIL) a.ctl[SC_FAIL] = 1u, r = T_DEAD;
+        atomicAdd(&a.ctl[SC_TRANS], 1u);
+        *reinterpret_cast<volatile uint16_t*>(tr) = (r == T_DEAD) ? T16_DEAD : (uint16_t)r;
+        return (r == T_DEAD) ? (uint32_t)ST_DEAD : r;
+      }
       const uint32_t at = atomicAdd(&a.ctl[SC_Q_N], 1u);
       if (at < SW_QUEUE) queue[at] = (ps << 8) | byte;
       else *reinterpret_cast<volatile uint16_t*>(tr) = T16_UNKNOWN;  // no room in this round: somebody claims it again in the next
@@ -627,7 +755,7 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
             const uint32_t node = first + 32u * u;
             const bool v = node < hi;
             uint32_t t = ST_DEAD;
-            if (ps[u] != ST_DEAD) t = step_node(G, a, queue, ps[u], byte[u]);
+            if (ps[u] != ST_DEAD) t = step_node(G, S, a, queue, ps[u], byte[u]);
             if (v) st_cur[node - lo] = (uint16_t)t;
             const bool alive = t != ST_DEAD, waits = t == ST_PENDING;
             if (alive && !waits) set_tokens(G, mask, node);
@@ -651,7 +779,8 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
       // ---- compute the queued transitions, settle the nodes that waited; again while some still wait
       for (uint32_t rounds = 0;; ++rounds) {
         const uint32_t nq = min(ctl[SC_Q_N], SW_QUEUE), np = ctl[SC_PEND_N];
-        if (nq == 0) break;
+        // (nodes may wait although nothing is queued: a thread computed their transition meanwhile)
+        if (nq == 0 && !(rounds == 0 ? np > 0 : ctl[SC_AGAIN] != 0u)) break;
         if (rounds > (1u << 16)) {  // cannot happen (every round settles at least one transition); never spin
           if (tid == 0) ctl[SC_FAIL] = 1u;
           break;
@@ -683,14 +812,17 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
           }
         }
         __syncthreads();
-        if (tid == 0) ctl[SC_Q_N] = 0u;
+        if (tid == 0) ctl[SC_Q_N] = 0u, ctl[SC_AGAIN] = 0u;
         __syncthreads();
         for (uint32_t i = tid; i < np; i += SW_THREADS) {
           const uint32_t node = pend[i];
           if (node == 0xFFFFFFFFu) continue;  // settled in an earlier round
           const uint32_t ps = st_prev[__ldg(&G.parent[node]) - lo_prev];
-          const uint32_t t = step_node(G, a, queue, ps, __ldg(&G.node_byte[node]));
-          if (t == ST_PENDING) continue;
+          const uint32_t t = step_node(G, S, a, queue, ps, __ldg(&G.node_byte[node]));
+          if (t == ST_PENDING) {
+            ctl[SC_AGAIN] = 1u;
+            continue;
+          }
           st_cur[node - lo] = (uint16_t)t;
           if (t != ST_DEAD) set_tokens(G, mask, node);
           pend[i] = 0xFFFFFFFFu;
