@@ -138,8 +138,6 @@ fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out);
  *          9 tok_node [V] u32 (node where a token ends, 0xFFFFFFFF if it has no bytes)
  *         10 byte class of each byte [256] u8
  *         11 node_tok [T] u32: the token ending at a node, 0xFFFFFFFF none, 0xFFFFFFFE several (see tok_off)
- *         12 chunk_par [chunks][2] u32: first and last parent of each block of 128 consecutive nodes of
- *            one trie depth         13 chunk offsets [depth+2] u32: blocks of depth L are [13][L]..[13][L+1]-1
  * Writes min(cap_bytes, size) bytes to `out` (may be NULL) and the full size to *size_bytes.
  */
 fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, size_t cap_bytes, size_t* size_bytes);

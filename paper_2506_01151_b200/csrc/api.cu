@@ -191,12 +191,7 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
     UP(node_tok);
     UP(tok_off);
     UP(tok_ids);
-    UP(lvl_chunk_off);
-    {
-      const uint32_t* cp = nullptr;
-      if (e == cudaSuccess) e = g->bufs.upload(h.chunk_par, &cp);
-      d.chunk_par = reinterpret_cast<const uint2*>(cp);
-    }
+    UP(child_off);
     d.max_level = h.max_level;
     UP(vocab_off);
     UP(vocab_bytes);
@@ -250,8 +245,6 @@ fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, si
     case 9: src = h.tok_node.data(), n = h.tok_node.size() * 4; break;
     case 10: src = h.eq_of_byte.data(), n = 256; break;
     case 11: src = h.node_tok.data(), n = h.node_tok.size() * 4; break;
-    case 12: src = h.chunk_par.data(), n = h.chunk_par.size() * 4; break;
-    case 13: src = h.lvl_chunk_off.data(), n = h.lvl_chunk_off.size() * 4; break;
     default: return fail(FMT_ERR_INVALID_ARG, "unknown table");
   }
   *size_bytes = n;
@@ -324,8 +317,7 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(au.recs, (size_t)au.grid * (au.cap - au.sm_states) * au.rec_words, 0);
   AL(au.hash, (size_t)au.grid * hs, 0);
   AL(au.items, au.items_cap, 0);
-  AL(au.st, (size_t)au.grid * 2u * au.level_pad, 0xFF);
-  AL(au.pend, (size_t)au.grid * au.level_pad, 0);
+  AL(au.front, (size_t)au.grid * 3u * au.level_pad, 0);
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);

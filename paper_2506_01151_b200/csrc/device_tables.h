@@ -30,8 +30,7 @@ struct GrammarDev {
   const uint32_t* node_tok;      // [T] token ending at the node, NODE_TOK_NONE or NODE_TOK_MANY
   const uint32_t* tok_off;       // [T+1] \ all tokens ending at a node (needed for NODE_TOK_MANY only)
   const uint32_t* tok_ids;       //       /
-  const uint2* chunk_par;        // [chunks] first and last parent of each chunk of TRIE_CHUNK nodes
-  const uint32_t* lvl_chunk_off; // [depth+2]
+  const uint32_t* child_off;     // [T+1] children of node n are nodes child_off[n] .. child_off[n+1]-1
   uint32_t max_level;            // nodes of the most populous depth
   const uint32_t* vocab_off;     // [V+1]
   const uint8_t* vocab_bytes;
@@ -92,7 +91,6 @@ struct AutoDev {
   uint32_t chart_sm_words;  // a base chart up to this many words is staged in shared memory
   uint32_t mask_in_smem;    // 1: the mask row is assembled in shared memory
   uint32_t tables_in_smem;  // 1: the grammar's hot tables are staged in shared memory
-  uint32_t bit_words;       // words of one "32 nodes alive" bitmap over a trie depth
   uint32_t smem_bytes;      // dynamic shared memory of the sweep kernel
   uint32_t grid;            // CTAs of the sweep; the per-CTA areas below are sized for it
   uint32_t level_pad;       // entries of one per-depth buffer (>= max_level)
@@ -101,10 +99,10 @@ struct AutoDev {
   uint32_t* recs;           // [grid][cap - sm_states][rec_words]
   uint32_t* hash;           // [grid][gl_hash_mask + 1] id + 1 or 0; all zero between jobs
   uint32_t* items;          // [items_cap]
-  uint16_t* st;             // [grid][2][level_pad] state reached at every node of the previous / current depth
-  uint32_t* pend;           // [grid][level_pad] nodes of the current depth that wait for a transition
+  uint2* front;             // [grid][3][level_pad] (node, set) lists beyond their shared-memory part: the alive
+                            // nodes of the current and of the next depth, and the nodes that wait for a transition
 };
-constexpr uint16_t ST_DEAD = 0xFFFFu, ST_PENDING = 0xFFFEu;
+constexpr uint16_t ST_DEAD = 0xFFFFu;
 constexpr uint16_t T16_UNKNOWN = 0xFFFFu, T16_DEAD = 0xFFFEu, T16_PENDING = 0xFFFDu;
 constexpr uint32_t T_DEAD = 0xfffffffeu, T_FAIL = 0xfffffffdu;
 constexpr uint32_t ORIGIN_SELF = 0xFFFFu;

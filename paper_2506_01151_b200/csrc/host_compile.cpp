@@ -588,22 +588,8 @@ void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t 
       if (cnt == 1) out.node_tok[n] = out.tok_ids[out.tok_off[n]];
       else if (cnt > 1) out.node_tok[n] = NODE_TOK_MANY;
     }
-  // per depth, chunks of TRIE_CHUNK consecutive nodes with the range of their parents: a chunk
-  // none of whose parents is alive needs no visit
-  out.lvl_chunk_off.assign(out.depth + 2, 0);
-  out.chunk_par.clear();
   out.max_level = 1;
-  for (uint32_t L = 0; L <= out.depth; ++L) {
-    out.lvl_chunk_off[L] = (uint32_t)(out.chunk_par.size() / 2);
-    const uint32_t lo = out.lvl_off[L], hi = out.lvl_off[L + 1];
-    out.max_level = std::max(out.max_level, hi - lo);
-    for (uint32_t a = lo; a < hi; a += TRIE_CHUNK) {
-      const uint32_t b = std::min(hi, a + TRIE_CHUNK);
-      out.chunk_par.push_back(out.parent[a]);
-      out.chunk_par.push_back(out.parent[b - 1]);
-    }
-  }
-  out.lvl_chunk_off[out.depth + 1] = (uint32_t)(out.chunk_par.size() / 2);
+  for (uint32_t L = 0; L <= out.depth; ++L) out.max_level = std::max(out.max_level, out.lvl_off[L + 1] - out.lvl_off[L]);
 }
 
 }  // namespace fmt

@@ -473,12 +473,11 @@ void sweep_plan(const GrammarDev& G, AutoDev& A) {
   A.mask_in_smem = G.Wm * 4u <= 48u * 1024u ? 1u : 0u;
   A.chart_sm_words = SW_CHART_SM;
   A.level_pad = (G.max_level + 63u) & ~63u;
-  A.bit_words = (A.level_pad / 32u + 31u) / 32u + 1u;
   A.sm_states = 0;
   A.sm_items = 0;
   const uint32_t budget = SW_SMEM_BUDGET / 4u;
   uint32_t fixed = sweep_smem(G, A).total;
-  if (fixed + 4096u > budget && A.mask_in_smem) {  // a huge trie depth: give the room to the bitmaps
+  if (fixed + 4096u > budget && A.mask_in_smem) {  // a huge vocabulary: assemble the mask row in global memory
     A.mask_in_smem = 0;
     fixed = sweep_smem(G, A).total;
   }

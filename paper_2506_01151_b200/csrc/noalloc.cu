@@ -18,7 +18,7 @@ namespace {
 using namespace fmt;
 
 constexpr uint32_t NA_MAX = FMT_NOALLOC_MAX_CHARTS;
-constexpr uint32_t NA_GRID = 16;            // CTAs of the sweep, one chart at a time each
+constexpr uint32_t NA_GRID = 8;             // CTAs of the sweep, one chart at a time each
 constexpr uint32_t NA_WARPS_PER_CTA = 16;
 constexpr uint32_t NA_ARENA_ITEMS = 8192;   // per-warp overflow area for Earley sets (items)
 constexpr uint32_t NA_HSET_SLOTS = 2048;    // per-warp overflow uniqueness hash
@@ -37,21 +37,20 @@ constexpr size_t NA_BIG_WORDS = NA_WARPS * (NA_ARENA_ITEMS + NA_HSET_SLOTS);
 constexpr uint32_t NA_REC_WORDS_PER_CTA = 65536;
 constexpr uint32_t NA_HASH_SLOTS = 8192;
 constexpr uint32_t NA_ITEM_WORDS = 2u << 20;
-// per CTA and trie depth: the Earley set reached at every node of the previous and the current depth
-// (uint16) and the list of nodes that wait for a transition (uint32)
+// per CTA three lists of (trie node, Earley set) pairs of up to one trie depth each: the alive nodes of
+// the current and of the next depth and the nodes that wait for a transition
 constexpr uint32_t NA_LEVEL_MAX = 128u << 10;
 constexpr size_t NA_OFF_BIG = NA_HEADER_WORDS;
 constexpr size_t NA_OFF_RECS = NA_OFF_BIG + NA_BIG_WORDS;
 constexpr size_t NA_OFF_HASH = NA_OFF_RECS + (size_t)NA_GRID * NA_REC_WORDS_PER_CTA;
 constexpr size_t NA_OFF_ITEMS = NA_OFF_HASH + (size_t)NA_GRID * NA_HASH_SLOTS;
-constexpr size_t NA_OFF_ST = NA_OFF_ITEMS + NA_ITEM_WORDS;
-constexpr size_t NA_OFF_PEND = NA_OFF_ST + (size_t)NA_GRID * NA_LEVEL_MAX;  // 2 x NA_LEVEL_MAX uint16 per CTA
-constexpr size_t NA_WORDS = NA_OFF_PEND + (size_t)NA_GRID * NA_LEVEL_MAX;
+constexpr size_t NA_OFF_FRONT = NA_OFF_ITEMS + NA_ITEM_WORDS;  // 8-byte aligned: all sizes above are even
+constexpr size_t NA_WORDS = NA_OFF_FRONT + (size_t)NA_GRID * 3u * 2u * NA_LEVEL_MAX;
 static_assert(CNT_TOTAL <= NA_OFF_JOBS, "the counters overlap the job list");
 static_assert(NA_OFF_BAD + NA_MAX <= NA_HEADER_WORDS, "header too small");
 static_assert((NA_OFF_CHART % 2) == 0, "64-bit offsets must be 8-byte aligned");
 
-// ~39 MB, held by every GPU that loads the library until the process exits
+// ~41 MB, held by every GPU that loads the library until the process exits
 static __device__ __align__(256) uint32_t g_noalloc_scratch[NA_WORDS];
 
 struct Offsets {
@@ -181,8 +180,7 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   S.au.recs = scratch + NA_OFF_RECS;
   S.au.hash = scratch + NA_OFF_HASH;
   S.au.items = scratch + NA_OFF_ITEMS;
-  S.au.st = reinterpret_cast<uint16_t*>(scratch + NA_OFF_ST);
-  S.au.pend = scratch + NA_OFF_PEND;
+  S.au.front = reinterpret_cast<uint2*>(scratch + NA_OFF_FRONT);
   cudaStream_t st = (cudaStream_t)stream;
   noalloc_prepare_kernel<<<256, 256, 0, st>>>(*G, S, scratch, charts_dev, off, n, mask_dev);
   noalloc_jobs_kernel<<<1, 32, 0, st>>>(S, scratch, n);

@@ -3,19 +3,21 @@
 // For its job the CTA answers, for every trie node, "is the Earley set reached by this node's bytes
 // non-empty?" (Sections 3.3 and 4.1: a token is valid iff every Earley set along its bytes stays
 // non-empty).  Sets are hash-consed per job (AutoDev): a transition (set, byte class) is computed
-// once, with the warp-cooperative scan / complete / predict of earley_device.cuh, and every other
-// node that needs it reads it from the set's record.  The automaton (records, items, hash), the
-// job's base chart, the grammar's hot tables and the mask row under construction live in the CTA's
-// shared memory; only automata that outgrow it spill into the CTA's slice of global memory.
+// once, and every other node that needs it reads it from the set's record.  The automaton (records,
+// items, hash), the job's base chart, the grammar's hot tables and the mask row under construction
+// live in the CTA's shared memory; only automata that outgrow it spill into the CTA's slice of
+// global memory.
 //
-// The trie is processed one depth at a time, one THREAD per node: st[node] =
-// transition(st[parent], byte).  Nodes are numbered breadth first, so a depth is a contiguous
-// range, the children of consecutive parents are consecutive, and whole chunks of TRIE_CHUNK nodes
-// whose parents are all dead are skipped after one look at a bitmap ("some node of this group of
-// 32 is alive").  A transition nobody has computed yet is claimed by the first thread that meets
-// it and queued; after the pass the warps take the queued transitions, one each, then the nodes
-// that waited are settled.  Only __syncthreads() separates the phases: nothing waits on another
-// CTA, and jobs are handed out through an atomic ticket.
+// The trie is explored breadth first over the ALIVE nodes only: the frontier of a depth is a list of
+// (node, Earley set) pairs; a warp takes some consecutive entries, lays their children out side by
+// side (nodes are numbered breadth first, so the children of a node are consecutive) and gives each
+// lane one child: next set = transition(parent's set, child's byte).  A transition nobody has
+// computed yet belongs to the lane that claims it first: a step along a literal it takes on the
+// spot (thread_step); anything else it queues for the warps (SweepWarp), which take the queued
+// transitions, one each, once the depth has been laid out.  A child whose transition is queued or
+// claimed by somebody else goes on a retry list, settled right after.  Only __syncthreads()
+// separates the phases: nothing waits on another CTA or spins, and jobs are handed out through an
+// atomic ticket.
 #pragma once
 #include "chart_step.cuh"
 
@@ -25,36 +27,36 @@ constexpr int SW_WARPS = 16;
 constexpr int SW_THREADS = SW_WARPS * 32;
 constexpr uint32_t SW_CUR = 256;        // items of a set under construction per warp (fast mode, power of two)
 constexpr uint32_t SW_HSET = 512;       // uniqueness hash slots per warp (fast mode)
-constexpr uint32_t SW_QUEUE = 512;      // transitions queued per round
+constexpr uint32_t SW_QUEUE = 512;      // transitions queued for the warps per round
 constexpr uint32_t SW_HASH = 4096;      // slots of the shared-memory hash of Earley sets
 constexpr uint32_t SW_HASH_MAX = 2560;  // sets it may hold; later ones go to the CTA's overflow hash
-constexpr uint32_t SW_CHUNKS = SW_THREADS;  // chunks tested per round, one per thread
+constexpr uint32_t SW_FRONT_SM = 256;   // entries of each frontier list kept in shared memory
 constexpr uint32_t SW_SMEM_BUDGET = 227u * 1024u;
 constexpr uint32_t SW_CHART_SM = 4096;  // words of a base chart staged in shared memory
-constexpr uint32_t SW_PER_LANE = TRIE_CHUNK / 32;
 
 // control words in shared memory
 enum : uint32_t {
   SC_N_STATES = 0,   // Earley sets of the job so far
   SC_ITEMS_TOP,      // top of the shared-memory item pool
-  SC_Q_N,            // queued transitions
-  SC_PEND_N,         // waiting nodes of the current depth
-  SC_CH_N0,          // alive chunks of the round (two counters, used alternately)
-  SC_CH_N1,
-  SC_ALIVE,          // some node of the current depth is alive
+  SC_F_N0,           // entries of the frontier lists: three counters used in turn (depth mod 3), so that
+  SC_F_N1,           // the one needed two depths ahead can be cleared while the other two are in use
+  SC_F_N2,
+  SC_RETRY_N0,       // entries of the retry list (two counters, by depth parity)
+  SC_RETRY_N1,
   SC_FAIL,           // a capacity was exceeded: the row's mask cannot be trusted
   SC_GL_HASH,        // the overflow hash is in use
   SC_N_SMHASH,       // sets entered into the shared-memory hash
   SC_TRANS,          // transitions computed (statistics)
   SC_JOB,            // the job in hand
   SC_BIG,            // warps that switched to their large scratch (statistics)
+  SC_Q_N,            // transitions queued for the warps
   SC_AGAIN,          // some node still waits after this round
   SC_TOTAL = 16
 };
 
 // word offsets into the dynamic shared memory
 struct SweepSmem {
-  uint32_t tables, mask, warps, warp_words, chart, hash, queue, chunks, bits, ctl, recs, items, total;
+  uint32_t tables, mask, warps, warp_words, chart, hash, front, queue, ctl, recs, items, total;
 };
 
 __host__ __device__ inline uint32_t sw_pad4(uint32_t words) { return (words + 3u) & ~3u; }
@@ -68,9 +70,8 @@ __host__ __device__ inline SweepSmem sweep_smem(const GrammarDev& G, const AutoD
   L.warps = at, at += SW_WARPS * L.warp_words;
   L.chart = at, at += sw_pad4(A.chart_sm_words);
   L.hash = at, at += SW_HASH;
+  L.front = at, at += 3u * 2u * SW_FRONT_SM;  // three lists of (node, set) pairs
   L.queue = at, at += SW_QUEUE;
-  L.chunks = at, at += SW_CHUNKS;
-  L.bits = at, at += sw_pad4(2u * A.bit_words);
   L.ctl = at, at += SC_TOTAL;
   L.recs = at, at += sw_pad4(A.sm_states * A.rec_words);
   L.items = at, at += sw_pad4(A.sm_items);
@@ -561,35 +562,6 @@ __device__ uint32_t thread_step(const GrammarDev& G, const StateDev& S, const Ct
   return T_FAIL;
 }
 
-// The state a node reaches from parent state `ps` on `byte`: ST_DEAD, ST_PENDING (the transition
-// is not known yet: it has been queued, by this thread if nobody did before) or the state's id.
-__device__ __forceinline__ uint32_t step_node(const GrammarDev& G, const StateDev& S, const CtaAuto& a, uint32_t* queue,
-                                              uint32_t ps, uint32_t byte) {
-  const uint32_t* rec = a.rec(ps);
-  // one 256-bit test rejects most bytes without touching the transition table
-  if (!((rec[AR_SCAN + (byte >> 5)] >> (byte & 31u)) & 1u)) return ST_DEAD;
-  uint16_t* tr = a.trans(ps) + G.eq_of_byte[byte];
-  uint32_t t = *reinterpret_cast<volatile uint16_t*>(tr);
-  if (t == T16_UNKNOWN) {
-    t = atomicCAS(tr, (unsigned short)T16_UNKNOWN, (unsigned short)T16_PENDING);
-    if (t == T16_UNKNOWN) {  // ours: compute it here if it is a step along a literal, else queue it for a warp
-      uint32_t r = thread_step(G, S, a, ps, byte);
-      if (r != TS_WARP) {
-        if (r == T_FAIL) a.ctl[SC_FAIL] = 1u, r = T_DEAD;
-        atomicAdd(&a.ctl[SC_TRANS], 1u);
-        *reinterpret_cast<volatile uint16_t*>(tr) = (r == T_DEAD) ? T16_DEAD : (uint16_t)r;
-        return (r == T_DEAD) ? (uint32_t)ST_DEAD : r;
-      }
-      const uint32_t at = atomicAdd(&a.ctl[SC_Q_N], 1u);
-      if (at < SW_QUEUE) queue[at] = (ps << 8) | byte;
-      else *reinterpret_cast<volatile uint16_t*>(tr) = T16_UNKNOWN;  // no room in this round: somebody claims it again in the next
-      return ST_PENDING;
-    }
-  }
-  if (t == T16_PENDING || t == T16_UNKNOWN) return ST_PENDING;
-  return (t == T16_DEAD) ? (uint32_t)ST_DEAD : t;
-}
-
 __device__ __forceinline__ void set_tokens(const GrammarDev& G, uint32_t* mask, uint32_t node) {
   const uint32_t tok = __ldg(&G.node_tok[node]);
   if (tok == NODE_TOK_NONE) return;
@@ -603,6 +575,60 @@ __device__ __forceinline__ void set_tokens(const GrammarDev& G, uint32_t* mask, 
   }
 }
 
+constexpr uint32_t ST_WAIT = 0xFFFEu;  // the transition is not known yet: the node goes on the retry list
+
+// The set a node reaches from its parent's set `ps` on `byte`: ST_DEAD, ST_WAIT or the set's id.  An
+// unknown transition is claimed: the claimer takes a step along a literal itself, here and now, and
+// queues anything else for the warps.
+__device__ __forceinline__ uint32_t step_node(const GrammarDev& G, const StateDev& S, const CtaAuto& a, uint32_t* queue,
+                                              uint32_t ps, uint32_t byte) {
+  const uint32_t* rec = a.rec(ps);
+  // one 256-bit test rejects most bytes without touching the transition table
+  if (!((rec[AR_SCAN + (byte >> 5)] >> (byte & 31u)) & 1u)) return ST_DEAD;
+  uint16_t* tr = a.trans(ps) + G.eq_of_byte[byte];
+  uint32_t t = *reinterpret_cast<volatile uint16_t*>(tr);
+  if (t == T16_UNKNOWN) {
+    t = atomicCAS(tr, (unsigned short)T16_UNKNOWN, (unsigned short)T16_PENDING);
+    if (t == T16_UNKNOWN) {  // ours
+      uint32_t r = thread_step(G, S, a, ps, byte);
+      if (r != TS_WARP) {
+        if (r == T_FAIL) a.ctl[SC_FAIL] = 1u, r = T_DEAD;
+        atomicAdd(&a.ctl[SC_TRANS], 1u);
+        *reinterpret_cast<volatile uint16_t*>(tr) = (r == T_DEAD) ? T16_DEAD : (uint16_t)r;
+        return (r == T_DEAD) ? (uint32_t)ST_DEAD : r;
+      }
+      const uint32_t at = atomicAdd(&a.ctl[SC_Q_N], 1u);
+      if (at < SW_QUEUE) queue[at] = (ps << 8) | byte;
+      else *reinterpret_cast<volatile uint16_t*>(tr) = T16_UNKNOWN;  // no room in this round: somebody claims it again in the next
+      return ST_WAIT;
+    }
+  }
+  if (t == T16_PENDING || t == T16_UNKNOWN) return ST_WAIT;
+  return (t == T16_DEAD) ? (uint32_t)ST_DEAD : t;
+}
+
+// A list of (node, Earley set) pairs: the first SW_FRONT_SM entries in shared memory, the rest in the
+// CTA's slice of global memory.
+struct NodeList {
+  uint2* sm;
+  uint2* gl;
+  __device__ __forceinline__ uint2 get(uint32_t i) const { return i < SW_FRONT_SM ? sm[i] : gl[i - SW_FRONT_SM]; }
+  __device__ __forceinline__ void put(uint32_t i, uint2 v) const {
+    if (i < SW_FRONT_SM) sm[i] = v;
+    else gl[i - SW_FRONT_SM] = v;
+  }
+  // (all lanes) append the pairs of the lanes with `v` set
+  __device__ __forceinline__ void push(uint32_t* counter, bool v, uint32_t node, uint32_t set) const {
+    const uint32_t bal = __ballot_sync(FULL, v);
+    if (!bal) return;
+    const uint32_t lane = lane_id();
+    uint32_t at = 0;
+    if (lane == 0) at = atomicAdd(counter, (uint32_t)__popc(bal));
+    at = __shfl_sync(FULL, at, 0);
+    if (v) put(at + __popc(bal & ((1u << lane) - 1u)), make_uint2(node, set));
+  }
+};
+
 __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, StateDev S) {
   const uint32_t n_jobs = S.counters[CNT_N_JOBS];
   if (blockIdx.x >= n_jobs) return;  // more CTAs than jobs
@@ -614,8 +640,6 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
   if (A.tables_in_smem) G = stage_hot_tables(Gg, smem + L.tables);
   uint32_t* const ctl = smem + L.ctl;
   uint32_t* const queue = smem + L.queue;
-  uint32_t* const chunks = smem + L.chunks;
-  uint32_t* const bits = smem + L.bits;
   uint32_t* const chart_sm = smem + L.chart;
   uint32_t* const mask_sm = smem + L.mask;
 
@@ -629,8 +653,11 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
   a.gl_hash = A.hash + (size_t)blockIdx.x * (A.gl_hash_mask + 1u);
   a.gl_hash_mask = A.gl_hash_mask;
   a.gl_items = A.items;
-  uint16_t* const st_base = A.st + (size_t)blockIdx.x * 2u * A.level_pad;
-  uint32_t* const pend = A.pend + (size_t)blockIdx.x * A.level_pad;
+  // two frontiers (used by depth parity) and the retry list
+  uint2* const front_sm = reinterpret_cast<uint2*>(smem + L.front);
+  uint2* const front_gl = A.front + (size_t)blockIdx.x * 3u * A.level_pad;
+  const NodeList list_even{front_sm, front_gl}, list_odd{front_sm + SW_FRONT_SM, front_gl + A.level_pad};
+  const NodeList retry{front_sm + 2u * SW_FRONT_SM, front_gl + 2u * (size_t)A.level_pad};
 
   uint32_t* mine = smem + L.warps + (size_t)warp * L.warp_words;
   SweepWarp sw{G, S, a};
@@ -648,6 +675,30 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
   for (uint32_t i = lane; i < ntw; i += 32) sw.w.nt[i] = 0u;
   if (tid < SC_TOTAL) ctl[tid] = 0u;
   uint32_t stat_trans = 0, stat_states = 0;  // thread 0's copies count
+
+  // (all lanes) the transition of set ps on byte pb, by the whole warp
+  auto warp_transition = [&](uint32_t ps, uint32_t pb) -> uint32_t {
+    uint32_t r = big_mode ? T_RETRY : sw.compute_small(ps, pb);
+    if (r == T_RETRY) r = sw.compute_general(ps, pb);
+    if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
+      big_mode = true;
+      hset_clear_all(sw.w.hset, sw.w.hset_mask);
+      clear_nt(G, sw.w);
+      sw.w.cur = big;
+      sw.w.cur_cap = S.big_arena_items;
+      sw.w.hset = big + S.big_arena_items;
+      sw.w.hset_mask = S.big_hset_slots - 1;
+      if (lane == 0) atomicAdd(&ctl[SC_BIG], 1u);
+      r = sw.compute_general(ps, pb);
+    }
+    if (r == T_FAIL) {  // a capacity was exceeded: the row's mask cannot be trusted
+      hset_clear_all(sw.w.hset, sw.w.hset_mask);
+      clear_nt(G, sw.w);
+      if (lane == 0) ctl[SC_FAIL] = 1u;
+      r = T_DEAD;  // lets the sweep go on
+    }
+    return r;
+  };
 
   for (;;) {
     __syncthreads();
@@ -681,7 +732,6 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
     if (gl_hash_dirty)
       for (uint32_t i = tid; i <= a.gl_hash_mask; i += SW_THREADS) a.gl_hash[i] = 0u;
     for (uint32_t i = tid; i < G.Wm; i += SW_THREADS) mask[i] = 0u;
-    for (uint32_t i = tid; i < 2u * A.bit_words; i += SW_THREADS) bits[i] = 0u;
     if (tid < SC_TOTAL && tid != SC_JOB) ctl[tid] = 0u;
     uint32_t* rec0 = a.rec(0);
     for (uint32_t i = tid; i < a.rec_words; i += SW_THREADS)
@@ -692,120 +742,72 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
       if (lane < 8) rec0[AR_SCAN + lane] = sw.tmp8[lane];
       if (lane == 0) {
         ctl[SC_N_STATES] = 1u;
-        bits[0] = 1u;    // depth 0 is the root alone, alive,
-        st_base[0] = 0;  // in state 0
+        list_even.put(0, make_uint2(0u, 0u));  // depth 0: the root, in state 0
+        ctl[SC_F_N0] = 1u;
         if (accepting && G.eos >= 0) mask[(uint32_t)G.eos >> 5] = 1u << ((uint32_t)G.eos & 31u);
       }
     }
     __syncthreads();
 
-    uint32_t round = 0;
-    for (uint32_t Lv = 1; Lv <= G.depth; ++Lv) {
-      const uint32_t lo_prev = __ldg(&G.lvl_off[Lv - 1]), lo = __ldg(&G.lvl_off[Lv]), hi = __ldg(&G.lvl_off[Lv + 1]);
-      if (hi == lo) break;
-      const uint32_t coff = __ldg(&G.lvl_chunk_off[Lv]), nch = __ldg(&G.lvl_chunk_off[Lv + 1]) - coff;
-      const uint16_t* st_prev = st_base + (size_t)((Lv - 1) & 1u) * A.level_pad;
-      uint16_t* st_cur = st_base + (size_t)(Lv & 1u) * A.level_pad;
-      const uint32_t* bits_prev = bits + ((Lv - 1) & 1u) * A.bit_words;
-      uint32_t* bits_cur = bits + (Lv & 1u) * A.bit_words;
-      for (uint32_t i = tid; i < A.bit_words; i += SW_THREADS) bits_cur[i] = 0u;
-      if (tid == 0) ctl[SC_ALIVE] = 0u, ctl[SC_PEND_N] = 0u, ctl[SC_Q_N] = 0u;
-      __syncthreads();
-
-      // ---- the pass over this depth
-      for (uint32_t base = 0; base < nch; base += SW_CHUNKS, ++round) {
-        uint32_t* const n_alive_ctr = &ctl[SC_CH_N0 + (round & 1u)];
-        if (tid == 0) ctl[SC_CH_N0 + ((round + 1u) & 1u)] = 0u;  // the other counter, for the next round
-        const uint32_t c = base + tid;
-        bool visit = false;
-        if (c < nch) {  // is any parent of this chunk's nodes alive?
-          const uint2 pr = __ldg(&G.chunk_par[coff + c]);
-          const uint32_t g0 = (pr.x - lo_prev) >> 5, g1 = (pr.y - lo_prev) >> 5;
-          for (uint32_t wd = g0 >> 5; wd <= (g1 >> 5) && !visit; ++wd) {
-            uint32_t b = bits_prev[wd];
-            if (wd == (g0 >> 5)) b &= 0xFFFFFFFFu << (g0 & 31u);
-            if (wd == (g1 >> 5)) b &= 0xFFFFFFFFu >> (31u - (g1 & 31u));
-            visit = b != 0u;
-          }
+    for (uint32_t Lv = 0; Lv <= G.depth; ++Lv) {
+      const uint32_t F = ctl[SC_F_N0 + Lv % 3u];  // nodes of depth Lv that are alive
+      if (F == 0) break;
+      uint32_t* const next_n = &ctl[SC_F_N0 + (Lv + 1u) % 3u];
+      uint32_t* const retry_n = &ctl[SC_RETRY_N0 + (Lv & 1u)];
+      if (tid == 0) ctl[SC_F_N0 + (Lv + 2u) % 3u] = 0u, ctl[SC_RETRY_N0 + ((Lv + 1u) & 1u)] = 0u;  // for the next depth
+      const NodeList cur = (Lv & 1u) ? list_odd : list_even, next = (Lv & 1u) ? list_even : list_odd;
+      // a warp takes `grp` consecutive entries at a time: one when there are few, so that their
+      // transitions are computed by different warps
+      const uint32_t grp = (F <= (uint32_t)SW_WARPS) ? 1u : min(32u, (F + 2u * SW_WARPS - 1u) / (2u * SW_WARPS));
+      for (uint32_t p0 = warp * grp; p0 < F; p0 += SW_WARPS * grp) {
+        const uint32_t np = min(grp, F - p0);
+        uint32_t pst = ST_DEAD, c0 = 0, cnt = 0;
+        if (lane < np) {
+          const uint2 e = cur.get(p0 + lane);
+          pst = e.y;
+          c0 = __ldg(&G.child_off[e.x]);
+          cnt = __ldg(&G.child_off[e.x + 1u]) - c0;
+          if (e.x != 0u) set_tokens(G, mask, e.x);  // the node is alive: so are the tokens that end there
         }
-        const uint32_t bal = __ballot_sync(FULL, visit);
-        uint32_t at = 0;
-        if (lane == 0 && bal) at = atomicAdd(n_alive_ctr, (uint32_t)__popc(bal));
-        at = __shfl_sync(FULL, at, 0);
-        if (visit) chunks[at + __popc(bal & ((1u << lane) - 1u))] = c;
-        __syncthreads();
-        const uint32_t n_alive = *n_alive_ctr;
-        for (uint32_t k = warp; k < n_alive; k += SW_WARPS) {
-          const uint32_t first = lo + chunks[k] * TRIE_CHUNK + lane;
-          uint32_t byte[SW_PER_LANE], par[SW_PER_LANE], ps[SW_PER_LANE];
-#pragma unroll
-          for (uint32_t u = 0; u < SW_PER_LANE; ++u) {
-            const uint32_t node = first + 32u * u;
-            const bool v = node < hi;
-            byte[u] = v ? __ldg(&G.node_byte[node]) : 0u;
-            par[u] = v ? __ldg(&G.parent[node]) - lo_prev : 0xFFFFFFFFu;
-          }
-#pragma unroll
-          for (uint32_t u = 0; u < SW_PER_LANE; ++u) {
-            ps[u] = ST_DEAD;
-            if (par[u] != 0xFFFFFFFFu && ((bits_prev[par[u] >> 10] >> ((par[u] >> 5) & 31u)) & 1u)) ps[u] = st_prev[par[u]];
-          }
-#pragma unroll
-          for (uint32_t u = 0; u < SW_PER_LANE; ++u) {
-            const uint32_t node = first + 32u * u;
-            const bool v = node < hi;
-            uint32_t t = ST_DEAD;
-            if (ps[u] != ST_DEAD) t = step_node(G, S, a, queue, ps[u], byte[u]);
-            if (v) st_cur[node - lo] = (uint16_t)t;
-            const bool alive = t != ST_DEAD, waits = t == ST_PENDING;
-            if (alive && !waits) set_tokens(G, mask, node);
-            const uint32_t wb = __ballot_sync(FULL, waits);
-            if (wb) {
-              uint32_t pa = 0;
-              if (lane == 0) pa = atomicAdd(&ctl[SC_PEND_N], (uint32_t)__popc(wb));
-              pa = __shfl_sync(FULL, pa, 0);
-              if (waits) pend[pa + __popc(wb & ((1u << lane) - 1u))] = node;
-            }
-            if (__ballot_sync(FULL, alive) && lane == 0) {
-              const uint32_t g = (node - lo) >> 5;
-              atomicOr(&bits_cur[g >> 5], 1u << (g & 31u));
-              ctl[SC_ALIVE] = 1u;
-            }
-          }
+        uint32_t incl = cnt;
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t t = __shfl_up_sync(FULL, incl, d);
+          if ((int)lane >= d) incl += t;
         }
-        __syncthreads();
+        const uint32_t total = __shfl_sync(FULL, incl, 31);
+        for (uint32_t base = 0; base < total; base += 32) {
+          const uint32_t idx = base + lane;
+          const bool valid = idx < total;
+          uint32_t p = 0;  // the parent whose children include the idx-th child: how many prefix sums are <= idx
+#pragma unroll
+          for (uint32_t sft = 16; sft > 0; sft >>= 1) {
+            const uint32_t v = __shfl_sync(FULL, incl, (p + sft - 1u) & 31u);
+            if (v <= idx && p + sft <= 32u) p += sft;
+          }
+          p &= 31u;
+          const uint32_t p_incl = __shfl_sync(FULL, incl, p), p_cnt = __shfl_sync(FULL, cnt, p);
+          const uint32_t p_c0 = __shfl_sync(FULL, c0, p), ps = __shfl_sync(FULL, pst, p);
+          const uint32_t child = p_c0 + (idx - (p_incl - p_cnt));
+          const uint32_t byte = valid ? __ldg(&G.node_byte[child]) : 0u;
+          const uint32_t t = valid ? step_node(G, S, a, queue, ps, byte) : (uint32_t)ST_DEAD;
+          next.push(next_n, valid && t != ST_DEAD && t != ST_WAIT, child, t);
+          retry.push(retry_n, t == ST_WAIT, child, ps);
+        }
       }
-
-      // ---- compute the queued transitions, settle the nodes that waited; again while some still wait
+      __syncthreads();
+      // ---- the warps compute the queued transitions, then the children that waited are settled;
+      // again while some still wait (only when more transitions were queued than the queue holds)
+      const uint32_t R = *retry_n;
       for (uint32_t rounds = 0;; ++rounds) {
-        const uint32_t nq = min(ctl[SC_Q_N], SW_QUEUE), np = ctl[SC_PEND_N];
-        // (nodes may wait although nothing is queued: a thread computed their transition meanwhile)
-        if (nq == 0 && !(rounds == 0 ? np > 0 : ctl[SC_AGAIN] != 0u)) break;
+        const uint32_t nq = min(ctl[SC_Q_N], SW_QUEUE);
+        if (nq == 0 && !(rounds == 0 ? R > 0 : ctl[SC_AGAIN] != 0u)) break;
         if (rounds > (1u << 16)) {  // cannot happen (every round settles at least one transition); never spin
           if (tid == 0) ctl[SC_FAIL] = 1u;
           break;
         }
         for (uint32_t i = warp; i < nq; i += SW_WARPS) {
           const uint32_t ps = queue[i] >> 8, pb = queue[i] & 0xFFu;
-          uint32_t r = big_mode ? T_RETRY : sw.compute_small(ps, pb);
-          if (r == T_RETRY) r = sw.compute_general(ps, pb);
-          if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
-            big_mode = true;
-            hset_clear_all(sw.w.hset, sw.w.hset_mask);
-            clear_nt(G, sw.w);
-            sw.w.cur = big;
-            sw.w.cur_cap = S.big_arena_items;
-            sw.w.hset = big + S.big_arena_items;
-            sw.w.hset_mask = S.big_hset_slots - 1;
-            if (lane == 0) atomicAdd(&ctl[SC_BIG], 1u);
-            r = sw.compute_general(ps, pb);
-          }
-          if (r == T_FAIL) {  // a capacity was exceeded: the row's mask cannot be trusted
-            hset_clear_all(sw.w.hset, sw.w.hset_mask);
-            clear_nt(G, sw.w);
-            if (lane == 0) ctl[SC_FAIL] = 1u;
-            r = T_DEAD;  // lets the sweep go on
-          }
+          const uint32_t r = warp_transition(ps, pb);
           if (lane == 0) {
             *reinterpret_cast<volatile uint16_t*>(a.trans(ps) + G.eq_of_byte[pb]) = (r == T_DEAD) ? T16_DEAD : (uint16_t)r;
             atomicAdd(&ctl[SC_TRANS], 1u);
@@ -814,24 +816,23 @@ __global__ void __launch_bounds__(SW_THREADS, 1) sweep_kernel(GrammarDev Gg, Sta
         __syncthreads();
         if (tid == 0) ctl[SC_Q_N] = 0u, ctl[SC_AGAIN] = 0u;
         __syncthreads();
-        for (uint32_t i = tid; i < np; i += SW_THREADS) {
-          const uint32_t node = pend[i];
-          if (node == 0xFFFFFFFFu) continue;  // settled in an earlier round
-          const uint32_t ps = st_prev[__ldg(&G.parent[node]) - lo_prev];
-          const uint32_t t = step_node(G, S, a, queue, ps, __ldg(&G.node_byte[node]));
-          if (t == ST_PENDING) {
-            ctl[SC_AGAIN] = 1u;
-            continue;
+        for (uint32_t base = 0; base < R; base += SW_THREADS) {
+          const uint32_t i = base + tid;
+          uint32_t child = 0xFFFFFFFFu, t = ST_DEAD;
+          if (i < R) {
+            const uint2 e = retry.get(i);
+            child = e.x;
+            if (child != 0xFFFFFFFFu) {  // not settled in an earlier round
+              t = step_node(G, S, a, queue, e.y, __ldg(&G.node_byte[child]));
+              if (t == ST_WAIT) ctl[SC_AGAIN] = 1u;
+              else retry.put(i, make_uint2(0xFFFFFFFFu, 0u));
+            }
           }
-          st_cur[node - lo] = (uint16_t)t;
-          if (t != ST_DEAD) set_tokens(G, mask, node);
-          pend[i] = 0xFFFFFFFFu;
+          next.push(next_n, t != ST_DEAD && t != ST_WAIT, child, t);
         }
         __syncthreads();
       }
-      const bool any_alive = ctl[SC_ALIVE] != 0u;
-      __syncthreads();  // everybody has read the flag before the next depth resets it
-      if (!any_alive) break;  // nothing survives this depth
+      __syncthreads();  // everybody has seen this depth's counters before the next depth changes them
     }
 
     // ---- the job's result

@@ -82,20 +82,14 @@ def test_trie_is_a_valid_csr_trie(config, kw):
             assert tok_node[t] == walk(child_off, node_byte, vocab[t])
         else:
             assert tok_node[t] == 0xFFFFFFFF
-    # per node: the token that ends there; per block of 128 nodes of one depth: the range of their parents
-    node_tok, chunk_par, chunk_off = g.table(11), g.table(12).reshape(-1, 2), g.table(13)
-    assert len(node_tok) == T and len(chunk_off) == info.trie_depth + 2 and chunk_off[-1] == len(chunk_par)
+    # per node: the token that ends there
+    node_tok = g.table(11)
+    assert len(node_tok) == T
     for n in range(T):
         ids = tok_ids[tok_off[n]:tok_off[n + 1]]
         want = 0xFFFFFFFF if len(ids) == 0 else (int(ids[0]) if len(ids) == 1 else 0xFFFFFFFE)
         assert node_tok[n] == want
     assert node_tok[walk(child_off, node_byte, vocab[300])] == 0xFFFFFFFE
-    for L in range(info.trie_depth + 1):
-        nodes = np.arange(lvl[L], lvl[L + 1])
-        assert chunk_off[L + 1] - chunk_off[L] == (len(nodes) + 127) // 128
-        for c in range(chunk_off[L], chunk_off[L + 1]):
-            blk = nodes[(c - chunk_off[L]) * 128:(c - chunk_off[L] + 1) * 128]
-            assert chunk_par[c, 0] == parent[blk].min() and chunk_par[c, 1] == parent[blk].max()
     # bytes in one class behave alike: for this grammar digits must share a class, '(' and ')' must not
     eq = g.table(10)
     assert info.n_byte_classes == len(set(eq.tolist()))
