@@ -137,7 +137,6 @@ fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out);
  *          6 nullable flags [N] u8      7 item info [D] u32        8 item lhs [D] u16
  *          9 tok_node [V] u32 (node where a token ends, 0xFFFFFFFF if it has no bytes)
  *         10 byte class of each byte [256] u8
- *         11 node_tok [T] u32: the token ending at a node, 0xFFFFFFFF none, 0xFFFFFFFE several (see tok_off)
  * Writes min(cap_bytes, size) bytes to `out` (may be NULL) and the full size to *size_bytes.
  */
 fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, size_t cap_bytes, size_t* size_bytes);

@@ -119,7 +119,7 @@ def _ptr(x) -> Optional[int]:
 
 
 _TABLE_DTYPES = {0: np.uint32, 1: np.uint8, 2: np.uint32, 3: np.uint32, 4: np.uint32, 5: np.uint32, 6: np.uint8,
-                 7: np.uint32, 8: np.uint16, 9: np.uint32, 10: np.uint8, 11: np.uint32}
+                 7: np.uint32, 8: np.uint16, 9: np.uint32, 10: np.uint8}
 
 
 class Grammar:

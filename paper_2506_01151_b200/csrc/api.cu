@@ -110,6 +110,7 @@ struct fmt_state {
   int32_t* init_state_dev = nullptr;
   int32_t* result_dev = nullptr;
   uint8_t* query_dev = nullptr;  // scratch for fmt_state_query
+  int sweep_grid = 1;
 };
 
 namespace fmt {
@@ -188,11 +189,6 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
     UP(node_depth);
     UP(lvl_off);
     UP(tok_node);
-    UP(node_tok);
-    UP(tok_off);
-    UP(tok_ids);
-    UP(child_off);
-    d.max_level = h.max_level;
     UP(vocab_off);
     UP(vocab_bytes);
 #undef UP
@@ -244,7 +240,6 @@ fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, si
     case 8: src = h.lhs.data(), n = (size_t)h.D * 2; break;
     case 9: src = h.tok_node.data(), n = h.tok_node.size() * 4; break;
     case 10: src = h.eq_of_byte.data(), n = 256; break;
-    case 11: src = h.node_tok.data(), n = h.node_tok.size() * 4; break;
     default: return fail(FMT_ERR_INVALID_ARG, "unknown table");
   }
   *size_bytes = n;
@@ -281,25 +276,30 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   d.ht_mask = ht - 1;
   d.init_off = (uint64_t)batch * 3u * d.chart_words;
   d.pool_base = d.init_off + d.chart_words;
-  d.big_arena_items = 1u << 15;
+  d.big_arena_items = 1u << 16;
   d.big_hset_slots = 1u << 14;
   AutoDev& au = d.au;
-  au.cap = (opt && opt->sweep_states) ? opt->sweep_states : 16384u;
+  au.cap = (opt && opt->sweep_states) ? opt->sweep_states : std::min(32768u, std::max(2048u, (4u << 20) / batch));
   if (au.cap < 16) au.cap = 16;
-  if (au.cap > AUTO_MAX_STATES) au.cap = AUTO_MAX_STATES;
-  sweep_plan(g->dev, au);
+  if (au.cap > 60000) au.cap = 60000;
+  au.rec_words = (AR_TRANS + g->dev.n_eq + 31u) & ~31u;
   uint32_t hs = 64;
   while (hs < au.cap * 2u) hs <<= 1;
-  au.gl_hash_mask = hs - 1;
+  au.hash_mask = hs - 1;
   au.items_cap = 128u << 20;
 
+  sweep_layout(g->dev, &au.smem_bytes, &au.tables_in_smem);
   cudaError_t e = configure_kernels();
-  int sms = 0, dev = 0;
+  int per_sm = 0, sms = 0, dev = 0;
+  if (e == cudaSuccess) e = sweep_blocks_per_sm(&per_sm, au.smem_bytes);
   if (e == cudaSuccess) e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  // one CTA per job and per SM; a call with more jobs than SMs hands them out as CTAs finish
-  au.grid = std::max(1u, std::min(batch, (uint32_t)std::max(1, sms)));
-  const size_t big_words = (size_t)au.grid * sweep_warps() * ((size_t)d.big_arena_items + d.big_hset_slots);
+  if (e == cudaSuccess && per_sm < 1) {
+    delete s;
+    return fail(FMT_ERR_CUDA, "the sweep kernel does not fit on this device");
+  }
+  s->sweep_grid = std::max(1, per_sm * sms);
+  const size_t big_words = (size_t)s->sweep_grid * sweep_warps() * ((size_t)d.big_arena_items + d.big_hset_slots);
 #define AL(ptr, count, fill) if (e == cudaSuccess) e = s->bufs.alloc((size_t)(count), &(ptr), (fill))
   AL(d.arena, d.pool_base + d.pool_words, 0);
   AL(d.row_chart, batch, 0);
@@ -314,10 +314,15 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(d.jobs, batch, 0);
   AL(d.counters, CNT_TOTAL, 0);
   AL(d.big_scratch, big_words, 0xFF);
-  AL(au.recs, (size_t)au.grid * (au.cap - au.sm_states) * au.rec_words, 0);
-  AL(au.hash, (size_t)au.grid * hs, 0);
+  AL(au.recs, (size_t)batch * au.cap * au.rec_words, 0);
+  AL(au.hash, (size_t)batch * hs, 0);
   AL(au.items, au.items_cap, 0);
-  AL(au.front, (size_t)au.grid * 3u * au.level_pad, 0);
+  AL(au.n_states, batch, 0);
+  au.st_stride = (g->dev.T + 63u) & ~63u;
+  AL(au.st, (size_t)batch * au.st_stride, 0xFF);
+  au.req_cap = 1u << 20;
+  AL(au.req, au.req_cap, 0);
+  AL(au.job_info, batch, 0);
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);
@@ -378,7 +383,7 @@ fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, 
   cudaStream_t st = (cudaStream_t)stream;
   cudaEvent_t w0, w1;
   s->prof.next(1, &w0, &w1);
-  launch_fill(s->g->dev, s->dev, st, w0, w1);
+  launch_fill(s->g->dev, s->dev, s->sweep_grid, st, w0, w1);
   launch_gather(s->g->dev, s->dev, mask_dev, stride_words, st);
   return launched("fmt_fill_mask");
 }
@@ -404,7 +409,7 @@ fmt_status fmt_fill_and_apply(fmt_state* s, uint32_t* mask_dev_or_null, size_t s
   cudaEvent_t w0, w1, a0, a1;
   s->prof.next(1, &w0, &w1);
   s->prof.next(2, &a0, &a1);
-  launch_fill(s->g->dev, s->dev, st, w0, w1);
+  launch_fill(s->g->dev, s->dev, s->sweep_grid, st, w0, w1);
   if (a0) cudaEventRecord(a0, st);
   launch_gather_apply(s->g->dev, s->dev, logits_dev, (int)dtype, row_stride_elems, mask_dev_or_null, stride_words, st);
   if (a1) cudaEventRecord(a1, st);

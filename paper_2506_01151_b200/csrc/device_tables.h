@@ -27,11 +27,6 @@ struct GrammarDev {
   uint32_t hot_words;
   const uint32_t* lvl_off;       // [depth+2]
   const uint32_t* tok_node;      // [V]
-  const uint32_t* node_tok;      // [T] token ending at the node, NODE_TOK_NONE or NODE_TOK_MANY
-  const uint32_t* tok_off;       // [T+1] \ all tokens ending at a node (needed for NODE_TOK_MANY only)
-  const uint32_t* tok_ids;       //       /
-  const uint32_t* child_off;     // [T+1] children of node n are nodes child_off[n] .. child_off[n+1]-1
-  uint32_t max_level;            // nodes of the most populous depth
   const uint32_t* vocab_off;     // [V+1]
   const uint8_t* vocab_bytes;
 };
@@ -66,48 +61,44 @@ enum : uint32_t {
   CNT_STAT_BIG = 24,
   CNT_STAT_TRANS = 26,  // transitions computed by the trie sweep (Earley steps)
   CNT_STAT_LOCAL = 28,  // local states created by the trie sweep
-  CNT_JOB_NEXT = 30,    // next job to hand to a CTA of the trie sweep, reset by every fill
-  CNT_TOTAL = 32
+  CNT_BAR = 30,         // grid barrier of the trie sweep: arrivals
+  CNT_BAR_ERR = 31,     // a block gave up waiting at the barrier
+  CNT_LEVEL_ALIVE = 32, // [MAX_TOKEN_BYTES + 2] per trie depth: some node of some job was alive
+  CNT_LEVEL_REQ = 68,   // [MAX_TOKEN_BYTES + 2] per trie depth: transitions queued for computation
+  CNT_TOTAL = 104
 };
 
-// Per-job automaton of hash-consed Earley sets, built on demand by the trie sweep.  A "local
+// Per-job automaton of hash-consed Earley sets, built on demand by the trie walk.  A "local
 // state" is the Earley set reached from the job's base chart by some byte string; equal sets get
 // one id, so a transition (state, byte class) is computed once per job, whatever the number of
 // trie nodes that need it.  Items of a local state name their origin as: a set index of the base
 // chart (< m), m + k for local state k, or ORIGIN_SELF for the state itself.
-// One CTA builds the automaton of one job.  The first sm_states records and the first sm_items
-// item words live in that CTA's shared memory, the rest in the CTA's slice of the global areas
-// below, so small automata (the common case) never leave the SM.
-// Record of a state (rec_words uint32):
-//   [0] first item (word offset: < sm_items shared memory, else sm_items + offset into `items`)
-//   [1] item count  [2] hash of the kernel  [3] items of the kernel (they come first)  [4..11] scannable bytes
-//   [12 ..) one uint16 per byte class: T16_UNKNOWN, T16_PENDING (queued for computation),
-//           T16_DEAD or the next state's id
+// Record of a state (rec_words uint32, a multiple of 32, so records never share a 128-byte line):
+//   [0] first item (word offset into items)  [1] item count  [2] hash of the kernel  [3] items of the
+//   kernel (they come first)  [4..11] scannable bytes
+//   [16 .. 16+n_eq) transition per byte class: T_UNKNOWN, T_PENDING (a warp is computing it),
+//                   T_DEAD or the next state's id
 struct AutoDev {
-  uint32_t cap;             // Earley sets one job may create (state 0 is the base chart's last set)
+  uint32_t cap;        // states per job, state 0 being the base chart's last set
   uint32_t rec_words;
-  uint32_t sm_states;       // records kept in shared memory
-  uint32_t sm_items;        // item words kept in shared memory
-  uint32_t chart_sm_words;  // a base chart up to this many words is staged in shared memory
-  uint32_t mask_in_smem;    // 1: the mask row is assembled in shared memory
-  uint32_t tables_in_smem;  // 1: the grammar's hot tables are staged in shared memory
+  uint32_t hash_mask;  // hash slots per job - 1
+  uint32_t items_cap;  // words of the item pool shared by all jobs
+  uint32_t* recs;      // [jobs][cap][rec_words]
+  uint32_t* hash;      // [jobs][hash_mask + 1], id + 1 or 0
+  uint32_t* items;     // [items_cap]
+  uint32_t* n_states;  // [jobs]
+  uint16_t* st;        // [jobs][st_stride] local state reached at every trie node (ST_DEAD if none)
+  uint32_t st_stride;
+  unsigned long long* req;  // [req_cap] transitions to compute at the current depth: job << 32 | state << 8 | byte
+  uint32_t req_cap;
   uint32_t smem_bytes;      // dynamic shared memory of the sweep kernel
-  uint32_t grid;            // CTAs of the sweep; the per-CTA areas below are sized for it
-  uint32_t level_pad;       // entries of one per-depth buffer (>= max_level)
-  uint32_t gl_hash_mask;    // slots - 1 of a CTA's overflow hash
-  uint32_t items_cap;       // words of the item pool shared by all CTAs
-  uint32_t* recs;           // [grid][cap - sm_states][rec_words]
-  uint32_t* hash;           // [grid][gl_hash_mask + 1] id + 1 or 0; all zero between jobs
-  uint32_t* items;          // [items_cap]
-  uint2* front;             // [grid][3][level_pad] (node, set) lists beyond their shared-memory part: the alive
-                            // nodes of the current and of the next depth, and the nodes that wait for a transition
+  uint32_t tables_in_smem;  // 1: the grammar's hot tables are staged in shared memory
+  uint4* job_info;          // [jobs] x: chart offset low, y: chart offset high, z: live sets m, w: row | accepting << 31
 };
-constexpr uint16_t ST_DEAD = 0xFFFFu;
-constexpr uint16_t T16_UNKNOWN = 0xFFFFu, T16_DEAD = 0xFFFEu, T16_PENDING = 0xFFFDu;
-constexpr uint32_t T_DEAD = 0xfffffffeu, T_FAIL = 0xfffffffdu;
+constexpr uint16_t ST_DEAD = 0xFFFFu, ST_PENDING = 0xFFFEu;
+constexpr uint32_t T_UNKNOWN = 0xffffffffu, T_DEAD = 0xfffffffeu, T_FAIL = 0xfffffffdu, T_PENDING = 0xfffffffcu;
 constexpr uint32_t ORIGIN_SELF = 0xFFFFu;
-constexpr uint32_t AUTO_MAX_STATES = 0xFF00u;  // ids stay below the uint16 marks above and, plus m, below ORIGIN_SELF
-constexpr uint32_t AR_ITEMS = 0, AR_N = 1, AR_HASH = 2, AR_NK = 3, AR_SCAN = 4, AR_TRANS = 12;
+constexpr uint32_t AR_ITEMS = 0, AR_N = 1, AR_HASH = 2, AR_NK = 3, AR_SCAN = 4, AR_TRANS = 16;
 
 struct StateDev {
   uint32_t B;

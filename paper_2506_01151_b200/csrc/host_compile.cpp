@@ -580,16 +580,6 @@ void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t 
   out.tok_node.assign(V, 0xFFFFFFFFu);
   for (uint32_t n = 0; n < out.T; ++n)
     for (uint32_t i = out.tok_off[n]; i < out.tok_off[n + 1] && i < (uint32_t)order.size(); ++i) out.tok_node[out.tok_ids[i]] = n;
-  // per node: the token that ends there (the common cases need no second lookup)
-  out.node_tok.assign(out.T, NODE_TOK_NONE);
-  if (!order.empty())
-    for (uint32_t n = 0; n < out.T; ++n) {
-      const uint32_t cnt = out.tok_off[n + 1] - out.tok_off[n];
-      if (cnt == 1) out.node_tok[n] = out.tok_ids[out.tok_off[n]];
-      else if (cnt > 1) out.node_tok[n] = NODE_TOK_MANY;
-    }
-  out.max_level = 1;
-  for (uint32_t L = 0; L <= out.depth; ++L) out.max_level = std::max(out.max_level, out.lvl_off[L + 1] - out.lvl_off[L]);
 }
 
 }  // namespace fmt

@@ -21,7 +21,6 @@ constexpr uint32_t ITEM_START = 0;   // $ -> . start
 constexpr uint32_t ITEM_ACCEPT = 1;  // $ -> start .
 constexpr uint32_t MAX_TOKEN_BYTES = 32;
 constexpr uint32_t MAX_NONTERMINALS = 4096;
-constexpr uint32_t NODE_TOK_NONE = 0xFFFFFFFFu, NODE_TOK_MANY = 0xFFFFFFFEu;
 
 struct CompileError {
   int code;
@@ -55,8 +54,6 @@ struct HostTables {
   std::vector<uint32_t> tok_ids;
   std::vector<uint32_t> lvl_off;    // [depth+2] nodes of depth L are lvl_off[L]..lvl_off[L+1]-1
   std::vector<uint32_t> tok_node;   // [V] node where the token's bytes end, 0xFFFFFFFF for empty tokens
-  std::vector<uint32_t> node_tok;   // [T] the token ending at the node, NODE_TOK_NONE, or NODE_TOK_MANY (use tok_off / tok_ids)
-  uint32_t max_level = 0;           // nodes of the most populous depth
   std::vector<uint32_t> vocab_off;  // [V+1] byte offsets (32-bit) into vocab_bytes
   std::vector<uint8_t> vocab_bytes;
 };

@@ -222,10 +222,10 @@ __global__ void __launch_bounds__(ADV_WARPS * 32) advance_kernel(GrammarDev Gg, 
 // One block decides, row by row, where each mask comes from: the state cache, another row of
 // this call with the same chart, or a fresh computation (a "job").
 __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
+  if (threadIdx.x < CNT_TOTAL - CNT_BAR) S.counters[CNT_BAR + threadIdx.x] = 0u;  // barrier and level counters
   if (threadIdx.x == 0) {
     S.counters[CNT_N_JOBS] = 0u;
     S.counters[CNT_AUTO_ITEMS] = 0u;
-    S.counters[CNT_JOB_NEXT] = 0u;
   }
   __syncthreads();
   for (uint32_t row = threadIdx.x; row < S.B; row += blockDim.x) {
@@ -269,10 +269,621 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
 }
 
 // ===================================================================================== fill: sweep
+//
+// For every job (a row whose mask must be computed) and every trie node the sweep answers "is the
+// Earley set reached by this node's bytes non-empty?".  Sets are hash-consed per job (AutoDev): a
+// transition (set, byte class) is computed once, by whichever warp needs it first, with the
+// warp-cooperative scan / complete / predict of earley_device.cuh; everybody else reads it from
+// the set's record.  The trie is processed one depth at a time by the whole grid, one THREAD per
+// (job, node): st[node] = transition(st[parent], byte).  Reads of parent, byte and writes of st
+// are coalesced because nodes are numbered breadth first.  A grid barrier separates the depths;
+// the kernel is launched cooperatively so that all CTAs are resident, and the barrier gives up
+// (and flags an error) after a bounded number of polls instead of hanging.
 
-}  // namespace fmt
-#include "sweep_cta.cuh"
-namespace fmt {
+constexpr int SWEEP_WARPS = 8;
+constexpr uint32_t SWEEP_CUR = 512;     // items of a set under construction per warp (fast mode, power of two)
+constexpr uint32_t SWEEP_HSET = 1024;   // uniqueness hash slots per warp (fast mode)
+
+struct JobCtx {
+  const uint32_t* base_off;
+  const uint32_t* base_items;
+  uint32_t m;         // live sets of the base chart
+  uint32_t* recs;     // this job's state records
+  uint32_t* hash;
+  uint32_t* n_states;
+  uint32_t cap;       // states this job may create (ids stay below ORIGIN_SELF - m)
+  uint16_t* st;
+  uint32_t row;
+  bool accepting;
+};
+
+// (phase 0 of the sweep) what later phases need to know about job j, in one 16-byte record
+__device__ __forceinline__ void make_job_info(const StateDev& S, uint32_t j) {
+  const uint32_t row = S.jobs[j];
+  const uint64_t off = S.row_chart[row];
+  const uint32_t* chart = S.arena + off;
+  const uint32_t acc = (chart[CH_FLAGS] & CHART_ACCEPTING) ? 0x80000000u : 0u;
+  S.au.job_info[j] = make_uint4((uint32_t)off, (uint32_t)(off >> 32), chart[CH_SETS], row | acc);
+}
+
+__device__ __forceinline__ JobCtx job_ctx(const StateDev& S, uint32_t j) {
+  const AutoDev& A = S.au;
+  const uint4 ji = __ldcg(A.job_info + j);
+  JobCtx J;
+  J.row = ji.w & 0x7FFFFFFFu;
+  J.accepting = (ji.w >> 31) != 0u;
+  const uint32_t* chart = S.arena + (((uint64_t)ji.y << 32) | ji.x);
+  J.m = ji.z;
+  J.base_off = chart + CH_HDR;
+  J.base_items = chart + CH_HDR + J.m + 1;
+  J.recs = A.recs + (size_t)j * A.cap * A.rec_words;
+  J.hash = A.hash + (size_t)j * (A.hash_mask + 1);
+  J.n_states = A.n_states + j;
+  J.cap = min(A.cap, (ORIGIN_SELF - 1u > J.m) ? ORIGIN_SELF - 1u - J.m : 0u);
+  J.st = A.st + (size_t)j * A.st_stride;
+  return J;
+}
+
+struct AutoView {
+  const JobCtx& J;
+  const AutoDev& A;
+  __device__ __forceinline__ void operator()(uint32_t o, const uint32_t*& p, uint32_t& n) const {
+    if (o < J.m) {
+      uint32_t a = J.base_off[o], b = J.base_off[o + 1];
+      p = J.base_items + a;
+      n = b - a;
+    } else {
+      const uint32_t* rec = J.recs + (size_t)(o - J.m) * A.rec_words;
+      p = A.items + rec[AR_ITEMS];
+      n = rec[AR_N];
+    }
+  }
+  // an item of local state o that names its own state as origin means "origin o"
+  __device__ __forceinline__ uint32_t fix(uint32_t item, uint32_t o) const {
+    return ((item >> 16) == ORIGIN_SELF) ? ((o << 16) | (item & 0xFFFFu)) : item;
+  }
+};
+
+// The Earley step of one warp.  Two forms of the same step (Section 3.2: scan, complete to a
+// fixpoint, predict): while the scanned and completed items ("kernel") number at most 32 they sit
+// one per lane and uniqueness is a matter of shuffles and ballots; larger sets go through the
+// hash-based primitives of earley_device.cuh.  Either way the predicted items are a function of
+// the kernel, so a set is looked up by its kernel alone (an order-independent hash, then an exact
+// comparison as sets) BEFORE anything is predicted, and a set already known costs no prediction.
+// A set's items are stored kernel first; nothing is sorted.
+constexpr uint32_t T_RETRY = 0xfffffffbu;  // the lane-resident form does not apply: take the general one
+
+struct SweepWarp {
+  const GrammarDev& G;
+  const StateDev& S;
+  WarpCtx w;
+  uint32_t* tmp8;     // shared
+  uint32_t n_computed = 0, n_created = 0;  // statistics, flushed once at the end of the kernel
+  uint32_t chunk_at = 0, chunk_left = 0;   // this warp's private piece of the item pool (lane 0's copy counts)
+
+  // A new set of job J with the items w.cur[0..n), the first nk of them its kernel: its id or T_FAIL.
+  __device__ uint32_t create_set(const JobCtx& J, uint32_t n, uint32_t nk, uint32_t hash) {
+    const uint32_t lane = lane_id();
+    const AutoDev& A = S.au;
+    uint32_t id = T_FAIL, ioff = 0;
+    if (lane == 0) {
+      const uint32_t got = atomicAdd(J.n_states, 1u);
+      const uint32_t need = (max(n, 1u) + 31u) & ~31u;
+      if (got < J.cap) {
+        if (need > chunk_left) {  // take a new piece of the pool: one atomic per ~4 Ki item words
+          const uint32_t take = max(need, 4096u);
+          chunk_at = atomicAdd(&S.counters[CNT_AUTO_ITEMS], take);
+          chunk_left = (chunk_at <= A.items_cap && take <= A.items_cap - chunk_at) ? take : 0u;
+        }
+        if (need <= chunk_left) {
+          ioff = chunk_at;
+          chunk_at += need;
+          chunk_left -= need;
+          id = got;
+        }
+      }
+    }
+    id = __shfl_sync(FULL, id, 0);
+    ioff = __shfl_sync(FULL, ioff, 0);
+    if (id == T_FAIL) return T_FAIL;
+    uint32_t* rec = J.recs + (size_t)id * A.rec_words;
+    uint32_t* items = A.items + ioff;
+    for (uint32_t i = lane; i < n; i += 32) items[i] = w.cur[i];
+    for (uint32_t i = lane; i < A.rec_words; i += 32) {
+      uint32_t v2 = 0u;
+      if (i == AR_ITEMS) v2 = ioff;
+      else if (i == AR_N) v2 = n;
+      else if (i == AR_HASH) v2 = hash;
+      else if (i == AR_NK) v2 = nk;
+      else if (i >= AR_SCAN && i < AR_SCAN + 8) v2 = tmp8[i - AR_SCAN];
+      else if (i >= AR_TRANS) v2 = T_UNKNOWN;
+      rec[i] = v2;
+    }
+    __syncwarp();
+    __threadfence();
+    ++n_created;
+    return id;
+  }
+
+  // Is set `sid` the one with this hash and a kernel of nk items for which `member` holds?
+  // member(x, valid) is called by all lanes.
+  template <class Member>
+  __device__ __forceinline__ bool same_set(const JobCtx& J, uint32_t sid, uint32_t nk, uint32_t hash, Member member) {
+    const uint32_t lane = lane_id();
+    const uint32_t* rec = J.recs + (size_t)sid * S.au.rec_words;
+    if (__ldcg(rec + AR_HASH) != hash || __ldcg(rec + AR_NK) != nk) return false;
+    const uint32_t* items = S.au.items + __ldcg(rec + AR_ITEMS);
+    bool ok = true;
+    for (uint32_t base = 0; base < nk; base += 32) {
+      const bool valid = base + lane < nk;
+      const uint32_t x = valid ? __ldcg(items + base + lane) : 0u;
+      ok = member(x, valid) && ok;
+    }
+    return __all_sync(FULL, ok);
+  }
+
+  // The set of job J with this kernel: its id, or T_FAIL if there is none yet.
+  template <class Member>
+  __device__ uint32_t lookup_set(const JobCtx& J, uint32_t nk, uint32_t hash, Member member) {
+    const uint32_t lane = lane_id();
+    const uint32_t mask = S.au.hash_mask;
+    uint32_t slot = hash & mask;
+    for (uint32_t probe = 0; probe <= mask && probe < 4096u; ++probe) {
+      uint32_t v = 0;
+      if (lane == 0) v = ld_acquire(&J.hash[slot]);
+      v = __shfl_sync(FULL, v, 0);
+      if (v == 0) break;
+      if (same_set(J, v - 1u, nk, hash, member)) return v - 1u;
+      slot = (slot + 1u) & mask;
+    }
+    return T_FAIL;
+  }
+
+  // Enter the freshly created set `id` into the job's hash, unless an equal set got there first
+  // (several warps often reach the same new set at the same moment): returns the id to use.
+  template <class Member>
+  __device__ uint32_t insert_set(const JobCtx& J, uint32_t id, uint32_t nk, uint32_t hash, Member member) {
+    const uint32_t lane = lane_id();
+    const uint32_t mask = S.au.hash_mask;
+    uint32_t slot = hash & mask;
+    for (uint32_t probe = 0; probe <= mask && probe < 4096u; ++probe) {
+      uint32_t old = 0;
+      if (lane == 0) old = atomicCAS(&J.hash[slot], 0u, id + 1u);
+      old = __shfl_sync(FULL, old, 0);
+      if (old == 0u) return id;
+      __threadfence();
+      if (same_set(J, old - 1u, nk, hash, member)) return old - 1u;
+      slot = (slot + 1u) & mask;
+    }
+    return T_FAIL;
+  }
+
+  // The kernel w.cur[0..nk) is new: predict, describe, store and enter the set.
+  template <class Member>
+  __device__ uint32_t finish_new(const JobCtx& J, uint32_t nk, uint32_t hash, Member member) {
+    const uint32_t lane = lane_id();
+    __syncwarp();
+    if (lane == 0) w.ctr[W_NCUR] = nk, w.ctr[W_OVERFLOW] = 0u;
+    predict_into_cur(G, w, ORIGIN_SELF);
+    if (w.ctr[W_OVERFLOW]) return T_RETRY;
+    const uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
+    scannable_bytes(G, w.cur, n, tmp8);
+    const uint32_t id = create_set(J, n, nk, hash);
+    return id == T_FAIL ? T_FAIL : insert_set(J, id, nk, hash, member);
+  }
+
+  // (lane-resident form) The candidates c .. c + skip of the lanes with `v` set join cur[0..n)
+  // unless already there.  `mine` is cur[lane].  Returns the new count, above 32 when they do not fit.
+  __device__ __forceinline__ uint32_t append_small(uint32_t c, bool v, uint32_t skip, uint32_t n, uint32_t& mine) {
+    const uint32_t lane = lane_id();
+    const uint32_t maxskip = __reduce_max_sync(FULL, v ? skip : 0u);
+    for (uint32_t j = 0; j <= maxskip; ++j) {
+      const bool vj = v && j <= skip;
+      const uint32_t cj = c + j;
+      const uint32_t vm = __ballot_sync(FULL, vj);
+      if (!vm) continue;
+      bool keep = vj;
+      if (vj) keep = (uint32_t)(__ffs(__match_any_sync(vm, cj)) - 1) == lane;  // one of equal candidates
+      for (uint32_t i = 0; i < n; ++i)
+        if (__shfl_sync(FULL, mine, i) == cj) keep = false;
+      const uint32_t kb = __ballot_sync(FULL, keep);
+      const uint32_t nn = n + __popc(kb);
+      if (nn > 32u) return nn;
+      if (keep) w.cur[n + __popc(kb & ((1u << lane) - 1u))] = cj;
+      __syncwarp();
+      n = nn;
+      mine = lane < n ? w.cur[lane] : 0u;
+    }
+    return n;
+  }
+
+  __device__ uint32_t compute_small(const JobCtx& J, uint32_t ps, uint32_t byte) {
+    const uint32_t lane = lane_id();
+    const uint32_t* pitems;
+    uint32_t plen;
+    AutoView view{J, S.au};
+    view(ps == 0 ? J.m - 1 : J.m + ps, pitems, plen);
+    const uint32_t self_code = J.m + ps;
+    uint32_t n = 0, mine = 0;
+    __syncwarp();
+    // ---- scan
+    for (uint32_t base = 0; base < plen; base += 32) {
+      const uint32_t k = base + lane;
+      uint32_t it = k < plen ? pitems[k] : 0u;
+      const uint32_t inf = k < plen ? G.info[it & 0xFFFFu] : 0u;
+      const bool hit = (inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte);
+      if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
+      const uint32_t skip = hit ? (G.info[(it + 1u) & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
+      if (__any_sync(FULL, hit)) n = append_small(it + 1u, hit, skip, n, mine);
+      if (n > 32u) return T_RETRY;
+    }
+    if (n == 0) return T_DEAD;
+    // ---- complete to a fixpoint: lanes [head, n) hold the items not looked at yet
+    uint32_t head = 0;
+    while (head < n) {
+      const bool have = lane >= head && lane < n;
+      const uint32_t inf = have ? G.info[mine & 0xFFFFu] : 0u;
+      const uint32_t kind = inf >> INFO_KIND_SHIFT;
+      if (have && kind == KIND_NT) {
+        const uint32_t y = inf & INFO_ARG_MASK;
+        atomicOr(&w.nt[y >> 5], 1u << (y & 31u));
+      }
+      uint32_t bal = __ballot_sync(FULL, have && kind == KIND_END && (mine >> 16) != ORIGIN_SELF);
+      const uint32_t it = mine;
+      head = n;
+      while (bal) {
+        const int src = __ffs(bal) - 1;
+        bal &= bal - 1;
+        const uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, src);
+        const uint32_t o = __shfl_sync(FULL, it >> 16, src);
+        const uint32_t* sp;
+        uint32_t sl;
+        view(o, sp, sl);
+        for (uint32_t base = 0; base < sl; base += 32) {
+          const uint32_t k = base + lane;
+          const uint32_t wi = k < sl ? sp[k] : 0u;
+          const uint32_t winf = k < sl ? G.info[wi & 0xFFFFu] : 0u;
+          const bool match = (winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X;
+          const uint32_t cand = view.fix(wi, o) + 1u;
+          const uint32_t skip = match ? (G.info[cand & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
+          if (__any_sync(FULL, match)) n = append_small(cand, match, skip, n, mine);
+          if (n > 32u) {
+            clear_nt(G, w);
+            return T_RETRY;
+          }
+        }
+      }
+    }
+    // ---- the kernel: what is left when the completed items go
+    const bool keep = lane < n && (G.info[mine & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
+    const uint32_t kb = __ballot_sync(FULL, keep);
+    const uint32_t nk = __popc(kb);
+    uint32_t h = keep ? mix32(mine) : 0u;
+    for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
+    h = mix32(h + nk * 0x9E3779B9u);
+    __syncwarp();
+    if (keep) w.cur[__popc(kb & ((1u << lane) - 1u))] = mine;
+    __syncwarp();
+    mine = lane < nk ? w.cur[lane] : 0u;
+    auto member = [&](uint32_t x, bool valid) {  // the kernel sits one item per lane
+      bool found = false;
+      for (uint32_t i = 0; i < nk; ++i)
+        if (__shfl_sync(FULL, mine, i) == x) found = true;
+      return found || !valid;
+    };
+    const uint32_t id = lookup_set(J, nk, h, member);
+    if (id != T_FAIL) {
+      clear_nt(G, w);
+      return id;
+    }
+    return finish_new(J, nk, h, member);
+  }
+
+  // The general form, for sets of any size (w.cur may be the warp's large area).
+  __device__ uint32_t compute_general(const JobCtx& J, uint32_t ps, uint32_t byte) {
+    const uint32_t lane = lane_id();
+    const uint32_t* pitems;
+    uint32_t plen;
+    AutoView view{J, S.au};
+    view(ps == 0 ? J.m - 1 : J.m + ps, pitems, plen);
+    __syncwarp();
+    if (lane < W_CTRS) w.ctr[lane] = 0u;
+    __syncwarp();
+    const uint32_t self_code = J.m + ps;
+    for (uint32_t k = lane; k < plen; k += 32) {
+      uint32_t it = pitems[k];
+      uint32_t inf = G.info[it & 0xFFFFu];
+      if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) {
+        if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
+        add_item(G, w, it + 1u);
+      }
+    }
+    __syncwarp();
+    if (w.ctr[W_OVERFLOW]) {
+      hset_clear_all(w.hset, w.hset_mask);
+      return T_FAIL;
+    }
+    if (w.ctr[W_NCUR] == 0u) return T_DEAD;
+    complete_fixpoint(G, w, view, ORIGIN_SELF, 0u);
+    const uint32_t hashed = min(w.ctr[W_NCUR], w.cur_cap);
+    if (w.ctr[W_OVERFLOW]) {
+      hset_clear_all(w.hset, w.hset_mask);
+      clear_nt(G, w);
+      return T_FAIL;
+    }
+    // the kernel: the items that are not completed; all of cur[0..hashed) are in the uniqueness hash
+    uint32_t nk = 0, h = 0;
+    for (uint32_t base = 0; base < hashed; base += 32) {
+      const uint32_t i = base + lane;
+      const uint32_t it = i < hashed ? w.cur[i] : 0u;
+      const bool keep = i < hashed && (G.info[it & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
+      if (keep) h += mix32(it);
+      nk += __popc(__ballot_sync(FULL, keep));
+    }
+    for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
+    h = mix32(h + nk * 0x9E3779B9u);
+    const uint32_t id = lookup_set(J, nk, h, [&](uint32_t x, bool valid) { return !valid || hset_contains(w.hset, w.hset_mask, x); });
+    hset_clear_items(w, hashed);
+    if (id != T_FAIL) {
+      clear_nt(G, w);
+      return id;
+    }
+    drop_completed(G, w, hashed);
+    // the kernel is cur[0..nk) now and no longer in the hash: a set met while entering this one is compared item by item
+    const uint32_t r = finish_new(J, nk, h, [&](uint32_t x, bool valid) {
+      bool found = !valid;
+      for (uint32_t i = 0; i < nk && !found; ++i) found = w.cur[i] == x;
+      return found;
+    });
+    return r == T_RETRY ? T_FAIL : r;
+  }
+
+  // Compute, publish and return the transition of local state `ps` on `byte`: T_DEAD, a state id,
+  // or T_FAIL when a capacity was exceeded (the caller may switch to the large scratch and ask
+  // again).  The transition has been claimed (T_PENDING) by whoever queued it.
+  __device__ uint32_t compute(const JobCtx& J, uint32_t ps, uint32_t byte, bool small_ok) {
+    uint32_t r = small_ok ? compute_small(J, ps, byte) : T_RETRY;
+    if (r == T_RETRY) r = compute_general(J, ps, byte);
+    if (r == T_FAIL) return T_FAIL;
+    uint32_t* slot = J.recs + (size_t)ps * S.au.rec_words + AR_TRANS + G.eq_of_byte[byte];
+    if (lane_id() == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(slot), "r"(r) : "memory");
+    ++n_computed;
+    return r;
+  }
+};
+
+// All CTAs of the (cooperatively launched) grid meet here.  Returns false if the sweep must be
+// abandoned: some CTA waited longer than the limit, which only a fault elsewhere can cause.
+__device__ __forceinline__ bool grid_barrier(const StateDev& S, uint32_t& phase) {
+  __shared__ uint32_t ok_s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    ++phase;
+    __threadfence();
+    atomicAdd(&S.counters[CNT_BAR], 1u);
+    const uint32_t target = phase * gridDim.x;
+    uint32_t ok = 1u;
+    for (uint32_t polls = 0;; ++polls) {
+      if (ld_acquire(&S.counters[CNT_BAR]) >= target) break;
+      if (polls > (1u << 24) || ld_acquire(&S.counters[CNT_BAR_ERR])) {
+        atomicExch(&S.counters[CNT_BAR_ERR], 1u);
+        ok = 0u;
+        break;
+      }
+      __nanosleep(40);
+    }
+    __threadfence();
+    ok_s = ok;
+  }
+  __syncthreads();
+  const bool ok = ok_s != 0u;
+  __syncthreads();
+  return ok;
+}
+
+// What the Earley set at `node` is, given that its mark says "pending": the transition it waited
+// for has been computed meanwhile.  `parent_state` is the (final) state of its parent.
+__device__ __forceinline__ uint32_t settled(const GrammarDev& G, const AutoDev& A, const JobCtx& J, uint32_t parent_state,
+                                            uint32_t byte) {
+  const uint32_t* slot = J.recs + (size_t)parent_state * A.rec_words + AR_TRANS + G.eq_of_byte[byte];
+  return __ldcg(slot);
+}
+
+constexpr uint32_t SWEEP_PER_LANE = 4;  // trie nodes per lane and pass iteration (independent loads in flight)
+
+__global__ void __launch_bounds__(SWEEP_WARPS * 32, 3) sweep_kernel(GrammarDev Gg, StateDev S) {
+  const uint32_t n_jobs = S.counters[CNT_N_JOBS];
+  if (n_jobs == 0) return;  // every CTA sees the same count: nobody is left at a barrier
+  extern __shared__ __align__(16) uint32_t smem[];
+  const uint32_t warp = threadIdx.x >> 5, lane = lane_id();
+  const AutoDev& A = S.au;
+  const uint32_t ntw = (2u * Gg.Nw + 7u) & ~7u;
+  const uint32_t warp_words = SWEEP_CUR + SWEEP_HSET + ntw + W_CTRS + 8;
+  uint32_t* mine = smem + (size_t)warp * warp_words;
+  uint32_t* sm_cur = mine;
+  uint32_t* sm_hset = sm_cur + SWEEP_CUR;
+  uint32_t* nt = sm_hset + SWEEP_HSET;
+  uint32_t* ctr = nt + ntw;
+  uint32_t* tmp8 = ctr + W_CTRS;
+  // ---- the small grammar tables every Earley step reads go to shared memory when they fit
+  GrammarDev G = Gg;
+  if (A.tables_in_smem) G = stage_hot_tables(Gg, smem + (size_t)SWEEP_WARPS * warp_words);
+  uint32_t* big = S.big_scratch + ((size_t)blockIdx.x * SWEEP_WARPS + warp) * ((size_t)S.big_arena_items + S.big_hset_slots);
+  const uint32_t gw = blockIdx.x * SWEEP_WARPS + warp, GW = gridDim.x * SWEEP_WARPS;
+  uint32_t bar_phase = 0;
+
+  hset_clear_all(sm_hset, SWEEP_HSET - 1);
+  for (uint32_t i = lane; i < ntw; i += 32) nt[i] = 0u;
+  __syncthreads();
+
+  // ---- the automata start with one state each: the base chart's last set
+  for (uint32_t j = blockIdx.x; j < n_jobs; j += gridDim.x) {
+    uint32_t* hash = A.hash + (size_t)j * (A.hash_mask + 1);
+    for (uint32_t i = threadIdx.x; i <= A.hash_mask; i += blockDim.x) hash[i] = 0u;
+    uint32_t* rec0 = A.recs + (size_t)j * A.cap * A.rec_words;
+    for (uint32_t i = threadIdx.x; i < A.rec_words; i += blockDim.x)
+      if (i < AR_SCAN || i >= AR_SCAN + 8) rec0[i] = (i >= AR_TRANS) ? T_UNKNOWN : 0u;
+    if (threadIdx.x == 0) A.n_states[j] = 1u;
+    if (warp == 0) {
+      if (lane == 0) make_job_info(S, j);
+      __syncwarp();
+      __threadfence_block();
+      JobCtx J = job_ctx(S, j);
+      scannable_bytes(G, J.base_items + J.base_off[J.m - 1], J.base_off[J.m] - J.base_off[J.m - 1], tmp8);
+      if (lane < 8) rec0[AR_SCAN + lane] = tmp8[lane];
+    }
+  }
+  if (!grid_barrier(S, bar_phase)) return;
+
+  SweepWarp sw{G, S};
+  sw.w.nt = nt;
+  sw.w.ctr = ctr;
+  sw.tmp8 = tmp8;
+  sw.w.cur = sm_cur;
+  sw.w.cur_cap = SWEEP_CUR;
+  sw.w.hset = sm_hset;
+  sw.w.hset_mask = SWEEP_HSET - 1;
+  bool big_mode = false;
+
+  uint32_t last_level = 0;
+  for (uint32_t L = 1; L <= G.depth; ++L) {
+    const uint32_t lo = __ldg(&G.lvl_off[L]), hi = __ldg(&G.lvl_off[L + 1]);
+    constexpr uint32_t CH = 32 * SWEEP_PER_LANE;
+    const uint32_t nL = hi - lo, cpj = (nL + CH - 1) / CH;
+    const uint32_t chunks = n_jobs * cpj;
+    // ---- the pass: one thread per (job, node).  Known transitions are final; an unknown one is
+    // claimed by the first thread that meets it, which queues it for the compute phase below, and
+    // the node is marked pending.  A pending PARENT (marked at the previous depth, computed since)
+    // is settled on the way; pending leaves are settled when the mask words are formed.
+    bool any_alive = false;
+    for (uint32_t c = gw; c < chunks; c += GW) {
+      const uint32_t j = c / cpj;
+      const uint32_t first = lo + (c % cpj) * CH + lane;
+      const JobCtx J = job_ctx(S, j);
+      uint32_t node[SWEEP_PER_LANE], byte[SWEEP_PER_LANE], par[SWEEP_PER_LANE], ps[SWEEP_PER_LANE];
+#pragma unroll
+      for (uint32_t u = 0; u < SWEEP_PER_LANE; ++u) {
+        node[u] = first + 32u * u;
+        const bool v = node[u] < hi;
+        byte[u] = v ? __ldg(&G.node_byte[node[u]]) : 0u;
+        par[u] = (v && L > 1) ? __ldg(&G.parent[node[u]]) : 0u;
+      }
+#pragma unroll
+      for (uint32_t u = 0; u < SWEEP_PER_LANE; ++u)
+        ps[u] = (node[u] < hi) ? ((L == 1) ? 0u : (uint32_t)__ldcg(J.st + par[u])) : (uint32_t)ST_DEAD;  // written by other SMs: bypass L1
+#pragma unroll
+      for (uint32_t u = 0; u < SWEEP_PER_LANE; ++u) {
+        if (node[u] >= hi) continue;
+        uint32_t p_state = ps[u];
+        if (p_state == ST_PENDING) {  // settle the parent first
+          const uint32_t gp_state = (L == 2) ? 0u : (uint32_t)__ldcg(J.st + __ldg(&G.parent[par[u]]));
+          const uint32_t t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
+          if (t2 == T_UNKNOWN || t2 == T_PENDING) {  // only if the queue overflowed: give the row up rather than guess
+            atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+            atomicExch(&S.counters[CNT_ERR], 1u);
+            p_state = ST_DEAD;
+          } else {
+            p_state = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+          }
+          J.st[par[u]] = (uint16_t)p_state;
+        }
+        uint32_t t = T_DEAD;
+        if (p_state != ST_DEAD) {
+          const uint32_t* rec = J.recs + (size_t)p_state * A.rec_words;
+          // one 256-bit test rejects most bytes without touching the transition table
+          if ((rec[AR_SCAN + (byte[u] >> 5)] >> (byte[u] & 31u)) & 1u) {
+            uint32_t* slot = J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[byte[u]];
+            t = *slot;
+            if (t == T_UNKNOWN || t == T_PENDING) t = __ldcg(slot);
+            if (t == T_UNKNOWN) {
+              t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
+              if (t == T_UNKNOWN) {  // ours to queue
+                const uint32_t at = atomicAdd(&S.counters[CNT_LEVEL_REQ + L], 1u);
+                if (at < A.req_cap) A.req[at] = ((unsigned long long)j << 32) | ((unsigned long long)p_state << 8) | byte[u];
+                t = T_PENDING;
+              }
+            }
+          }
+        }
+        J.st[node[u]] = (t == T_PENDING) ? ST_PENDING : (t == T_DEAD) ? ST_DEAD : (uint16_t)t;
+        any_alive |= (t != T_DEAD);
+      }
+    }
+    __syncwarp();
+    if (__any_sync(FULL, any_alive) && lane == 0) atomicOr(&S.counters[CNT_LEVEL_ALIVE + L], 1u);
+    if (!grid_barrier(S, bar_phase)) return;
+    last_level = L;
+    if (ld_acquire(&S.counters[CNT_LEVEL_ALIVE + L]) == 0u) break;  // nothing survives this depth in any job
+    const uint32_t n_req = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), A.req_cap);
+    if (n_req == 0) continue;  // nothing was unknown at this depth
+    // ---- compute phase: one queued transition per warp at a time, all warps of the grid in parallel
+    for (uint32_t i = gw; i < n_req; i += GW) {
+      const unsigned long long rq = __ldcg(A.req + i);
+      const uint32_t j = (uint32_t)(rq >> 32), p_state = (uint32_t)(rq >> 8) & 0xFFFFu, pb = (uint32_t)rq & 0xFFu;
+      const JobCtx J = job_ctx(S, j);
+      uint32_t r = sw.compute(J, p_state, pb, !big_mode);
+      if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
+        big_mode = true;
+        hset_clear_all(sw.w.hset, sw.w.hset_mask);
+        clear_nt(G, sw.w);
+        sw.w.cur = big;
+        sw.w.cur_cap = S.big_arena_items;
+        sw.w.hset = big + S.big_arena_items;
+        sw.w.hset_mask = S.big_hset_slots - 1;
+        if (lane == 0) stat_add(S, CNT_STAT_BIG, 1u);
+        r = sw.compute(J, p_state, pb, false);
+      }
+      if (r == T_FAIL) {  // a capacity was exceeded: the row's mask cannot be trusted
+        hset_clear_all(sw.w.hset, sw.w.hset_mask);
+        clear_nt(G, sw.w);
+        if (lane == 0) {
+          atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+          atomicExch(&S.counters[CNT_ERR], 1u);
+          stat_add(S, CNT_STAT_CAPERR, 1u);
+          atomicExch(J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[pb], T_DEAD);  // lets the sweep go on
+        }
+      }
+    }
+    if (!grid_barrier(S, bar_phase)) return;
+  }
+  if (big_mode) hset_clear_all(sw.w.hset, sw.w.hset_mask);
+  if (lane == 0 && (sw.n_computed | sw.n_created)) {
+    stat_add(S, CNT_STAT_TRANS, sw.n_computed);
+    stat_add(S, CNT_STAT_LOCAL, sw.n_created);
+  }
+
+  // ---- mask words: 32 tokens per warp pass, one ballot per word (token t is valid iff the node
+  // where its bytes end was reached alive; EOS iff the chart is accepting)
+  const uint32_t Wm = G.Wm;
+  for (uint32_t c = gw; c < n_jobs * Wm; c += GW) {
+    const uint32_t j = c / Wm, wd = c % Wm;
+    const JobCtx J = job_ctx(S, j);
+    const uint32_t tok = wd * 32 + lane;
+    bool ok = false;
+    if (tok < G.V) {
+      const uint32_t node = __ldg(&G.tok_node[tok]);
+      if (node == 0xFFFFFFFFu) {
+        ok = ((int32_t)tok == G.eos) && J.accepting;
+      } else if (__ldg(&G.node_depth[node]) <= last_level) {
+        uint32_t s = __ldcg(J.st + node);
+        if (s == ST_PENDING) {  // a leaf that waited for a transition: its parent is final by now
+          const uint32_t p = __ldg(&G.parent[node]);
+          const uint32_t p_state = (p == 0) ? 0u : (uint32_t)__ldcg(J.st + p);
+          const uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node]));
+          if (t2 == T_UNKNOWN || t2 == T_PENDING || p_state == ST_PENDING) {
+            atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+            s = ST_DEAD;
+          } else {
+            s = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+          }
+        }
+        ok = s != ST_DEAD;
+      }
+    }
+    const uint32_t word = __ballot_sync(FULL, ok);
+    if (lane == 0) S.mask_rows[(size_t)S.row_mask[J.row] * Wm + wd] = word;
+  }
+}
 
 // Publish the masks computed in this call to the cache (or release the claim when the row had
 // no cache row, or broke).
@@ -282,7 +893,8 @@ __global__ void publish_kernel(StateDev S) {
   if (j < n_jobs) {
     const uint32_t row = S.jobs[j];
     const int32_t sid = S.row_state[row];
-    const bool broken = (S.row_flags[row] & ROW_BROKEN) != 0u;
+    const bool broken = (S.row_flags[row] & ROW_BROKEN) || S.counters[CNT_BAR_ERR];
+    if (S.counters[CNT_BAR_ERR]) atomicOr(&S.row_flags[row], ROW_BROKEN);
     if (sid >= 0) {
       const int32_t mrow = S.row_mask[row];
       S.st_mask[sid] = (!broken && mrow >= (int32_t)S.B) ? mrow : -1;
@@ -463,38 +1075,29 @@ static size_t adv_smem_bytes(const GrammarDev& G) {
   return (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + (G.hot_words * 4u <= HOT_TABLE_BYTES ? G.hot_words * 4u : 0u);
 }
 static size_t init_smem_bytes() { return (size_t)ADV_WARP_WORDS * 4; }
-// Decide what of a sweep CTA's working set lives in shared memory for this grammar and fill in
-// the layout fields of `A` (cap must be set): the grammar's hot tables and the mask row when they
-// are small enough, a staged base chart, and as many automaton records and item words as the
-// rest of the budget holds.
-void sweep_plan(const GrammarDev& G, AutoDev& A) {
-  A.rec_words = (AR_TRANS + (G.n_eq + 1u) / 2u + 3u) & ~3u;
-  A.tables_in_smem = G.hot_words * 4u <= HOT_TABLE_BYTES ? 1u : 0u;
-  A.mask_in_smem = G.Wm * 4u <= 48u * 1024u ? 1u : 0u;
-  A.chart_sm_words = SW_CHART_SM;
-  A.level_pad = (G.max_level + 63u) & ~63u;
-  A.sm_states = 0;
-  A.sm_items = 0;
-  const uint32_t budget = SW_SMEM_BUDGET / 4u;
-  uint32_t fixed = sweep_smem(G, A).total;
-  if (fixed + 4096u > budget && A.mask_in_smem) {  // a huge vocabulary: assemble the mask row in global memory
-    A.mask_in_smem = 0;
-    fixed = sweep_smem(G, A).total;
-  }
-  const uint32_t rest = budget > fixed + 64u ? budget - fixed - 64u : 0u;
-  A.sm_items = std::min(rest / 3u, 16384u) & ~3u;
-  A.sm_states = std::min(std::min((rest - A.sm_items) / A.rec_words, A.cap), AUTO_MAX_STATES);
-  if (A.sm_states < 1u) A.sm_states = 0u, A.sm_items = 0u;
-  A.smem_bytes = sweep_smem(G, A).total * 4u;
+// Dynamic shared memory of the sweep for a grammar: per-warp scratch plus, if they fit the
+// budget, the item-info / byte-class / byte-class-number tables.
+void sweep_layout(const GrammarDev& G, uint32_t* smem_bytes, uint32_t* tables_in_smem) {
+  const uint32_t ntw = (2u * G.Nw + 7u) & ~7u;
+  const uint32_t warp_words = SWEEP_CUR + SWEEP_HSET + ntw + W_CTRS + 8;
+  uint32_t bytes = SWEEP_WARPS * warp_words * 4u;
+  const uint32_t tab = G.hot_words * 4u;
+  *tables_in_smem = tab <= HOT_TABLE_BYTES ? 1u : 0u;
+  if (*tables_in_smem) bytes += tab;
+  *smem_bytes = bytes;
 }
-int sweep_warps() { return SW_WARPS; }
+int sweep_warps() { return SWEEP_WARPS; }
 
 cudaError_t configure_kernels() {
   cudaError_t e;
   if ((e = opt_in_smem((const void*)init_kernel, init_smem_bytes())) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)advance_kernel, (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + HOT_TABLE_BYTES)) != cudaSuccess) return e;
-  if ((e = opt_in_smem((const void*)sweep_kernel, SW_SMEM_BUDGET)) != cudaSuccess) return e;
+  if ((e = opt_in_smem((const void*)sweep_kernel, 160 * 1024)) != cudaSuccess) return e;
   return cudaSuccess;
+}
+
+cudaError_t sweep_blocks_per_sm(int* out, uint32_t smem_bytes) {
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, sweep_kernel, SWEEP_WARPS * 32, smem_bytes);
 }
 
 void launch_init(const GrammarDev& G, const StateDev& S, int32_t* result_dev, cudaStream_t st) {
@@ -510,16 +1113,23 @@ void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const
 void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st) {
   advance_kernel<<<(S.B + ADV_WARPS - 1) / ADV_WARPS, ADV_WARPS * 32, adv_smem_bytes(G), st>>>(G, S, tokens, status);
 }
-void launch_sweep(const GrammarDev& G, const StateDev& S, cudaStream_t st) {
-  sweep_kernel<<<S.au.grid, SW_THREADS, S.au.smem_bytes, st>>>(G, S);
+static void launch_sweep_coop(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) {
+  GrammarDev g = G;
+  StateDev s = S;
+  void* args[] = {&g, &s};
+  cudaLaunchCooperativeKernel((const void*)sweep_kernel, dim3((unsigned)grid), dim3(SWEEP_WARPS * 32), args,
+                              S.au.smem_bytes, st);
 }
-void launch_fill(const GrammarDev& G, const StateDev& S, cudaStream_t st, cudaEvent_t before_sweep, cudaEvent_t after_sweep) {
+void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_sweep,
+                 cudaEvent_t after_sweep) {
   plan_kernel<<<1, 1024, 0, st>>>(G, S);
   if (before_sweep) cudaEventRecord(before_sweep, st);
-  launch_sweep(G, S, st);
+  launch_sweep_coop(G, S, sweep_grid, st);
   if (after_sweep) cudaEventRecord(after_sweep, st);
   publish_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(S);
 }
+// the sweep alone, for jobs the caller has already listed (used by the allocation-free entry point)
+void launch_sweep(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) { launch_sweep_coop(G, S, grid, st); }
 void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st) {
   dim3 grid((unsigned)std::min<size_t>((stride_words + 255) / 256, 64), S.B);
   gather_kernel<<<grid, 256, 0, st>>>(G, S, out, stride_words);

@@ -7,14 +7,15 @@
 namespace fmt {
 
 cudaError_t configure_kernels();
-void sweep_plan(const GrammarDev& G, AutoDev& A);  // fills the layout fields of A (A.cap must be set)
+cudaError_t sweep_blocks_per_sm(int* out, uint32_t smem_bytes);
+void sweep_layout(const GrammarDev& G, uint32_t* smem_bytes, uint32_t* tables_in_smem);
 int sweep_warps();
 
 void launch_init(const GrammarDev& G, const StateDev& S, int32_t* result_dev, cudaStream_t st);
 void launch_intern_init(const StateDev& S, int32_t* init_state_dev, cudaStream_t st);
 void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const int32_t* init_state_dev, cudaStream_t st);
 void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st);
-void launch_fill(const GrammarDev& G, const StateDev& S, cudaStream_t st, cudaEvent_t before_sweep = nullptr,
+void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_sweep = nullptr,
                  cudaEvent_t after_sweep = nullptr);
 void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st);
 void launch_apply(const uint32_t* mask, size_t stride_words, void* logits, int dtype, uint32_t batch, uint32_t V,
@@ -26,8 +27,8 @@ void launch_reintern(const StateDev& S, int32_t* init_state_dev, cudaStream_t st
 void launch_query(const StateDev& S, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets, uint32_t* n_items,
                   int32_t* state_id, cudaStream_t st);
 
-// the trie sweep alone, for jobs the caller has already listed (used by the allocation-free entry point)
-void launch_sweep(const GrammarDev& G, const StateDev& S, cudaStream_t st);
+// the trie-walk kernel alone, on an arbitrary grid (used by the allocation-free entry point)
+void launch_sweep(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st);
 
 }  // namespace fmt
 

@@ -18,39 +18,42 @@ namespace {
 using namespace fmt;
 
 constexpr uint32_t NA_MAX = FMT_NOALLOC_MAX_CHARTS;
-constexpr uint32_t NA_GRID = 8;             // CTAs of the sweep, one chart at a time each
-constexpr uint32_t NA_WARPS_PER_CTA = 16;
+constexpr uint32_t NA_GRID = 32;            // CTAs of the sweep
 constexpr uint32_t NA_ARENA_ITEMS = 8192;   // per-warp overflow area for Earley sets (items)
 constexpr uint32_t NA_HSET_SLOTS = 2048;    // per-warp overflow uniqueness hash
 // header: counters, then per-chart arrays
 constexpr uint32_t NA_OFF_COUNTERS = 0;                          // [CNT_TOTAL]
 constexpr uint32_t NA_OFF_JOBS = 128;                            // [NA_MAX]
+constexpr uint32_t NA_REQ_CAP = 1u << 16;                        // transitions queued per trie depth
 constexpr uint32_t NA_OFF_FLAGS = NA_OFF_JOBS + NA_MAX;          // [NA_MAX]
 constexpr uint32_t NA_OFF_MASKROW = NA_OFF_FLAGS + NA_MAX;       // [NA_MAX] int32
 constexpr uint32_t NA_OFF_CHART = NA_OFF_MASKROW + NA_MAX;       // [NA_MAX] uint64 (8-byte aligned)
 constexpr uint32_t NA_OFF_BAD = NA_OFF_CHART + 2 * NA_MAX;       // [NA_MAX] header check failed
+constexpr uint32_t NA_OFF_NSTATES = NA_OFF_BAD + NA_MAX;         // [NA_MAX] Earley sets created per chart
+constexpr uint32_t NA_OFF_JOBINFO = NA_OFF_NSTATES + NA_MAX;     // [NA_MAX] uint4 (16-byte aligned)
 constexpr uint32_t NA_HEADER_WORDS = 1024;
-constexpr size_t NA_WARPS = (size_t)NA_GRID * NA_WARPS_PER_CTA;
+constexpr size_t NA_WARPS = (size_t)NA_GRID * 8;
 constexpr size_t NA_BIG_WORDS = NA_WARPS * (NA_ARENA_ITEMS + NA_HSET_SLOTS);
-// what a CTA's automaton of Earley sets may use beyond its shared memory: 64 Ki words of records and
-// 8192 hash slots per CTA, and one pool of 2 Mi item words for all charts of a call
-constexpr uint32_t NA_REC_WORDS_PER_CTA = 65536;
-constexpr uint32_t NA_HASH_SLOTS = 8192;
+// the sweep's tables of Earley sets: per chart 64 Ki words of records and 2048 hash slots, and one
+// pool of 2 Mi item words for all charts of a call
+constexpr uint32_t NA_REC_WORDS_PER_CHART = 65536;
+constexpr uint32_t NA_HASH_SLOTS = 2048;
 constexpr uint32_t NA_ITEM_WORDS = 2u << 20;
-// per CTA three lists of (trie node, Earley set) pairs of up to one trie depth each: the alive nodes of
-// the current and of the next depth and the nodes that wait for a transition
-constexpr uint32_t NA_LEVEL_MAX = 128u << 10;
 constexpr size_t NA_OFF_BIG = NA_HEADER_WORDS;
 constexpr size_t NA_OFF_RECS = NA_OFF_BIG + NA_BIG_WORDS;
-constexpr size_t NA_OFF_HASH = NA_OFF_RECS + (size_t)NA_GRID * NA_REC_WORDS_PER_CTA;
-constexpr size_t NA_OFF_ITEMS = NA_OFF_HASH + (size_t)NA_GRID * NA_HASH_SLOTS;
-constexpr size_t NA_OFF_FRONT = NA_OFF_ITEMS + NA_ITEM_WORDS;  // 8-byte aligned: all sizes above are even
-constexpr size_t NA_WORDS = NA_OFF_FRONT + (size_t)NA_GRID * 3u * 2u * NA_LEVEL_MAX;
+constexpr size_t NA_OFF_HASH = NA_OFF_RECS + (size_t)NA_MAX * NA_REC_WORDS_PER_CHART;
+constexpr size_t NA_OFF_ITEMS = NA_OFF_HASH + (size_t)NA_MAX * NA_HASH_SLOTS;
+// per (chart, trie node) one uint16: which Earley set the node's bytes lead to
+constexpr size_t NA_ST_ENTRIES = 8u << 20;
+constexpr size_t NA_OFF_ST = NA_OFF_ITEMS + NA_ITEM_WORDS;
+constexpr size_t NA_OFF_REQ = NA_OFF_ST + NA_ST_ENTRIES / 2;       // 8-byte aligned: all sizes above are even
+constexpr size_t NA_WORDS = NA_OFF_REQ + 2 * (size_t)NA_REQ_CAP;
 static_assert(CNT_TOTAL <= NA_OFF_JOBS, "the counters overlap the job list");
-static_assert(NA_OFF_BAD + NA_MAX <= NA_HEADER_WORDS, "header too small");
+static_assert(NA_OFF_JOBINFO + 4 * NA_MAX <= NA_HEADER_WORDS, "header too small");
+static_assert((NA_OFF_JOBINFO % 4) == 0, "job records must be 16-byte aligned");
 static_assert((NA_OFF_CHART % 2) == 0, "64-bit offsets must be 8-byte aligned");
 
-// ~41 MB, held by every GPU that loads the library until the process exits
+// ~52 MB, held by every GPU that loads the library until the process exits
 static __device__ __align__(256) uint32_t g_noalloc_scratch[NA_WORDS];
 
 struct Offsets {
@@ -80,11 +83,11 @@ __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scrat
     S.row_flags[r] = 0u;
   }
   for (size_t i = tid; i < (size_t)n * G.Wm; i += nth) mask[i] = 0u;
+  if (tid == 0) S.counters[CNT_AUTO_ITEMS] = 0u;
   uint32_t* big = S.big_scratch;
   const size_t per_warp = (size_t)NA_ARENA_ITEMS + NA_HSET_SLOTS;
   for (size_t i = tid; i < NA_WARPS * NA_HSET_SLOTS; i += nth)
     big[(i / NA_HSET_SLOTS) * per_warp + NA_ARENA_ITEMS + (i % NA_HSET_SLOTS)] = 0xffffffffu;
-  for (size_t i = tid; i < (size_t)NA_GRID * NA_HASH_SLOTS; i += nth) S.au.hash[i] = 0u;  // the overflow hashes start empty
 }
 
 // One thread: the job list holds the charts whose header was accepted.
@@ -144,9 +147,10 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   if (!G) return fail(FMT_ERR_INVALID_ARG, "the grammar was compiled host_only");
   if (cudaGetDevice(&dev) != cudaSuccess || dev != gdev || dev < 0 || dev >= kMaxDevices)
     return fail(FMT_ERR_INVALID_ARG, "the grammar belongs to another device than the current one");
-  if (G->max_level > NA_LEVEL_MAX)
+  const size_t st_stride = ((size_t)G->T + 63u) & ~(size_t)63u;
+  if ((size_t)n * st_stride > NA_ST_ENTRIES)
     return fail(FMT_ERR_CAPACITY,
-                "fmt_fill_mask_noalloc: a depth of the vocabulary trie has more than 128 Ki nodes, beyond the built-in scratch");
+                "fmt_fill_mask_noalloc: charts x trie nodes exceeds the built-in scratch (8 Mi entries); pass fewer charts per call");
   Offsets off;
   for (uint32_t r = 0; r <= n; ++r) {
     off.v[r] = chart_offsets[r];
@@ -170,21 +174,24 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   S.big_scratch = scratch + NA_OFF_BIG;
   S.big_arena_items = NA_ARENA_ITEMS;
   S.big_hset_slots = NA_HSET_SLOTS;
-  S.au.cap = 4096;  // with the overflow hash of 8192 slots; lowered below to what the record area holds
-  sweep_plan(*G, S.au);
-  S.au.cap = std::min<uint32_t>(S.au.cap, S.au.sm_states + NA_REC_WORDS_PER_CTA / S.au.rec_words);
-  S.au.grid = NA_GRID;
-  S.au.level_pad = NA_LEVEL_MAX;
-  S.au.gl_hash_mask = NA_HASH_SLOTS - 1;
+  S.au.rec_words = (AR_TRANS + G->n_eq + 31u) & ~31u;
+  S.au.cap = std::min<uint32_t>(1024u, NA_REC_WORDS_PER_CHART / S.au.rec_words);
+  S.au.hash_mask = NA_HASH_SLOTS - 1;
   S.au.items_cap = NA_ITEM_WORDS;
   S.au.recs = scratch + NA_OFF_RECS;
   S.au.hash = scratch + NA_OFF_HASH;
   S.au.items = scratch + NA_OFF_ITEMS;
-  S.au.front = reinterpret_cast<uint2*>(scratch + NA_OFF_FRONT);
+  S.au.n_states = scratch + NA_OFF_NSTATES;
+  S.au.st = reinterpret_cast<uint16_t*>(scratch + NA_OFF_ST);
+  S.au.st_stride = (uint32_t)st_stride;
+  S.au.req = reinterpret_cast<unsigned long long*>(scratch + NA_OFF_REQ);
+  S.au.req_cap = NA_REQ_CAP;
+  S.au.job_info = reinterpret_cast<uint4*>(scratch + NA_OFF_JOBINFO);
+  sweep_layout(*G, &S.au.smem_bytes, &S.au.tables_in_smem);
   cudaStream_t st = (cudaStream_t)stream;
   noalloc_prepare_kernel<<<256, 256, 0, st>>>(*G, S, scratch, charts_dev, off, n, mask_dev);
   noalloc_jobs_kernel<<<1, 32, 0, st>>>(S, scratch, n);
-  launch_sweep(*G, S, st);
+  launch_sweep(*G, S, (int)NA_GRID, st);
   noalloc_finish_kernel<<<n, 128, 0, st>>>(*G, S, scratch, n, mask_dev, status_dev);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(FMT_ERR_CUDA, cudaGetErrorString(e));

@@ -82,14 +82,6 @@ def test_trie_is_a_valid_csr_trie(config, kw):
             assert tok_node[t] == walk(child_off, node_byte, vocab[t])
         else:
             assert tok_node[t] == 0xFFFFFFFF
-    # per node: the token that ends there
-    node_tok = g.table(11)
-    assert len(node_tok) == T
-    for n in range(T):
-        ids = tok_ids[tok_off[n]:tok_off[n + 1]]
-        want = 0xFFFFFFFF if len(ids) == 0 else (int(ids[0]) if len(ids) == 1 else 0xFFFFFFFE)
-        assert node_tok[n] == want
-    assert node_tok[walk(child_off, node_byte, vocab[300])] == 0xFFFFFFFE
     # bytes in one class behave alike: for this grammar digits must share a class, '(' and ')' must not
     eq = g.table(10)
     assert info.n_byte_classes == len(set(eq.tolist()))
