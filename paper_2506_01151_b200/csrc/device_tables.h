@@ -65,7 +65,9 @@ enum : uint32_t {
   CNT_BAR_ERR = 31,     // a block gave up waiting at the barrier
   CNT_LEVEL_ALIVE = 32, // [MAX_TOKEN_BYTES + 2] per trie depth: some node of some job was alive
   CNT_LEVEL_REQ = 68,   // [MAX_TOKEN_BYTES + 2] per trie depth: transitions queued for computation
-  CNT_TOTAL = 104
+  CNT_HASH_GEN = 104,   // generation of the sweep's per-job hashes (1 .. 65535), advanced by every fill
+  CNT_HASH_CLEAR = 105, // this fill starts the generations over: the sweep clears the hashes first
+  CNT_TOTAL = 106
 };
 
 // Per-job automaton of hash-consed Earley sets, built on demand by the trie walk.  A "local

@@ -222,10 +222,14 @@ __global__ void __launch_bounds__(ADV_WARPS * 32) advance_kernel(GrammarDev Gg, 
 // One block decides, row by row, where each mask comes from: the state cache, another row of
 // this call with the same chart, or a fresh computation (a "job").
 __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
-  if (threadIdx.x < CNT_TOTAL - CNT_BAR) S.counters[CNT_BAR + threadIdx.x] = 0u;  // barrier and level counters
+  if (threadIdx.x < CNT_HASH_GEN - CNT_BAR) S.counters[CNT_BAR + threadIdx.x] = 0u;  // barrier and level counters
   if (threadIdx.x == 0) {
     S.counters[CNT_N_JOBS] = 0u;
     S.counters[CNT_AUTO_ITEMS] = 0u;
+    // a new generation for the sweep's hashes (1 .. 65535); when the numbers start over, this fill clears them
+    const uint32_t g = (S.counters[CNT_HASH_GEN] & 0xFFFFu) % 65535u + 1u;
+    S.counters[CNT_HASH_CLEAR] = (g == 1u && S.counters[CNT_HASH_GEN] != 0u) ? 1u : 0u;
+    S.counters[CNT_HASH_GEN] = g;
   }
   __syncthreads();
   for (uint32_t row = threadIdx.x; row < S.B; row += blockDim.x) {
@@ -360,6 +364,7 @@ struct SweepWarp {
   uint32_t* tmp8;     // shared
   uint32_t n_computed = 0, n_created = 0;  // statistics, flushed once at the end of the kernel
   uint32_t chunk_at = 0, chunk_left = 0;   // this warp's private piece of the item pool (lane 0's copy counts)
+  uint32_t gen = 1;                        // this fill's generation of the per-job hashes
 
   // A new set of job J with the items w.cur[0..n), the first nk of them its kernel: its id or T_FAIL.
   __device__ uint32_t create_set(const JobCtx& J, uint32_t n, uint32_t nk, uint32_t hash) {
@@ -423,6 +428,8 @@ struct SweepWarp {
   }
 
   // The set of job J with this kernel: its id, or T_FAIL if there is none yet.
+  // (A hash slot holds generation << 16 | id + 1; a slot of another generation, left by an earlier
+  // fill, counts as empty, so the tables are never cleared between fills.)
   template <class Member>
   __device__ uint32_t lookup_set(const JobCtx& J, uint32_t nk, uint32_t hash, Member member) {
     const uint32_t lane = lane_id();
@@ -432,8 +439,8 @@ struct SweepWarp {
       uint32_t v = 0;
       if (lane == 0) v = ld_acquire(&J.hash[slot]);
       v = __shfl_sync(FULL, v, 0);
-      if (v == 0) break;
-      if (same_set(J, v - 1u, nk, hash, member)) return v - 1u;
+      if ((v >> 16) != gen) break;
+      if (same_set(J, (v & 0xFFFFu) - 1u, nk, hash, member)) return (v & 0xFFFFu) - 1u;
       slot = (slot + 1u) & mask;
     }
     return T_FAIL;
@@ -448,11 +455,18 @@ struct SweepWarp {
     uint32_t slot = hash & mask;
     for (uint32_t probe = 0; probe <= mask && probe < 4096u; ++probe) {
       uint32_t old = 0;
-      if (lane == 0) old = atomicCAS(&J.hash[slot], 0u, id + 1u);
+      if (lane == 0) {
+        old = ld_acquire(&J.hash[slot]);
+        if ((old >> 16) != gen) {  // empty: take it, unless somebody is faster
+          const uint32_t seen = old;
+          old = atomicCAS(&J.hash[slot], seen, (gen << 16) | (id + 1u));
+          if (old == seen) old = 0u;
+        }
+      }
       old = __shfl_sync(FULL, old, 0);
       if (old == 0u) return id;
       __threadfence();
-      if (same_set(J, old - 1u, nk, hash, member)) return old - 1u;
+      if (same_set(J, (old & 0xFFFFu) - 1u, nk, hash, member)) return (old & 0xFFFFu) - 1u;
       slot = (slot + 1u) & mask;
     }
     return T_FAIL;
@@ -716,10 +730,13 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 3) sweep_kernel(GrammarDev G
   for (uint32_t i = lane; i < ntw; i += 32) nt[i] = 0u;
   __syncthreads();
 
+  // ---- the per-job hashes of Earley sets are cleared only when the 16-bit generation starts over
+  if (S.counters[CNT_HASH_CLEAR]) {
+    const size_t words = (size_t)S.B * (A.hash_mask + 1u);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += (size_t)gridDim.x * blockDim.x) A.hash[i] = 0u;
+  }
   // ---- the automata start with one state each: the base chart's last set
   for (uint32_t j = blockIdx.x; j < n_jobs; j += gridDim.x) {
-    uint32_t* hash = A.hash + (size_t)j * (A.hash_mask + 1);
-    for (uint32_t i = threadIdx.x; i <= A.hash_mask; i += blockDim.x) hash[i] = 0u;
     uint32_t* rec0 = A.recs + (size_t)j * A.cap * A.rec_words;
     for (uint32_t i = threadIdx.x; i < A.rec_words; i += blockDim.x)
       if (i < AR_SCAN || i >= AR_SCAN + 8) rec0[i] = (i >= AR_TRANS) ? T_UNKNOWN : 0u;
@@ -736,6 +753,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 3) sweep_kernel(GrammarDev G
   if (!grid_barrier(S, bar_phase)) return;
 
   SweepWarp sw{G, S};
+  sw.gen = S.counters[CNT_HASH_GEN] & 0xFFFFu;
   sw.w.nt = nt;
   sw.w.ctr = ctr;
   sw.tmp8 = tmp8;
@@ -855,33 +873,50 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 3) sweep_kernel(GrammarDev G
   // ---- mask words: 32 tokens per warp pass, one ballot per word (token t is valid iff the node
   // where its bytes end was reached alive; EOS iff the chart is accepting)
   const uint32_t Wm = G.Wm;
-  for (uint32_t c = gw; c < n_jobs * Wm; c += GW) {
-    const uint32_t j = c / Wm, wd = c % Wm;
-    const JobCtx J = job_ctx(S, j);
-    const uint32_t tok = wd * 32 + lane;
-    bool ok = false;
-    if (tok < G.V) {
-      const uint32_t node = __ldg(&G.tok_node[tok]);
-      if (node == 0xFFFFFFFFu) {
-        ok = ((int32_t)tok == G.eos) && J.accepting;
-      } else if (__ldg(&G.node_depth[node]) <= last_level) {
-        uint32_t s = __ldcg(J.st + node);
-        if (s == ST_PENDING) {  // a leaf that waited for a transition: its parent is final by now
-          const uint32_t p = __ldg(&G.parent[node]);
-          const uint32_t p_state = (p == 0) ? 0u : (uint32_t)__ldcg(J.st + p);
-          const uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node]));
-          if (t2 == T_UNKNOWN || t2 == T_PENDING || p_state == ST_PENDING) {
-            atomicOr(&S.row_flags[J.row], ROW_BROKEN);
-            s = ST_DEAD;
-          } else {
-            s = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
-          }
-        }
-        ok = s != ST_DEAD;
+  constexpr uint32_t MW = 4;  // mask words per warp and iteration: their loads are in flight together
+  for (uint32_t c0 = gw; c0 < n_jobs * Wm; c0 += MW * GW) {
+    uint32_t node[MW], s_[MW];
+    bool valid[MW], eos_ok[MW];
+#pragma unroll
+    for (uint32_t u = 0; u < MW; ++u) {
+      const uint32_t c = c0 + u * GW;
+      valid[u] = c < n_jobs * Wm;
+      const uint32_t tok = (c % Wm) * 32 + lane;
+      node[u] = (valid[u] && tok < G.V) ? __ldg(&G.tok_node[tok]) : 0xFFFFFFFEu;
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < MW; ++u) {
+      const uint32_t c = c0 + u * GW;
+      s_[u] = ST_DEAD;
+      eos_ok[u] = false;
+      if (node[u] == 0xFFFFFFFFu) {  // a token without bytes: only EOS can be valid
+        const uint32_t tok = (c % Wm) * 32 + lane;
+        eos_ok[u] = ((int32_t)tok == G.eos) && job_ctx(S, c / Wm).accepting;
+      } else if (node[u] != 0xFFFFFFFEu && __ldg(&G.node_depth[node[u]]) <= last_level) {
+        s_[u] = __ldcg(A.st + (size_t)(c / Wm) * A.st_stride + node[u]);
       }
     }
-    const uint32_t word = __ballot_sync(FULL, ok);
-    if (lane == 0) S.mask_rows[(size_t)S.row_mask[J.row] * Wm + wd] = word;
+#pragma unroll
+    for (uint32_t u = 0; u < MW; ++u) {
+      if (!valid[u]) continue;  // (uniform)
+      const uint32_t c = c0 + u * GW;
+      const uint32_t j = c / Wm, wd = c % Wm;
+      const JobCtx J = job_ctx(S, j);
+      uint32_t s = s_[u];
+      if (s == ST_PENDING) {  // a leaf that waited for a transition: its parent is final by now
+        const uint32_t p = __ldg(&G.parent[node[u]]);
+        const uint32_t p_state = (p == 0) ? 0u : (uint32_t)__ldcg(J.st + p);
+        const uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
+        if (t2 == T_UNKNOWN || t2 == T_PENDING || p_state == ST_PENDING) {
+          atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+          s = ST_DEAD;
+        } else {
+          s = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+        }
+      }
+      const uint32_t word = __ballot_sync(FULL, s != ST_DEAD || eos_ok[u]);
+      if (lane == 0) S.mask_rows[(size_t)S.row_mask[J.row] * Wm + wd] = word;
+    }
   }
 }
 

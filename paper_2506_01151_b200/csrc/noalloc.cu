@@ -67,7 +67,7 @@ __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scrat
                                        uint32_t n, uint32_t* mask) {
   const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t nth = (size_t)gridDim.x * blockDim.x;
-  if (tid < CNT_TOTAL) S.counters[tid] = 0u;
+  if (tid < CNT_TOTAL) S.counters[tid] = (tid == CNT_HASH_GEN) ? 1u : 0u;  // the hashes are cleared below: every call is generation 1
   if (tid < n) {
     const uint32_t r = (uint32_t)tid;
     const uint32_t* ch = charts + off.v[r];
@@ -83,7 +83,7 @@ __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scrat
     S.row_flags[r] = 0u;
   }
   for (size_t i = tid; i < (size_t)n * G.Wm; i += nth) mask[i] = 0u;
-  if (tid == 0) S.counters[CNT_AUTO_ITEMS] = 0u;
+  for (size_t i = tid; i < (size_t)NA_MAX * NA_HASH_SLOTS; i += nth) S.au.hash[i] = 0u;
   uint32_t* big = S.big_scratch;
   const size_t per_warp = (size_t)NA_ARENA_ITEMS + NA_HSET_SLOTS;
   for (size_t i = tid; i < NA_WARPS * NA_HSET_SLOTS; i += nth)
