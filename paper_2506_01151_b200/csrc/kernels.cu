@@ -517,6 +517,7 @@ struct SweepWarp {
     uint32_t plen;
     AutoView view{J, S.au};
     view(ps == 0 ? J.m - 1 : J.m + ps, pitems, plen);
+    if (plen > 8u * 32u) return T_RETRY;  // a large set seldom scans into a small one
     const uint32_t self_code = J.m + ps;
     uint32_t n = 0, mine = 0;
     __syncwarp();
