@@ -58,12 +58,6 @@ struct ChartView {
   __device__ __forceinline__ uint32_t fix(uint32_t item, uint32_t) const { return item; }
 };
 
-__device__ __forceinline__ void clear_nt(const GrammarDev& G, const WarpCtx& w) {
-  __syncwarp();
-  for (uint32_t i = lane_id(); i < 2 * G.Nw; i += 32) w.nt[i] = 0u;
-  __syncwarp();
-}
-
 __device__ __forceinline__ void push_need(const AdvScratch& s, uint32_t o, uint32_t A) {
   uint32_t key = (o << 16) | A;
   int r = hset_insert(s.w.hset, s.w.hset_mask, key);
@@ -204,25 +198,41 @@ __device__ int token_step(const GrammarDev& G, AdvScratch& s, const uint32_t* sr
     __syncwarp();
     if (lane < W_CTRS) s.w.ctr[lane] = 0u;
     __syncwarp();
-    uint32_t n = scan_into_cur(G, s.w, prev, prev_len, __ldg(&bytes[L - 1]));
-    if (s.w.ctr[W_OVERFLOW]) {
-      hset_clear_all(s.w.hset, s.w.hset_mask);
-      return -2;
-    }
-    if (n == 0) return 0;
+    const uint32_t byte = __ldg(&bytes[L - 1]);
     const uint32_t index = m - 1 + L;
-    complete_fixpoint(G, s.w, view, index, 0u);
-    uint32_t hashed = min(s.w.ctr[W_NCUR], s.w.cur_cap);
-    if (s.w.ctr[W_OVERFLOW]) {
-      hset_clear_all(s.w.hset, s.w.hset_mask);
-      clear_nt(G, s.w);
-      return -2;
+    uint32_t n;
+    // sets of up to 32 scanned and completed items (nearly all) are built in lanes ...
+    uint32_t mine;
+    const uint32_t ns = (prev_len <= 96u) ? small_scan_complete(G, s.w, view, prev, prev_len, byte, index,
+                                                                 [](uint32_t it) { return it; }, mine, accepting)
+                                           : SMALL_OVERFLOW;
+    if (ns == 0) return 0;
+    if (ns != SMALL_OVERFLOW) {
+      const uint32_t nk = small_drop_completed(G, s.w, ns, mine);
+      if (lane == 0) s.w.ctr[W_NCUR] = nk;
+      predict_into_cur(G, s.w, index);
+      if (s.w.ctr[W_OVERFLOW]) return -2;
+      n = min(s.w.ctr[W_NCUR], s.w.cur_cap);
+    } else {  // ... larger ones with the uniqueness hash
+      n = scan_into_cur(G, s.w, prev, prev_len, byte);
+      if (s.w.ctr[W_OVERFLOW]) {
+        hset_clear_all(s.w.hset, s.w.hset_mask);
+        return -2;
+      }
+      if (n == 0) return 0;
+      complete_fixpoint(G, s.w, view, index, 0u);
+      uint32_t hashed = min(s.w.ctr[W_NCUR], s.w.cur_cap);
+      if (s.w.ctr[W_OVERFLOW]) {
+        hset_clear_all(s.w.hset, s.w.hset_mask);
+        clear_nt(G, s.w);
+        return -2;
+      }
+      hset_clear_items(s.w, hashed);
+      accepting = s.w.ctr[W_ACCEPT] != 0u;
+      predict_into_cur(G, s.w, index);
+      if (s.w.ctr[W_OVERFLOW]) return -2;
+      n = drop_completed(G, s.w, min(s.w.ctr[W_NCUR], s.w.cur_cap));
     }
-    hset_clear_items(s.w, hashed);
-    accepting = s.w.ctr[W_ACCEPT] != 0u;
-    predict_into_cur(G, s.w, index);
-    if (s.w.ctr[W_OVERFLOW]) return -2;
-    n = drop_completed(G, s.w, min(s.w.ctr[W_NCUR], s.w.cur_cap));
     prev = arena + top;
     prev_len = n;
     top += n;
@@ -241,29 +251,45 @@ __device__ int token_step(const GrammarDev& G, AdvScratch& s, const uint32_t* sr
     uint32_t it = arena[last_at + i];
     if ((it >> 16) < last) push_need(s, it >> 16, __ldg(&G.lhs[it & 0xFFFFu]));
   }
-  for (uint32_t head = 0;;) {  // needs are served a wave at a time, one lane per (set, non-terminal) need
+  // needs are served a wave at a time: a need whose set is short is served by its own lane, the
+  // needs of long sets (alternations of many literals predicted at once) by the whole warp in turn
+  constexpr uint32_t NEED_SHORT = 8;
+  for (uint32_t head = 0;;) {
     __syncwarp();
     const uint32_t np = min(s.w.ctr[W_NPAIRS], ADV_PAIRS);
     __syncwarp();
     if (head >= np) break;
     const uint32_t mine = head + lane;
+    uint32_t o = 0, A = 0, sl = 0, base = 0;
+    const uint32_t* sp = nullptr;
     if (mine < np) {
       const uint32_t key = s.pairs[mine];
-      const uint32_t o = key >> 16, A = key & 0xFFFFu;
-      const uint32_t* sp;
-      uint32_t sl;
+      o = key >> 16, A = key & 0xFFFFu;
       view(o, sp, sl);
-      const uint32_t base = view.bit_base(o, n_items);
-      for (uint32_t k = 0; k < sl; ++k) {
-        const uint32_t wi = sp[k];
-        const uint32_t inf = G.info[wi & 0xFFFFu];
-        if ((inf >> INFO_KIND_SHIFT) == KIND_NT && (inf & INFO_ARG_MASK) == A) {
-          const uint32_t pos = base + k;
-          const uint32_t bit = 1u << (pos & 31u);
-          const uint32_t old = atomicOr(&s.live[pos >> 5], bit);
-          if (!(old & bit)) push_need(s, wi >> 16, __ldg(&G.lhs[wi & 0xFFFFu]));
-        }
+      base = view.bit_base(o, n_items);
+    }
+    auto serve = [&](const uint32_t* set, uint32_t k, uint32_t bit_base, uint32_t want) {
+      const uint32_t wi = set[k];
+      const uint32_t inf = G.info[wi & 0xFFFFu];
+      if ((inf >> INFO_KIND_SHIFT) == KIND_NT && (inf & INFO_ARG_MASK) == want) {
+        const uint32_t pos = bit_base + k;
+        const uint32_t bit = 1u << (pos & 31u);
+        const uint32_t old = atomicOr(&s.live[pos >> 5], bit);
+        if (!(old & bit)) push_need(s, wi >> 16, __ldg(&G.lhs[wi & 0xFFFFu]));
       }
+    };
+    if (sl <= NEED_SHORT)
+      for (uint32_t k = 0; k < sl; ++k) serve(sp, k, base, A);
+    uint32_t longs = __ballot_sync(FULL, sl > NEED_SHORT);
+    while (longs) {
+      const int src = __ffs(longs) - 1;
+      longs &= longs - 1;
+      const uint32_t so = __shfl_sync(FULL, o, src), sA = __shfl_sync(FULL, A, src);
+      const uint32_t* lp;
+      uint32_t ll;
+      view(so, lp, ll);
+      const uint32_t lbase = view.bit_base(so, n_items);
+      for (uint32_t k = lane; k < ll; k += 32) serve(lp, k, lbase, sA);
     }
     head = min(head + 32u, np);
   }

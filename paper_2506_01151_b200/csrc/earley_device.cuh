@@ -239,6 +239,123 @@ __device__ __forceinline__ bool hset_contains(const uint32_t* hset, uint32_t mas
   return false;
 }
 
+__device__ __forceinline__ void clear_nt(const GrammarDev& G, const WarpCtx& w) {
+  __syncwarp();
+  for (uint32_t i = lane_id(); i < 2 * G.Nw; i += 32) w.nt[i] = 0u;
+  __syncwarp();
+}
+
+// ---- The lane-resident form of Scan and Complete, for sets of at most 32 items: the set under
+// construction sits one item per lane (and in w.cur[0..n)), uniqueness is a matter of shuffles and
+// ballots, and neither the uniqueness hash nor a shared-memory counter is touched.
+constexpr uint32_t SMALL_OVERFLOW = 0xffffffffu;
+
+// The candidates c .. c + skip of the lanes with `v` set join cur[0..n) unless already there.
+// `mine` is cur[lane].  Returns the new count, above 32 when they do not fit.
+__device__ __forceinline__ uint32_t append_small(const WarpCtx& w, uint32_t c, bool v, uint32_t skip, uint32_t n,
+                                                 uint32_t& mine) {
+  const uint32_t lane = lane_id();
+  const uint32_t maxskip = __reduce_max_sync(FULL, v ? skip : 0u);
+  for (uint32_t j = 0; j <= maxskip; ++j) {
+    const bool vj = v && j <= skip;
+    const uint32_t cj = c + j;
+    const uint32_t vm = __ballot_sync(FULL, vj);
+    if (!vm) continue;
+    bool keep = vj;
+    if (vj) keep = (uint32_t)(__ffs(__match_any_sync(vm, cj)) - 1) == lane;  // one of equal candidates
+    for (uint32_t i = 0; i < n; ++i)
+      if (__shfl_sync(FULL, mine, i) == cj) keep = false;
+    const uint32_t kb = __ballot_sync(FULL, keep);
+    const uint32_t nn = n + __popc(kb);
+    if (nn > 32u) return nn;
+    if (keep) w.cur[n + __popc(kb & ((1u << lane) - 1u))] = cj;
+    __syncwarp();
+    n = nn;
+    mine = lane < n ? w.cur[lane] : 0u;
+  }
+  return n;
+}
+
+// Scan the items of `set` over `byte`, then Complete to a fixpoint (Section 3.2), all in lanes.
+// `rename(item)` rewrites an item of `set` into the naming of the new set (identity for plain
+// charts); `view` and `cur_index` are as for complete_fixpoint.  On return the lanes' `mine` and
+// w.cur[0..n) hold the n <= 32 items (completed ones included), the non-terminals found after a
+// dot are collected in w.nt[0..Nw), and `accept` tells whether the accept item is among them.
+// Returns n (0: the byte cannot follow), or SMALL_OVERFLOW when the set outgrows 32 items (w.nt is
+// clean then and the caller takes the general path).
+template <class View, class Rename>
+__device__ __forceinline__ uint32_t small_scan_complete(const GrammarDev& G, const WarpCtx& w, const View& view,
+                                                        const uint32_t* set, uint32_t len, uint32_t byte, uint32_t cur_index,
+                                                        Rename rename, uint32_t& mine, bool& accept) {
+  const uint32_t lane = lane_id();
+  uint32_t n = 0;
+  mine = 0;
+  accept = false;
+  __syncwarp();
+  for (uint32_t base = 0; base < len; base += 32) {
+    const uint32_t k = base + lane;
+    uint32_t it = k < len ? set[k] : 0u;
+    const uint32_t inf = k < len ? G.info[it & 0xFFFFu] : 0u;
+    const bool hit = (inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte);
+    it = rename(it);
+    const uint32_t skip = hit ? (G.info[(it + 1u) & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
+    if (__any_sync(FULL, hit)) n = append_small(w, it + 1u, hit, skip, n, mine);
+    if (n > 32u) return SMALL_OVERFLOW;
+  }
+  if (n == 0) return 0;
+  uint32_t head = 0;  // lanes [head, n) hold the items not looked at yet
+  while (head < n) {
+    const bool have = lane >= head && lane < n;
+    const uint32_t inf = have ? G.info[mine & 0xFFFFu] : 0u;
+    const uint32_t kind = inf >> INFO_KIND_SHIFT;
+    if (have && kind == KIND_NT) {
+      const uint32_t y = inf & INFO_ARG_MASK;
+      atomicOr(&w.nt[y >> 5], 1u << (y & 31u));
+    }
+    if (__any_sync(FULL, have && kind == KIND_END && (mine & 0xFFFFu) == ITEM_ACCEPT)) accept = true;
+    uint32_t bal = __ballot_sync(FULL, have && kind == KIND_END && (mine >> 16) != cur_index);
+    const uint32_t it = mine;
+    head = n;
+    while (bal) {
+      const int src = __ffs(bal) - 1;
+      bal &= bal - 1;
+      const uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, src);
+      const uint32_t o = __shfl_sync(FULL, it >> 16, src);
+      const uint32_t* sp;
+      uint32_t sl;
+      view(o, sp, sl);
+      for (uint32_t base = 0; base < sl; base += 32) {
+        const uint32_t k = base + lane;
+        const uint32_t wi = k < sl ? sp[k] : 0u;
+        const uint32_t winf = k < sl ? G.info[wi & 0xFFFFu] : 0u;
+        const bool match = (winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X;
+        const uint32_t cand = view.fix(wi, o) + 1u;
+        const uint32_t skip = match ? (G.info[cand & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
+        if (__any_sync(FULL, match)) n = append_small(w, cand, match, skip, n, mine);
+        if (n > 32u) {
+          clear_nt(G, w);
+          return SMALL_OVERFLOW;
+        }
+      }
+    }
+  }
+  return n;
+}
+
+// Drop the completed items of a lane-resident set: the others move to cur[0..count) and to the
+// first lanes' `mine`.  Returns their count.
+__device__ __forceinline__ uint32_t small_drop_completed(const GrammarDev& G, const WarpCtx& w, uint32_t n, uint32_t& mine) {
+  const uint32_t lane = lane_id();
+  const bool keep = lane < n && (G.info[mine & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
+  const uint32_t kb = __ballot_sync(FULL, keep);
+  __syncwarp();
+  if (keep) w.cur[__popc(kb & ((1u << lane) - 1u))] = mine;
+  __syncwarp();
+  const uint32_t nk = __popc(kb);
+  mine = lane < nk ? w.cur[lane] : 0u;
+  return nk;
+}
+
 // Copy the grammar's hot tables into shared memory (all threads of the block take part, the
 // caller synchronizes) and return a view of the grammar that reads them from there.
 __device__ __forceinline__ GrammarDev stage_hot_tables(const GrammarDev& Gg, uint32_t* dst) {

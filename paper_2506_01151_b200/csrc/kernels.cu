@@ -138,7 +138,7 @@ constexpr int ADV_WARPS = 4;
 
 constexpr uint32_t HOT_TABLE_BYTES = 24 * 1024;  // grammar tables up to this size are staged in shared memory
 
-__global__ void __launch_bounds__(ADV_WARPS * 32) advance_kernel(GrammarDev Gg, StateDev S, const int32_t* tokens,
+__global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev Gg, StateDev S, const int32_t* tokens,
                                                                   int32_t* status) {
   extern __shared__ __align__(16) uint32_t smem[];
   const uint32_t warp = threadIdx.x >> 5, lane = lane_id();
@@ -486,31 +486,7 @@ struct SweepWarp {
     return id == T_FAIL ? T_FAIL : insert_set(J, id, nk, hash, member);
   }
 
-  // (lane-resident form) The candidates c .. c + skip of the lanes with `v` set join cur[0..n)
-  // unless already there.  `mine` is cur[lane].  Returns the new count, above 32 when they do not fit.
-  __device__ __forceinline__ uint32_t append_small(uint32_t c, bool v, uint32_t skip, uint32_t n, uint32_t& mine) {
-    const uint32_t lane = lane_id();
-    const uint32_t maxskip = __reduce_max_sync(FULL, v ? skip : 0u);
-    for (uint32_t j = 0; j <= maxskip; ++j) {
-      const bool vj = v && j <= skip;
-      const uint32_t cj = c + j;
-      const uint32_t vm = __ballot_sync(FULL, vj);
-      if (!vm) continue;
-      bool keep = vj;
-      if (vj) keep = (uint32_t)(__ffs(__match_any_sync(vm, cj)) - 1) == lane;  // one of equal candidates
-      for (uint32_t i = 0; i < n; ++i)
-        if (__shfl_sync(FULL, mine, i) == cj) keep = false;
-      const uint32_t kb = __ballot_sync(FULL, keep);
-      const uint32_t nn = n + __popc(kb);
-      if (nn > 32u) return nn;
-      if (keep) w.cur[n + __popc(kb & ((1u << lane) - 1u))] = cj;
-      __syncwarp();
-      n = nn;
-      mine = lane < n ? w.cur[lane] : 0u;
-    }
-    return n;
-  }
-
+  // The lane-resident form (see small_scan_complete).
   __device__ uint32_t compute_small(const JobCtx& J, uint32_t ps, uint32_t byte) {
     const uint32_t lane = lane_id();
     const uint32_t* pitems;
@@ -519,67 +495,18 @@ struct SweepWarp {
     view(ps == 0 ? J.m - 1 : J.m + ps, pitems, plen);
     if (plen > 8u * 32u) return T_RETRY;  // a large set seldom scans into a small one
     const uint32_t self_code = J.m + ps;
-    uint32_t n = 0, mine = 0;
-    __syncwarp();
-    // ---- scan
-    for (uint32_t base = 0; base < plen; base += 32) {
-      const uint32_t k = base + lane;
-      uint32_t it = k < plen ? pitems[k] : 0u;
-      const uint32_t inf = k < plen ? G.info[it & 0xFFFFu] : 0u;
-      const bool hit = (inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte);
-      if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
-      const uint32_t skip = hit ? (G.info[(it + 1u) & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
-      if (__any_sync(FULL, hit)) n = append_small(it + 1u, hit, skip, n, mine);
-      if (n > 32u) return T_RETRY;
-    }
+    uint32_t mine;
+    bool accept;
+    const uint32_t n = small_scan_complete(
+        G, w, view, pitems, plen, byte, ORIGIN_SELF,
+        [&](uint32_t it) { return ((it >> 16) == ORIGIN_SELF) ? ((self_code << 16) | (it & 0xFFFFu)) : it; }, mine, accept);
+    if (n == SMALL_OVERFLOW) return T_RETRY;
     if (n == 0) return T_DEAD;
-    // ---- complete to a fixpoint: lanes [head, n) hold the items not looked at yet
-    uint32_t head = 0;
-    while (head < n) {
-      const bool have = lane >= head && lane < n;
-      const uint32_t inf = have ? G.info[mine & 0xFFFFu] : 0u;
-      const uint32_t kind = inf >> INFO_KIND_SHIFT;
-      if (have && kind == KIND_NT) {
-        const uint32_t y = inf & INFO_ARG_MASK;
-        atomicOr(&w.nt[y >> 5], 1u << (y & 31u));
-      }
-      uint32_t bal = __ballot_sync(FULL, have && kind == KIND_END && (mine >> 16) != ORIGIN_SELF);
-      const uint32_t it = mine;
-      head = n;
-      while (bal) {
-        const int src = __ffs(bal) - 1;
-        bal &= bal - 1;
-        const uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, src);
-        const uint32_t o = __shfl_sync(FULL, it >> 16, src);
-        const uint32_t* sp;
-        uint32_t sl;
-        view(o, sp, sl);
-        for (uint32_t base = 0; base < sl; base += 32) {
-          const uint32_t k = base + lane;
-          const uint32_t wi = k < sl ? sp[k] : 0u;
-          const uint32_t winf = k < sl ? G.info[wi & 0xFFFFu] : 0u;
-          const bool match = (winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X;
-          const uint32_t cand = view.fix(wi, o) + 1u;
-          const uint32_t skip = match ? (G.info[cand & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
-          if (__any_sync(FULL, match)) n = append_small(cand, match, skip, n, mine);
-          if (n > 32u) {
-            clear_nt(G, w);
-            return T_RETRY;
-          }
-        }
-      }
-    }
     // ---- the kernel: what is left when the completed items go
-    const bool keep = lane < n && (G.info[mine & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
-    const uint32_t kb = __ballot_sync(FULL, keep);
-    const uint32_t nk = __popc(kb);
-    uint32_t h = keep ? mix32(mine) : 0u;
+    const uint32_t nk = small_drop_completed(G, w, n, mine);
+    uint32_t h = lane < nk ? mix32(mine) : 0u;
     for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
     h = mix32(h + nk * 0x9E3779B9u);
-    __syncwarp();
-    if (keep) w.cur[__popc(kb & ((1u << lane) - 1u))] = mine;
-    __syncwarp();
-    mine = lane < nk ? w.cur[lane] : 0u;
     auto member = [&](uint32_t x, bool valid) {  // the kernel sits one item per lane
       bool found = false;
       for (uint32_t i = 0; i < nk; ++i)
