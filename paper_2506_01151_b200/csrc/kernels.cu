@@ -284,7 +284,6 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
 // the kernel is launched cooperatively so that all CTAs are resident, and the barrier gives up
 // (and flags an error) after a bounded number of polls instead of hanging.
 
-constexpr int SWEEP_WARPS = 8;
 constexpr uint32_t SWEEP_CUR = 512;     // items of a set under construction per warp (fast mode, power of two)
 constexpr uint32_t SWEEP_HSET = 1024;   // uniqueness hash slots per warp (fast mode)
 
@@ -633,7 +632,7 @@ __device__ __forceinline__ uint32_t settled(const GrammarDev& G, const AutoDev& 
 
 constexpr uint32_t SWEEP_PER_LANE = 4;  // trie nodes per lane and pass iteration (independent loads in flight)
 
-__global__ void __launch_bounds__(SWEEP_WARPS * 32, 3) sweep_kernel(GrammarDev Gg, StateDev S) {
+__global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev Gg, StateDev S) {
   const uint32_t n_jobs = S.counters[CNT_N_JOBS];
   if (n_jobs == 0) return;  // every CTA sees the same count: nobody is left at a barrier
   extern __shared__ __align__(16) uint32_t smem[];
@@ -1055,7 +1054,7 @@ cudaError_t configure_kernels() {
   cudaError_t e;
   if ((e = opt_in_smem((const void*)init_kernel, init_smem_bytes())) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)advance_kernel, (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + HOT_TABLE_BYTES)) != cudaSuccess) return e;
-  if ((e = opt_in_smem((const void*)sweep_kernel, 160 * 1024)) != cudaSuccess) return e;
+  if ((e = opt_in_smem((const void*)sweep_kernel, 224 * 1024)) != cudaSuccess) return e;
   return cudaSuccess;
 }
 

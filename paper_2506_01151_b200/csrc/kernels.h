@@ -6,6 +6,8 @@
 
 namespace fmt {
 
+constexpr int SWEEP_WARPS = 24;  // warps of a CTA of the trie sweep: one CTA per SM, so that the grid barrier has few arrivals
+
 cudaError_t configure_kernels();
 cudaError_t sweep_blocks_per_sm(int* out, uint32_t smem_bytes);
 void sweep_layout(const GrammarDev& G, uint32_t* smem_bytes, uint32_t* tables_in_smem);

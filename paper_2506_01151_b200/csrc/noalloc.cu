@@ -18,7 +18,7 @@ namespace {
 using namespace fmt;
 
 constexpr uint32_t NA_MAX = FMT_NOALLOC_MAX_CHARTS;
-constexpr uint32_t NA_GRID = 32;            // CTAs of the sweep
+constexpr uint32_t NA_GRID = 12;            // CTAs of the sweep
 constexpr uint32_t NA_ARENA_ITEMS = 8192;   // per-warp overflow area for Earley sets (items)
 constexpr uint32_t NA_HSET_SLOTS = 2048;    // per-warp overflow uniqueness hash
 // header: counters, then per-chart arrays
@@ -32,7 +32,7 @@ constexpr uint32_t NA_OFF_BAD = NA_OFF_CHART + 2 * NA_MAX;       // [NA_MAX] hea
 constexpr uint32_t NA_OFF_NSTATES = NA_OFF_BAD + NA_MAX;         // [NA_MAX] Earley sets created per chart
 constexpr uint32_t NA_OFF_JOBINFO = NA_OFF_NSTATES + NA_MAX;     // [NA_MAX] uint4 (16-byte aligned)
 constexpr uint32_t NA_HEADER_WORDS = 1024;
-constexpr size_t NA_WARPS = (size_t)NA_GRID * 8;
+constexpr size_t NA_WARPS = (size_t)NA_GRID * SWEEP_WARPS;
 constexpr size_t NA_BIG_WORDS = NA_WARPS * (NA_ARENA_ITEMS + NA_HSET_SLOTS);
 // the sweep's tables of Earley sets: per chart 64 Ki words of records and 2048 hash slots, and one
 // pool of 2 Mi item words for all charts of a call
