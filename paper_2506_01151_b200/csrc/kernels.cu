@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
     S.counters[CNT_AUTO_ITEMS] = 0u;
     // a new generation for the sweep's hashes (1 .. 65535); when the numbers start over, this fill clears them
     const uint32_t g = (S.counters[CNT_HASH_GEN] & 0xFFFFu) % 65535u + 1u;
-    S.counters[CNT_HASH_CLEAR] = (g == 1u && S.counters[CNT_HASH_GEN] != 0u) ? 1u : 0u;
+    if (g == 1u && S.counters[CNT_HASH_GEN] != 0u) S.counters[CNT_HASH_CLEAR] = 1u;  // stays set until a sweep has done it
     S.counters[CNT_HASH_GEN] = g;
   }
   __syncthreads();
@@ -678,6 +678,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     }
   }
   if (!grid_barrier(S, bar_phase)) return;
+  if (blockIdx.x == 0 && threadIdx.x == 0) S.counters[CNT_HASH_CLEAR] = 0u;  // done above, if it was asked for
 
   SweepWarp sw{G, S};
   sw.gen = S.counters[CNT_HASH_GEN] & 0xFFFFu;

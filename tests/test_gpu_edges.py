@@ -261,3 +261,34 @@ def test_capacity_overflow_is_reported_not_guessed():
         assert _advance(st2, [c]) == [0]
     _mask_of(st2, g, 1)
     assert st2.stats()["capacity_errors"] == 0 or not _mask_of(st2, g, 1).any()
+
+
+def test_sweep_hash_generations_start_over():
+    """The sweep's per-job hashes of Earley sets are never cleared between fills: every fill has a
+    16-bit generation and takes slots of other generations for empty.  After 65535 fills the numbers
+    start over, and that fill must clear the hashes first or it would meet its own old entries.
+    Two rows with the cache off (every fill sweeps) go through more than 65535 fills; the masks
+    before, at and after the turn must equal the oracle's."""
+    import paper_2506_01151_b200 as fmt
+
+    torch, dev = _torch()
+    w = workloads.build(1, steps=4)
+    g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
+    og, ov = oracle.Grammar(w.ebnf, w.start), oracle.Vocab(w.vocab, w.eos)
+    st = fmt.State(g, 2, cache=False)
+    seqs = [oracle.Sequence_(og) for _ in range(2)]
+    for b, text in enumerate([b"(1+", b"12*(3"]):
+        toks = [w.vocab.index(bytes([c])) for c in text]  # the single bytes are tokens 0..255
+        for t in toks:
+            ids = [-1, -1]
+            ids[b] = t
+            assert _advance(st, ids)[b] == fmt.FMT_OK
+        assert seqs[b].advance(text)
+    want = np.stack([s.mask(ov) for s in seqs])
+    m = torch.zeros((2, g.mask_words), dtype=torch.int32, device=dev)
+    total = 65535 + 40
+    for i in range(total):
+        st.fill_mask(m)
+        if i in (0, 65533, 65534, 65535, 65536, total - 1):
+            assert np.array_equal(m.cpu().numpy().view(np.uint32), want), i
+    assert st.stats()["capacity_errors"] == 0
