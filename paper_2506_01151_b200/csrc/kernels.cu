@@ -563,19 +563,18 @@ struct SweepWarp {
     }
     for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
     h = mix32(h + nk * 0x9E3779B9u);
-    const uint32_t id = lookup_set(J, nk, h, [&](uint32_t x, bool valid) { return !valid || hset_contains(w.hset, w.hset_mask, x); });
-    hset_clear_items(w, hashed);
+    auto member = [&](uint32_t x, bool valid) { return !valid || hset_contains(w.hset, w.hset_mask, x); };
+    const uint32_t id = lookup_set(J, nk, h, member);
     if (id != T_FAIL) {
+      hset_clear_items(w, hashed);
       clear_nt(G, w);
       return id;
     }
+    // a new set: its items stay in the uniqueness hash, for the comparisons that entering the set
+    // may need (the completed items among them do no harm: no stored kernel holds one)
     drop_completed(G, w, hashed);
-    // the kernel is cur[0..nk) now and no longer in the hash: a set met while entering this one is compared item by item
-    const uint32_t r = finish_new(J, nk, h, [&](uint32_t x, bool valid) {
-      bool found = !valid;
-      for (uint32_t i = 0; i < nk && !found; ++i) found = w.cur[i] == x;
-      return found;
-    });
+    const uint32_t r = finish_new(J, nk, h, member);
+    hset_clear_all(w.hset, w.hset_mask);
     return r == T_RETRY ? T_FAIL : r;
   }
 
