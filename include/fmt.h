@@ -225,7 +225,7 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
  * but it needs an fmt_state, whose creation allocates hundreds of megabytes.  This call needs no
  * fmt_state: it sweeps the vocabulary trie for charts the caller already holds in device memory
  * (in the layout fmt_state_copy_chart documents) and uses a fixed scratch array that is part of
- * the loaded library image (about 52 MB of device memory on every GPU that loads the library,
+ * the loaded library image (about 55 MB of device memory on every GPU that loads the library,
  * held until the process exits).
  *
  *   g              a grammar compiled for the current device

@@ -53,7 +53,7 @@ static_assert(NA_OFF_JOBINFO + 4 * NA_MAX <= NA_HEADER_WORDS, "header too small"
 static_assert((NA_OFF_JOBINFO % 4) == 0, "job records must be 16-byte aligned");
 static_assert((NA_OFF_CHART % 2) == 0, "64-bit offsets must be 8-byte aligned");
 
-// ~52 MB, held by every GPU that loads the library until the process exits
+// ~55 MB, held by every GPU that loads the library until the process exits
 static __device__ __align__(256) uint32_t g_noalloc_scratch[NA_WORDS];
 
 struct Offsets {
