@@ -301,7 +301,9 @@ def run_ours(args):
                   "capacity_errors": stats1["capacity_errors"],
                   "sweep_transitions": stats1["sweep_transitions"] - stats0["sweep_transitions"],
                   "sweep_states": stats1["sweep_states"] - stats0["sweep_states"],
-                  "big_mode": stats1["big_mode_units"] - stats0["big_mode_units"]},
+                  "big_mode": stats1["big_mode_units"] - stats0["big_mode_units"],
+                  "advances": stats1["steps_advanced"] - stats0["steps_advanced"],
+                  "advances_from_cache": stats1["advances_cached"] - stats0["advances_cached"]},
         "cold": cold,
         "grammar": {"nonterminals": info.n_nonterminals, "rules": info.n_rules, "dotted": info.n_dotted,
                     "trie_nodes": info.trie_nodes, "byte_classes": info.n_byte_classes},

@@ -105,6 +105,7 @@ typedef struct {
   uint64_t big_mode_units;     /* times a warp of the trie sweep switched to its large scratch area */
   uint64_t sweep_transitions;   /* Earley steps (scan + complete + predict) done by the trie sweep */
   uint64_t sweep_states;        /* distinct Earley sets created by the trie sweep */
+  uint64_t advances_cached;     /* row-advances answered by the transition cache (no Earley step run) */
 } fmt_stats;
 
 /*
@@ -155,7 +156,9 @@ fmt_status fmt_state_reset(fmt_state* s, const uint32_t* rows_dev, uint32_t n, v
 /*
  * Advance every row by its chosen token (Section 3.2 scan / complete / predict per byte, with
  * the Compact step of Section 4.2.3 between complete and predict; the resulting pruned chart
- * is looked up in the state cache, Section 5.2 "state cache").
+ * is looked up in the state cache, Section 5.2 "state cache").  With the cache on, the outcome of
+ * advancing a cached chart by a token - the next chart's cache id, or "rejected" - is remembered
+ * too, so the same (chart, token) pair later costs one table look-up instead of Earley steps.
  *   token_ids_dev  [batch] int32 on the device; -1 leaves the row alone
  *   status_dev     [batch] int32 on the device or NULL; receives FMT_OK, FMT_ERR_TOKEN_REJECTED
  *                  (row unchanged), FMT_ERR_FINISHED, FMT_ERR_INVALID_ARG (id out of range) or

@@ -55,7 +55,7 @@ class Stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "steps_advanced", "fills", "fills_computed", "fills_from_cache", "fills_shared", "states_cached",
         "mask_rows_cached", "pool_words_used", "chart_items_max", "chart_sets_max", "capacity_errors",
-        "big_mode_units", "sweep_transitions", "sweep_states")]
+        "big_mode_units", "sweep_transitions", "sweep_states", "advances_cached")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}

@@ -311,6 +311,11 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(d.st_off, d.max_states, 0);
   AL(d.st_mask, d.max_states, 0xFF);
   AL(d.mask_rows, ((size_t)batch + d.max_mask_rows) * g->dev.Wm, 0);
+  uint32_t trn = 1024;
+  while (trn < d.max_states * 4u) trn <<= 1;
+  d.tr_mask = trn - 1;
+  AL(d.tr_key, trn, 0);
+  AL(d.tr_val, trn, 0x80);
   AL(d.jobs, batch, 0);
   AL(d.counters, CNT_TOTAL, 0);
   AL(d.big_scratch, big_words, 0xFF);
@@ -423,6 +428,9 @@ fmt_status fmt_state_cache_clear(fmt_state* s, void* stream) {
   StateDev& d = s->dev;
   launch_evacuate(d, st);
   cudaError_t e = cudaMemsetAsync(d.ht, 0, ((size_t)d.ht_mask + 1) * 4, st);
+  // the cache ids are handed out anew: what was learnt about (id, token) pairs goes too
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.tr_key, 0, ((size_t)d.tr_mask + 1) * 8, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.tr_val, 0x80, ((size_t)d.tr_mask + 1) * 4, st);
   // counters: states, mask rows, jobs, work, error flag, pool top
   if (e == cudaSuccess) e = cudaMemsetAsync(d.counters, 0, 8 * 4, st);
   if (e != cudaSuccess) return cuda_fail(e, "fmt_state_cache_clear");
@@ -521,6 +529,7 @@ fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   out->big_mode_units = u64(CNT_STAT_BIG);
   out->sweep_transitions = u64(CNT_STAT_TRANS);
   out->sweep_states = u64(CNT_STAT_LOCAL);
+  out->advances_cached = u64(CNT_STAT_ADV_HIT);
   return FMT_OK;
 }
 

@@ -67,7 +67,8 @@ enum : uint32_t {
   CNT_LEVEL_REQ = 68,   // [MAX_TOKEN_BYTES + 2] per trie depth: transitions queued for computation
   CNT_HASH_GEN = 104,   // generation of the sweep's per-job hashes (1 .. 65535), advanced by every fill
   CNT_HASH_CLEAR = 105, // this fill starts the generations over: the sweep clears the hashes first
-  CNT_TOTAL = 106
+  CNT_STAT_ADV_HIT = 106,  // 64-bit: advances answered by the transition cache
+  CNT_TOTAL = 108
 };
 
 // Per-job automaton of hash-consed Earley sets, built on demand by the trie walk.  A "local
@@ -119,6 +120,11 @@ struct StateDev {
   uint64_t* st_off;           // [max_states] word offset of the cached chart
   int32_t* st_mask;           // [max_states] -1 none, >= 0 mask row, <= -2 claimed by row -(x+2)
   uint32_t* mask_rows;        // [B + max_mask_rows][Wm]; rows 0..B-1 are per-row scratch
+  // transition cache of advance: (cache id of a chart, token) -> cache id of the next chart, or TR_REJECT.
+  // Open addressing; tr_key holds (id + 1) << 32 | token, 0 = empty; tr_val is TR_UNSET until the value is there.
+  unsigned long long* tr_key; // [tr_mask + 1]
+  int32_t* tr_val;            // [tr_mask + 1]
+  uint32_t tr_mask;
   uint32_t* jobs;             // [B] rows whose mask must be computed
   uint32_t* counters;         // [CNT_TOTAL]
   uint32_t* big_scratch;      // per-warp large scratch areas of the trie walk
@@ -126,6 +132,8 @@ struct StateDev {
   AutoDev au;
 };
 
+constexpr int32_t TR_REJECT = -2;                 // tr_val: the token cannot follow
+constexpr int32_t TR_UNSET = (int32_t)0x80808080;  // tr_val: not written yet (the arrays are filled with byte 0x80)
 constexpr int32_t MASK_ZERO = -1;       // row_mask: all-zero mask (broken row)
 constexpr int32_t MASK_EOS_ONLY = -2;   // row_mask: finished row
 constexpr int32_t MASK_ALIAS0 = -10;    // row_mask <= MASK_ALIAS0: same mask as row (MASK_ALIAS0 - x)

@@ -101,6 +101,43 @@ __device__ int32_t intern_chart(const StateDev& S, const uint32_t* ch, uint64_t&
   return -1;
 }
 
+// ===================================================================================== transition cache
+//
+// What advancing the chart with cache id `sid` by `tok` leads to, if that is known: the next chart's
+// cache id, TR_REJECT, or TR_UNSET (not known).  Called by one lane.
+__device__ __forceinline__ uint32_t tr_slot(const StateDev& S, unsigned long long key) {
+  return (mix32((uint32_t)key) ^ mix32((uint32_t)(key >> 32) * 0x9E3779B9u)) & S.tr_mask;
+}
+__device__ int32_t tr_lookup(const StateDev& S, int32_t sid, uint32_t tok) {
+  const unsigned long long key = ((unsigned long long)((uint32_t)sid + 1u) << 32) | tok;
+  uint32_t slot = tr_slot(S, key);
+  for (uint32_t probe = 0; probe < 32; ++probe) {
+    const unsigned long long k = __ldcg(S.tr_key + slot);
+    if (k == 0ull) return TR_UNSET;
+    if (k == key) {
+      const int32_t v = (int32_t)ld_acquire(reinterpret_cast<const uint32_t*>(S.tr_val + slot));
+      return (v >= 0 || v == TR_REJECT) ? v : TR_UNSET;
+    }
+    slot = (slot + 1u) & S.tr_mask;
+  }
+  return TR_UNSET;
+}
+// Remember the outcome (one lane).  The first to claim a slot for the key writes the value; a full
+// neighbourhood simply leaves the pair unrecorded.
+__device__ void tr_insert(const StateDev& S, int32_t sid, uint32_t tok, int32_t val) {
+  const unsigned long long key = ((unsigned long long)((uint32_t)sid + 1u) << 32) | tok;
+  uint32_t slot = tr_slot(S, key);
+  for (uint32_t probe = 0; probe < 32; ++probe) {
+    const unsigned long long k = atomicCAS(S.tr_key + slot, 0ull, key);
+    if (k == 0ull) {
+      asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(S.tr_val + slot), "r"(val) : "memory");
+      return;
+    }
+    if (k == key) return;
+    slot = (slot + 1u) & S.tr_mask;
+  }
+}
+
 // ===================================================================================== start chart
 
 __global__ void __launch_bounds__(32) init_kernel(GrammarDev G, StateDev S, int32_t* result) {
@@ -169,6 +206,24 @@ __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev G
     return finish(FMT_ERR_TOKEN_REJECTED);
   }
   if (b1 == b0) return finish(FMT_ERR_TOKEN_REJECTED);
+  // ---- has this chart been advanced by this token before?  (Section 5.2: the state cache)
+  const int32_t sid = S.cache_on ? S.row_state[row] : -1;
+  if (sid >= 0) {
+    int32_t known = TR_UNSET;
+    if (lane == 0) known = tr_lookup(S, sid, (uint32_t)tok);
+    known = __shfl_sync(FULL, known, 0);
+    if (known == TR_REJECT) return finish(FMT_ERR_TOKEN_REJECTED);
+    if (known >= 0 && (uint32_t)known < S.max_states) {
+      if (lane == 0) {
+        S.row_state[row] = known;
+        S.row_chart[row] = ld_cg64(&S.st_off[known]);
+        S.row_buf[row] = 255;
+        stat_add(S, CNT_STAT_ADV, 1u);
+        stat_add(S, CNT_STAT_ADV_HIT, 1u);
+      }
+      return finish(FMT_OK);
+    }
+  }
 
   hset_clear_all(s.w.hset, s.w.hset_mask);
   for (uint32_t i = lane; i < ADV_NT_WORDS; i += 32) s.w.nt[i] = 0u;
@@ -188,7 +243,10 @@ __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev G
     __syncwarp();
     r = (held == 2) ? -1 : token_step(G, s, cur, G.vocab_bytes + b0, b1 - b0, dst, S.chart_words, big, cap);
   }
-  if (r == 0) return finish(FMT_ERR_TOKEN_REJECTED);
+  if (r == 0) {
+    if (sid >= 0 && lane == 0) tr_insert(S, sid, (uint32_t)tok, TR_REJECT);
+    return finish(FMT_ERR_TOKEN_REJECTED);
+  }
   if (r < 0) {
     if (lane == 0) {
       S.row_flags[row] = flags | ROW_BROKEN;
@@ -205,6 +263,7 @@ __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev G
   uint64_t off;
   int32_t id = intern_chart(S, dst, off);
   if (lane == 0) {
+    if (sid >= 0 && id >= 0) tr_insert(S, sid, (uint32_t)tok, id);
     S.row_state[row] = id;
     if (id >= 0) {
       S.row_chart[row] = off;

@@ -292,3 +292,51 @@ def test_sweep_hash_generations_start_over():
         if i in (0, 65533, 65534, 65535, 65536, total - 1):
             assert np.array_equal(m.cpu().numpy().view(np.uint32), want), i
     assert st.stats()["capacity_errors"] == 0
+
+
+def test_advance_transition_cache_replays_exactly():
+    """Advancing a cached chart by a token it has been advanced by before is answered from the
+    transition cache.  The same token streams are fed twice (rows reset in between) with a
+    rejected token slipped in: statuses, masks, charts and cache ids of the second pass, which
+    runs no Earley step, must equal those of the first, and the masks the oracle's."""
+    import paper_2506_01151_b200 as fmt
+    from helpers import OracleBatch
+
+    torch, dev = _torch()
+    w = workloads.build(2, V=6000, batch=4, steps=20)
+    g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
+    st = fmt.State(g, w.batch)
+    bad = ord("}")  # ids 0..255 are the single bytes; "}" cannot open a JSON document
+
+    def run():
+        ob = OracleBatch(w)
+        st.reset()
+        seen = []
+        assert _advance(st, [bad] * w.batch) == [fmt.ERR_TOKEN_REJECTED] * w.batch
+        for p in range(w.prefix.shape[0]):
+            toks = w.prefix[p].tolist()
+            want = [ob.advance(b, t) for b, t in enumerate(toks)]
+            assert _advance(st, toks) == want
+        for i in range(w.steps):
+            if w.reset_before[i].any():
+                break
+            toks = w.tokens[i].tolist()
+            want = [ob.advance(b, t) for b, t in enumerate(toks)]
+            assert _advance(st, toks) == want, i
+            got = _mask_of(st, g, w.batch)
+            for b in range(w.batch):
+                assert np.array_equal(got[b], ob.mask(b)), (i, b)
+            q = st.query()
+            seen.append((got.copy(), [st.chart_words(b).tolist() for b in range(w.batch)], list(q["state_id"])))
+        return seen
+
+    first = run()
+    s0 = st.stats()
+    second = run()
+    s1 = st.stats()
+    assert len(first) == len(second) and len(first) > 4
+    for a, b in zip(first, second):
+        assert np.array_equal(a[0], b[0]) and a[1] == b[1] and a[2] == b[2]
+    replayed = s1["steps_advanced"] - s0["steps_advanced"]
+    assert replayed > 0 and s1["advances_cached"] - s0["advances_cached"] == replayed
+    assert s1["states_cached"] == s0["states_cached"]
