@@ -128,6 +128,26 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
                        const fmt_compile_options* opt, fmt_grammar** out);
 void fmt_grammar_destroy(fmt_grammar* g);
 
+/*
+ * A JSON schema as the grammar (the paper's JSON-Schema task, Section 5.1, takes schemas; it leaves
+ * the translation to its front end and fixes none, so the rules below are this library's).
+ * fmt_json_schema_to_ebnf writes grammar text in the dialect fmt_compile reads, start rule "root":
+ * min(cap_bytes, size) bytes to `out` (may be NULL; no terminating NUL) and the full size to
+ * *size_bytes.  fmt_compile_json_schema is that followed by fmt_compile.
+ * A schema node may hold: "type" (object, array, string, number, integer, boolean, null, or a list
+ * of them), "properties" with "required" (members come in the order written; a member that is not
+ * required may be left out; no other member is allowed), "items" and "minItems" (0 or 1), "enum",
+ * "const", "anyOf" / "oneOf" (both read as "any of"), "$ref" to "#/$defs/NAME" or
+ * "#/definitions/NAME" (may be recursive).  A node with none of these accepts any JSON value.
+ * Annotations (title, description, default, examples, $schema, $id) are skipped; any other
+ * keyword is refused with FMT_ERR_GRAMMAR_SYNTAX rather than silently ignored.  White space is
+ * allowed wherever JSON allows it; strings are RFC 8259 strings in well-formed UTF-8.
+ */
+fmt_status fmt_json_schema_to_ebnf(const char* schema, size_t schema_len, char* out, size_t cap_bytes, size_t* size_bytes);
+fmt_status fmt_compile_json_schema(const char* schema, size_t schema_len, const uint8_t* vocab_bytes,
+                                   const uint64_t* vocab_offsets, uint32_t V, int32_t eos_token_id,
+                                   const fmt_compile_options* opt, fmt_grammar** out);
+
 /* Sizes of the compiled grammar (host data; works for host_only grammars too). */
 fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out);
 

@@ -7,5 +7,5 @@ from ._build import build  # noqa: F401
 from .binding import (  # noqa: F401
     BF16, FP32, FMT_OK, ERR_CAPACITY, ERR_FINISHED, ERR_INVALID_ARG, ERR_TOKEN_REJECTED, ERR_GRAMMAR_SYNTAX,
     ERR_UNDEFINED_SYMBOL, ERR_EMPTY_LANGUAGE, EXPORTS, NOALLOC_MAX_CHARTS, FmtError, Grammar, State, apply_mask,
-    fill_mask_noalloc, lib,
+    fill_mask_noalloc, json_schema_to_ebnf, lib,
 )

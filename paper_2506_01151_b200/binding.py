@@ -20,7 +20,7 @@ ERR_OOM, ERR_CUDA, ERR_CAPACITY, ERR_TOKEN_REJECTED, ERR_FINISHED = 5, 6, 7, 8, 
 BF16, FP32 = 0, 1
 
 EXPORTS = [
-    "fmt_compile", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table",
+    "fmt_compile", "fmt_json_schema_to_ebnf", "fmt_compile_json_schema", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table",
     "fmt_state_create", "fmt_state_destroy", "fmt_state_reset", "fmt_state_advance", "fmt_fill_mask",
     "fmt_apply_mask", "fmt_fill_and_apply", "fmt_state_cache_clear", "fmt_state_query", "fmt_state_copy_chart", "fmt_get_stats",
     "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_fill_mask_noalloc", "fmt_last_error",
@@ -122,8 +122,37 @@ _TABLE_DTYPES = {0: np.uint32, 1: np.uint8, 2: np.uint32, 3: np.uint32, 4: np.ui
                  7: np.uint32, 8: np.uint16, 9: np.uint32, 10: np.uint8}
 
 
+def json_schema_to_ebnf(schema) -> str:
+    """fmt_json_schema_to_ebnf: grammar text (start rule "root") for the instances of a JSON schema."""
+    src = schema.encode("utf-8") if isinstance(schema, str) else bytes(schema)
+    n = C.c_size_t()
+    _check(lib().fmt_json_schema_to_ebnf(src, len(src), None, 0, C.byref(n)))
+    buf = C.create_string_buffer(max(n.value, 1))
+    _check(lib().fmt_json_schema_to_ebnf(src, len(src), buf, n.value, C.byref(n)))
+    return buf.raw[: n.value].decode("latin-1")
+
+
 class Grammar:
     """fmt_compile: grammar text + vocabulary -> device tables and byte trie."""
+
+    @classmethod
+    def from_json_schema(cls, schema, vocab: Sequence[bytes], eos: int = -1, host_only: bool = False) -> "Grammar":
+        """fmt_compile_json_schema: the instances of a JSON schema as the grammar."""
+        self = cls.__new__(cls)
+        src = schema.encode("utf-8") if isinstance(schema, str) else bytes(schema)
+        offs = np.zeros(len(vocab) + 1, dtype=np.uint64)
+        offs[1:] = np.cumsum([len(t) for t in vocab], dtype=np.uint64)
+        blob = np.frombuffer(b"".join(vocab) + b"\0", dtype=np.uint8).copy()
+        opt = CompileOptions()
+        opt.host_only = 1 if host_only else 0
+        h = C.c_void_p()
+        _check(lib().fmt_compile_json_schema(src, len(src), blob.ctypes.data, offs.ctypes.data, len(vocab), eos,
+                                             C.byref(opt), C.byref(h)))
+        self._h = h
+        self.V = len(vocab)
+        self.eos = eos
+        self.mask_words = (self.V + 31) // 32
+        return self
 
     def __init__(self, ebnf, start: str, vocab: Sequence[bytes], eos: int = -1, host_only: bool = False):
         src = ebnf.encode("latin-1") if isinstance(ebnf, str) else bytes(ebnf)

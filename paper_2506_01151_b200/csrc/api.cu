@@ -205,6 +205,37 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
 
 void fmt_grammar_destroy(fmt_grammar* g) { delete g; }
 
+fmt_status fmt_json_schema_to_ebnf(const char* schema, size_t schema_len, char* out, size_t cap_bytes, size_t* size_bytes) {
+  if (!schema || !size_bytes) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  try {
+    const std::string text = json_schema_to_ebnf(schema, schema_len);
+    *size_bytes = text.size();
+    if (out && cap_bytes) memcpy(out, text.data(), std::min(text.size(), cap_bytes));
+  } catch (const CompileError& e) {
+    return fail((fmt_status)e.code, e.msg);
+  } catch (const std::bad_alloc&) {
+    return fail(FMT_ERR_OOM, "out of host memory");
+  }
+  return FMT_OK;
+}
+
+fmt_status fmt_compile_json_schema(const char* schema, size_t schema_len, const uint8_t* vocab_bytes,
+                                   const uint64_t* vocab_offsets, uint32_t V, int32_t eos_token_id,
+                                   const fmt_compile_options* opt, fmt_grammar** out) {
+  if (!out) return fail(FMT_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (!schema) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  std::string text;
+  try {
+    text = json_schema_to_ebnf(schema, schema_len);
+  } catch (const CompileError& e) {
+    return fail((fmt_status)e.code, e.msg);
+  } catch (const std::bad_alloc&) {
+    return fail(FMT_ERR_OOM, "out of host memory");
+  }
+  return fmt_compile(text.data(), text.size(), "root", vocab_bytes, vocab_offsets, V, eos_token_id, opt, out);
+}
+
 fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out) {
   if (!g || !out) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
   const HostTables& h = g->host;

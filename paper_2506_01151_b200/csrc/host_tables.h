@@ -58,6 +58,9 @@ struct HostTables {
   std::vector<uint8_t> vocab_bytes;
 };
 
+// Grammar text (start rule "root") for the instances of a JSON schema; throws CompileError.
+std::string json_schema_to_ebnf(const char* schema, size_t len);
+
 // Both throw CompileError.
 void compile_grammar(const char* text, size_t len, const std::string& start, HostTables& out);
 void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t eos, HostTables& out);
