@@ -68,7 +68,9 @@ enum : uint32_t {
   CNT_HASH_GEN = 104,   // generation of the sweep's per-job hashes (1 .. 65535), advanced by every fill
   CNT_HASH_CLEAR = 105, // this fill starts the generations over: the sweep clears the hashes first
   CNT_STAT_ADV_HIT = 106,  // 64-bit: advances answered by the transition cache
-  CNT_TOTAL = 108
+  CNT_LEVEL_TAKEN = 108,   // [MAX_TOKEN_BYTES + 2] per trie depth: tickets drawn for the queued transitions
+  CNT_PASS_DONE = 144,     // CTAs that have finished their part of a depth's pass (summed over the depths)
+  CNT_TOTAL = 146
 };
 
 // Per-job automaton of hash-consed Earley sets, built on demand by the trie walk.  A "local

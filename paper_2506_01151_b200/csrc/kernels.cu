@@ -282,6 +282,7 @@ __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev G
 // this call with the same chart, or a fresh computation (a "job").
 __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
   if (threadIdx.x < CNT_HASH_GEN - CNT_BAR) S.counters[CNT_BAR + threadIdx.x] = 0u;  // barrier and level counters
+  if (threadIdx.x < CNT_TOTAL - CNT_LEVEL_TAKEN) S.counters[CNT_LEVEL_TAKEN + threadIdx.x] = 0u;
   if (threadIdx.x == 0) {
     S.counters[CNT_N_JOBS] = 0u;
     S.counters[CNT_AUTO_ITEMS] = 0u;
@@ -680,6 +681,21 @@ __device__ __forceinline__ bool grid_barrier(const StateDev& S, uint32_t& phase)
   return ok;
 }
 
+// A CTA reports that its part of a depth's pass is done (its writes are visible to whoever then sees
+// the count) and goes on without waiting.  Returns false if the sweep is being abandoned.
+__device__ __forceinline__ bool pass_arrive(const StateDev& S, uint32_t& phase) {
+  __shared__ uint32_t go_s;
+  __syncthreads();
+  ++phase;  // (every thread keeps the count: the warps compare it with the global one on their own)
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(&S.counters[CNT_PASS_DONE], 1u);
+    go_s = ld_acquire(&S.counters[CNT_BAR_ERR]) == 0u ? 1u : 0u;
+  }
+  __syncthreads();
+  return go_s != 0u;
+}
+
 // What the Earley set at `node` is, given that its mark says "pending": the transition it waited
 // for has been computed meanwhile.  `parent_state` is the (final) state of its parent.
 __device__ __forceinline__ uint32_t settled(const GrammarDev& G, const AutoDev& A, const JobCtx& J, uint32_t parent_state,
@@ -709,7 +725,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
   if (A.tables_in_smem) G = stage_hot_tables(Gg, smem + (size_t)SWEEP_WARPS * warp_words);
   uint32_t* big = S.big_scratch + ((size_t)blockIdx.x * SWEEP_WARPS + warp) * ((size_t)S.big_arena_items + S.big_hset_slots);
   const uint32_t gw = blockIdx.x * SWEEP_WARPS + warp, GW = gridDim.x * SWEEP_WARPS;
-  uint32_t bar_phase = 0;
+  uint32_t bar_phase = 0, pass_phase = 0;
 
   hset_clear_all(sm_hset, SWEEP_HSET - 1);
   for (uint32_t i = lane; i < ntw; i += 32) nt[i] = 0u;
@@ -719,6 +735,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
   if (S.counters[CNT_HASH_CLEAR]) {
     const size_t words = (size_t)S.B * (A.hash_mask + 1u);
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += (size_t)gridDim.x * blockDim.x) A.hash[i] = 0u;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < A.req_cap; i += (size_t)gridDim.x * blockDim.x) A.req[i] = 0ull;  // their tags too
   }
   // ---- the automata start with one state each: the base chart's last set
   for (uint32_t j = blockIdx.x; j < n_jobs; j += gridDim.x) {
@@ -760,6 +777,8 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     // the node is marked pending.  A pending PARENT (marked at the previous depth, computed since)
     // is settled on the way; pending leaves are settled when the mask words are formed.
     bool any_alive = false;
+    // a queued transition carries the fill's generation and the depth, so that whoever takes it can tell when it has landed
+    const unsigned long long req_tag = ((unsigned long long)sw.gen << 48) | ((unsigned long long)L << 24);
     for (uint32_t c = gw; c < chunks; c += GW) {
       const uint32_t j = c / cpj;
       const uint32_t first = lo + (c % cpj) * CH + lane;
@@ -803,7 +822,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
               t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
               if (t == T_UNKNOWN) {  // ours to queue
                 const uint32_t at = atomicAdd(&S.counters[CNT_LEVEL_REQ + L], 1u);
-                if (at < A.req_cap) A.req[at] = ((unsigned long long)j << 32) | ((unsigned long long)p_state << 8) | byte[u];
+                if (at < A.req_cap) A.req[at] = req_tag | ((unsigned long long)j << 32) | ((unsigned long long)p_state << 8) | byte[u];
                 t = T_PENDING;
               }
             }
@@ -815,15 +834,51 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     }
     __syncwarp();
     if (__any_sync(FULL, any_alive) && lane == 0) atomicOr(&S.counters[CNT_LEVEL_ALIVE + L], 1u);
-    if (!grid_barrier(S, bar_phase)) return;
-    last_level = L;
-    if (ld_acquire(&S.counters[CNT_LEVEL_ALIVE + L]) == 0u) break;  // nothing survives this depth in any job
-    const uint32_t n_req = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), A.req_cap);
-    if (n_req == 0) continue;  // nothing was unknown at this depth
-    // ---- compute phase: one queued transition per warp at a time, all warps of the grid in parallel
-    for (uint32_t i = gw; i < n_req; i += GW) {
-      const unsigned long long rq = __ldcg(A.req + i);
-      const uint32_t j = (uint32_t)(rq >> 32), p_state = (uint32_t)(rq >> 8) & 0xFFFFu, pb = (uint32_t)rq & 0xFFu;
+    // ---- this CTA's part of the pass is done.  The queued transitions are computed WHILE the other
+    // CTAs finish theirs: every warp draws a ticket and serves the transition with that number as
+    // soon as it has been queued; a ticket beyond the last transition queued, once all CTAs are
+    // done with the pass, is void.  One transition per warp at a time, all warps of the grid in parallel.
+    if (!pass_arrive(S, pass_phase)) return;
+    const uint32_t all_passed = pass_phase * gridDim.x;
+    bool have_ticket = false, gave_up = false;
+    uint32_t ticket = 0;
+    for (uint32_t polls = 0;;) {
+      if (!have_ticket) {
+        if (lane == 0) ticket = atomicAdd(&S.counters[CNT_LEVEL_TAKEN + L], 1u);
+        ticket = __shfl_sync(FULL, ticket, 0);
+        have_ticket = true;
+      }
+      uint32_t passed = 0, queued = 0;
+      if (lane == 0) {  // in this order: once all have passed, the number queued is final
+        passed = ld_acquire(&S.counters[CNT_PASS_DONE]) >= all_passed ? 1u : 0u;
+        queued = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), A.req_cap);
+      }
+      passed = __shfl_sync(FULL, passed, 0);
+      queued = __shfl_sync(FULL, queued, 0);
+      if (ticket >= queued) {
+        if (passed) break;
+        if (++polls > (1u << 21) || ((polls & 63u) == 0u && lane == 0 && ld_acquire(&S.counters[CNT_BAR_ERR]))) gave_up = true;
+        gave_up = __any_sync(FULL, gave_up);
+        if (gave_up) break;
+        __nanosleep(polls < 8u ? 100 : 400);  // thousands of warps read the same two counters: back off
+        continue;
+      }
+      polls = 0;
+      unsigned long long rq = 0;
+      if (lane == 0) {  // the entry is written right after its number was drawn: wait for it to land
+        for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+          rq = __ldcg(A.req + ticket);
+          if ((rq >> 48) == sw.gen && ((rq >> 24) & 0xFFu) == L) break;
+          rq = 0;
+        }
+      }
+      rq = __shfl_sync(FULL, rq, 0);
+      have_ticket = false;
+      if (rq == 0) {
+        gave_up = true;
+        break;
+      }
+      const uint32_t j = (uint32_t)(rq >> 32) & 0xFFFFu, p_state = (uint32_t)(rq >> 8) & 0xFFFFu, pb = (uint32_t)rq & 0xFFu;
       const JobCtx J = job_ctx(S, j);
       uint32_t r = sw.compute(J, p_state, pb, !big_mode);
       if (r == T_FAIL && !big_mode) {  // a set outgrew the shared-memory scratch: use the large area from now on
@@ -848,7 +903,23 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
         }
       }
     }
-    if (!grid_barrier(S, bar_phase)) return;
+    if (gave_up && lane == 0) atomicExch(&S.counters[CNT_BAR_ERR], 1u);  // cannot happen short of a fault elsewhere
+    // all CTAs have passed this depth: how it went is read once per CTA, so that all its warps agree
+    __shared__ uint32_t lvl_s[3];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      lvl_s[0] = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), A.req_cap);
+      lvl_s[1] = ld_acquire(&S.counters[CNT_LEVEL_ALIVE + L]);
+      lvl_s[2] = ld_acquire(&S.counters[CNT_BAR_ERR]);
+    }
+    __syncthreads();
+    const uint32_t n_req = lvl_s[0];
+    const bool alive = lvl_s[1] != 0u;
+    if (lvl_s[2]) return;
+    last_level = L;
+    // if transitions were computed, wait until all of them are in
+    if (n_req != 0 && !grid_barrier(S, bar_phase)) return;
+    if (!alive) break;  // nothing survives this depth in any job
   }
   if (big_mode) hset_clear_all(sw.w.hset, sw.w.hset_mask);
   if (lane == 0 && (sw.n_computed | sw.n_created)) {

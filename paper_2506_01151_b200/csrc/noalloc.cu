@@ -23,7 +23,7 @@ constexpr uint32_t NA_ARENA_ITEMS = 8192;   // per-warp overflow area for Earley
 constexpr uint32_t NA_HSET_SLOTS = 2048;    // per-warp overflow uniqueness hash
 // header: counters, then per-chart arrays
 constexpr uint32_t NA_OFF_COUNTERS = 0;                          // [CNT_TOTAL]
-constexpr uint32_t NA_OFF_JOBS = 128;                            // [NA_MAX]
+constexpr uint32_t NA_OFF_JOBS = 256;                            // [NA_MAX]
 constexpr uint32_t NA_REQ_CAP = 1u << 16;                        // transitions queued per trie depth
 constexpr uint32_t NA_OFF_FLAGS = NA_OFF_JOBS + NA_MAX;          // [NA_MAX]
 constexpr uint32_t NA_OFF_MASKROW = NA_OFF_FLAGS + NA_MAX;       // [NA_MAX] int32
@@ -84,6 +84,7 @@ __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scrat
   }
   for (size_t i = tid; i < (size_t)n * G.Wm; i += nth) mask[i] = 0u;
   for (size_t i = tid; i < (size_t)NA_MAX * NA_HASH_SLOTS; i += nth) S.au.hash[i] = 0u;
+  for (size_t i = tid; i < NA_REQ_CAP; i += nth) S.au.req[i] = 0ull;  // no stale tags: every call is generation 1
   uint32_t* big = S.big_scratch;
   const size_t per_warp = (size_t)NA_ARENA_ITEMS + NA_HSET_SLOTS;
   for (size_t i = tid; i < NA_WARPS * NA_HSET_SLOTS; i += nth)
