@@ -701,7 +701,7 @@ __device__ __forceinline__ bool pass_arrive(const StateDev& S, uint32_t& phase) 
 __device__ __forceinline__ uint32_t settled(const GrammarDev& G, const AutoDev& A, const JobCtx& J, uint32_t parent_state,
                                             uint32_t byte) {
   const uint32_t* slot = J.recs + (size_t)parent_state * A.rec_words + AR_TRANS + G.eq_of_byte[byte];
-  return __ldcg(slot);
+  return ld_acquire(slot);  // (the set it names was written before the transition was published)
 }
 
 constexpr uint32_t SWEEP_PER_LANE = 4;  // trie nodes per lane and pass iteration (independent loads in flight)
@@ -779,6 +779,9 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     bool any_alive = false;
     // a queued transition carries the fill's generation and the depth, so that whoever takes it can tell when it has landed
     const unsigned long long req_tag = ((unsigned long long)sw.gen << 48) | ((unsigned long long)L << 24);
+    // the queue has two halves, used by odd and even depths in turn: a depth's transitions may still be
+    // in the making while the next depth queues its own
+    const uint32_t req_half = A.req_cap / 2u, req_base = (L & 1u) * req_half;
     for (uint32_t c = gw; c < chunks; c += GW) {
       const uint32_t j = c / cpj;
       const uint32_t first = lo + (c % cpj) * CH + lane;
@@ -800,7 +803,12 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
         uint32_t p_state = ps[u];
         if (p_state == ST_PENDING) {  // settle the parent first
           const uint32_t gp_state = (L == 2) ? 0u : (uint32_t)__ldcg(J.st + __ldg(&G.parent[par[u]]));
-          const uint32_t t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
+          uint32_t t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
+          // the transition was queued at the previous depth; the warp that drew it may still be at it
+          for (uint32_t spin = 0; t2 == T_PENDING && spin < (1u << 20); ++spin) {
+            __nanosleep(100);
+            t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
+          }
           if (t2 == T_UNKNOWN || t2 == T_PENDING) {  // only if the queue overflowed: give the row up rather than guess
             atomicOr(&S.row_flags[J.row], ROW_BROKEN);
             atomicExch(&S.counters[CNT_ERR], 1u);
@@ -817,12 +825,12 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
           if ((rec[AR_SCAN + (byte[u] >> 5)] >> (byte[u] & 31u)) & 1u) {
             uint32_t* slot = J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[byte[u]];
             t = *slot;
-            if (t == T_UNKNOWN || t == T_PENDING) t = __ldcg(slot);
+            if (t == T_UNKNOWN || t == T_PENDING) t = ld_acquire(slot);
             if (t == T_UNKNOWN) {
               t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
               if (t == T_UNKNOWN) {  // ours to queue
                 const uint32_t at = atomicAdd(&S.counters[CNT_LEVEL_REQ + L], 1u);
-                if (at < A.req_cap) A.req[at] = req_tag | ((unsigned long long)j << 32) | ((unsigned long long)p_state << 8) | byte[u];
+                if (at < req_half) A.req[req_base + at] = req_tag | ((unsigned long long)j << 32) | ((unsigned long long)p_state << 8) | byte[u];
                 t = T_PENDING;
               }
             }
@@ -851,7 +859,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       uint32_t passed = 0, queued = 0;
       if (lane == 0) {  // in this order: once all have passed, the number queued is final
         passed = ld_acquire(&S.counters[CNT_PASS_DONE]) >= all_passed ? 1u : 0u;
-        queued = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), A.req_cap);
+        queued = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), req_half);
       }
       passed = __shfl_sync(FULL, passed, 0);
       queued = __shfl_sync(FULL, queued, 0);
@@ -867,7 +875,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       unsigned long long rq = 0;
       if (lane == 0) {  // the entry is written right after its number was drawn: wait for it to land
         for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
-          rq = __ldcg(A.req + ticket);
+          rq = __ldcg(A.req + req_base + ticket);
           if ((rq >> 48) == sw.gen && ((rq >> 24) & 0xFFu) == L) break;
           rq = 0;
         }
@@ -905,22 +913,22 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     }
     if (gave_up && lane == 0) atomicExch(&S.counters[CNT_BAR_ERR], 1u);  // cannot happen short of a fault elsewhere
     // all CTAs have passed this depth: how it went is read once per CTA, so that all its warps agree
-    __shared__ uint32_t lvl_s[3];
+    // (The next depth's pass starts at once: a node whose parent waits for a transition that is still
+    // being computed waits for that one transition, see above.)
+    __shared__ uint32_t lvl_s[2];
     __syncthreads();
     if (threadIdx.x == 0) {
-      lvl_s[0] = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), A.req_cap);
-      lvl_s[1] = ld_acquire(&S.counters[CNT_LEVEL_ALIVE + L]);
-      lvl_s[2] = ld_acquire(&S.counters[CNT_BAR_ERR]);
+      lvl_s[0] = ld_acquire(&S.counters[CNT_LEVEL_ALIVE + L]);
+      lvl_s[1] = ld_acquire(&S.counters[CNT_BAR_ERR]);
     }
     __syncthreads();
-    const uint32_t n_req = lvl_s[0];
-    const bool alive = lvl_s[1] != 0u;
-    if (lvl_s[2]) return;
+    const bool alive = lvl_s[0] != 0u;
+    if (lvl_s[1]) return;
     last_level = L;
-    // if transitions were computed, wait until all of them are in
-    if (n_req != 0 && !grid_barrier(S, bar_phase)) return;
     if (!alive) break;  // nothing survives this depth in any job
   }
+  // every transition queued must be in before the mask words are formed
+  if (!grid_barrier(S, bar_phase)) return;
   if (big_mode) hset_clear_all(sw.w.hset, sw.w.hset_mask);
   if (lane == 0 && (sw.n_computed | sw.n_created)) {
     stat_add(S, CNT_STAT_TRANS, sw.n_computed);
