@@ -340,9 +340,12 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
 // warp-cooperative scan / complete / predict of earley_device.cuh; everybody else reads it from
 // the set's record.  The trie is processed one depth at a time by the whole grid, one THREAD per
 // (job, node): st[node] = transition(st[parent], byte).  Reads of parent, byte and writes of st
-// are coalesced because nodes are numbered breadth first.  A grid barrier separates the depths;
-// the kernel is launched cooperatively so that all CTAs are resident, and the barrier gives up
-// (and flags an error) after a bounded number of polls instead of hanging.
+// are coalesced because nodes are numbered breadth first.  The depths are not separated by grid
+// barriers: a CTA reports the end of its part of a depth's pass, its warps then serve the queued
+// transitions (tickets) while the other CTAs finish, and go on to the next depth once all have
+// reported; a node whose parent's transition is still being computed waits for that transition
+// alone.  The kernel is launched cooperatively so that all CTAs are resident, and every wait is a
+// poll with an iteration limit that flags an error instead of hanging.
 
 constexpr uint32_t SWEEP_CUR = 512;     // items of a set under construction per warp (fast mode, power of two)
 constexpr uint32_t SWEEP_HSET = 1024;   // uniqueness hash slots per warp (fast mode)
