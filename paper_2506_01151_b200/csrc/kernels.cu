@@ -808,8 +808,8 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
           const uint32_t gp_state = (L == 2) ? 0u : (uint32_t)__ldcg(J.st + __ldg(&G.parent[par[u]]));
           uint32_t t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
           // the transition was queued at the previous depth; the warp that drew it may still be at it
-          for (uint32_t spin = 0; t2 == T_PENDING && spin < (1u << 20); ++spin) {
-            __nanosleep(100);
+          for (uint32_t spin = 0; t2 == T_PENDING && spin < (1u << 21); ++spin) {
+            __nanosleep(40);
             t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
           }
           if (t2 == T_UNKNOWN || t2 == T_PENDING) {  // only if the queue overflowed: give the row up rather than guess
@@ -871,7 +871,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
         if (++polls > (1u << 21) || ((polls & 63u) == 0u && lane == 0 && ld_acquire(&S.counters[CNT_BAR_ERR]))) gave_up = true;
         gave_up = __any_sync(FULL, gave_up);
         if (gave_up) break;
-        __nanosleep(polls < 8u ? 100 : 400);  // thousands of warps read the same two counters: back off
+        __nanosleep(polls < 16u ? 40 : 200);  // thousands of warps read the same two counters: back off
         continue;
       }
       polls = 0;
