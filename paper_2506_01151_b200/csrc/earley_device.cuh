@@ -246,40 +246,36 @@ __device__ __forceinline__ void clear_nt(const GrammarDev& G, const WarpCtx& w) 
 }
 
 // ---- The lane-resident form of Scan and Complete, for sets of at most 32 items: the set under
-// construction sits one item per lane (and in w.cur[0..n)), uniqueness is a matter of shuffles and
+// construction sits one item per lane, uniqueness is a matter of shuffles and
 // ballots, and neither the uniqueness hash nor a shared-memory counter is touched.
 constexpr uint32_t SMALL_OVERFLOW = 0xffffffffu;
 
-// The candidates c .. c + skip of the lanes with `v` set join cur[0..n) unless already there.
-// `mine` is cur[lane].  Returns the new count, above 32 when they do not fit.
-__device__ __forceinline__ uint32_t append_small(const WarpCtx& w, uint32_t c, bool v, uint32_t skip, uint32_t n,
-                                                 uint32_t& mine) {
+// The candidates c .. c + skip of the lanes with `v` set join the set unless already there.  The
+// set sits one item per lane: `mine` is item `lane` for lane < n.  One candidate at a time (there
+// are seldom more than one or two per call): a broadcast, and a ballot of "is it mine?".  Returns
+// the new count, above 32 when they do not fit.
+__device__ __forceinline__ uint32_t append_small(uint32_t c, bool v, uint32_t skip, uint32_t n, uint32_t& mine) {
   const uint32_t lane = lane_id();
-  const uint32_t maxskip = __reduce_max_sync(FULL, v ? skip : 0u);
-  for (uint32_t j = 0; j <= maxskip; ++j) {
-    const bool vj = v && j <= skip;
-    const uint32_t cj = c + j;
-    const uint32_t vm = __ballot_sync(FULL, vj);
-    if (!vm) continue;
-    bool keep = vj;
-    if (vj) keep = (uint32_t)(__ffs(__match_any_sync(vm, cj)) - 1) == lane;  // one of equal candidates
-    for (uint32_t i = 0; i < n; ++i)
-      if (__shfl_sync(FULL, mine, i) == cj) keep = false;
-    const uint32_t kb = __ballot_sync(FULL, keep);
-    const uint32_t nn = n + __popc(kb);
-    if (nn > 32u) return nn;
-    if (keep) w.cur[n + __popc(kb & ((1u << lane) - 1u))] = cj;
-    __syncwarp();
-    n = nn;
-    mine = lane < n ? w.cur[lane] : 0u;
+  uint32_t vm = __ballot_sync(FULL, v);
+  while (vm) {
+    const int src = __ffs(vm) - 1;
+    vm &= vm - 1;
+    const uint32_t c0 = __shfl_sync(FULL, c, src), sk = __shfl_sync(FULL, skip, src);
+    for (uint32_t j = 0; j <= sk; ++j) {
+      const uint32_t cj = c0 + j;
+      if (__ballot_sync(FULL, lane < n && mine == cj)) continue;  // already there
+      if (n == 32u) return 33u;
+      if (lane == n) mine = cj;
+      ++n;
+    }
   }
   return n;
 }
 
 // Scan the items of `set` over `byte`, then Complete to a fixpoint (Section 3.2), all in lanes.
 // `rename(item)` rewrites an item of `set` into the naming of the new set (identity for plain
-// charts); `view` and `cur_index` are as for complete_fixpoint.  On return the lanes' `mine` and
-// w.cur[0..n) hold the n <= 32 items (completed ones included), the non-terminals found after a
+// charts); `view` and `cur_index` are as for complete_fixpoint.  On return the lanes' `mine`
+// hold the n <= 32 items (completed ones included), the non-terminals found after a
 // dot are collected in w.nt[0..Nw), and `accept` tells whether the accept item is among them.
 // Returns n (0: the byte cannot follow), or SMALL_OVERFLOW when the set outgrows 32 items (w.nt is
 // clean then and the caller takes the general path).
@@ -299,7 +295,7 @@ __device__ __forceinline__ uint32_t small_scan_complete(const GrammarDev& G, con
     const bool hit = (inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte);
     it = rename(it);
     const uint32_t skip = hit ? (G.info[(it + 1u) & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
-    if (__any_sync(FULL, hit)) n = append_small(w, it + 1u, hit, skip, n, mine);
+    if (__any_sync(FULL, hit)) n = append_small(it + 1u, hit, skip, n, mine);
     if (n > 32u) return SMALL_OVERFLOW;
   }
   if (n == 0) return 0;
@@ -331,7 +327,7 @@ __device__ __forceinline__ uint32_t small_scan_complete(const GrammarDev& G, con
         const bool match = (winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X;
         const uint32_t cand = view.fix(wi, o) + 1u;
         const uint32_t skip = match ? (G.info[cand & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
-        if (__any_sync(FULL, match)) n = append_small(w, cand, match, skip, n, mine);
+        if (__any_sync(FULL, match)) n = append_small(cand, match, skip, n, mine);
         if (n > 32u) {
           clear_nt(G, w);
           return SMALL_OVERFLOW;
