@@ -941,9 +941,11 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
   // ---- mask words: 32 tokens per warp pass, one ballot per word (token t is valid iff the node
   // where its bytes end was reached alive; EOS iff the chart is accepting)
   const uint32_t Wm = G.Wm;
-  constexpr uint32_t MW = 4;  // mask words per warp and iteration: their loads are in flight together
+  constexpr uint32_t MW = 6;  // mask words per warp and iteration: their loads are in flight together
+  // nodes are numbered breadth first: a node was visited iff it comes before the first node of depth last_level + 1
+  const uint32_t visited_end = __ldg(&G.lvl_off[last_level + 1]);
   for (uint32_t c0 = gw; c0 < n_jobs * Wm; c0 += MW * GW) {
-    uint32_t node[MW], s_[MW];
+    uint32_t node[MW], s_[MW], dst[MW];
     bool valid[MW], eos_ok[MW];
 #pragma unroll
     for (uint32_t u = 0; u < MW; ++u) {
@@ -951,6 +953,8 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       valid[u] = c < n_jobs * Wm;
       const uint32_t tok = (c % Wm) * 32 + lane;
       node[u] = (valid[u] && tok < G.V) ? __ldg(&G.tok_node[tok]) : 0xFFFFFFFEu;
+      // where the word goes (needed last, asked for first: one lane, off the chain of the loads below)
+      dst[u] = (valid[u] && lane == 0) ? (uint32_t)S.row_mask[__ldcg(A.job_info + c / Wm).w & 0x7FFFFFFFu] : 0u;
     }
 #pragma unroll
     for (uint32_t u = 0; u < MW; ++u) {
@@ -960,7 +964,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       if (node[u] == 0xFFFFFFFFu) {  // a token without bytes: only EOS can be valid
         const uint32_t tok = (c % Wm) * 32 + lane;
         eos_ok[u] = ((int32_t)tok == G.eos) && job_ctx(S, c / Wm).accepting;
-      } else if (node[u] != 0xFFFFFFFEu && __ldg(&G.node_depth[node[u]]) <= last_level) {
+      } else if (node[u] < visited_end) {
         s_[u] = __ldcg(A.st + (size_t)(c / Wm) * A.st_stride + node[u]);
       }
     }
@@ -969,21 +973,23 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       if (!valid[u]) continue;  // (uniform)
       const uint32_t c = c0 + u * GW;
       const uint32_t j = c / Wm, wd = c % Wm;
-      const JobCtx J = job_ctx(S, j);
       uint32_t s = s_[u];
-      if (s == ST_PENDING) {  // a leaf that waited for a transition: its parent is final by now
-        const uint32_t p = __ldg(&G.parent[node[u]]);
-        const uint32_t p_state = (p == 0) ? 0u : (uint32_t)__ldcg(J.st + p);
-        const uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
-        if (t2 == T_UNKNOWN || t2 == T_PENDING || p_state == ST_PENDING) {
-          atomicOr(&S.row_flags[J.row], ROW_BROKEN);
-          s = ST_DEAD;
-        } else {
-          s = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+      if (__any_sync(FULL, s == ST_PENDING)) {  // leaves that waited for a transition: their parents are final by now
+        const JobCtx J = job_ctx(S, j);
+        if (s == ST_PENDING) {
+          const uint32_t p = __ldg(&G.parent[node[u]]);
+          const uint32_t p_state = (p == 0) ? 0u : (uint32_t)__ldcg(J.st + p);
+          const uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
+          if (t2 == T_UNKNOWN || t2 == T_PENDING || p_state == ST_PENDING) {
+            atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+            s = ST_DEAD;
+          } else {
+            s = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+          }
         }
       }
       const uint32_t word = __ballot_sync(FULL, s != ST_DEAD || eos_ok[u]);
-      if (lane == 0) S.mask_rows[(size_t)S.row_mask[J.row] * Wm + wd] = word;
+      if (lane == 0) S.mask_rows[(size_t)dst[u] * Wm + wd] = word;
     }
   }
 }
