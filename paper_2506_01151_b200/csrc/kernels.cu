@@ -770,6 +770,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
   bool big_mode = false;
 
   uint32_t last_level = 0;
+  uint32_t expect_req = n_jobs * Gg.n_eq;  // transitions likely to be queued at the next depth (depth 1: every byte class of every job)
   for (uint32_t L = 1; L <= G.depth; ++L) {
     const uint32_t lo = __ldg(&G.lvl_off[L]), hi = __ldg(&G.lvl_off[L + 1]);
     constexpr uint32_t CH = 32 * SWEEP_PER_LANE;
@@ -851,9 +852,14 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     // done with the pass, is void.  One transition per warp at a time, all warps of the grid in parallel.
     if (!pass_arrive(S, pass_phase)) return;
     const uint32_t all_passed = pass_phase * gridDim.x;
+    // When few transitions are being queued (as many as at the depth before, roughly), eight warps of
+    // every CTA stand by for tickets and the others simply wait for them at the CTA's barrier below:
+    // thousands of warps polling the same counters slow down the few that work.  A heavy fill
+    // needs all hands.
+    const uint32_t takers = (expect_req > 4u * gridDim.x) ? (uint32_t)SWEEP_WARPS : 8u;
     bool have_ticket = false, gave_up = false;
     uint32_t ticket = 0;
-    for (uint32_t polls = 0;;) {
+    for (uint32_t polls = 0; warp < takers;) {
       if (!have_ticket) {
         if (lane == 0) ticket = atomicAdd(&S.counters[CNT_LEVEL_TAKEN + L], 1u);
         ticket = __shfl_sync(FULL, ticket, 0);
@@ -918,15 +924,17 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     // all CTAs have passed this depth: how it went is read once per CTA, so that all its warps agree
     // (The next depth's pass starts at once: a node whose parent waits for a transition that is still
     // being computed waits for that one transition, see above.)
-    __shared__ uint32_t lvl_s[2];
+    __shared__ uint32_t lvl_s[3];
     __syncthreads();
     if (threadIdx.x == 0) {
       lvl_s[0] = ld_acquire(&S.counters[CNT_LEVEL_ALIVE + L]);
       lvl_s[1] = ld_acquire(&S.counters[CNT_BAR_ERR]);
+      lvl_s[2] = ld_acquire(&S.counters[CNT_LEVEL_REQ + L]);
     }
     __syncthreads();
     const bool alive = lvl_s[0] != 0u;
     if (lvl_s[1]) return;
+    expect_req = lvl_s[2];
     last_level = L;
     if (!alive) break;  // nothing survives this depth in any job
   }
