@@ -938,8 +938,13 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     last_level = L;
     if (!alive) break;  // nothing survives this depth in any job
   }
-  // every transition queued must be in before the mask words are formed
-  if (!grid_barrier(S, bar_phase)) return;
+  // All CTAs have passed the last depth.  Transitions queued there may still be in the making: a
+  // leaf that waits for one waits for it below, so no barrier is needed here either.
+  {
+    uint32_t abandoned = 0;
+    if (lane == 0) abandoned = ld_acquire(&S.counters[CNT_BAR_ERR]);
+    if (__shfl_sync(FULL, abandoned, 0) != 0u) return;  // the rows are marked broken when the masks are published
+  }
   if (big_mode) hset_clear_all(sw.w.hset, sw.w.hset_mask);
   if (lane == 0 && (sw.n_computed | sw.n_created)) {
     stat_add(S, CNT_STAT_TRANS, sw.n_computed);
@@ -987,7 +992,11 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
         if (s == ST_PENDING) {
           const uint32_t p = __ldg(&G.parent[node[u]]);
           const uint32_t p_state = (p == 0) ? 0u : (uint32_t)__ldcg(J.st + p);
-          const uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
+          uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
+          for (uint32_t spin = 0; t2 == T_PENDING && spin < (1u << 21); ++spin) {  // some warp is still at it
+            __nanosleep(40);
+            t2 = settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
+          }
           if (t2 == T_UNKNOWN || t2 == T_PENDING || p_state == ST_PENDING) {
             atomicOr(&S.row_flags[J.row], ROW_BROKEN);
             s = ST_DEAD;
