@@ -72,7 +72,14 @@ typedef struct {
   uint64_t pool_words;        /* uint32 words of chart storage for the cache (default 64 Mi) */
   uint32_t sweep_states;       /* distinct Earley sets one mask computation may create while it
                                  sweeps the vocabulary (default: 4 Mi / batch, within 2048..32768) */
-  uint32_t reserved[5];
+  uint32_t roots_disable;      /* 1: no context-independent mask cache: every computed row walks the
+                                 whole vocabulary trie against its own chart */
+  uint32_t max_roots;          /* entries of the context-independent mask cache (default 4096; each
+                                 holds one mask row of ceil(V/32) words) */
+  uint32_t root_max_items;     /* a last Earley set with more items than this gets no entry (default 256) */
+  uint32_t root_max_origins;   /* nor one whose items start in more distinct earlier sets (default 16) */
+  uint32_t wait_limit_log2;    /* every wait inside a kernel is a poll that gives up after 2^this many
+                                 polls (0 = defaults, 2^21..2^24); see fmt_state_set_wait_limit */
 } fmt_state_options;
 
 typedef struct {
@@ -106,6 +113,25 @@ typedef struct {
   uint64_t sweep_transitions;   /* Earley steps (scan + complete + predict) done by the trie sweep */
   uint64_t sweep_states;        /* distinct Earley sets created by the trie sweep */
   uint64_t advances_cached;     /* row-advances answered by the transition cache (no Earley step run) */
+  uint64_t roots;               /* entries of the context-independent mask cache */
+  uint64_t root_sweeps;         /* vocabulary sweeps done to fill such entries (one per entry) */
+  uint64_t rows_from_root;      /* computed rows that started from such an entry */
+  uint64_t rows_plain;          /* computed rows that walked the whole trie against their own chart */
+  uint64_t walk_transitions;    /* Earley steps of the context-dependent walks */
+  uint64_t walk_states;         /* distinct Earley sets they created */
+  uint64_t frontier_entries;    /* trie nodes at which a walk started (context-dependent transitions) */
+  uint64_t walk_tasks;          /* trie nodes expanded below them */
+  uint64_t fills_aborted;       /* fills given up because a bounded wait ran out (their rows got all-zero masks) */
+  uint64_t device_bytes;        /* device memory fmt_state_create allocated for this state */
+  uint64_t earley_step_cycles;  /* SM cycles spent inside the Earley steps of fills, summed over warps
+                                   (divide by sweep_transitions + walk_transitions for a step's latency) */
+  uint64_t advance_chart_words; /* uint32 words of charts read and written by fmt_state_advance */
+  uint64_t diag[16];            /* where capacity errors and expired waits came from: [0] a row's table of
+                                   Earley sets full, [1] the fill's item pool full, [2] a set beyond the large
+                                   per-warp scratch, [3] a work queue full, [4] wait for a transition another
+                                   warp computes, [5] wait for queued work, [6] wait for the other thread
+                                   blocks, [7] a context-independent entry that could not be kept;
+                                   [8..15] the same for the sweeps that fill such entries */
 } fmt_stats;
 
 /*
@@ -206,8 +232,18 @@ fmt_status fmt_apply_mask(const uint32_t* mask_dev, size_t stride_words, void* l
 fmt_status fmt_fill_and_apply(fmt_state* s, uint32_t* mask_dev_or_null, size_t stride_words, void* logits_dev,
                               fmt_dtype dtype, size_t row_stride_elems, void* stream);
 
-/* Forget every cached chart and mask (rows keep their current charts). */
+/* Forget every cached chart and mask of the state cache (rows keep their current charts).  The
+ * context-independent mask cache (Section 4.3) is knowledge about the grammar and the vocabulary,
+ * not about the sequences, and stays; fmt_state_ci_cache_clear forgets that one. */
 fmt_status fmt_state_cache_clear(fmt_state* s, void* stream);
+fmt_status fmt_state_ci_cache_clear(fmt_state* s, void* stream);
+
+/* Every wait inside a kernel of this library (for another thread block, for a queued work item, for
+ * a transition another warp is computing) is a poll with an iteration limit; a wait that runs out
+ * makes the fill give up: its computed rows get all-zero masks, fmt_stats.fills_aborted counts it,
+ * nothing hangs and the next fill starts afresh.  log2_polls = 0 restores the defaults.  (A test
+ * aid: with a tiny limit the give-up path can be taken without anything being wrong.) */
+fmt_status fmt_state_set_wait_limit(fmt_state* s, uint32_t log2_polls);
 
 /* Per-row summary, written to host arrays (any may be NULL); synchronizes `stream`.
  *   accepting[batch] u8, finished[batch] u8 (1 finished, 2 broken by a capacity error),
@@ -221,6 +257,11 @@ fmt_status fmt_state_query(fmt_state* s, uint8_t* accepting, uint8_t* finished, 
  * Writes min(cap_words, total) words to `out` (may be NULL) and the total to *n_words. */
 fmt_status fmt_state_copy_chart(fmt_state* s, uint32_t row, uint32_t* out, size_t cap_words, size_t* n_words,
                                 void* stream);
+
+/* Raw device counters of the state (which = 0) or of its sweeps of context-independent entries
+ * (which = 1), for inspection and tests: min(cap_words, total) uint32 words to `out`, the total to
+ * *n_words; synchronizes `stream`.  The layout is the library's own (csrc/device_tables.h). */
+fmt_status fmt_state_copy_counters(fmt_state* s, int which, uint32_t* out, size_t cap_words, size_t* n_words, void* stream);
 
 /* Counters since creation; synchronizes `stream`. */
 fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream);

@@ -7,10 +7,10 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfmt.so")
-SOURCES = ["api.cu", "kernels.cu", "noalloc.cu", "host_compile.cpp", "json_schema.cpp"]
+SOURCES = ["api.cu", "kernels.cu", "ctx_kernels.cu", "noalloc.cu", "host_compile.cpp", "json_schema.cpp"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-    "-shared", "-Xcompiler", "-fPIC",
+    "-shared", "-Xcompiler", "-fPIC", "--threads", "4",
 ]
 
 

@@ -22,7 +22,7 @@ BF16, FP32 = 0, 1
 EXPORTS = [
     "fmt_compile", "fmt_json_schema_to_ebnf", "fmt_compile_json_schema", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table",
     "fmt_state_create", "fmt_state_destroy", "fmt_state_reset", "fmt_state_advance", "fmt_fill_mask",
-    "fmt_apply_mask", "fmt_fill_and_apply", "fmt_state_cache_clear", "fmt_state_query", "fmt_state_copy_chart", "fmt_get_stats",
+    "fmt_apply_mask", "fmt_fill_and_apply", "fmt_state_cache_clear", "fmt_state_ci_cache_clear", "fmt_state_set_wait_limit", "fmt_state_copy_counters", "fmt_state_query", "fmt_state_copy_chart", "fmt_get_stats",
     "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_fill_mask_noalloc", "fmt_last_error",
 ]
 
@@ -41,7 +41,8 @@ class StateOptions(C.Structure):
     _fields_ = [
         ("cache_disable", C.c_uint32), ("max_states", C.c_uint32), ("max_mask_rows", C.c_uint32),
         ("chart_words", C.c_uint32), ("pool_words", C.c_uint64), ("sweep_states", C.c_uint32),
-        ("reserved", C.c_uint32 * 5),
+        ("roots_disable", C.c_uint32), ("max_roots", C.c_uint32), ("root_max_items", C.c_uint32),
+        ("root_max_origins", C.c_uint32), ("wait_limit_log2", C.c_uint32),
     ]
 
 
@@ -55,10 +56,14 @@ class Stats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "steps_advanced", "fills", "fills_computed", "fills_from_cache", "fills_shared", "states_cached",
         "mask_rows_cached", "pool_words_used", "chart_items_max", "chart_sets_max", "capacity_errors",
-        "big_mode_units", "sweep_transitions", "sweep_states", "advances_cached")]
+        "big_mode_units", "sweep_transitions", "sweep_states", "advances_cached", "roots", "root_sweeps",
+        "rows_from_root", "rows_plain", "walk_transitions", "walk_states", "frontier_entries", "walk_tasks",
+        "fills_aborted", "device_bytes", "earley_step_cycles", "advance_chart_words")] + [("diag", C.c_uint64 * 16)]
 
     def as_dict(self):
-        return {n: int(getattr(self, n)) for n, _ in self._fields_}
+        d = {n: int(getattr(self, n)) for n, _ in self._fields_ if n != "diag"}
+        d["diag"] = [int(x) for x in self.diag]
+        return d
 
 
 class Profile(C.Structure):
@@ -90,6 +95,9 @@ def lib():
         L.fmt_apply_mask.argtypes = [vp, sz, vp, C.c_int, u32, u32, sz, vp]
         L.fmt_fill_and_apply.argtypes = [vp, vp, sz, vp, C.c_int, sz, vp]
         L.fmt_state_cache_clear.argtypes = [vp, vp]
+        L.fmt_state_ci_cache_clear.argtypes = [vp, vp]
+        L.fmt_state_set_wait_limit.argtypes = [vp, u32]
+        L.fmt_state_copy_counters.argtypes = [vp, C.c_int, vp, sz, C.POINTER(sz), vp]
         L.fmt_state_query.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.fmt_state_copy_chart.argtypes = [vp, u32, vp, sz, C.POINTER(sz), vp]
         L.fmt_get_stats.argtypes = [vp, C.POINTER(Stats), vp]
@@ -193,7 +201,9 @@ class State:
     """fmt_state_*: a batch of sequences on the device."""
 
     def __init__(self, grammar: Grammar, batch: int, stream=None, cache: bool = True, max_states: int = 0,
-                 max_mask_rows: int = 0, pool_words: int = 0, chart_words: int = 0, sweep_states: int = 0):
+                 max_mask_rows: int = 0, pool_words: int = 0, chart_words: int = 0, sweep_states: int = 0,
+                 roots: bool = True, max_roots: int = 0, root_max_items: int = 0, root_max_origins: int = 0,
+                 wait_limit_log2: int = 0):
         self.grammar = grammar
         self.batch = batch
         opt = StateOptions()
@@ -203,6 +213,11 @@ class State:
         opt.pool_words = pool_words
         opt.chart_words = chart_words
         opt.sweep_states = sweep_states
+        opt.roots_disable = 0 if roots else 1
+        opt.max_roots = max_roots
+        opt.root_max_items = root_max_items
+        opt.root_max_origins = root_max_origins
+        opt.wait_limit_log2 = wait_limit_log2
         h = C.c_void_p()
         _check(lib().fmt_state_create(grammar._h, batch, C.byref(opt), _ptr(stream), C.byref(h)))
         self._h = h
@@ -237,6 +252,20 @@ class State:
 
     def cache_clear(self, stream=None):
         _check(lib().fmt_state_cache_clear(self._h, _ptr(stream)))
+
+    def ci_cache_clear(self, stream=None):
+        _check(lib().fmt_state_ci_cache_clear(self._h, _ptr(stream)))
+
+    def counters(self, which: int = 0, stream=None) -> np.ndarray:
+        """fmt_state_copy_counters: the raw device counters (0: the state's, 1: its root sweeps')."""
+        n = C.c_size_t()
+        _check(lib().fmt_state_copy_counters(self._h, which, None, 0, C.byref(n), _ptr(stream)))
+        buf = np.zeros(n.value, dtype=np.uint32)
+        _check(lib().fmt_state_copy_counters(self._h, which, buf.ctypes.data, n.value, C.byref(n), _ptr(stream)))
+        return buf
+
+    def set_wait_limit(self, log2_polls: int):
+        _check(lib().fmt_state_set_wait_limit(self._h, log2_polls))
 
     def query(self, stream=None):
         B = self.batch

@@ -29,6 +29,7 @@ fmt_status cuda_fail(cudaError_t e, const char* what) {
 
 struct DeviceBuffers {
   std::vector<void*> ptrs;
+  size_t bytes = 0;
   ~DeviceBuffers() {
     for (void* p : ptrs) cudaFree(p);
   }
@@ -53,6 +54,7 @@ struct DeviceBuffers {
     cudaError_t e = cudaMalloc(&p, bytes);
     if (e != cudaSuccess) return e;
     ptrs.push_back(p);
+    this->bytes += bytes;
     e = cudaMemset(p, fill_byte, bytes);
     if (e != cudaSuccess) return e;
     *out = static_cast<T*>(p);
@@ -111,7 +113,27 @@ struct fmt_state {
   int32_t* result_dev = nullptr;
   uint8_t* query_dev = nullptr;  // scratch for fmt_state_query
   int sweep_grid = 1;
+  uint32_t next_gen = 1;      // generations handed to the fills: two per fill, 1 .. 65534
+  size_t device_bytes = 0;    // what fmt_state_create allocated
 };
+
+// Two fresh generations for a fill (its root sweep and its walk).  Tables tagged with a generation
+// are never cleared between fills; when the 16-bit numbers start over they all are.
+static cudaError_t next_generations(fmt_state* s, cudaStream_t st) {
+  StateDev& d = s->dev;
+  cudaError_t e = cudaSuccess;
+  if (s->next_gen + 1u > 65534u) {
+    e = cudaMemsetAsync(d.au.hash, 0, (size_t)d.B * (d.au.hash_mask + 1u) * 4, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d.au.req, 0, (size_t)d.au.req_cap * 8, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d.cx.ctab, 0, (size_t)d.B * CT_SLOTS * 8, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d.cx.queue, 0, (size_t)d.cx.q_cap * 16, st);
+    s->next_gen = 1;
+  }
+  d.gen = s->next_gen;
+  d.gen_ctx = s->next_gen + 1u;
+  s->next_gen += 2u;
+  return e;
+}
 
 namespace fmt {
 const GrammarDev* grammar_device_tables(const ::fmt_grammar* g, int* device) {
@@ -189,6 +211,9 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
     UP(node_depth);
     UP(lvl_off);
     UP(tok_node);
+    UP(child_off);
+    UP(tok_off);
+    UP(tok_ids);
     UP(vocab_off);
     UP(vocab_bytes);
 #undef UP
@@ -318,6 +343,20 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   while (hs < au.cap * 2u) hs <<= 1;
   au.hash_mask = hs - 1;
   au.items_cap = 128u << 20;
+  d.poll_limit_shift = (opt && opt->wait_limit_log2) ? std::min(opt->wait_limit_log2, 30u) : 0u;
+  RootDev& rt = d.rt;
+  rt.on = (opt && opt->roots_disable) ? 0u : 1u;
+  rt.max_roots = (opt && opt->max_roots) ? opt->max_roots : 4096u;
+  rt.max_items = (opt && opt->root_max_items) ? opt->root_max_items : 256u;
+  rt.max_ph = (opt && opt->root_max_origins) ? std::min(opt->root_max_origins, 1024u) : 16u;
+  uint32_t rh = 256;
+  while (rh < rt.max_roots * 4u) rh <<= 1;
+  rt.hash_mask = rh - 1;
+  rt.charts_cap = rt.max_roots * 512u;
+  rt.fr_cap = 8u << 20;
+  rt.st_cap = 8u << 20;
+  rt.it_cap = 64u << 20;
+  d.cx.q_cap = 4u << 20;
 
   sweep_layout(g->dev, &au.smem_bytes, &au.tables_in_smem);
   cudaError_t e = configure_kernels();
@@ -359,6 +398,26 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   au.req_cap = 1u << 20;
   AL(au.req, au.req_cap, 0);
   AL(au.job_info, batch, 0);
+  AL(rt.hash, rh, 0);
+  AL(rt.info, (size_t)rt.max_roots * RI_WORDS, 0);
+  AL(rt.n_roots, 4, 0);
+  AL(rt.charts, rt.charts_cap, 0);
+  AL(rt.ci_rows, (size_t)rt.max_roots * g->dev.Wm, 0);
+  AL(rt.frontier, rt.fr_cap, 0);
+  AL(rt.states, rt.st_cap, 0);
+  AL(rt.items, rt.it_cap, 0);
+  AL(rt.tops, 4, 0);
+  AL(rt.counters, CNT_TOTAL, 0);
+  AL(rt.rj_chart, batch, 0);
+  AL(rt.rj_mask, batch, 0);
+  AL(rt.rj_flags, batch, 0);
+  AL(rt.rj_jobs, batch, 0);
+  AL(d.cx.bind, (size_t)batch * rt.max_ph, 0);
+  AL(d.cx.jobs, batch, 0);
+  AL(d.cx.ctab, (size_t)batch * CT_SLOTS, 0);
+  AL(d.cx.chunk_off, (size_t)batch + 1, 0);
+  AL(d.cx.queue, d.cx.q_cap, 0);
+  AL(d.cx.qctr, Q_WORDS, 0);
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);
@@ -384,6 +443,7 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
     delete s;
     return fail(FMT_ERR_CAPACITY, "the start chart does not fit the configured capacities");
   }
+  s->device_bytes = s->bufs.bytes;
   *out = s;
   return FMT_OK;
 }
@@ -419,6 +479,7 @@ fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, 
   cudaStream_t st = (cudaStream_t)stream;
   cudaEvent_t w0, w1;
   s->prof.next(1, &w0, &w1);
+  if (cudaError_t e = next_generations(s, st)) return cuda_fail(e, "fmt_fill_mask");
   launch_fill(s->g->dev, s->dev, s->sweep_grid, st, w0, w1);
   launch_gather(s->g->dev, s->dev, mask_dev, stride_words, st);
   return launched("fmt_fill_mask");
@@ -445,6 +506,7 @@ fmt_status fmt_fill_and_apply(fmt_state* s, uint32_t* mask_dev_or_null, size_t s
   cudaEvent_t w0, w1, a0, a1;
   s->prof.next(1, &w0, &w1);
   s->prof.next(2, &a0, &a1);
+  if (cudaError_t e = next_generations(s, st)) return cuda_fail(e, "fmt_fill_and_apply");
   launch_fill(s->g->dev, s->dev, s->sweep_grid, st, w0, w1);
   if (a0) cudaEventRecord(a0, st);
   launch_gather_apply(s->g->dev, s->dev, logits_dev, (int)dtype, row_stride_elems, mask_dev_or_null, stride_words, st);
@@ -467,6 +529,23 @@ fmt_status fmt_state_cache_clear(fmt_state* s, void* stream) {
   if (e != cudaSuccess) return cuda_fail(e, "fmt_state_cache_clear");
   launch_reintern(d, s->init_state_dev, st);
   return launched("fmt_state_cache_clear");
+}
+
+fmt_status fmt_state_ci_cache_clear(fmt_state* s, void* stream) {
+  if (!s) return fail(FMT_ERR_INVALID_ARG, "NULL state");
+  cudaStream_t st = (cudaStream_t)stream;
+  RootDev& r = s->dev.rt;
+  cudaError_t e = cudaMemsetAsync(r.hash, 0, ((size_t)r.hash_mask + 1) * 4, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(r.n_roots, 0, 4, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(r.tops, 0, 16, st);
+  if (e != cudaSuccess) return cuda_fail(e, "fmt_state_ci_cache_clear");
+  return FMT_OK;
+}
+
+fmt_status fmt_state_set_wait_limit(fmt_state* s, uint32_t log2_polls) {
+  if (!s) return fail(FMT_ERR_INVALID_ARG, "NULL state");
+  s->dev.poll_limit_shift = std::min(log2_polls, 30u);
+  return FMT_OK;
 }
 
 fmt_status fmt_state_query(fmt_state* s, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets, uint32_t* n_items,
@@ -538,6 +617,19 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out) {
   return FMT_OK;
 }
 
+fmt_status fmt_state_copy_counters(fmt_state* s, int which, uint32_t* out, size_t cap_words, size_t* n_words, void* stream) {
+  if (!s || !n_words || which < 0 || which > 1) return fail(FMT_ERR_INVALID_ARG, "bad argument");
+  *n_words = CNT_TOTAL;
+  const size_t n = std::min<size_t>(cap_words, CNT_TOTAL);
+  if (out && n) {
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(out, which ? s->dev.rt.counters : s->dev.counters, n * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "fmt_state_copy_counters");
+  }
+  return FMT_OK;
+}
+
 fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   if (!s || !out) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
   cudaStream_t st = (cudaStream_t)stream;
@@ -561,6 +653,30 @@ fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   out->sweep_transitions = u64(CNT_STAT_TRANS);
   out->sweep_states = u64(CNT_STAT_LOCAL);
   out->advances_cached = u64(CNT_STAT_ADV_HIT);
+  out->rows_from_root = u64(CNT_STAT_JOBS_ROOT);
+  out->rows_plain = u64(CNT_STAT_JOBS_PLAIN);
+  out->walk_transitions = u64(CNT_STAT_CTX_TRANS);
+  out->walk_states = u64(CNT_STAT_CTX_STATES);
+  out->frontier_entries = u64(CNT_STAT_FRONTIER);
+  out->walk_tasks = u64(CNT_STAT_TASKS);
+  out->root_sweeps = u64(CNT_STAT_ROOT_SWEEPS);
+  out->fills_aborted = u64(CNT_STAT_ABORTS);
+  out->device_bytes = s->device_bytes;
+  out->earley_step_cycles = u64(CNT_STAT_STEP_CYCLES);
+  out->advance_chart_words = u64(CNT_STAT_ADV_WORDS);
+  for (int i = 0; i < 8; ++i) out->diag[i] = c[CNT_DIAG + i];
+  // the root sweeps count their Earley steps in counters of their own
+  uint32_t n_roots = 0;
+  e = cudaMemcpyAsync(c, s->dev.rt.counters, sizeof(c), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&n_roots, s->dev.rt.n_roots, 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e, "fmt_get_stats");
+  out->sweep_transitions = u64(CNT_STAT_TRANS);
+  out->sweep_states = u64(CNT_STAT_LOCAL);
+  out->big_mode_units += u64(CNT_STAT_BIG);
+  out->earley_step_cycles += u64(CNT_STAT_STEP_CYCLES);
+  for (int i = 0; i < 8; ++i) out->diag[8 + i] = c[CNT_DIAG + i];
+  out->roots = std::min<uint64_t>(n_roots, s->dev.rt.max_roots);
   return FMT_OK;
 }
 

@@ -366,9 +366,35 @@ __device__ int token_step(const GrammarDev& G, AdvScratch& s, const uint32_t* sr
       uint32_t it = (i < n_items) ? sitems[i] : arena[i - n_items];
       uint32_t no = s.sets[it >> 16];
       if (no == 0xffffffffu) bad = 1;
-      put(dst, h, items_at + out + __popc(bal & ((1u << lane) - 1u)), (no << 16) | (it & 0xFFFFu));
+      const uint32_t at = items_at + out + __popc(bal & ((1u << lane) - 1u)), v = (no << 16) | (it & 0xFFFFu);
+      if (i < n_items) put(dst, h, at, v);  // the source chart's sets are sorted and stay so
+      else dst[at] = v;                     // the token's own sets are in the order they were built: sorted below
     }
     out += __popc(bal);
+  }
+  // ---- the kept items of the token's earlier sets, ascending like every other set: the chart is
+  // the cache key, and the same bytes fed as other tokens must give the same words
+  __syncwarp();
+  for (uint32_t L = 1; L < len; ++L) {
+    const uint32_t nw = s.sets[m - 1 + L];
+    if (nw == 0xffffffffu) continue;  // (uniform)
+    const uint32_t a = dst[CH_HDR + nw], b = (nw + 1 < m_new) ? dst[CH_HDR + nw + 1] : kept;
+    uint32_t* set = dst + items_at + a;
+    const uint32_t ns = b - a;
+    if (ns <= 32) {
+      sort_items(set, ns, 32);
+    } else {  // rare: by rank, through the part of the arena whose sets have been copied out by now
+      for (uint32_t i = lane; i < ns; i += 32) arena[i] = set[i];
+      __syncwarp();
+      for (uint32_t i = lane; i < ns; i += 32) {
+        const uint32_t x = arena[i];
+        uint32_t rank = 0;
+        for (uint32_t k = 0; k < ns; ++k) rank += arena[k] < x ? 1u : 0u;
+        set[rank] = x;  // (the items of a set are distinct)
+      }
+      __syncwarp();
+    }
+    for (uint32_t i = lane; i < ns; i += 32) h.add(items_at + a + i, set[i]);
   }
   // ---- the last set: renumber origins (its own index becomes m_new), move it to the front of the
   // arena region it occupies so that it can be sorted in place

@@ -27,6 +27,9 @@ struct GrammarDev {
   uint32_t hot_words;
   const uint32_t* lvl_off;       // [depth+2]
   const uint32_t* tok_node;      // [V]
+  const uint32_t* child_off;     // [T+1] children of node n are nodes child_off[n] .. child_off[n+1]-1
+  const uint32_t* tok_off;       // [T+1] tokens whose bytes end at node n (duplicates included)
+  const uint32_t* tok_ids;
   const uint32_t* vocab_off;     // [V+1]
   const uint8_t* vocab_bytes;
 };
@@ -70,7 +73,31 @@ enum : uint32_t {
   CNT_STAT_ADV_HIT = 106,  // 64-bit: advances answered by the transition cache
   CNT_LEVEL_TAKEN = 108,   // [MAX_TOKEN_BYTES + 2] per trie depth: tickets drawn for the queued transitions
   CNT_PASS_DONE = 144,     // CTAs that have finished their part of a depth's pass (summed over the depths)
-  CNT_TOTAL = 146
+  CNT_LAST_LEVEL = 145,    // deepest trie depth the last sweep visited
+  CNT_STAT_CTX_TRANS = 146,    // 64-bit: Earley steps of the context-dependent walk
+  CNT_STAT_CTX_STATES = 148,   // 64-bit: Earley sets it created
+  CNT_STAT_ROOT_SWEEPS = 150,  // 64-bit: roots whose context-independent part was swept
+  CNT_STAT_JOBS_ROOT = 152,    // 64-bit: computed rows that started from a swept root
+  CNT_STAT_JOBS_PLAIN = 154,   // 64-bit: computed rows that walked the whole trie themselves
+  CNT_STAT_FRONTIER = 156,     // 64-bit: frontier entries looked at
+  CNT_STAT_TASKS = 158,        // 64-bit: node expansions queued
+  CNT_STAT_ABORTS = 160,       // 64-bit: fills abandoned because a bounded wait ran out
+  CNT_STAT_STEP_CYCLES = 162,  // 64-bit: SM cycles spent inside Earley steps of the fill (summed over warps)
+  CNT_STAT_ADV_WORDS = 164,    // 64-bit: chart words read and written by advance
+  CNT_DIAG = 166,              // [16] where capacity errors and expired waits came from (see DIAG_*)
+  CNT_TOTAL = 182
+};
+
+enum : uint32_t {
+  DIAG_SET_TABLE = 0,    // a job's table of Earley sets is full
+  DIAG_ITEM_POOL = 1,    // the fill's item pool is full
+  DIAG_SET_SCRATCH = 2,  // a set outgrew even the large per-warp scratch
+  DIAG_QUEUE_FULL = 3,   // the walk's queue (or a depth's queue of the sweep) is full
+  DIAG_WAIT_VALUE = 4,   // a wait for a transition another warp was computing ran out
+  DIAG_WAIT_QUEUE = 5,   // a wait for queued work ran out
+  DIAG_WAIT_GRID = 6,    // a wait for the other thread blocks ran out
+  DIAG_ROOT_FAILED = 7,  // a root's sweep could not be kept
+  DIAG_N = 16
 };
 
 // Per-job automaton of hash-consed Earley sets, built on demand by the trie walk.  A "local
@@ -102,11 +129,91 @@ struct AutoDev {
 };
 constexpr uint16_t ST_DEAD = 0xFFFFu, ST_PENDING = 0xFFFEu;
 constexpr uint32_t T_UNKNOWN = 0xffffffffu, T_DEAD = 0xfffffffeu, T_FAIL = 0xfffffffdu, T_PENDING = 0xfffffffcu;
+constexpr uint32_t T_CTX = 0xfffffffau;  // the transition needs the sequence's own chart (context-dependent)
+constexpr uint16_t ST_CTX = 0xFFFDu;
 constexpr uint32_t ORIGIN_SELF = 0xFFFFu;
 constexpr uint32_t AR_ITEMS = 0, AR_N = 1, AR_HASH = 2, AR_NK = 3, AR_SCAN = 4, AR_TRANS = 16;
 
+// ---- Context-independent part of a mask, computed once per "root" (Section 4.3).
+// A root is the last Earley set of a chart with its origins made anonymous: the k distinct origins
+// of its scanned / completed items become placeholders 0..k-1 (ascending), the set's own index
+// becomes k.  The trie sweep over the root's one-set chart, in which a completion that would have
+// to read a placeholder set answers T_CTX instead, yields
+//   - the tokens valid whatever the rest of the chart holds (one mask row per root),
+//   - the frontier: every trie node whose transition is the first T_CTX on its path, with the
+//     Earley set of its parent,
+//   - the Earley sets met on the way ("region": item lists only), which a sequence's own walk reads
+//     with the placeholders bound to its chart's set indices.
+// Origin codes inside a sequence's walk: [0, LBASE) a set of its chart, [LBASE, RBASE) a set the
+// walk made, [RBASE, ORIGIN_SELF) set (code - RBASE) of the root's region (0 = the root set).
+constexpr uint32_t LBASE = 0x800u, RBASE = 0x8000u;
+constexpr uint32_t ROOT_NONE = 0xffffffffu;
+enum : uint32_t { ROOT_NEW = 0, ROOT_READY = 1, ROOT_FAILED = 2 };
+enum : uint32_t {  // words of a root's directory entry
+  RI_STATUS = 0, RI_P = 1, RI_NK = 2, RI_N = 3, RI_HASH = 4, RI_CHART = 5, RI_FR_OFF = 6, RI_FR_N = 7,
+  RI_ST_OFF = 8, RI_NSTATES = 9, RI_USES = 10, RI_WORDS = 16
+};
+enum : uint32_t { TOP_CHARTS = 0, TOP_FRONTIER = 1, TOP_STATES = 2, TOP_ITEMS = 3 };
+
+struct RootDev {
+  uint32_t on;           // 0: every computed row walks the whole trie itself
+  uint32_t max_roots, hash_mask;
+  uint32_t max_items;    // a last set with more items than this is not made a root
+  uint32_t max_ph;       // nor one with more distinct origins than this
+  uint32_t* hash;        // [hash_mask + 1] root id + 1, 0 = empty
+  uint32_t* info;        // [max_roots][RI_WORDS]
+  uint32_t* n_roots;
+  uint32_t* charts;      // pool of one-set charts, the key of a root (the scanned / completed items come first)
+  uint32_t charts_cap;
+  uint32_t* ci_rows;     // [max_roots][Wm]
+  uint2* frontier;       // pool: x = node, y = parent's region set | byte class << 16
+  uint32_t fr_cap;
+  uint2* states;         // pool: per region set x = first item (in `items`), y = item count
+  uint32_t st_cap;
+  uint32_t* items;       // pool
+  uint32_t it_cap;
+  uint32_t* tops;        // [4] tops of the four pools
+  uint32_t* counters;    // [CNT_TOTAL] counters of the root sweep (its own barrier, queue and job counts)
+  // the roots to sweep in this fill, as the rows of the sweep's view of the state
+  uint64_t* rj_chart;    // [B] word offset of the root's chart in `charts`
+  int32_t* rj_mask;      // [B] root id = its row in ci_rows
+  uint32_t* rj_flags;    // [B]
+  uint32_t* rj_jobs;     // [B] identity
+};
+
+// What the context-dependent walk needs to know about a job (a row whose mask is computed).
+struct CtxJob {
+  uint64_t chart_off;    // the row's chart (word offset into the arena)
+  uint32_t m;            // its live sets
+  uint32_t row_acc;      // row | accepting << 31
+  uint32_t root;         // root id or ROOT_NONE (the walk starts at the trie's first level from the chart's last set)
+  uint32_t P;            // placeholders of the root
+  uint32_t fr_off, fr_n; // frontier entries (or first node / node count of depth 1 when root is ROOT_NONE)
+  uint32_t st_off;       // the region's sets in RootDev::states
+  int32_t mrow;          // mask row to write
+  uint32_t pad[2];
+};
+
+constexpr uint32_t CT_SLOTS = 1024;  // per job: remembered transitions out of region sets (power of two)
+enum : uint32_t { Q_TAIL = 0, Q_HEAD = 32, Q_OUT = 64, Q_CHUNK = 96, Q_CHUNKS = 97, Q_WORDS = 128 };
+
+struct CtxDev {
+  uint32_t* job_root;          // [B] root of job j (ROOT_NONE: none)
+  uint16_t* bind;              // [B][max_ph] the chart set each placeholder stands for
+  CtxJob* jobs;                // [B]
+  unsigned long long* ctab;    // [B][CT_SLOTS] generation << 48 | (region set << 8 | byte class) << 24 | value
+  uint32_t* chunk_off;         // [B + 1] first chunk (32 frontier entries) of each job
+  uint4* queue;                // [q_cap] x: node, y: set the node leads to, z: job, w: tag (generation << 16 | 1), written last
+  uint32_t q_cap;
+  uint32_t* qctr;              // [Q_WORDS] tail, head, outstanding work, next chunk: one 128-byte line each
+};
+
 struct StateDev {
   uint32_t B;
+  uint32_t ctx_mode;          // 1: this is the view of a root sweep (see RootDev)
+  uint32_t gen;               // generation of the sweep's per-job hashes and queue tags (1 .. 65535)
+  uint32_t gen_ctx;           // generation of the context-dependent walk's tables
+  uint32_t poll_limit_shift;  // bounded waits give up after 2^shift polls
   uint32_t chart_words;       // capacity of one private chart buffer
   uint32_t cache_on;
   uint32_t max_states, ht_mask, max_mask_rows;
@@ -132,6 +239,8 @@ struct StateDev {
   uint32_t* big_scratch;      // per-warp large scratch areas of the trie walk
   uint32_t big_arena_items, big_hset_slots;
   AutoDev au;
+  RootDev rt;
+  CtxDev cx;
 };
 
 constexpr int32_t TR_REJECT = -2;                 // tr_val: the token cannot follow

@@ -3,7 +3,7 @@
 //
 // An item is one uint32: (origin << 16) | dotted-rule id.  Moving the dot is "+1" on the id.
 // A set under construction lives in `cur` with a small open-addressing hash for uniqueness
-// ("each state set maintains only unique states").  Rules that derive the empty string never
+// (Section 3.2: an Earley set holds every item once).  Rules that derive the empty string never
 // appear as items: every item whose post-dot non-terminal is nullable is accompanied by the
 // item with the dot moved over it (table `skip`), and prediction uses precomputed closures.
 #pragma once
@@ -138,7 +138,7 @@ __device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const War
       atomicOr(&w.nt[y >> 5], 1u << (y & 31u));
     }
     if (have && kind == KIND_END && (it & 0xFFFFu) == ITEM_ACCEPT) w.ctr[W_ACCEPT] = 1u;
-    bool done_item = have && kind == KIND_END && (it >> 16) != cur_index;
+    bool done_item = have && kind == KIND_END && (it >> 16) != cur_index && (it & 0xFFFFu) != ITEM_ACCEPT;  // (nothing waits for the augmented start symbol)
     uint32_t bal = __ballot_sync(FULL, done_item);
     while (bal) {
       int src = __ffs(bal) - 1;
@@ -309,7 +309,7 @@ __device__ __forceinline__ uint32_t small_scan_complete(const GrammarDev& G, con
       atomicOr(&w.nt[y >> 5], 1u << (y & 31u));
     }
     if (__any_sync(FULL, have && kind == KIND_END && (mine & 0xFFFFu) == ITEM_ACCEPT)) accept = true;
-    uint32_t bal = __ballot_sync(FULL, have && kind == KIND_END && (mine >> 16) != cur_index);
+    uint32_t bal = __ballot_sync(FULL, have && kind == KIND_END && (mine >> 16) != cur_index && (mine & 0xFFFFu) != ITEM_ACCEPT);
     const uint32_t it = mine;
     head = n;
     while (bal) {

@@ -6,24 +6,13 @@
 
 #include "../../include/fmt.h"
 #include "chart_step.cuh"
+#include "sweep_warp.cuh"
 #include "kernels.h"
 
 namespace fmt {
 
 // ===================================================================================== helpers
 
-__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ uint64_t ld_cg64(const uint64_t* p) {
-  return (uint64_t)__ldcg(reinterpret_cast<const unsigned long long*>(p));
-}
-__device__ __forceinline__ void stat_add(const StateDev& S, uint32_t slot, uint32_t v) {
-  atomicAdd(reinterpret_cast<unsigned long long*>(S.counters + slot), (unsigned long long)v);
-}
-__device__ __forceinline__ void stat_max(const StateDev& S, uint32_t slot, uint32_t v) { atomicMax(S.counters + slot, v); }
 
 __device__ __forceinline__ uint32_t* private_buf(const StateDev& S, uint32_t row, uint32_t which) {
   return S.arena + ((size_t)row * 3u + which) * S.chart_words;
@@ -173,7 +162,6 @@ __global__ void reset_kernel(StateDev S, const uint32_t* rows, uint32_t n, const
 
 constexpr int ADV_WARPS = 4;
 
-constexpr uint32_t HOT_TABLE_BYTES = 24 * 1024;  // grammar tables up to this size are staged in shared memory
 
 __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev Gg, StateDev S, const int32_t* tokens,
                                                                   int32_t* status) {
@@ -259,6 +247,7 @@ __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev G
     stat_add(S, CNT_STAT_ADV, 1u);
     stat_max(S, CNT_STAT_ITEMS_MAX, dst[CH_ITEMS]);
     stat_max(S, CNT_STAT_SETS_MAX, dst[CH_SETS]);
+    stat_add(S, CNT_STAT_ADV_WORDS, cur[CH_WORDS] + dst[CH_WORDS]);
   }
   uint64_t off;
   int32_t id = intern_chart(S, dst, off);
@@ -282,14 +271,15 @@ __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev G
 // this call with the same chart, or a fresh computation (a "job").
 __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
   if (threadIdx.x < CNT_HASH_GEN - CNT_BAR) S.counters[CNT_BAR + threadIdx.x] = 0u;  // barrier and level counters
-  if (threadIdx.x < CNT_TOTAL - CNT_LEVEL_TAKEN) S.counters[CNT_LEVEL_TAKEN + threadIdx.x] = 0u;
+  if (threadIdx.x < CNT_LAST_LEVEL + 1 - CNT_LEVEL_TAKEN) S.counters[CNT_LEVEL_TAKEN + threadIdx.x] = 0u;
   if (threadIdx.x == 0) {
     S.counters[CNT_N_JOBS] = 0u;
     S.counters[CNT_AUTO_ITEMS] = 0u;
-    // a new generation for the sweep's hashes (1 .. 65535); when the numbers start over, this fill clears them
-    const uint32_t g = (S.counters[CNT_HASH_GEN] & 0xFFFFu) % 65535u + 1u;
-    if (g == 1u && S.counters[CNT_HASH_GEN] != 0u) S.counters[CNT_HASH_CLEAR] = 1u;  // stays set until a sweep has done it
-    S.counters[CNT_HASH_GEN] = g;
+  }
+  if (S.rt.counters) {  // the root sweep of this fill starts from clean counters, too
+    if (threadIdx.x < CNT_HASH_GEN - CNT_BAR) S.rt.counters[CNT_BAR + threadIdx.x] = 0u;
+    if (threadIdx.x < CNT_LAST_LEVEL + 1 - CNT_LEVEL_TAKEN) S.rt.counters[CNT_LEVEL_TAKEN + threadIdx.x] = 0u;
+    if (threadIdx.x == 0) S.rt.counters[CNT_N_JOBS] = 0u, S.rt.counters[CNT_AUTO_ITEMS] = 0u;
   }
   __syncthreads();
   for (uint32_t row = threadIdx.x; row < S.B; row += blockDim.x) {
@@ -347,22 +337,6 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
 // alone.  The kernel is launched cooperatively so that all CTAs are resident, and every wait is a
 // poll with an iteration limit that flags an error instead of hanging.
 
-constexpr uint32_t SWEEP_CUR = 512;     // items of a set under construction per warp (fast mode, power of two)
-constexpr uint32_t SWEEP_HSET = 1024;   // uniqueness hash slots per warp (fast mode)
-
-struct JobCtx {
-  const uint32_t* base_off;
-  const uint32_t* base_items;
-  uint32_t m;         // live sets of the base chart
-  uint32_t* recs;     // this job's state records
-  uint32_t* hash;
-  uint32_t* n_states;
-  uint32_t cap;       // states this job may create (ids stay below ORIGIN_SELF - m)
-  uint16_t* st;
-  uint32_t row;
-  bool accepting;
-};
-
 // (phase 0 of the sweep) what later phases need to know about job j, in one 16-byte record
 __device__ __forceinline__ void make_job_info(const StateDev& S, uint32_t j) {
   const uint32_t row = S.jobs[j];
@@ -386,274 +360,16 @@ __device__ __forceinline__ JobCtx job_ctx(const StateDev& S, uint32_t j) {
   J.hash = A.hash + (size_t)j * (A.hash_mask + 1);
   J.n_states = A.n_states + j;
   J.cap = min(A.cap, (ORIGIN_SELF - 1u > J.m) ? ORIGIN_SELF - 1u - J.m : 0u);
+  if (S.ctx_mode) J.cap = min(J.cap, ORIGIN_SELF - 16u - RBASE);  // a root's sets are named RBASE + id later on
   J.st = A.st + (size_t)j * A.st_stride;
   return J;
 }
 
-struct AutoView {
-  const JobCtx& J;
-  const AutoDev& A;
-  __device__ __forceinline__ void operator()(uint32_t o, const uint32_t*& p, uint32_t& n) const {
-    if (o < J.m) {
-      uint32_t a = J.base_off[o], b = J.base_off[o + 1];
-      p = J.base_items + a;
-      n = b - a;
-    } else {
-      const uint32_t* rec = J.recs + (size_t)(o - J.m) * A.rec_words;
-      p = A.items + rec[AR_ITEMS];
-      n = rec[AR_N];
-    }
-  }
-  // an item of local state o that names its own state as origin means "origin o"
-  __device__ __forceinline__ uint32_t fix(uint32_t item, uint32_t o) const {
-    return ((item >> 16) == ORIGIN_SELF) ? ((o << 16) | (item & 0xFFFFu)) : item;
-  }
-};
-
-// The Earley step of one warp.  Two forms of the same step (Section 3.2: scan, complete to a
-// fixpoint, predict): while the scanned and completed items ("kernel") number at most 32 they sit
-// one per lane and uniqueness is a matter of shuffles and ballots; larger sets go through the
-// hash-based primitives of earley_device.cuh.  Either way the predicted items are a function of
-// the kernel, so a set is looked up by its kernel alone (an order-independent hash, then an exact
-// comparison as sets) BEFORE anything is predicted, and a set already known costs no prediction.
-// A set's items are stored kernel first; nothing is sorted.
-constexpr uint32_t T_RETRY = 0xfffffffbu;  // the lane-resident form does not apply: take the general one
-
-struct SweepWarp {
-  const GrammarDev& G;
-  const StateDev& S;
-  WarpCtx w;
-  uint32_t* tmp8;     // shared
-  uint32_t n_computed = 0, n_created = 0;  // statistics, flushed once at the end of the kernel
-  uint32_t chunk_at = 0, chunk_left = 0;   // this warp's private piece of the item pool (lane 0's copy counts)
-  uint32_t gen = 1;                        // this fill's generation of the per-job hashes
-
-  // A new set of job J with the items w.cur[0..n), the first nk of them its kernel: its id or T_FAIL.
-  __device__ uint32_t create_set(const JobCtx& J, uint32_t n, uint32_t nk, uint32_t hash) {
-    const uint32_t lane = lane_id();
-    const AutoDev& A = S.au;
-    uint32_t id = T_FAIL, ioff = 0;
-    if (lane == 0) {
-      const uint32_t got = atomicAdd(J.n_states, 1u);
-      const uint32_t need = (max(n, 1u) + 31u) & ~31u;
-      if (got < J.cap) {
-        if (need > chunk_left) {  // take a new piece of the pool: one atomic per ~4 Ki item words
-          const uint32_t take = max(need, 4096u);
-          chunk_at = atomicAdd(&S.counters[CNT_AUTO_ITEMS], take);
-          chunk_left = (chunk_at <= A.items_cap && take <= A.items_cap - chunk_at) ? take : 0u;
-        }
-        if (need <= chunk_left) {
-          ioff = chunk_at;
-          chunk_at += need;
-          chunk_left -= need;
-          id = got;
-        }
-      }
-    }
-    id = __shfl_sync(FULL, id, 0);
-    ioff = __shfl_sync(FULL, ioff, 0);
-    if (id == T_FAIL) return T_FAIL;
-    uint32_t* rec = J.recs + (size_t)id * A.rec_words;
-    uint32_t* items = A.items + ioff;
-    for (uint32_t i = lane; i < n; i += 32) items[i] = w.cur[i];
-    for (uint32_t i = lane; i < A.rec_words; i += 32) {
-      uint32_t v2 = 0u;
-      if (i == AR_ITEMS) v2 = ioff;
-      else if (i == AR_N) v2 = n;
-      else if (i == AR_HASH) v2 = hash;
-      else if (i == AR_NK) v2 = nk;
-      else if (i >= AR_SCAN && i < AR_SCAN + 8) v2 = tmp8[i - AR_SCAN];
-      else if (i >= AR_TRANS) v2 = T_UNKNOWN;
-      rec[i] = v2;
-    }
-    __syncwarp();
-    __threadfence();
-    ++n_created;
-    return id;
-  }
-
-  // Is set `sid` the one with this hash and a kernel of nk items for which `member` holds?
-  // member(x, valid) is called by all lanes.
-  template <class Member>
-  __device__ __forceinline__ bool same_set(const JobCtx& J, uint32_t sid, uint32_t nk, uint32_t hash, Member member) {
-    const uint32_t lane = lane_id();
-    const uint32_t* rec = J.recs + (size_t)sid * S.au.rec_words;
-    if (__ldcg(rec + AR_HASH) != hash || __ldcg(rec + AR_NK) != nk) return false;
-    const uint32_t* items = S.au.items + __ldcg(rec + AR_ITEMS);
-    bool ok = true;
-    for (uint32_t base = 0; base < nk; base += 32) {
-      const bool valid = base + lane < nk;
-      const uint32_t x = valid ? __ldcg(items + base + lane) : 0u;
-      ok = member(x, valid) && ok;
-    }
-    return __all_sync(FULL, ok);
-  }
-
-  // The set of job J with this kernel: its id, or T_FAIL if there is none yet.
-  // (A hash slot holds generation << 16 | id + 1; a slot of another generation, left by an earlier
-  // fill, counts as empty, so the tables are never cleared between fills.)
-  template <class Member>
-  __device__ uint32_t lookup_set(const JobCtx& J, uint32_t nk, uint32_t hash, Member member) {
-    const uint32_t lane = lane_id();
-    const uint32_t mask = S.au.hash_mask;
-    uint32_t slot = hash & mask;
-    for (uint32_t probe = 0; probe <= mask && probe < 4096u; ++probe) {
-      uint32_t v = 0;
-      if (lane == 0) v = ld_acquire(&J.hash[slot]);
-      v = __shfl_sync(FULL, v, 0);
-      if ((v >> 16) != gen) break;
-      if (same_set(J, (v & 0xFFFFu) - 1u, nk, hash, member)) return (v & 0xFFFFu) - 1u;
-      slot = (slot + 1u) & mask;
-    }
-    return T_FAIL;
-  }
-
-  // Enter the freshly created set `id` into the job's hash, unless an equal set got there first
-  // (several warps often reach the same new set at the same moment): returns the id to use.
-  template <class Member>
-  __device__ uint32_t insert_set(const JobCtx& J, uint32_t id, uint32_t nk, uint32_t hash, Member member) {
-    const uint32_t lane = lane_id();
-    const uint32_t mask = S.au.hash_mask;
-    uint32_t slot = hash & mask;
-    for (uint32_t probe = 0; probe <= mask && probe < 4096u; ++probe) {
-      uint32_t old = 0;
-      if (lane == 0) {
-        old = ld_acquire(&J.hash[slot]);
-        if ((old >> 16) != gen) {  // empty: take it, unless somebody is faster
-          const uint32_t seen = old;
-          old = atomicCAS(&J.hash[slot], seen, (gen << 16) | (id + 1u));
-          if (old == seen) old = 0u;
-        }
-      }
-      old = __shfl_sync(FULL, old, 0);
-      if (old == 0u) return id;
-      __threadfence();
-      if (same_set(J, (old & 0xFFFFu) - 1u, nk, hash, member)) return (old & 0xFFFFu) - 1u;
-      slot = (slot + 1u) & mask;
-    }
-    return T_FAIL;
-  }
-
-  // The kernel w.cur[0..nk) is new: predict, describe, store and enter the set.
-  template <class Member>
-  __device__ uint32_t finish_new(const JobCtx& J, uint32_t nk, uint32_t hash, Member member) {
-    const uint32_t lane = lane_id();
-    __syncwarp();
-    if (lane == 0) w.ctr[W_NCUR] = nk, w.ctr[W_OVERFLOW] = 0u;
-    predict_into_cur(G, w, ORIGIN_SELF);
-    if (w.ctr[W_OVERFLOW]) return T_RETRY;
-    const uint32_t n = min(w.ctr[W_NCUR], w.cur_cap);
-    scannable_bytes(G, w.cur, n, tmp8);
-    const uint32_t id = create_set(J, n, nk, hash);
-    return id == T_FAIL ? T_FAIL : insert_set(J, id, nk, hash, member);
-  }
-
-  // The lane-resident form (see small_scan_complete).
-  __device__ uint32_t compute_small(const JobCtx& J, uint32_t ps, uint32_t byte) {
-    const uint32_t lane = lane_id();
-    const uint32_t* pitems;
-    uint32_t plen;
-    AutoView view{J, S.au};
-    view(ps == 0 ? J.m - 1 : J.m + ps, pitems, plen);
-    if (plen > 8u * 32u) return T_RETRY;  // a large set seldom scans into a small one
-    const uint32_t self_code = J.m + ps;
-    uint32_t mine;
-    bool accept;
-    const uint32_t n = small_scan_complete(
-        G, w, view, pitems, plen, byte, ORIGIN_SELF,
-        [&](uint32_t it) { return ((it >> 16) == ORIGIN_SELF) ? ((self_code << 16) | (it & 0xFFFFu)) : it; }, mine, accept);
-    if (n == SMALL_OVERFLOW) return T_RETRY;
-    if (n == 0) return T_DEAD;
-    // ---- the kernel: what is left when the completed items go
-    const uint32_t nk = small_drop_completed(G, w, n, mine);
-    uint32_t h = lane < nk ? mix32(mine) : 0u;
-    for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
-    h = mix32(h + nk * 0x9E3779B9u);
-    auto member = [&](uint32_t x, bool valid) {  // the kernel sits one item per lane
-      bool found = false;
-      for (uint32_t i = 0; i < nk; ++i)
-        if (__shfl_sync(FULL, mine, i) == x) found = true;
-      return found || !valid;
-    };
-    const uint32_t id = lookup_set(J, nk, h, member);
-    if (id != T_FAIL) {
-      clear_nt(G, w);
-      return id;
-    }
-    return finish_new(J, nk, h, member);
-  }
-
-  // The general form, for sets of any size (w.cur may be the warp's large area).
-  __device__ uint32_t compute_general(const JobCtx& J, uint32_t ps, uint32_t byte) {
-    const uint32_t lane = lane_id();
-    const uint32_t* pitems;
-    uint32_t plen;
-    AutoView view{J, S.au};
-    view(ps == 0 ? J.m - 1 : J.m + ps, pitems, plen);
-    __syncwarp();
-    if (lane < W_CTRS) w.ctr[lane] = 0u;
-    __syncwarp();
-    const uint32_t self_code = J.m + ps;
-    for (uint32_t k = lane; k < plen; k += 32) {
-      uint32_t it = pitems[k];
-      uint32_t inf = G.info[it & 0xFFFFu];
-      if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) {
-        if ((it >> 16) == ORIGIN_SELF) it = (self_code << 16) | (it & 0xFFFFu);
-        add_item(G, w, it + 1u);
-      }
-    }
-    __syncwarp();
-    if (w.ctr[W_OVERFLOW]) {
-      hset_clear_all(w.hset, w.hset_mask);
-      return T_FAIL;
-    }
-    if (w.ctr[W_NCUR] == 0u) return T_DEAD;
-    complete_fixpoint(G, w, view, ORIGIN_SELF, 0u);
-    const uint32_t hashed = min(w.ctr[W_NCUR], w.cur_cap);
-    if (w.ctr[W_OVERFLOW]) {
-      hset_clear_all(w.hset, w.hset_mask);
-      clear_nt(G, w);
-      return T_FAIL;
-    }
-    // the kernel: the items that are not completed; all of cur[0..hashed) are in the uniqueness hash
-    uint32_t nk = 0, h = 0;
-    for (uint32_t base = 0; base < hashed; base += 32) {
-      const uint32_t i = base + lane;
-      const uint32_t it = i < hashed ? w.cur[i] : 0u;
-      const bool keep = i < hashed && (G.info[it & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
-      if (keep) h += mix32(it);
-      nk += __popc(__ballot_sync(FULL, keep));
-    }
-    for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
-    h = mix32(h + nk * 0x9E3779B9u);
-    auto member = [&](uint32_t x, bool valid) { return !valid || hset_contains(w.hset, w.hset_mask, x); };
-    const uint32_t id = lookup_set(J, nk, h, member);
-    if (id != T_FAIL) {
-      hset_clear_items(w, hashed);
-      clear_nt(G, w);
-      return id;
-    }
-    // a new set: its items stay in the uniqueness hash, for the comparisons that entering the set
-    // may need (the completed items among them do no harm: no stored kernel holds one)
-    drop_completed(G, w, hashed);
-    const uint32_t r = finish_new(J, nk, h, member);
-    hset_clear_all(w.hset, w.hset_mask);
-    return r == T_RETRY ? T_FAIL : r;
-  }
-
-  // Compute, publish and return the transition of local state `ps` on `byte`: T_DEAD, a state id,
-  // or T_FAIL when a capacity was exceeded (the caller may switch to the large scratch and ask
-  // again).  The transition has been claimed (T_PENDING) by whoever queued it.
-  __device__ uint32_t compute(const JobCtx& J, uint32_t ps, uint32_t byte, bool small_ok) {
-    uint32_t r = small_ok ? compute_small(J, ps, byte) : T_RETRY;
-    if (r == T_RETRY) r = compute_general(J, ps, byte);
-    if (r == T_FAIL) return T_FAIL;
-    uint32_t* slot = J.recs + (size_t)ps * S.au.rec_words + AR_TRANS + G.eq_of_byte[byte];
-    if (lane_id() == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(slot), "r"(r) : "memory");
-    ++n_computed;
-    return r;
-  }
-};
+// How often a bounded wait polls before it gives up: 2^dflt times, or 2^poll_limit_shift when the state
+// was created with a limit of its own (tests use a tiny one to take the give-up path).
+__device__ __forceinline__ uint32_t poll_limit(const StateDev& S, uint32_t dflt) {
+  return 1u << (S.poll_limit_shift ? S.poll_limit_shift : dflt);
+}
 
 // All CTAs of the (cooperatively launched) grid meet here.  Returns false if the sweep must be
 // abandoned: some CTA waited longer than the limit, which only a fault elsewhere can cause.
@@ -668,7 +384,8 @@ __device__ __forceinline__ bool grid_barrier(const StateDev& S, uint32_t& phase)
     uint32_t ok = 1u;
     for (uint32_t polls = 0;; ++polls) {
       if (ld_acquire(&S.counters[CNT_BAR]) >= target) break;
-      if (polls > (1u << 24) || ld_acquire(&S.counters[CNT_BAR_ERR])) {
+      if (polls > poll_limit(S, 24) || ld_acquire(&S.counters[CNT_BAR_ERR])) {
+        if (polls > poll_limit(S, 24)) diag(S, DIAG_WAIT_GRID);
         atomicExch(&S.counters[CNT_BAR_ERR], 1u);
         ok = 0u;
         break;
@@ -734,12 +451,6 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
   for (uint32_t i = lane; i < ntw; i += 32) nt[i] = 0u;
   __syncthreads();
 
-  // ---- the per-job hashes of Earley sets are cleared only when the 16-bit generation starts over
-  if (S.counters[CNT_HASH_CLEAR]) {
-    const size_t words = (size_t)S.B * (A.hash_mask + 1u);
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < words; i += (size_t)gridDim.x * blockDim.x) A.hash[i] = 0u;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < A.req_cap; i += (size_t)gridDim.x * blockDim.x) A.req[i] = 0ull;  // their tags too
-  }
   // ---- the automata start with one state each: the base chart's last set
   for (uint32_t j = blockIdx.x; j < n_jobs; j += gridDim.x) {
     uint32_t* rec0 = A.recs + (size_t)j * A.cap * A.rec_words;
@@ -756,10 +467,9 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
     }
   }
   if (!grid_barrier(S, bar_phase)) return;
-  if (blockIdx.x == 0 && threadIdx.x == 0) S.counters[CNT_HASH_CLEAR] = 0u;  // done above, if it was asked for
 
   SweepWarp sw{G, S};
-  sw.gen = S.counters[CNT_HASH_GEN] & 0xFFFFu;
+  sw.gen = S.gen & 0xFFFFu;  // (a slot of the per-job hashes written under another generation counts as empty)
   sw.w.nt = nt;
   sw.w.ctr = ctr;
   sw.tmp8 = tmp8;
@@ -809,39 +519,54 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
           const uint32_t gp_state = (L == 2) ? 0u : (uint32_t)__ldcg(J.st + __ldg(&G.parent[par[u]]));
           uint32_t t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
           // the transition was queued at the previous depth; the warp that drew it may still be at it
-          for (uint32_t spin = 0; t2 == T_PENDING && spin < (1u << 21); ++spin) {
+          for (uint32_t spin = 0; t2 == T_PENDING && spin < poll_limit(S, 21); ++spin) {
             __nanosleep(40);
             t2 = settled(G, A, J, gp_state, __ldg(&G.node_byte[par[u]]));
           }
-          if (t2 == T_UNKNOWN || t2 == T_PENDING) {  // only if the queue overflowed: give the row up rather than guess
-            atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+          if (t2 == T_UNKNOWN || t2 == T_PENDING) {  // the wait ran out: give the row up rather than guess
+            diag(S, DIAG_WAIT_VALUE);
+            if (!(atomicOr(&S.row_flags[J.row], ROW_BROKEN) & ROW_BROKEN)) stat_add(S, CNT_STAT_CAPERR, 1u);
             atomicExch(&S.counters[CNT_ERR], 1u);
             p_state = ST_DEAD;
           } else {
-            p_state = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+            p_state = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : (t2 == T_CTX) ? (uint32_t)ST_CTX : t2;
           }
           J.st[par[u]] = (uint16_t)p_state;
         }
         uint32_t t = T_DEAD;
-        if (p_state != ST_DEAD) {
+        if (p_state != ST_DEAD && p_state != ST_CTX) {  // (what lies below a context-dependent node is not this sweep's business)
+          // records are written by other SMs while the sweep runs: read them past L1.  A record is complete
+          // before its id appears anywhere (the writer fences, then publishes the transition that names it).
           const uint32_t* rec = J.recs + (size_t)p_state * A.rec_words;
           // one 256-bit test rejects most bytes without touching the transition table
-          if ((rec[AR_SCAN + (byte[u] >> 5)] >> (byte[u] & 31u)) & 1u) {
+          if ((__ldcg(rec + AR_SCAN + (byte[u] >> 5)) >> (byte[u] & 31u)) & 1u) {
             uint32_t* slot = J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[byte[u]];
-            t = *slot;
-            if (t == T_UNKNOWN || t == T_PENDING) t = ld_acquire(slot);
+            t = ld_acquire(slot);
             if (t == T_UNKNOWN) {
               t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
               if (t == T_UNKNOWN) {  // ours to queue
                 const uint32_t at = atomicAdd(&S.counters[CNT_LEVEL_REQ + L], 1u);
-                if (at < req_half) A.req[req_base + at] = req_tag | ((unsigned long long)j << 32) | ((unsigned long long)p_state << 8) | byte[u];
-                t = T_PENDING;
+                if (at < req_half) {
+                  A.req[req_base + at] = req_tag | ((unsigned long long)j << 32) | ((unsigned long long)p_state << 8) | byte[u];
+                  t = T_PENDING;
+                } else {
+                  // the depth's queue is full: nobody will compute this transition.  Settle it here so that
+                  // nobody waits for it: the root sweep calls it context-dependent (always a safe answer),
+                  // a row's own sweep gives the row up.
+                  t = S.ctx_mode ? T_CTX : T_DEAD;
+                  diag(S, DIAG_QUEUE_FULL);
+                  if (!S.ctx_mode) {
+                    if (!(atomicOr(&S.row_flags[J.row], ROW_BROKEN) & ROW_BROKEN)) stat_add(S, CNT_STAT_CAPERR, 1u);
+                    atomicExch(&S.counters[CNT_ERR], 1u);
+                  }
+                  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(slot), "r"(t) : "memory");
+                }
               }
             }
           }
         }
-        J.st[node[u]] = (t == T_PENDING) ? ST_PENDING : (t == T_DEAD) ? ST_DEAD : (uint16_t)t;
-        any_alive |= (t != T_DEAD);
+        J.st[node[u]] = (t == T_PENDING) ? ST_PENDING : (t == T_DEAD) ? ST_DEAD : (t == T_CTX) ? ST_CTX : (uint16_t)t;
+        any_alive |= (t != T_DEAD && t != T_CTX);
       }
     }
     __syncwarp();
@@ -874,7 +599,11 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       queued = __shfl_sync(FULL, queued, 0);
       if (ticket >= queued) {
         if (passed) break;
-        if (++polls > (1u << 21) || ((polls & 63u) == 0u && lane == 0 && ld_acquire(&S.counters[CNT_BAR_ERR]))) gave_up = true;
+        if (++polls > poll_limit(S, 21)) {
+          gave_up = true;
+          if (lane == 0) diag(S, DIAG_WAIT_QUEUE);
+        }
+        if ((polls & 63u) == 0u && lane == 0 && ld_acquire(&S.counters[CNT_BAR_ERR])) gave_up = true;
         gave_up = __any_sync(FULL, gave_up);
         if (gave_up) break;
         __nanosleep(polls < 16u ? 40 : 200);  // thousands of warps read the same two counters: back off
@@ -883,8 +612,8 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       polls = 0;
       unsigned long long rq = 0;
       if (lane == 0) {  // the entry is written right after its number was drawn: wait for it to land
-        for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
-          rq = __ldcg(A.req + req_base + ticket);
+        for (uint32_t spin = 0; spin < poll_limit(S, 22); ++spin) {
+          rq = ld_acquire64(A.req + req_base + ticket);  // (a volatile access: a plain load may be hoisted out of the loop)
           if ((rq >> 48) == sw.gen && ((rq >> 24) & 0xFFu) == L) break;
           rq = 0;
         }
@@ -892,6 +621,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       rq = __shfl_sync(FULL, rq, 0);
       have_ticket = false;
       if (rq == 0) {
+        if (lane == 0) diag(S, DIAG_WAIT_QUEUE);
         gave_up = true;
         break;
       }
@@ -913,10 +643,15 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
         hset_clear_all(sw.w.hset, sw.w.hset_mask);
         clear_nt(G, sw.w);
         if (lane == 0) {
-          atomicOr(&S.row_flags[J.row], ROW_BROKEN);
-          atomicExch(&S.counters[CNT_ERR], 1u);
-          stat_add(S, CNT_STAT_CAPERR, 1u);
-          atomicExch(J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[pb], T_DEAD);  // lets the sweep go on
+          diag(S, DIAG_SET_SCRATCH);
+          uint32_t* slot = J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[pb];
+          if (S.ctx_mode) {  // the root sweep leaves what it cannot hold to the rows' own walks
+            atomicExch(slot, T_CTX);
+          } else {
+            if (!(atomicOr(&S.row_flags[J.row], ROW_BROKEN) & ROW_BROKEN)) stat_add(S, CNT_STAT_CAPERR, 1u);
+            atomicExch(&S.counters[CNT_ERR], 1u);
+            atomicExch(slot, T_DEAD);  // lets the sweep go on
+          }
         }
       }
     }
@@ -949,7 +684,9 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
   if (lane == 0 && (sw.n_computed | sw.n_created)) {
     stat_add(S, CNT_STAT_TRANS, sw.n_computed);
     stat_add(S, CNT_STAT_LOCAL, sw.n_created);
+    stat_add64(S, CNT_STAT_STEP_CYCLES, sw.cycles);
   }
+  if (blockIdx.x == 0 && threadIdx.x == 0) S.counters[CNT_LAST_LEVEL] = last_level;
 
   // ---- mask words: 32 tokens per warp pass, one ballot per word (token t is valid iff the node
   // where its bytes end was reached alive; EOS iff the chart is accepting)
@@ -976,7 +713,7 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
       eos_ok[u] = false;
       if (node[u] == 0xFFFFFFFFu) {  // a token without bytes: only EOS can be valid
         const uint32_t tok = (c % Wm) * 32 + lane;
-        eos_ok[u] = ((int32_t)tok == G.eos) && job_ctx(S, c / Wm).accepting;
+        eos_ok[u] = ((int32_t)tok == G.eos) && !S.ctx_mode && job_ctx(S, c / Wm).accepting;
       } else if (node[u] < visited_end) {
         s_[u] = __ldcg(A.st + (size_t)(c / Wm) * A.st_stride + node[u]);
       }
@@ -992,20 +729,22 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
         if (s == ST_PENDING) {
           const uint32_t p = __ldg(&G.parent[node[u]]);
           const uint32_t p_state = (p == 0) ? 0u : (uint32_t)__ldcg(J.st + p);
-          uint32_t t2 = (p_state == ST_DEAD || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
-          for (uint32_t spin = 0; t2 == T_PENDING && spin < (1u << 21); ++spin) {  // some warp is still at it
+          uint32_t t2 = (p_state == ST_DEAD || p_state == ST_CTX || p_state == ST_PENDING) ? T_DEAD : settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
+          for (uint32_t spin = 0; t2 == T_PENDING && spin < poll_limit(S, 21); ++spin) {  // some warp is still at it
             __nanosleep(40);
             t2 = settled(G, A, J, p_state, __ldg(&G.node_byte[node[u]]));
           }
           if (t2 == T_UNKNOWN || t2 == T_PENDING || p_state == ST_PENDING) {
-            atomicOr(&S.row_flags[J.row], ROW_BROKEN);
+            diag(S, DIAG_WAIT_VALUE);
+            if (!(atomicOr(&S.row_flags[J.row], ROW_BROKEN) & ROW_BROKEN)) stat_add(S, CNT_STAT_CAPERR, 1u);
             s = ST_DEAD;
           } else {
-            s = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : t2;
+            s = (t2 == T_DEAD) ? (uint32_t)ST_DEAD : (t2 == T_CTX) ? (uint32_t)ST_CTX : t2;
           }
+          if (S.ctx_mode) J.st[node[u]] = (uint16_t)s;  // the frontier is collected from st afterwards
         }
       }
-      const uint32_t word = __ballot_sync(FULL, s != ST_DEAD || eos_ok[u]);
+      const uint32_t word = __ballot_sync(FULL, (s != ST_DEAD && s != ST_CTX) || eos_ok[u]);
       if (lane == 0) S.mask_rows[(size_t)dst[u] * Wm + wd] = word;
     }
   }
@@ -1019,19 +758,29 @@ __global__ void publish_kernel(StateDev S) {
   if (j < n_jobs) {
     const uint32_t row = S.jobs[j];
     const int32_t sid = S.row_state[row];
-    const bool broken = (S.row_flags[row] & ROW_BROKEN) || S.counters[CNT_BAR_ERR];
-    if (S.counters[CNT_BAR_ERR]) atomicOr(&S.row_flags[row], ROW_BROKEN);
+    // a fill that was given up (a bounded wait ran out) hands out all-zero masks, never a guess; the
+    // rows themselves are fine and the next fill computes them afresh
+    const bool aborted = S.counters[CNT_BAR_ERR] != 0u;
+    const bool broken = (S.row_flags[row] & ROW_BROKEN) || aborted;
     if (sid >= 0) {
       const int32_t mrow = S.row_mask[row];
       S.st_mask[sid] = (!broken && mrow >= (int32_t)S.B) ? mrow : -1;
+    }
+    if (aborted) {
+      S.row_mask[row] = MASK_ZERO;
+      if (j == 0) stat_add(S, CNT_STAT_ABORTS, 1u);
     }
   }
 }
 
 __device__ __forceinline__ int32_t resolve_mask_row(const StateDev& S, uint32_t row) {
   int32_t r = S.row_mask[row];
-  if (r <= MASK_ALIAS0) r = S.row_mask[(uint32_t)(MASK_ALIAS0 - r)];
-  if (S.row_flags[row] & ROW_BROKEN) r = MASK_ZERO;
+  if (S.row_flags[row] & ROW_BROKEN) return MASK_ZERO;
+  if (r <= MASK_ALIAS0) {  // the mask another row of this call computed: not to be used if that row broke
+    const uint32_t other = (uint32_t)(MASK_ALIAS0 - r);
+    if (S.row_flags[other] & ROW_BROKEN) return MASK_ZERO;
+    r = S.row_mask[other];
+  }
   return r;
 }
 
@@ -1219,7 +968,7 @@ cudaError_t configure_kernels() {
   if ((e = opt_in_smem((const void*)init_kernel, init_smem_bytes())) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)advance_kernel, (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + HOT_TABLE_BYTES)) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)sweep_kernel, 224 * 1024)) != cudaSuccess) return e;
-  return cudaSuccess;
+  return configure_walk_kernels();
 }
 
 cudaError_t sweep_blocks_per_sm(int* out, uint32_t smem_bytes) {
@@ -1246,14 +995,8 @@ static void launch_sweep_coop(const GrammarDev& G, const StateDev& S, int grid, 
   cudaLaunchCooperativeKernel((const void*)sweep_kernel, dim3((unsigned)grid), dim3(SWEEP_WARPS * 32), args,
                               S.au.smem_bytes, st);
 }
-void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_sweep,
-                 cudaEvent_t after_sweep) {
-  plan_kernel<<<1, 1024, 0, st>>>(G, S);
-  if (before_sweep) cudaEventRecord(before_sweep, st);
-  launch_sweep_coop(G, S, sweep_grid, st);
-  if (after_sweep) cudaEventRecord(after_sweep, st);
-  publish_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(S);
-}
+void launch_plan(const GrammarDev& G, const StateDev& S, cudaStream_t st) { plan_kernel<<<1, 1024, 0, st>>>(G, S); }
+void launch_publish(const StateDev& S, cudaStream_t st) { publish_kernel<<<(S.B + 255) / 256, 256, 0, st>>>(S); }
 // the sweep alone, for jobs the caller has already listed (used by the allocation-free entry point)
 void launch_sweep(const GrammarDev& G, const StateDev& S, int grid, cudaStream_t st) { launch_sweep_coop(G, S, grid, st); }
 void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st) {

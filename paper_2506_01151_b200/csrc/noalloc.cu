@@ -165,6 +165,7 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   StateDev S{};
   S.B = n;
   S.cache_on = 0;
+  S.gen = 1;  // the hashes are cleared by every call
   S.arena = const_cast<uint32_t*>(charts_dev);  // the sweep only reads charts
   S.counters = scratch + NA_OFF_COUNTERS;
   S.jobs = scratch + NA_OFF_JOBS;

@@ -259,16 +259,22 @@ def test_capacity_overflow_is_reported_not_guessed():
     assert _advance(st2, [ord("[")]) == [0]
     for c in names[0].encode():
         assert _advance(st2, [c]) == [0]
-    _mask_of(st2, g, 1)
-    assert st2.stats()["capacity_errors"] == 0 or not _mask_of(st2, g, 1).any()
+    seq = oracle.Sequence_(og)
+    assert seq.advance(b"[" + names[0].encode())
+    got2 = _mask_of(st2, g, 1)[0]
+    if st2.stats()["capacity_errors"]:
+        assert not got2.any()  # reported: the mask is all-zero, never a partial one
+    else:
+        assert np.array_equal(got2, seq.mask(ov))
 
 
 def test_sweep_hash_generations_start_over():
     """The sweep's per-job hashes of Earley sets are never cleared between fills: every fill has a
-    16-bit generation and takes slots of other generations for empty.  After 65535 fills the numbers
-    start over, and that fill must clear the hashes first or it would meet its own old entries.
-    Two rows with the cache off (every fill sweeps) go through more than 65535 fills; the masks
-    before, at and after the turn must equal the oracle's."""
+    16-bit generation (two per fill: one for the sweep of new roots, one for the rows' own walks) and
+    takes slots of other generations for empty.  When the numbers start over (every 32767 fills) the
+    tables are cleared first, or a fill would meet its own old entries.  Two rows with the state cache
+    off (every fill computes them) go through more than 65535 fills; the masks before, at and after
+    every turn must equal the oracle's."""
     import paper_2506_01151_b200 as fmt
 
     torch, dev = _torch()
@@ -289,7 +295,7 @@ def test_sweep_hash_generations_start_over():
     total = 65535 + 40
     for i in range(total):
         st.fill_mask(m)
-        if i in (0, 65533, 65534, 65535, 65536, total - 1):
+        if i in (0, 32765, 32766, 32767, 32768, 32769, 65532, 65533, 65534, 65535, 65536, total - 1):
             assert np.array_equal(m.cpu().numpy().view(np.uint32), want), i
     assert st.stats()["capacity_errors"] == 0
 
