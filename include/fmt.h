@@ -76,7 +76,7 @@ typedef struct {
                                  whole vocabulary trie against its own chart */
   uint32_t max_roots;          /* entries of the context-independent mask cache (default 4096; each
                                  holds one mask row of ceil(V/32) words) */
-  uint32_t root_max_items;     /* a last Earley set with more items than this gets no entry (default 256) */
+  uint32_t root_max_items;     /* a last Earley set with more items than this gets no entry (default and maximum 1024) */
   uint32_t root_max_origins;   /* nor one whose items start in more distinct earlier sets (default 16) */
   uint32_t wait_limit_log2;    /* every wait inside a kernel is a poll that gives up after 2^this many
                                  polls (0 = defaults, 2^21..2^24); see fmt_state_set_wait_limit */
@@ -121,6 +121,9 @@ typedef struct {
   uint64_t walk_states;         /* distinct Earley sets they created */
   uint64_t frontier_entries;    /* trie nodes at which a walk started (context-dependent transitions) */
   uint64_t walk_tasks;          /* trie nodes expanded below them */
+  uint64_t walk_shared_nodes;   /* of those, nodes handed from one warp to another through the work queue */
+  uint64_t walk_frames;         /* sets met by a walk that were themselves known context-independent entries
+                                   (what follows them is looked up again instead of computed) */
   uint64_t fills_aborted;       /* fills given up because a bounded wait ran out (their rows got all-zero masks) */
   uint64_t device_bytes;        /* device memory fmt_state_create allocated for this state */
   uint64_t earley_step_cycles;  /* SM cycles spent inside the Earley steps of fills, summed over warps

@@ -347,7 +347,7 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   RootDev& rt = d.rt;
   rt.on = (opt && opt->roots_disable) ? 0u : 1u;
   rt.max_roots = (opt && opt->max_roots) ? opt->max_roots : 4096u;
-  rt.max_items = (opt && opt->root_max_items) ? opt->root_max_items : 256u;
+  rt.max_items = (opt && opt->root_max_items) ? std::min(opt->root_max_items, 1024u) : 1024u;
   rt.max_ph = (opt && opt->root_max_origins) ? std::min(opt->root_max_origins, 1024u) : 16u;
   uint32_t rh = 256;
   while (rh < rt.max_roots * 4u) rh <<= 1;
@@ -356,6 +356,11 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   rt.fr_cap = 8u << 20;
   rt.st_cap = 8u << 20;
   rt.it_cap = 64u << 20;
+  rt.tr_cap = 256u << 20;
+  rt.m_mask = (4u << 20) - 1;
+  rt.me_cap = 2u << 20;
+  rt.md_cap = 128u << 20;
+  rt.pend_cap = 4096;
   d.cx.q_cap = 4u << 20;
 
   sweep_layout(g->dev, &au.smem_bytes, &au.tables_in_smem);
@@ -406,7 +411,13 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(rt.frontier, rt.fr_cap, 0);
   AL(rt.states, rt.st_cap, 0);
   AL(rt.items, rt.it_cap, 0);
-  AL(rt.tops, 4, 0);
+  AL(rt.trans, rt.tr_cap, 0);
+  AL(rt.tops, TOP_N, 0);
+  AL(rt.mkey, (size_t)rt.m_mask + 1, 0);
+  AL(rt.mval, (size_t)rt.m_mask + 1, 0);
+  AL(rt.ment, rt.me_cap, 0);
+  AL(rt.mdata, rt.md_cap, 0);
+  AL(rt.pending, rt.pend_cap, 0);
   AL(rt.counters, CNT_TOTAL, 0);
   AL(rt.rj_chart, batch, 0);
   AL(rt.rj_mask, batch, 0);
@@ -418,6 +429,9 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(d.cx.chunk_off, (size_t)batch + 1, 0);
   AL(d.cx.queue, d.cx.q_cap, 0);
   AL(d.cx.qctr, Q_WORDS, 0);
+  AL(d.cx.frames, (size_t)batch * MAXF, 0);
+  AL(d.cx.fbind, (size_t)batch * MAXF * rt.max_ph, 0);
+  AL(d.cx.frame_ctr, batch, 0);
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);
@@ -537,7 +551,9 @@ fmt_status fmt_state_ci_cache_clear(fmt_state* s, void* stream) {
   RootDev& r = s->dev.rt;
   cudaError_t e = cudaMemsetAsync(r.hash, 0, ((size_t)r.hash_mask + 1) * 4, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(r.n_roots, 0, 4, st);
-  if (e == cudaSuccess) e = cudaMemsetAsync(r.tops, 0, 16, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(r.tops, 0, TOP_N * 4, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(r.mkey, 0, ((size_t)r.m_mask + 1) * 8, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(r.mval, 0, ((size_t)r.m_mask + 1) * 4, st);
   if (e != cudaSuccess) return cuda_fail(e, "fmt_state_ci_cache_clear");
   return FMT_OK;
 }
@@ -659,6 +675,8 @@ fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   out->walk_states = u64(CNT_STAT_CTX_STATES);
   out->frontier_entries = u64(CNT_STAT_FRONTIER);
   out->walk_tasks = u64(CNT_STAT_TASKS);
+  out->walk_shared_nodes = u64(CNT_STAT_SHARED_NODES);
+  out->walk_frames = u64(CNT_STAT_FRAMES);
   out->root_sweeps = u64(CNT_STAT_ROOT_SWEEPS);
   out->fills_aborted = u64(CNT_STAT_ABORTS);
   out->device_bytes = s->device_bytes;

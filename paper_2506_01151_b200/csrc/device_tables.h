@@ -84,8 +84,10 @@ enum : uint32_t {
   CNT_STAT_ABORTS = 160,       // 64-bit: fills abandoned because a bounded wait ran out
   CNT_STAT_STEP_CYCLES = 162,  // 64-bit: SM cycles spent inside Earley steps of the fill (summed over warps)
   CNT_STAT_ADV_WORDS = 164,    // 64-bit: chart words read and written by advance
+  CNT_STAT_SHARED_NODES = 182, // 64-bit: nodes handed from one warp to the others through the queue
+  CNT_STAT_FRAMES = 184,       // 64-bit: frames made (sets of a walk recognised as roots)
   CNT_DIAG = 166,              // [16] where capacity errors and expired waits came from (see DIAG_*)
-  CNT_TOTAL = 182
+  CNT_TOTAL = 186
 };
 
 enum : uint32_t {
@@ -151,9 +153,10 @@ constexpr uint32_t ROOT_NONE = 0xffffffffu;
 enum : uint32_t { ROOT_NEW = 0, ROOT_READY = 1, ROOT_FAILED = 2 };
 enum : uint32_t {  // words of a root's directory entry
   RI_STATUS = 0, RI_P = 1, RI_NK = 2, RI_N = 3, RI_HASH = 4, RI_CHART = 5, RI_FR_OFF = 6, RI_FR_N = 7,
-  RI_ST_OFF = 8, RI_NSTATES = 9, RI_USES = 10, RI_WORDS = 16
+  RI_ST_OFF = 8, RI_NSTATES = 9, RI_TR_OFF = 10, RI_WORDS = 16
 };
-enum : uint32_t { TOP_CHARTS = 0, TOP_FRONTIER = 1, TOP_STATES = 2, TOP_ITEMS = 3 };
+enum : uint32_t { TOP_CHARTS = 0, TOP_FRONTIER = 1, TOP_STATES = 2, TOP_ITEMS = 3, TOP_TRANS = 4, TOP_MENT = 5, TOP_MDATA = 6, TOP_PENDING = 7, TOP_N = 8 };
+constexpr uint16_t R_DEAD = 0xFFFFu, R_CTX = 0xFFFEu;  // values of a region's transition table besides set numbers
 
 struct RootDev {
   uint32_t on;           // 0: every computed row walks the whole trie itself
@@ -172,7 +175,23 @@ struct RootDev {
   uint32_t st_cap;
   uint32_t* items;       // pool
   uint32_t it_cap;
-  uint32_t* tops;        // [4] tops of the four pools
+  uint16_t* trans;       // pool: per region set one entry per byte class: the set reached, R_DEAD or R_CTX
+  uint32_t tr_cap;
+  uint32_t* tops;        // [TOP_N] tops of the pools
+  // What a root's region makes of the subtree of a trie node, when the walk of some row stands at that
+  // node in the root set: the tokens below that are valid whatever the chart holds, and the nodes where
+  // the chart is needed again (node, region set | byte class << 16).  Computed once per (root, node)
+  // by whoever needs it first, then shared by all rows and fills.
+  unsigned long long* mkey;  // [m_mask + 1] (root + 1) << 32 | node, 0 = empty
+  uint32_t* mval;            // [m_mask + 1] 0 while it is being computed, then entry + 1
+  uint32_t m_mask;
+  uint4* ment;               // pool: x = first word in mdata, y = tokens, z = frontier entries (two words each, after the tokens)
+  uint32_t me_cap;
+  uint32_t* mdata;           // pool
+  uint32_t md_cap;
+  // roots made by a walk (a set it met had no entry yet): swept by the next fill
+  uint32_t* pending;         // [pend_cap] root ids
+  uint32_t pend_cap;
   uint32_t* counters;    // [CNT_TOTAL] counters of the root sweep (its own barrier, queue and job counts)
   // the roots to sweep in this fill, as the rows of the sweep's view of the state
   uint64_t* rj_chart;    // [B] word offset of the root's chart in `charts`
@@ -194,6 +213,21 @@ struct CtxJob {
   uint32_t pad[2];
 };
 
+// A frame: a root's region as one job sees it, with the root's placeholders bound to sets of the job's
+// chart.  Frame 0 is the job's own root; further frames appear when a context-dependent step of the
+// walk lands on a set that is itself a known root (what follows it is context-independent again).
+// Set k of a frame is named by the code RBASE + k, in every frame: which frame is meant follows from
+// where the code stands.  A set made by a step out of a frame's set lives "in" that frame (the frame
+// codes among its origins mean that frame's sets), and so does every set made from it; a set whose
+// origins all lie in the chart depends on no frame, and only such a set can open a frame of its own.
+struct Frame {
+  uint32_t root, P, n, st_off, tr_off, pad0, pad1, pad2;
+};
+constexpr uint32_t MAXF = 255;        // frames per job
+constexpr uint32_t NOFRAME = 0xffffffffu;
+constexpr uint32_t AR_FRAME = 12;     // word of a walk's set record: 0 not looked up yet, NOFRAME, or frame + 1 (the frame it opens)
+constexpr uint32_t AR_SALT = 13;      // word of a set record: 0, or frame + 1 (the frame the set lives in)
+
 constexpr uint32_t CT_SLOTS = 1024;  // per job: remembered transitions out of region sets (power of two)
 enum : uint32_t { Q_TAIL = 0, Q_HEAD = 32, Q_OUT = 64, Q_CHUNK = 96, Q_CHUNKS = 97, Q_WORDS = 128 };
 
@@ -201,11 +235,14 @@ struct CtxDev {
   uint32_t* job_root;          // [B] root of job j (ROOT_NONE: none)
   uint16_t* bind;              // [B][max_ph] the chart set each placeholder stands for
   CtxJob* jobs;                // [B]
-  unsigned long long* ctab;    // [B][CT_SLOTS] generation << 48 | (region set << 8 | byte class) << 24 | value
+  unsigned long long* ctab;    // [B][CT_SLOTS] generation << 48 | (frame + 1) << 40 | set code << 24 | byte class << 16 | value
   uint32_t* chunk_off;         // [B + 1] first chunk (32 frontier entries) of each job
   uint4* queue;                // [q_cap] x: node, y: set the node leads to, z: job, w: tag (generation << 16 | 1), written last
   uint32_t q_cap;
   uint32_t* qctr;              // [Q_WORDS] tail, head, outstanding work, next chunk: one 128-byte line each
+  Frame* frames;               // [B][MAXF]
+  uint16_t* fbind;             // [B][MAXF][max_ph] what each frame's placeholders stand for (sets of the chart)
+  uint32_t* frame_ctr;         // [B] frames of the job so far
 };
 
 struct StateDev {

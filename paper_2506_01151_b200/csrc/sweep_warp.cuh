@@ -104,6 +104,7 @@ struct SweepWarp {
   unsigned long long cycles = 0;           // SM cycles inside step()
   uint32_t chunk_at = 0, chunk_left = 0;   // this warp's private piece of the item pool (lane 0's copy counts)
   uint32_t gen = 1;                        // this fill's generation of the per-job hashes
+  uint32_t salt = 0;                       // told apart by it: sets with equal items that mean different things (see Frame)
 
   // A new set of job J with the items w.cur[0..n), the first nk of them its kernel: its id or T_FAIL.
   __device__ uint32_t create_set(const JobCtx& J, uint32_t n, uint32_t nk, uint32_t hash) {
@@ -143,6 +144,7 @@ struct SweepWarp {
       else if (i == AR_N) v2 = n;
       else if (i == AR_HASH) v2 = hash;
       else if (i == AR_NK) v2 = nk;
+      else if (i == AR_SALT) v2 = salt;
       else if (i >= AR_SCAN && i < AR_SCAN + 8) v2 = tmp8[i - AR_SCAN];
       else if (i >= AR_TRANS) v2 = T_UNKNOWN;
       rec[i] = v2;
@@ -159,7 +161,7 @@ struct SweepWarp {
   __device__ __forceinline__ bool same_set(const JobCtx& J, uint32_t sid, uint32_t nk, uint32_t hash, Member member) {
     const uint32_t lane = lane_id();
     const uint32_t* rec = J.recs + (size_t)sid * S.au.rec_words;
-    if (__ldcg(rec + AR_HASH) != hash || __ldcg(rec + AR_NK) != nk) return false;
+    if (__ldcg(rec + AR_HASH) != hash || __ldcg(rec + AR_NK) != nk || __ldcg(rec + AR_SALT) != salt) return false;
     const uint32_t* items = S.au.items + __ldcg(rec + AR_ITEMS);
     bool ok = true;
     for (uint32_t base = 0; base < nk; base += 32) {
@@ -250,7 +252,7 @@ struct SweepWarp {
     const uint32_t nk = small_drop_completed(G, w, n, mine);
     uint32_t h = lane < nk ? mix32(mine) : 0u;
     for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
-    h = mix32(h + nk * 0x9E3779B9u);
+    h = mix32(h + nk * 0x9E3779B9u + salt * 0x85EBCA77u);
     auto member = [&](uint32_t x, bool valid) {  // the kernel sits one item per lane
       bool found = false;
       for (uint32_t i = 0; i < nk; ++i)
@@ -306,7 +308,7 @@ struct SweepWarp {
       nk += __popc(__ballot_sync(FULL, keep));
     }
     for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
-    h = mix32(h + nk * 0x9E3779B9u);
+    h = mix32(h + nk * 0x9E3779B9u + salt * 0x85EBCA77u);
     auto member = [&](uint32_t x, bool valid) { return !valid || hset_contains(w.hset, w.hset_mask, x); };
     const uint32_t id = lookup_set(J, nk, h, member);
     if (id != T_FAIL) {

@@ -60,7 +60,7 @@ def test_rows_with_different_charts_share_the_context_independent_part():
     for b in range(2):
         assert np.array_equal(got[b], seqs[b].mask(ov)), b
     s0 = st.stats()
-    assert s0["roots"] >= 2 and s0["root_sweeps"] == s0["roots"] and s0["sweep_transitions"] > 0
+    assert s0["roots"] >= 2 and s0["root_sweeps"] >= 2 and s0["sweep_transitions"] > 0
     # row 1 now reaches the inside of a string by another way
     _feed_bytes(st, seqs, [[], list(b'[[1, {"k": ["yz')])
     q = st.query()
@@ -69,8 +69,8 @@ def test_rows_with_different_charts_share_the_context_independent_part():
     for b in range(2):
         assert np.array_equal(got[b], seqs[b].mask(ov)), b
     s1 = st.stats()
-    assert s1["roots"] == s0["roots"] and s1["root_sweeps"] == s0["root_sweeps"]  # nothing new was swept
-    assert s1["sweep_transitions"] == s0["sweep_transitions"]
+    # the only sweeps since are of sets the first row's walk met on its way (entered then, swept now)
+    assert s1["root_sweeps"] - s0["root_sweeps"] <= s0["roots"] - s0["root_sweeps"]
     assert s1["rows_from_root"] - s0["rows_from_root"] == 2 and s1["rows_plain"] == s0["rows_plain"]
     # what is left per row is the closing quote and what may follow it in that row's context
     assert s1["walk_transitions"] - s0["walk_transitions"] < 1000
