@@ -115,15 +115,13 @@ typedef struct {
   uint64_t advances_cached;     /* row-advances answered by the transition cache (no Earley step run) */
   uint64_t roots;               /* entries of the context-independent mask cache */
   uint64_t root_sweeps;         /* vocabulary sweeps done to fill such entries (one per entry) */
-  uint64_t rows_from_root;      /* computed rows that started from such an entry */
-  uint64_t rows_plain;          /* computed rows that walked the whole trie against their own chart */
-  uint64_t walk_transitions;    /* Earley steps of the context-dependent walks */
+  uint64_t rows_mask_only;      /* computed rows answered by their entry's mask alone (nothing in their state mattered) */
+  uint64_t rows_from_root;      /* computed rows swept over the vocabulary starting from such an entry */
+  uint64_t rows_plain;          /* computed rows swept from their own chart's last set (no usable entry) */
+  uint64_t walk_transitions;    /* Earley steps run for context-dependent transitions of those sweeps */
   uint64_t walk_states;         /* distinct Earley sets they created */
-  uint64_t frontier_entries;    /* trie nodes at which a walk started (context-dependent transitions) */
-  uint64_t walk_tasks;          /* trie nodes expanded below them */
-  uint64_t walk_shared_nodes;   /* of those, nodes handed from one warp to another through the work queue */
-  uint64_t walk_frames;         /* sets met by a walk that were themselves known context-independent entries
-                                   (what follows them is looked up again instead of computed) */
+  uint64_t walk_frames;         /* of those, sets that were themselves known entries (what follows them is
+                                   looked up in the entry's transition table again instead of computed) */
   uint64_t fills_aborted;       /* fills given up because a bounded wait ran out (their rows got all-zero masks) */
   uint64_t device_bytes;        /* device memory fmt_state_create allocated for this state */
   uint64_t earley_step_cycles;  /* SM cycles spent inside the Earley steps of fills, summed over warps

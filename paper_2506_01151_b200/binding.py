@@ -57,8 +57,7 @@ class Stats(C.Structure):
         "steps_advanced", "fills", "fills_computed", "fills_from_cache", "fills_shared", "states_cached",
         "mask_rows_cached", "pool_words_used", "chart_items_max", "chart_sets_max", "capacity_errors",
         "big_mode_units", "sweep_transitions", "sweep_states", "advances_cached", "roots", "root_sweeps",
-        "rows_from_root", "rows_plain", "walk_transitions", "walk_states", "frontier_entries", "walk_tasks",
-        "walk_shared_nodes", "walk_frames",
+        "rows_mask_only", "rows_from_root", "rows_plain", "walk_transitions", "walk_states", "walk_frames",
         "fills_aborted", "device_bytes", "earley_step_cycles", "advance_chart_words")] + [("diag", C.c_uint64 * 16)]
 
     def as_dict(self):

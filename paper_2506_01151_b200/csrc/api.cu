@@ -126,7 +126,7 @@ static cudaError_t next_generations(fmt_state* s, cudaStream_t st) {
     e = cudaMemsetAsync(d.au.hash, 0, (size_t)d.B * (d.au.hash_mask + 1u) * 4, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(d.au.req, 0, (size_t)d.au.req_cap * 8, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(d.cx.ctab, 0, (size_t)d.B * CT_SLOTS * 8, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(d.cx.queue, 0, (size_t)d.cx.q_cap * 16, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d.cx.req2, 0, (size_t)d.cx.req2_cap * 16, st);
     s->next_gen = 1;
   }
   d.gen = s->next_gen;
@@ -353,15 +353,10 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   while (rh < rt.max_roots * 4u) rh <<= 1;
   rt.hash_mask = rh - 1;
   rt.charts_cap = rt.max_roots * 512u;
-  rt.fr_cap = 8u << 20;
   rt.st_cap = 8u << 20;
   rt.it_cap = 64u << 20;
   rt.tr_cap = 256u << 20;
-  rt.m_mask = (4u << 20) - 1;
-  rt.me_cap = 2u << 20;
-  rt.md_cap = 128u << 20;
   rt.pend_cap = 4096;
-  d.cx.q_cap = 4u << 20;
 
   sweep_layout(g->dev, &au.smem_bytes, &au.tables_in_smem);
   cudaError_t e = configure_kernels();
@@ -408,15 +403,10 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(rt.n_roots, 4, 0);
   AL(rt.charts, rt.charts_cap, 0);
   AL(rt.ci_rows, (size_t)rt.max_roots * g->dev.Wm, 0);
-  AL(rt.frontier, rt.fr_cap, 0);
   AL(rt.states, rt.st_cap, 0);
   AL(rt.items, rt.it_cap, 0);
   AL(rt.trans, rt.tr_cap, 0);
   AL(rt.tops, TOP_N, 0);
-  AL(rt.mkey, (size_t)rt.m_mask + 1, 0);
-  AL(rt.mval, (size_t)rt.m_mask + 1, 0);
-  AL(rt.ment, rt.me_cap, 0);
-  AL(rt.mdata, rt.md_cap, 0);
   AL(rt.pending, rt.pend_cap, 0);
   AL(rt.counters, CNT_TOTAL, 0);
   AL(rt.rj_chart, batch, 0);
@@ -426,12 +416,13 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   AL(d.cx.bind, (size_t)batch * rt.max_ph, 0);
   AL(d.cx.jobs, batch, 0);
   AL(d.cx.ctab, (size_t)batch * CT_SLOTS, 0);
-  AL(d.cx.chunk_off, (size_t)batch + 1, 0);
-  AL(d.cx.queue, d.cx.q_cap, 0);
-  AL(d.cx.qctr, Q_WORDS, 0);
+  AL(d.cx.fjobs, batch, 0);
   AL(d.cx.frames, (size_t)batch * MAXF, 0);
   AL(d.cx.fbind, (size_t)batch * MAXF * rt.max_ph, 0);
   AL(d.cx.frame_ctr, batch, 0);
+  AL(d.cx.st32, (size_t)batch * au.st_stride, 0xFF);
+  d.cx.req2_cap = 1u << 20;
+  AL(d.cx.req2, d.cx.req2_cap, 0);
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);
@@ -552,8 +543,7 @@ fmt_status fmt_state_ci_cache_clear(fmt_state* s, void* stream) {
   cudaError_t e = cudaMemsetAsync(r.hash, 0, ((size_t)r.hash_mask + 1) * 4, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(r.n_roots, 0, 4, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(r.tops, 0, TOP_N * 4, st);
-  if (e == cudaSuccess) e = cudaMemsetAsync(r.mkey, 0, ((size_t)r.m_mask + 1) * 8, st);
-  if (e == cudaSuccess) e = cudaMemsetAsync(r.mval, 0, ((size_t)r.m_mask + 1) * 4, st);
+
   if (e != cudaSuccess) return cuda_fail(e, "fmt_state_ci_cache_clear");
   return FMT_OK;
 }
@@ -673,9 +663,7 @@ fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   out->rows_plain = u64(CNT_STAT_JOBS_PLAIN);
   out->walk_transitions = u64(CNT_STAT_CTX_TRANS);
   out->walk_states = u64(CNT_STAT_CTX_STATES);
-  out->frontier_entries = u64(CNT_STAT_FRONTIER);
-  out->walk_tasks = u64(CNT_STAT_TASKS);
-  out->walk_shared_nodes = u64(CNT_STAT_SHARED_NODES);
+  out->rows_mask_only = u64(CNT_STAT_JOBS_MASK);
   out->walk_frames = u64(CNT_STAT_FRAMES);
   out->root_sweeps = u64(CNT_STAT_ROOT_SWEEPS);
   out->fills_aborted = u64(CNT_STAT_ABORTS);

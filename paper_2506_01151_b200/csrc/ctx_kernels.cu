@@ -1,13 +1,14 @@
-// The mask fill in two parts (Section 4.3 of the paper: tokens whose validity does not depend on the
-// context are looked up, only the context-dependent ones are checked against the parser state).
+// The mask fill (Sections 4.1, 4.3 of the paper: tokens whose validity does not depend on the context
+// are looked up, only the context-dependent ones are checked against the parser state).
 //
-//   root_kernel      per computed row: its chart's last set with anonymous origins (a "root") is
-//                    looked up in, or added to, the directory of roots
-//   sweep_kernel     (kernels.cu, root mode) the trie sweep of every new root, once for good
-//   collect_kernel   turns a finished root sweep into the root's frontier list and region of sets
-//   ctx_init_kernel  starts every job's mask row from its root's context-independent mask
-//   ctx_kernel       the context-dependent walk: from each frontier node on, Earley steps against the
-//                    row's own chart (Section 3.2), memoised per job, spread over the grid by a queue
+//   root_kernel       per computed row: its chart's last set with anonymous origins (a "root") is
+//                     looked up in, or added to, the directory of roots
+//   sweep_kernel      (kernels.cu, root mode) the trie sweep of every new root, once for good
+//   collect_kernel    keeps a finished root sweep: mask row, region of sets, transition table
+//   job_setup_kernel  rows whose root has no context-dependent trie node take the root's mask row;
+//                     the others get their frame 0 and go to
+//   fill_kernel       the level sweep over the trie, per (row, node): table look-ups inside frames,
+//                     Earley steps against the row's own chart (Section 3.2) where the context matters
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -23,9 +24,6 @@ __device__ __forceinline__ void st_release64(unsigned long long* p, unsigned lon
 }
 __device__ __forceinline__ void st_release32(uint32_t* p, uint32_t v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t ctx_poll_limit(const StateDev& S, uint32_t dflt) {
-  return 1u << (S.poll_limit_shift ? S.poll_limit_shift : dflt);
 }
 
 // ===================================================================================== roots
@@ -201,7 +199,7 @@ __global__ void __launch_bounds__(ROOT_WARPS * 32) root_kernel(GrammarDev G, Sta
       cj.row_acc = row | ((chart[CH_FLAGS] & CHART_ACCEPTING) ? 0x80000000u : 0u);
       cj.root = root;
       cj.P = P;
-      cj.fr_off = cj.fr_n = cj.st_off = 0;
+      cj.spare[0] = cj.spare[1] = cj.spare[2] = 0;
       cj.mrow = S.row_mask[row];
       cj.pad[0] = cj.pad[1] = 0;
       S.cx.jobs[j] = cj;
@@ -212,10 +210,11 @@ __global__ void __launch_bounds__(ROOT_WARPS * 32) root_kernel(GrammarDev G, Sta
 // ===================================================================================== collect
 //
 // After the root sweep: one CTA per swept root keeps what later fills need.  The sweep left, per trie
-// node, the set the node leads to (or dead / context-dependent) and, per set, its items.  Kept are
-// the frontier (nodes marked context-dependent, with the set of their parent), in node order, and
-// the items of every set (the walk of a row reads them with its own bindings); the transitions are
-// not needed again: the trie has been swept for good.
+// node, the set the node leads to (or dead / context-dependent) and, per set, its items and
+// transitions.  Kept are the root's mask row (written by the sweep itself), the number of trie nodes
+// marked context-dependent (none: the mask row is the whole answer for any row with this root), the
+// items of every set (an Earley step of a row reads them with the row's bindings) and the
+// transitions, as a table of 16-bit entries.
 
 constexpr int COLLECT_THREADS = 1024;
 
@@ -291,11 +290,10 @@ __global__ void __launch_bounds__(COLLECT_THREADS) collect_kernel(GrammarDev G, 
   if (threadIdx.x == 0) {
     uint32_t fo = 0, so = 0, io = 0, to = 0, f = failed ? 1u : 0u;
     if (!f) {
-      fo = atomicAdd(&R.tops[TOP_FRONTIER], fr_total);
       so = atomicAdd(&R.tops[TOP_STATES], nst);
       io = atomicAdd(&R.tops[TOP_ITEMS], it_total);
       to = atomicAdd(&R.tops[TOP_TRANS], tr_total);
-      if (fo > R.fr_cap || fr_total > R.fr_cap - fo || so > R.st_cap || nst > R.st_cap - so || io > R.it_cap || it_total > R.it_cap - io ||
+      if (so > R.st_cap || nst > R.st_cap - so || io > R.it_cap || it_total > R.it_cap - io ||
           to > R.tr_cap || tr_total > R.tr_cap - to)
         f = 1u;
     }
@@ -305,20 +303,9 @@ __global__ void __launch_bounds__(COLLECT_THREADS) collect_kernel(GrammarDev G, 
   __syncthreads();
   if (threadIdx.x < 256) rep_byte[G.eq_of_byte[threadIdx.x]] = (uint8_t)threadIdx.x;  // any byte of the class will do
   __syncthreads();
-  const uint32_t fr_off = sh[0], st_off = sh[1], it_off = sh[2], tr_off = sh[4];
+  const uint32_t st_off = sh[1], it_off = sh[2], tr_off = sh[4];
   failed = sh[3] != 0u;
   if (!failed) {
-    // ---- pass 2: the frontier in node order
-    uint32_t done = 0;
-    for (uint32_t base = 1; base < visited_end; base += blockDim.x) {
-      const uint32_t node = base + threadIdx.x;
-      uint32_t ps = 0;
-      const bool is_f = node < visited_end && frontier_at(node, ps);
-      uint32_t tile;
-      const uint32_t at = block_scan(is_f ? 1u : 0u, sums, tile);
-      if (is_f) R.frontier[fr_off + done + at] = make_uint2(node, ps | ((uint32_t)G.eq_of_byte[G.node_byte[node]] << 16));
-      done += tile;
-    }
     // ---- the region: where each set's items go, then the items
     uint32_t run = 0;
     for (uint32_t base = 0; base < nst; base += blockDim.x) {
@@ -353,7 +340,6 @@ __global__ void __launch_bounds__(COLLECT_THREADS) collect_kernel(GrammarDev G, 
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
-    info[RI_FR_OFF] = fr_off;
     info[RI_FR_N] = failed ? 0u : fr_total;
     info[RI_ST_OFF] = st_off;
     info[RI_TR_OFF] = tr_off;
@@ -365,79 +351,48 @@ __global__ void __launch_bounds__(COLLECT_THREADS) collect_kernel(GrammarDev G, 
   }
 }
 
-// ===================================================================================== walk: set-up
+// ===================================================================================== fill: set-up
 //
-// Every job's mask row starts as its root's context-independent mask (or empty), plus the EOS bit of
-// an accepting chart; block 0 also lists the work: the frontier of every job in chunks of 32 entries,
-// and gives every job with a usable root its frame 0.  A job without one starts at the trie's first
-// level with the chart's own last set.
+// One CTA per job.  A job whose root has been swept and has no context-dependent trie node at all
+// takes the root's mask row as it is (plus the EOS bit of an accepting chart): Section 4.3's
+// context-independent mask, and nothing else to do.  Every other job goes to the level sweep: with
+// frame 0 (its root's region, placeholders bound as root_kernel found them) if it has a root, from
+// the chart's own last set if not.
 
-__global__ void __launch_bounds__(1024) ctx_init_kernel(GrammarDev G, StateDev S) {
+__global__ void __launch_bounds__(256) job_setup_kernel(GrammarDev G, StateDev S) {
   const uint32_t n_jobs = S.counters[CNT_N_JOBS];
   const RootDev& R = S.rt;
   const uint32_t Wm = G.Wm;
-  auto ready = [&](const CtxJob& cj) { return cj.root != ROOT_NONE && __ldcg(R.info + (size_t)cj.root * RI_WORDS + RI_STATUS) == ROOT_READY; };
   for (uint32_t j = blockIdx.x; j < n_jobs; j += gridDim.x) {
     const CtxJob cj = S.cx.jobs[j];
-    const bool use = ready(cj);
-    const uint32_t* src = use ? R.ci_rows + (size_t)cj.root * Wm : nullptr;
-    uint32_t* dst = S.mask_rows + (size_t)cj.mrow * Wm;
-    const bool acc = (cj.row_acc >> 31) != 0u && G.eos >= 0;
-    for (uint32_t w = threadIdx.x; w < Wm; w += blockDim.x) {
-      uint32_t v = src ? src[w] : 0u;
-      if (acc && w == ((uint32_t)G.eos >> 5)) v |= 1u << ((uint32_t)G.eos & 31u);
-      dst[w] = v;
+    const uint32_t* info = R.info + (size_t)(cj.root != ROOT_NONE ? cj.root : 0u) * RI_WORDS;
+    const bool use = cj.root != ROOT_NONE && __ldcg(info + RI_STATUS) == ROOT_READY;
+    if (use && __ldcg(info + RI_FR_N) == 0u) {
+      const uint32_t* src = R.ci_rows + (size_t)cj.root * Wm;
+      uint32_t* dst = S.mask_rows + (size_t)cj.mrow * Wm;
+      const bool acc = (cj.row_acc >> 31) != 0u && G.eos >= 0;
+      for (uint32_t w = threadIdx.x; w < Wm; w += blockDim.x) {
+        uint32_t v = src[w];
+        if (acc && w == ((uint32_t)G.eos >> 5)) v |= 1u << ((uint32_t)G.eos & 31u);
+        dst[w] = v;
+      }
+      if (threadIdx.x == 0) stat_add(S, CNT_STAT_JOBS_MASK, 1u);
+      continue;
     }
-    // frame 0: the job's own root, its placeholders bound as root_kernel found them
-    const uint32_t* info = R.info + (size_t)(use ? cj.root : 0u) * RI_WORDS;
     if (threadIdx.x == 0) {
       Frame f;
       f.root = cj.root, f.P = cj.P, f.n = use ? info[RI_NSTATES] : 0u;
       f.st_off = use ? info[RI_ST_OFF] : 0u, f.tr_off = use ? info[RI_TR_OFF] : 0u, f.pad0 = f.pad1 = f.pad2 = 0u;
       S.cx.frames[(size_t)j * MAXF] = f;
       S.cx.frame_ctr[j] = use ? 1u : 0u;
+      S.cx.jobs[j].pad[0] = use ? 1u : 0u;
+      S.au.n_states[j] = 0u;
+      S.cx.fjobs[atomicAdd(&S.counters[CNT_N_FJOBS], 1u)] = j;
+      stat_add(S, use ? CNT_STAT_JOBS_ROOT : CNT_STAT_JOBS_PLAIN, 1u);
     }
     if (use)
       for (uint32_t i = threadIdx.x; i < cj.P && i < R.max_ph; i += blockDim.x)
         S.cx.fbind[(size_t)j * MAXF * R.max_ph + i] = S.cx.bind[(size_t)j * R.max_ph + i];
-  }
-  if (blockIdx.x != 0) return;
-  __shared__ uint32_t sums[33];
-  uint32_t run = 0;
-  for (uint32_t base = 0; base < n_jobs; base += blockDim.x) {
-    const uint32_t j = base + threadIdx.x;
-    uint32_t chunks = 0;
-    if (j < n_jobs) {
-      CtxJob cj = S.cx.jobs[j];
-      const bool use = ready(cj);
-      const uint32_t* info = R.info + (size_t)(use ? cj.root : 0u) * RI_WORDS;
-      uint32_t fr_off, fr_n, st_off = 0;
-      if (use) {
-        fr_off = info[RI_FR_OFF], fr_n = info[RI_FR_N], st_off = info[RI_ST_OFF];
-        stat_add(S, CNT_STAT_JOBS_ROOT, 1u);
-      } else {
-        fr_off = G.lvl_off[1], fr_n = G.lvl_off[2] - G.lvl_off[1];
-        stat_add(S, CNT_STAT_JOBS_PLAIN, 1u);
-      }
-      S.cx.jobs[j].fr_off = fr_off;
-      S.cx.jobs[j].fr_n = fr_n;
-      S.cx.jobs[j].st_off = st_off;
-      S.cx.jobs[j].pad[0] = use ? 1u : 0u;
-      S.au.n_states[j] = 0u;
-      chunks = (fr_n + 31u) / 32u;
-    }
-    uint32_t tile;
-    const uint32_t at = block_scan(chunks, sums, tile);
-    if (j < n_jobs) S.cx.chunk_off[j] = run + at;
-    run += tile;
-  }
-  if (threadIdx.x == 0) {
-    S.cx.chunk_off[n_jobs] = run;
-    S.cx.qctr[Q_TAIL] = 0u;
-    S.cx.qctr[Q_HEAD] = 0u;
-    S.cx.qctr[Q_OUT] = run;
-    S.cx.qctr[Q_CHUNK] = 0u;
-    S.cx.qctr[Q_CHUNKS] = run;
   }
 }
 
@@ -488,9 +443,6 @@ struct WalkView {
 };
 
 constexpr uint32_t NOF = 0xffffffffu;                       // "no frame"
-constexpr uint32_t STACK_NODES = 4096;                      // nodes a warp may hold for itself (node, set code | job << 16, frame)
-constexpr uint32_t STACK_WORDS = 3u * STACK_NODES;
-constexpr uint32_t SHARE_ABOVE = 6, SHARE_N = 32;           // a warp holding more nodes than this hands all but 4 (at most 32) to the queue
 constexpr uint32_t V_DEAD = 0xFFFFu, V_PEND = 0xFFFEu;      // values of a remembered transition (16 bits)
 constexpr uint32_t CODE_CHART = 0xFFFFu;                    // "parent set" of a job without a root: the chart's last set
 
@@ -500,11 +452,7 @@ struct Walker {
   SweepWarp& sw;
   uint32_t* big;
   bool big_mode = false;
-  uint32_t n_frontier = 0, n_tasks = 0, n_nodes = 0, n_frames = 0;
-  // Nodes waiting to be expanded by this warp: a stack at the top of the warp's large scratch area
-  // (the sets under construction use the part below).  Entry: node, set code | job << 16.
-  uint32_t held = 0;
-  __device__ __forceinline__ uint32_t* stack() const { return big + (S.big_arena_items - STACK_WORDS); }
+  uint32_t n_frames = 0;
 
   __device__ __forceinline__ JobCtx job(const CtxJob& cj, uint32_t j) const {
     const AutoDev& A = S.au;
@@ -548,6 +496,7 @@ struct Walker {
     const JobCtx J = job(cj, j);
     const WalkView v = view(J, j, frame);
     sw.salt = frame == NOF ? 0u : frame + 1u;
+    sw.region_base = LBASE;  // (a set that names sets of the walk's own may depend on the frame through them)
     const uint32_t* pitems;
     uint32_t plen;
     v(pcode, pitems, plen);
@@ -557,7 +506,7 @@ struct Walker {
       hset_clear_all(sw.w.hset, sw.w.hset_mask);
       clear_nt(G, sw.w);
       sw.w.cur = big;
-      sw.w.cur_cap = S.big_arena_items - STACK_WORDS;
+      sw.w.cur_cap = S.big_arena_items;
       sw.w.hset = big + S.big_arena_items;
       sw.w.hset_mask = S.big_hset_slots - 1;
       if (lane_id() == 0) stat_add(S, CNT_STAT_BIG, 1u);
@@ -572,180 +521,7 @@ struct Walker {
     }
     return r;
   }
-  // the tokens whose bytes end at `node` are valid
-  __device__ __forceinline__ void mark_tokens(const CtxJob& cj, uint32_t node) const {
-    uint32_t* row = S.mask_rows + (size_t)cj.mrow * G.Wm;
-    for (uint32_t i = __ldg(&G.tok_off[node]), e = __ldg(&G.tok_off[node + 1]); i < e; ++i) {
-      const uint32_t t = __ldg(&G.tok_ids[i]);
-      atomicOr(&row[t >> 5], 1u << (t & 31u));
-    }
-  }
-  // The nodes of the lanes with `want` (alive, reached in set `code`, with children) go onto this warp's stack.
-  __device__ void keep(const CtxJob& cj, uint32_t j, bool want, uint32_t node, uint32_t code, uint32_t frame) {
-    const uint32_t lane = lane_id();
-    const uint32_t wb = __ballot_sync(FULL, want);
-    if (!wb) return;
-    const uint32_t k = held + __popc(wb & ((1u << lane) - 1u));
-    bool gone = false;
-    if (want) {
-      if (k < STACK_NODES) {
-        uint32_t* st = stack();
-        st[3u * k] = node;
-        st[3u * k + 1u] = code | (j << 16);
-        st[3u * k + 2u] = frame;
-      } else {
-        gone = true;
-      }
-    }
-    held = min(held + __popc(wb), STACK_NODES);
-    __syncwarp();
-    if (__any_sync(FULL, gone)) {  // (the queue was full and the stack is, too)
-      if (lane == 0) diag(S, DIAG_QUEUE_FULL);
-      break_row(job(cj, j));
-    }
-  }
-  // A warp that holds many nodes hands the oldest ones (the largest subtrees) to the queue.
-  __device__ void share() {
-    if (held <= SHARE_ABOVE) return;
-    const uint32_t lane = lane_id();
-    uint32_t base = 0, fit = 0;
-    const uint32_t give = min(SHARE_N, held - 4u);
-    if (lane == 0) {
-      if (ld_acquire(&S.cx.qctr[Q_TAIL]) + give <= S.cx.q_cap) {
-        base = atomicAdd(&S.cx.qctr[Q_TAIL], give);
-        fit = base >= S.cx.q_cap ? 0u : min(give, S.cx.q_cap - base);
-        atomicAdd(&S.cx.qctr[Q_OUT], fit);  // (before this warp reports its own unit done)
-      }
-    }
-    base = __shfl_sync(FULL, base, 0);
-    fit = __shfl_sync(FULL, fit, 0);
-    if (fit == 0) return;
-    uint32_t* st = stack();
-    if (lane < fit) {
-      uint4* e = S.cx.queue + base + lane;
-      const uint32_t node = st[3u * lane], cj_ = st[3u * lane + 1u], fr_ = st[3u * lane + 2u];
-      e->x = node, e->y = (cj_ & 0xFFFFu) | (fr_ << 16), e->z = cj_ >> 16;
-      __threadfence();
-      st_release32(&e->w, (S.gen_ctx << 16) | 1u);
-    }
-    __syncwarp();
-    for (uint32_t i0 = 0; i0 + fit < held; i0 += 32) {  // close the gap
-      const uint32_t i = i0 + lane;
-      uint32_t a = 0, b = 0, c = 0;
-      if (i + fit < held) a = st[3u * (i + fit)], b = st[3u * (i + fit) + 1u], c = st[3u * (i + fit) + 2u];
-      __syncwarp();
-      if (i + fit < held) st[3u * i] = a, st[3u * i + 1u] = b, st[3u * i + 2u] = c;
-      __syncwarp();
-    }
-    held -= fit;
-    n_tasks += fit;
-  }
 };
-
-// The set that job j reaches from the set `code` of `frame` (or, with CODE_CHART and no frame, from
-// the chart's last set) on the byte class `eq`, for the lanes with `valid`: looked up in the job's
-// table of such transitions, computed by this warp if nobody has yet (one Earley step against the
-// row's chart).  Returns the walk's id of the set, or V_DEAD.  Called by all lanes.
-__device__ uint32_t ctx_transition(Walker& wk, const CtxJob& cj, uint32_t j, bool valid, uint32_t frame, uint32_t code, uint32_t eq,
-                                   uint32_t byte) {
-  const StateDev& S = wk.S;
-  const uint32_t lane = lane_id();
-  const unsigned long long key = ((unsigned long long)((frame + 1u) & 0xFFu) << 24) | (code << 8) | eq;  // 32 bits
-  const unsigned long long gen = S.gen_ctx & 0xFFFFu;
-  unsigned long long* tab = S.cx.ctab + (size_t)j * CT_SLOTS;
-  // ---- one lane per distinct key asks the table
-  const uint32_t peers = __match_any_sync(FULL, valid ? key : ((1ull << 40) | lane));  // (a key has 32 bits: idle lanes match nobody)
-  const bool leader = valid && (uint32_t)(__ffs(peers) - 1) == lane;
-  uint32_t val = V_PEND;
-  int slot = -1;       // >= 0: the slot that holds (or will hold) the value
-  bool mine = false;   // this lane computes the value
-  if (leader) {
-    uint32_t s = (mix32((uint32_t)key) & (CT_SLOTS - 1));
-    for (uint32_t probe = 0; probe < 64; ++probe) {
-      unsigned long long v = ld_acquire64(tab + s);
-      if ((v >> 48) != gen) {  // left by an earlier fill: free
-        const unsigned long long nv = (gen << 48) | (key << 16) | V_PEND;
-        const unsigned long long old = atomicCAS(tab + s, v, nv);
-        if (old == v) {
-          slot = (int)s;
-          mine = true;
-          break;
-        }
-        v = old;
-        if ((v >> 48) != gen) {
-          --probe;  // (taken and released again: look once more)
-          continue;
-        }
-      }
-      if (((v >> 16) & 0xFFFFFFFFull) == key) {
-        slot = (int)s;
-        val = (uint32_t)v & 0xFFFFu;
-        break;
-      }
-      s = (s + 1u) & (CT_SLOTS - 1);
-    }
-    if (slot < 0) mine = true;  // no room in the table: compute it all the same, it just is not remembered
-  }
-  // ---- the warp computes what its lanes have claimed, one transition at a time
-  uint32_t todo = __ballot_sync(FULL, mine);
-  while (todo) {
-    const int src = __ffs(todo) - 1;
-    todo &= todo - 1;
-    const uint32_t scode = __shfl_sync(FULL, code, src), sbyte = __shfl_sync(FULL, byte, src), sframe = __shfl_sync(FULL, frame, src);
-    const uint32_t r = wk.step(cj, j, scode == CODE_CHART ? cj.m - 1u : scode, sframe, sbyte);
-    if (lane == 0) diag(S, 11);
-    if ((int)lane == src) {
-      val = (r == T_DEAD) ? V_DEAD : r;
-      if (slot >= 0) st_release64(tab + slot, (gen << 48) | (key << 16) | val);
-    }
-  }
-  // ---- a value somebody else is computing: wait for it (the other warp is at it, it waits for nothing)
-  if (leader && val == V_PEND) {
-    const uint32_t limit = ctx_poll_limit(S, 22);
-    for (uint32_t spin = 0; spin < limit; ++spin) {
-      const unsigned long long v = ld_acquire64(tab + slot);
-      val = (uint32_t)v & 0xFFFFu;
-      if (val != V_PEND) break;
-      __nanosleep(100);
-    }
-    if (val == V_PEND) {
-      diag(S, DIAG_WAIT_VALUE);
-      atomicExch(&S.counters[CNT_BAR_ERR], 1u);
-      val = V_DEAD;
-    }
-  }
-  return __shfl_sync(FULL, val, __ffs(peers) - 1);
-}
-
-// A chunk of 32 frontier entries of job j, one per lane: nodes reached alive mark their tokens and
-// are kept for expansion if they have children.
-__device__ void walk_chunk(Walker& wk, uint32_t j, uint32_t e0) {
-  const GrammarDev& G = wk.G;
-  const StateDev& S = wk.S;
-  const uint32_t lane = lane_id();
-  const CtxJob cj = S.cx.jobs[j];
-  const bool use_root = cj.pad[0] != 0u;
-  const uint32_t e = e0 + lane;
-  const bool valid = e < cj.fr_n;
-  uint32_t node = 0, code = CODE_CHART, eq = 0;
-  const uint32_t frame = use_root ? 0u : NOF;  // (frame 0 is the job's own root)
-  if (valid) {
-    if (use_root) {
-      const uint2 fe = __ldg(S.rt.frontier + cj.fr_off + e);
-      node = fe.x, code = RBASE + (fe.y & 0xFFFFu), eq = fe.y >> 16;
-    } else {
-      node = cj.fr_off + e;
-      eq = G.eq_of_byte[__ldg(&G.node_byte[node])];
-    }
-  }
-  const uint32_t byte = valid ? __ldg(&G.node_byte[node]) : 0u;
-  const uint32_t val = ctx_transition(wk, cj, j, valid, frame, code, eq, byte);
-  const bool alive = valid && val != V_DEAD;
-  if (alive) wk.mark_tokens(cj, node);
-  const bool kids = alive && __ldg(&G.child_off[node + 1]) > __ldg(&G.child_off[node]);
-  wk.keep(cj, j, kids, node, LBASE + val, NOF);  // (a set of the walk's own knows the frame it lives in)
-  wk.n_frontier += __popc(__ballot_sync(FULL, valid));
-}
 
 // Is the set `id` this walk made itself a known root, with all its origins in the row's chart?  Then
 // what follows it is context-independent again: the job gets a frame for it (the root's region with
@@ -760,7 +536,7 @@ __device__ uint32_t resolve_frame(Walker& wk, const CtxJob& cj, uint32_t j, uint
   uint32_t* rec = A.recs + ((size_t)j * A.cap + id) * A.rec_words;
   const uint32_t nk = __ldcg(rec + AR_NK), n = __ldcg(rec + AR_N);
   const uint32_t* items = A.items + __ldcg(rec + AR_ITEMS);
-  uint32_t result = NOFRAME, why = 15;
+  uint32_t result = NOFRAME;
   constexpr uint32_t KMAX = 256;  // (the scratch has 512 words: the sorted kernel, then its anonymous form)
   if (R.on && nk >= 1 && nk <= KMAX && n <= R.max_items && wk.sw.w.cur_cap >= 2 * KMAX) {
     uint32_t* buf = wk.sw.w.cur;
@@ -773,9 +549,7 @@ __device__ uint32_t resolve_frame(Walker& wk, const CtxJob& cj, uint32_t j, uint
       if ((it >> 16) >= LBASE) ok = false;  // an origin inside the token: not a situation a chart can be in
     }
     ok = __all_sync(FULL, ok);
-    why = 13;
     if (ok) {
-      why = 15;
       sort_items(buf, nk, KMAX);
       __syncwarp();
       uint32_t P = 0, h = 0;
@@ -810,7 +584,6 @@ __device__ uint32_t resolve_frame(Walker& wk, const CtxJob& cj, uint32_t j, uint
           const uint32_t at = atomicAdd(&R.tops[TOP_PENDING], 1u);
           if (at < R.pend_cap) R.pending[at] = rid;
         }
-        why = 14;
         if (rid != ROOT_NONE) {
           const uint32_t* info = R.info + (size_t)rid * RI_WORDS;
           const uint32_t nst = __ldcg(info + RI_NSTATES);
@@ -834,7 +607,6 @@ __device__ uint32_t resolve_frame(Walker& wk, const CtxJob& cj, uint32_t j, uint
               __syncwarp();
               __threadfence();
               result = idx + 1u;
-              why = 0;
               ++wk.n_frames;
             }
           }
@@ -842,275 +614,125 @@ __device__ uint32_t resolve_frame(Walker& wk, const CtxJob& cj, uint32_t j, uint
       }
     }
   }
-  if (lane == 0 && why) diag(S, why);
   uint32_t old = 0;
   if (lane == 0) old = atomicCAS(rec + AR_FRAME, 0u, result);
   old = __shfl_sync(FULL, old, 0);
   return old != 0u ? old : result;  // (another warp may have looked the same set up meanwhile: use its answer)
 }
 
-// ---- What a root's region makes of the subtree of a node (see RootDev::mkey): computed once, by table
-// look-ups alone, by the first warp that needs it.  The warp's large scratch area holds the work:
-constexpr uint32_t MEMO_TOK = 24u * 1024u;   // tokens found                       [0, MEMO_TOK)
-constexpr uint32_t MEMO_FR = 4096u;          // frontier entries (two words each)  [MEMO_TOK, + 2 * MEMO_FR)
-constexpr uint32_t MEMO_STACK = 4096u;       // nodes to visit (two words each)    [.., + 2 * MEMO_STACK)
-static_assert(MEMO_TOK + 2 * MEMO_FR + 2 * MEMO_STACK + STACK_WORDS <= 65536, "the large scratch area is 64 Ki words");
+// ===================================================================================== fill: level sweep with frames
+//
+// The fill proper.  Like the root sweep it goes through the trie one depth at a time, one THREAD per
+// (job, node): node's set = transition(parent's set, byte), with coalesced reads of the trie and
+// writes of the per-node sets, the depths overlapped by tickets as in sweep_kernel.  The difference
+// is where a transition comes from.  A job starts in set 0 of its frame 0 (its root's region); inside
+// a frame a transition is ONE look-up in the root's table, shared by all rows and fills; only where
+// the table says "context-dependent" is an Earley step run against the row's chart (queued, computed
+// by a warp, remembered per job), and the set it yields usually opens the next frame.  Jobs without a
+// root start from the chart's last set and do everything by Earley steps, as does whatever set has
+// no frame.
+//
+// A node's word: SS_DEAD, SS_PENDING (its transition is queued), or (frame + 1) << 16 | code, with
+// frame + 1 = 0 for a set of the walk's own (code = LBASE + id) and for the chart's last set (CODE_CHART).
+constexpr uint32_t SS_DEAD = 0xffffffffu, SS_PENDING = 0xfffffffeu, SS_CLAIMED = 0xfffffffdu;
 
-// Returns entry + 1, or 0 when there is no entry to use (another warp is computing it, or it does not fit).
-__device__ uint32_t memo_get(Walker& wk, uint32_t rid, uint32_t tr_off, uint32_t node) {
-  const GrammarDev& G = wk.G;
-  const StateDev& S = wk.S;
-  const RootDev& R = S.rt;
-  const uint32_t lane = lane_id();
-  const unsigned long long key = ((unsigned long long)(rid + 1u) << 32) | node;
-  uint32_t slot = (mix32(node) ^ mix32(rid * 0x9E3779B9u + 1u)) & R.m_mask;
-  uint32_t state = 0;  // 1: ours to compute (slot), 2: there (val), 3: none
-  uint32_t val = 0;
-  if (lane == 0) {
-    state = 3;
-    for (uint32_t probe = 0; probe < 32; ++probe) {
-      unsigned long long k = ld_acquire64(R.mkey + slot);
-      if (k == 0ull) {
-        k = atomicCAS(R.mkey + slot, 0ull, key);
-        if (k == 0ull) {
-          state = 1;
-          break;
-        }
-      }
-      if (k == key) {
-        val = ld_acquire(R.mval + slot);
-        state = 2;
-        break;
-      }
-      slot = (slot + 1u) & R.m_mask;
-    }
-  }
-  state = __shfl_sync(FULL, state, 0);
-  val = __shfl_sync(FULL, val, 0);
-  slot = __shfl_sync(FULL, slot, 0);
-  if (state == 2) return val;
-  if (state != 1 || S.big_arena_items < 65536u) return 0;
-  // ---- depth first through the subtree, in the region's transition table
-  uint32_t* tok = wk.big;
-  uint32_t* fr = wk.big + MEMO_TOK;
-  uint32_t* stk = fr + 2 * MEMO_FR;
-  uint32_t n_tok = 0, n_fr = 0, n_stk = 1;
-  bool ok = true;
-  if (lane == 0) stk[0] = node, stk[1] = 0u;  // the walk stands in the root set
-  __syncwarp();
-  while (n_stk && ok) {
-    --n_stk;
-    const uint32_t nd = stk[2u * n_stk], k = stk[2u * n_stk + 1u];
-    __syncwarp();
-    const uint16_t* row = R.trans + tr_off + (size_t)k * G.n_eq;
-    const uint32_t c0 = __ldg(&G.child_off[nd]), c1 = __ldg(&G.child_off[nd + 1]);
-    for (uint32_t base = c0; base < c1 && ok; base += 32) {
-      const uint32_t c = base + lane;
-      const bool valid = c < c1;
-      const uint32_t eq = valid ? (uint32_t)G.eq_of_byte[__ldg(&G.node_byte[c])] : 0u;
-      const uint32_t t16 = valid ? (uint32_t)__ldg(row + eq) : (uint32_t)R_DEAD;
-      const bool alive = t16 < R_CTX, ctx = t16 == R_CTX;
-      // the tokens that end at the children reached alive
-      const uint32_t t0 = alive ? __ldg(&G.tok_off[c]) : 0u, cnt = alive ? __ldg(&G.tok_off[c + 1]) - t0 : 0u;
-      uint32_t incl = cnt;
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t t = __shfl_up_sync(FULL, incl, d);
-        if ((int)lane >= d) incl += t;
-      }
-      const uint32_t total = __shfl_sync(FULL, incl, 31);
-      const uint32_t fb = __ballot_sync(FULL, ctx);
-      const bool kids = alive && __ldg(&G.child_off[c + 1]) > __ldg(&G.child_off[c]);
-      const uint32_t kb = __ballot_sync(FULL, kids);
-      if (n_tok + total > MEMO_TOK || n_fr + __popc(fb) > MEMO_FR || n_stk + __popc(kb) > MEMO_STACK) {
-        ok = false;
-        break;
-      }
-      for (uint32_t i = 0; i < cnt; ++i) tok[n_tok + incl - cnt + i] = __ldg(&G.tok_ids[t0 + i]);
-      if (ctx) {
-        const uint32_t at = n_fr + __popc(fb & ((1u << lane) - 1u));
-        fr[2u * at] = c, fr[2u * at + 1u] = k | (eq << 16);
-      }
-      if (kids) {
-        const uint32_t at = n_stk + __popc(kb & ((1u << lane) - 1u));
-        stk[2u * at] = c, stk[2u * at + 1u] = t16;
-      }
-      n_tok += total, n_fr += __popc(fb), n_stk += __popc(kb);
-      __syncwarp();
-    }
-  }
-  // ---- keep it
-  uint32_t ent = 0;
-  if (ok) {
-    const uint32_t words = n_tok + 2u * n_fr;
-    uint32_t e = 0, d = 0;
-    if (lane == 0) {
-      e = atomicAdd(&R.tops[TOP_MENT], 1u);
-      d = atomicAdd(&R.tops[TOP_MDATA], words);
-      if (e >= R.me_cap || d > R.md_cap || words > R.md_cap - d) e = 0xffffffffu;
-    }
-    e = __shfl_sync(FULL, e, 0);
-    d = __shfl_sync(FULL, d, 0);
-    if (e != 0xffffffffu) {
-      for (uint32_t i = lane; i < n_tok; i += 32) R.mdata[d + i] = tok[i];
-      for (uint32_t i = lane; i < 2u * n_fr; i += 32) R.mdata[d + n_tok + i] = fr[i];
-      if (lane == 0) R.ment[e] = make_uint4(d, n_tok, n_fr, 0u);
-      __syncwarp();
-      __threadfence();
-      ent = e + 1u;
-      if (lane == 0) st_release32(R.mval + slot, ent);
-    }
-  }
-  return ent;
-}
+struct FillReq {
+  uint32_t frame1, code;  // the parent set of the transition this thread has just claimed
+};
 
-// Job j stands at `node` in the root set of frame `fi`: mark what the region alone decides below the
-// node and keep the nodes where the chart is needed again.
-__device__ void memo_apply(Walker& wk, const CtxJob& cj, uint32_t j, uint32_t frame, uint32_t ent) {
-  const GrammarDev& G = wk.G;
-  const StateDev& S = wk.S;
-  const RootDev& R = S.rt;
-  const uint32_t lane = lane_id();
-  const uint4 e = __ldcg(R.ment + ent - 1u);
-  const uint32_t* tok = R.mdata + e.x;
-  const uint32_t* fr = tok + e.y;
-  uint32_t* row = S.mask_rows + (size_t)cj.mrow * G.Wm;
-  for (uint32_t i = lane; i < e.y; i += 32) {
-    const uint32_t t = __ldcg(tok + i);
-    atomicOr(&row[t >> 5], 1u << (t & 31u));
-  }
-  for (uint32_t base = 0; base < e.z; base += 32) {
-    const uint32_t i = base + lane;
-    const bool valid = i < e.z;
-    const uint32_t node = valid ? __ldcg(fr + 2u * i) : 0u, ke = valid ? __ldcg(fr + 2u * i + 1u) : 0u;
-    const uint32_t byte = valid ? __ldg(&G.node_byte[node]) : 0u;
-    const uint32_t val = ctx_transition(wk, cj, j, valid, frame, RBASE + (ke & 0xFFFFu), ke >> 16, byte);
-    const bool alive = valid && val != V_DEAD;
-    if (alive) wk.mark_tokens(cj, node);
-    const bool kids = alive && __ldg(&G.child_off[node + 1]) > __ldg(&G.child_off[node]);
-    wk.keep(cj, j, kids, node, LBASE + val, NOF);
-  }
-  wk.n_frontier += e.z;
-}
-
-// The children of `node`, which job j reached in the set `code` (of `frame`, if it is a frame's set).
-__device__ void walk_expand(Walker& wk, uint32_t j, uint32_t node, uint32_t code, uint32_t frame) {
-  const GrammarDev& G = wk.G;
-  const StateDev& S = wk.S;
+// (one thread) The set job j reaches from `state` on `byte`; SS_PENDING if somebody is computing it;
+// SS_CLAIMED if nobody had asked yet and `claim` is set: the caller must queue `rq`.
+__device__ uint32_t fill_next(const GrammarDev& G, const StateDev& S, uint32_t j, uint32_t state, uint32_t byte, bool claim, FillReq& rq) {
   const AutoDev& A = S.au;
-  const uint32_t lane = lane_id();
-  const CtxJob cj = S.cx.jobs[j];
-  ++wk.n_nodes;
-  if (code < RBASE) {  // a set this walk made: it lives in some frame, and may be a root in its own right
-    const uint32_t id = code - LBASE;
-    const uint32_t* rec = A.recs + ((size_t)j * A.cap + id) * A.rec_words;
-    uint32_t fr = 0;  // (one lane looks, all lanes act on what it saw: another warp may be writing the answer just now)
-    if (lane == 0) fr = ld_acquire(rec + AR_FRAME);
-    fr = __shfl_sync(FULL, fr, 0);
-    if (fr == 0u) fr = resolve_frame(wk, cj, j, id);
-    if (fr != NOFRAME) {
-      frame = fr - 1u;
-      code = RBASE;  // set 0 of the frame it opens
-      if (!wk.big_mode) {  // (the look-up below works in the warp's large scratch area: not while sets are built there)
-        const Frame* f = S.cx.frames + (size_t)j * MAXF + frame;
-        const uint32_t ent = memo_get(wk, __ldcg(&f->root), __ldcg(&f->tr_off), node);
-        if (ent) {
-          if (lane == 0) diag(S, 8);
-          memo_apply(wk, cj, j, frame, ent);
-          return;
+  const uint32_t eq = G.eq_of_byte[byte];
+  uint32_t frame1 = state >> 16, code = state & 0xFFFFu;
+  if (frame1 == 0u && code != CODE_CHART) {  // a set of the walk's own
+    uint32_t* rec = A.recs + ((size_t)j * A.cap + (code - LBASE)) * A.rec_words;
+    const uint32_t fr = __ldcg(rec + AR_FRAME);  // (looked up by whoever made the set, before its id went anywhere)
+    if (fr != 0u && fr != NOFRAME) {
+      frame1 = fr, code = RBASE;  // it opens a frame: go on in that frame's table
+    } else {
+      if (!((__ldcg(rec + AR_SCAN + (byte >> 5)) >> (byte & 31u)) & 1u)) return SS_DEAD;
+      uint32_t* slot = rec + AR_TRANS + eq;
+      uint32_t t = ld_acquire(slot);
+      if (t == T_UNKNOWN && claim) {
+        t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
+        if (t == T_UNKNOWN) {
+          rq.frame1 = 0u, rq.code = code;
+          return SS_CLAIMED;
         }
       }
-    } else {
-      const uint32_t salt = __ldcg(rec + AR_SALT);
-      frame = salt ? salt - 1u : NOF;
+      if (t == T_PENDING || t == T_UNKNOWN) return SS_PENDING;
+      return t == T_DEAD ? SS_DEAD : LBASE + t;
     }
   }
-  const uint32_t c0 = __ldg(&G.child_off[node]), c1 = __ldg(&G.child_off[node + 1]);
-  if (code >= RBASE) {
-    // ---- a frame's set: one table look-up per child; only context-dependent transitions cost a step
-    if (lane == 0) diag(S, 9);
-    const Frame* f = S.cx.frames + (size_t)j * MAXF + frame;
-    const uint16_t* row = S.rt.trans + __ldcg(&f->tr_off) + (size_t)(code - RBASE) * G.n_eq;
-    for (uint32_t base = c0; base < c1; base += 32) {
-      const uint32_t c = base + lane;
-      const bool valid = c < c1;
-      const uint32_t byte = valid ? __ldg(&G.node_byte[c]) : 0u;
-      const uint32_t eq = G.eq_of_byte[byte];
-      const uint32_t t16 = valid ? (uint32_t)__ldg(row + eq) : (uint32_t)R_DEAD;
-      const bool is_ctx = valid && t16 == R_CTX;
-      uint32_t ccode = RBASE + t16;
-      bool alive = valid && t16 < R_CTX;
-      if (__any_sync(FULL, is_ctx)) {
-        const uint32_t val = ctx_transition(wk, cj, j, is_ctx, frame, code, eq, byte);
-        if (is_ctx && val != V_DEAD) alive = true, ccode = LBASE + val;
+  if (frame1 != 0u) {  // a frame's set: the root's table
+    const Frame* f = S.cx.frames + (size_t)j * MAXF + (frame1 - 1u);
+    const uint32_t t16 = __ldg(S.rt.trans + __ldcg(&f->tr_off) + (size_t)(code - RBASE) * G.n_eq + eq);
+    if (t16 == R_DEAD) return SS_DEAD;
+    if (t16 < R_CTX) return (frame1 << 16) | (RBASE + t16);
+  }
+  // ---- context-dependent (or out of the chart's last set): the job's own table
+  const unsigned long long gen = S.gen_ctx & 0xFFFFu;
+  const unsigned long long key = ((unsigned long long)(frame1 & 0xFFu) << 24) | (code << 8) | eq;
+  unsigned long long* tab = S.cx.ctab + (size_t)j * CT_SLOTS;
+  uint32_t s = mix32((uint32_t)key) & (CT_SLOTS - 1);
+  for (uint32_t probe = 0; probe < 128; ++probe) {
+    unsigned long long v = ld_acquire64(tab + s);
+    if ((v >> 48) != gen) {  // left by an earlier fill: free
+      if (!claim) return SS_PENDING;
+      const unsigned long long old = atomicCAS(tab + s, v, (gen << 48) | (key << 16) | V_PEND);
+      if (old == v) {
+        rq.frame1 = frame1, rq.code = code;
+        return SS_CLAIMED;
       }
-      if (alive) wk.mark_tokens(cj, c);
-      const bool kids = alive && __ldg(&G.child_off[c + 1]) > __ldg(&G.child_off[c]);
-      wk.keep(cj, j, kids, c, ccode, frame);
+      v = old;
+      if ((v >> 48) != gen) {
+        --probe;
+        continue;
+      }
     }
+    if (((v >> 16) & 0xFFFFFFFFull) == key) {
+      const uint32_t val = (uint32_t)v & 0xFFFFu;
+      return val == V_PEND ? SS_PENDING : val == V_DEAD ? SS_DEAD : LBASE + val;
+    }
+    s = (s + 1u) & (CT_SLOTS - 1);
+  }
+  // no room to remember the transition: give the row up rather than guess
+  const uint32_t row = S.cx.jobs[j].row_acc & 0x7FFFFFFFu;
+  if (!(atomicOr(&S.row_flags[row], ROW_BROKEN) & ROW_BROKEN)) stat_add(S, CNT_STAT_CAPERR, 1u);
+  atomicExch(&S.counters[CNT_ERR], 1u);
+  diag(S, DIAG_SET_TABLE);
+  return SS_DEAD;
+}
+
+// (one lane) The transition (frame1, code, eq) of job j, which some thread claimed, is `val` (a set id or V_DEAD).
+__device__ void fill_publish(const StateDev& S, uint32_t j, uint32_t frame1, uint32_t code, uint32_t eq, uint32_t val) {
+  const AutoDev& A = S.au;
+  if (frame1 == 0u && code != CODE_CHART) {
+    uint32_t* slot = A.recs + ((size_t)j * A.cap + (code - LBASE)) * A.rec_words + AR_TRANS + eq;
+    st_release32(slot, val == V_DEAD ? T_DEAD : val);
     return;
   }
-  // ---- a set of the walk's own: its transitions are Earley steps, remembered in its record
-  if (lane == 0) diag(S, 10);
-  const uint32_t state = code - LBASE;
-  uint32_t* rec = A.recs + ((size_t)j * A.cap + state) * A.rec_words;
-  for (uint32_t base = c0; base < c1; base += 32) {
-    const uint32_t c = base + lane;
-    const bool valid = c < c1;
-    const uint32_t byte = valid ? __ldg(&G.node_byte[c]) : 0u;
-    uint32_t t = T_DEAD;
-    uint32_t* slot = nullptr;
-    bool mine = false;
-    // one 256-bit test rejects most bytes without touching the transition table
-    if (valid && ((__ldcg(rec + AR_SCAN + (byte >> 5)) >> (byte & 31u)) & 1u)) {
-      slot = rec + AR_TRANS + G.eq_of_byte[byte];
-      t = ld_acquire(slot);
-      if (t == T_UNKNOWN) {
-        t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
-        if (t == T_UNKNOWN) mine = true, t = T_PENDING;
-      }
+  const unsigned long long gen = S.gen_ctx & 0xFFFFu;
+  const unsigned long long key = ((unsigned long long)(frame1 & 0xFFu) << 24) | (code << 8) | eq;
+  unsigned long long* tab = S.cx.ctab + (size_t)j * CT_SLOTS;
+  uint32_t s = mix32((uint32_t)key) & (CT_SLOTS - 1);
+  for (uint32_t probe = 0; probe < 128; ++probe) {
+    const unsigned long long v = ld_acquire64(tab + s);
+    if ((v >> 48) == gen && ((v >> 16) & 0xFFFFFFFFull) == key) {
+      st_release64(tab + s, (gen << 48) | (key << 16) | val);
+      return;
     }
-    uint32_t todo = __ballot_sync(FULL, mine);
-    while (todo) {
-      const int src = __ffs(todo) - 1;
-      todo &= todo - 1;
-      const uint32_t sbyte = __shfl_sync(FULL, byte, src);
-      const uint32_t r = wk.step(cj, j, code, frame, sbyte);
-      if (lane == 0) diag(S, 12);
-      if ((int)lane == src) {
-        t = r;
-        st_release32(slot, r);
-      }
-    }
-    if (t == T_PENDING) {  // another lane or warp claimed it before this lane asked
-      const uint32_t limit = ctx_poll_limit(S, 22);
-      for (uint32_t spin = 0; spin < limit; ++spin) {
-        t = ld_acquire(slot);
-        if (t != T_PENDING) break;
-        __nanosleep(100);
-      }
-      if (t == T_PENDING) {
-        diag(S, DIAG_WAIT_VALUE);
-        atomicExch(&S.counters[CNT_BAR_ERR], 1u);
-        t = T_DEAD;
-      }
-    }
-    const bool alive = valid && t != T_DEAD;
-    if (alive) wk.mark_tokens(cj, c);
-    const bool kids = alive && __ldg(&G.child_off[c + 1]) > __ldg(&G.child_off[c]);
-    wk.keep(cj, j, kids, c, LBASE + t, NOF);
+    s = (s + 1u) & (CT_SLOTS - 1);
   }
 }
 
-// The walk of all jobs of a fill.  Work units: first the chunks of frontier entries, handed out by
-// a counter; then nodes drawn from a queue.  A warp expands the nodes of its unit depth first from a
-// stack of its own and hands nodes to the queue only when it holds many, so that most nodes cost no
-// atomic operation; a warp that finds the queue empty waits for either a new entry or the count of
-// unfinished units to reach zero.  No unit ever waits for another unit, only for a single Earley step
-// that another warp is computing, so every wait ends; all the same each is a poll with a limit that
-// flags an error instead of hanging.
-__global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) ctx_kernel(GrammarDev Gg, StateDev S) {
-  const uint32_t n_jobs = S.counters[CNT_N_JOBS];
-  if (n_jobs == 0) return;
+constexpr uint32_t FILL_PER_LANE = 4;  // trie nodes per lane and pass iteration (independent loads in flight)
+
+__global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) fill_kernel(GrammarDev Gg, StateDev S) {
+  const uint32_t n_jobs = S.counters[CNT_N_FJOBS];  // (the jobs that need the sweep: S.cx.fjobs)
+  if (n_jobs == 0) return;  // every CTA sees the same count: nobody is left at a barrier
   extern __shared__ __align__(16) uint32_t smem[];
   const uint32_t warp = threadIdx.x >> 5, lane = lane_id();
   const AutoDev& A = S.au;
@@ -1133,86 +755,175 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) ctx_kernel(GrammarDev Gg,
   if (lane < W_CTRS) sw.w.ctr[lane] = 0u;
   __syncthreads();
   Walker wk{G, S, sw, S.big_scratch + ((size_t)blockIdx.x * SWEEP_WARPS + warp) * ((size_t)S.big_arena_items + S.big_hset_slots)};
-  uint32_t* q = S.cx.qctr;
-  const uint32_t n_chunks = q[Q_CHUNKS];
-  const uint32_t tag = (S.gen_ctx << 16) | 1u;
-  const uint32_t limit = ctx_poll_limit(S, 22);
-  bool chunks_left = true, abandoned = false;
+  const uint32_t gw = blockIdx.x * SWEEP_WARPS + warp, GW = gridDim.x * SWEEP_WARPS;
+  uint32_t pass_phase = 0;
+  const uint32_t stride = A.st_stride;
+  const unsigned long long gen = S.gen_ctx & 0xFFFFu;
 
-  for (;;) {
-    bool have = false;
-    if (chunks_left) {  // ---- a chunk of some job's frontier
-      uint32_t c = 0;
-      if (lane == 0) c = atomicAdd(&q[Q_CHUNK], 1u);
-      c = __shfl_sync(FULL, c, 0);
-      if (c < n_chunks) {
-        uint32_t lo = 0, hi = n_jobs;  // the job whose chunks include c: chunk_off[lo] <= c < chunk_off[lo + 1]
-        while (hi - lo > 1) {
-          const uint32_t mid = (lo + hi) >> 1;
-          if (__ldg(&S.cx.chunk_off[mid]) <= c) lo = mid;
-          else hi = mid;
+  uint32_t last_level = 0;
+  uint32_t expect_req = n_jobs * Gg.n_eq;
+  for (uint32_t L = 1; L <= G.depth; ++L) {
+    const uint32_t lo = __ldg(&G.lvl_off[L]), hi = __ldg(&G.lvl_off[L + 1]);
+    constexpr uint32_t CH = 32 * FILL_PER_LANE;
+    const uint32_t nL = hi - lo, cpj = (nL + CH - 1) / CH;
+    const uint32_t chunks = n_jobs * cpj;
+    bool any_alive = false;
+    const uint32_t req_half = S.cx.req2_cap / 2u, req_base = (L & 1u) * req_half;
+    for (uint32_t c = gw; c < chunks; c += GW) {
+      const uint32_t ji = c / cpj, j = __ldg(&S.cx.fjobs[ji]);
+      const uint32_t first = lo + (c % cpj) * CH + lane;
+      uint32_t* st = S.cx.st32 + (size_t)ji * stride;
+      const uint32_t start = __ldcg(&S.cx.jobs[j].pad[0]) ? ((1u << 16) | RBASE) : CODE_CHART;  // set 0 of frame 0, or the chart's last set
+      uint32_t node[FILL_PER_LANE], byte[FILL_PER_LANE], par[FILL_PER_LANE], ps[FILL_PER_LANE];
+#pragma unroll
+      for (uint32_t u = 0; u < FILL_PER_LANE; ++u) {
+        node[u] = first + 32u * u;
+        const bool v = node[u] < hi;
+        byte[u] = v ? __ldg(&G.node_byte[node[u]]) : 0u;
+        par[u] = (v && L > 1) ? __ldg(&G.parent[node[u]]) : 0u;
+      }
+#pragma unroll
+      for (uint32_t u = 0; u < FILL_PER_LANE; ++u) ps[u] = (node[u] < hi) ? ((L == 1) ? start : __ldcg(st + par[u])) : SS_DEAD;
+#pragma unroll
+      for (uint32_t u = 0; u < FILL_PER_LANE; ++u) {
+        if (node[u] >= hi) continue;
+        uint32_t p_state = ps[u];
+        FillReq rq;
+        if (p_state == SS_PENDING) {  // settle the parent first: its transition was queued at the depth before
+          const uint32_t gp_state = (L == 2) ? start : __ldcg(st + __ldg(&G.parent[par[u]]));
+          const uint32_t pbyte = __ldg(&G.node_byte[par[u]]);
+          uint32_t t2 = (gp_state == SS_DEAD || gp_state == SS_PENDING) ? SS_DEAD : fill_next(G, S, j, gp_state, pbyte, false, rq);
+          for (uint32_t spin = 0; t2 == SS_PENDING && spin < poll_limit(S, 21); ++spin) {
+            __nanosleep(40);
+            t2 = fill_next(G, S, j, gp_state, pbyte, false, rq);
+          }
+          if (t2 == SS_PENDING) {  // the wait ran out: give the row up rather than guess
+            diag(S, DIAG_WAIT_VALUE);
+            const uint32_t row = __ldcg(&S.cx.jobs[j].row_acc) & 0x7FFFFFFFu;
+            if (!(atomicOr(&S.row_flags[row], ROW_BROKEN) & ROW_BROKEN)) stat_add(S, CNT_STAT_CAPERR, 1u);
+            atomicExch(&S.counters[CNT_ERR], 1u);
+            t2 = SS_DEAD;
+          }
+          p_state = t2;
+          st[par[u]] = p_state;
         }
-        walk_chunk(wk, lo, (c - __ldg(&S.cx.chunk_off[lo])) * 32u);
-        have = true;
-      } else {
-        chunks_left = false;
-      }
-    }
-    if (!have) {  // ---- a node from the queue
-      uint32_t ticket = 0;
-      if (lane == 0) ticket = atomicAdd(&q[Q_HEAD], 1u);
-      ticket = __shfl_sync(FULL, ticket, 0);
-      uint32_t got = 0;  // 1: the entry is there, 2: all work is done, 3: gave up
-      if (lane == 0) {
-        for (uint32_t polls = 0;; ++polls) {
-          if (ticket < S.cx.q_cap && ld_acquire(&S.cx.queue[ticket].w) == tag) {
-            got = 1;
-            break;
+        uint32_t t = SS_DEAD;
+        if (p_state != SS_DEAD) {
+          t = fill_next(G, S, j, p_state, byte[u], true, rq);
+          if (t == SS_CLAIMED) {  // ours to queue
+            const uint32_t at = atomicAdd(&S.counters[CNT_LEVEL_REQ + L], 1u);
+            if (at < req_half) {
+              ulonglong2* e = S.cx.req2 + req_base + at;
+              e->y = ((unsigned long long)j << 32) | ((unsigned long long)rq.frame1 << 24) | (rq.code << 8) | byte[u];
+              __threadfence();
+              st_release64(&e->x, (gen << 48) | ((unsigned long long)L << 40) | 1ull);
+              t = SS_PENDING;
+            } else {  // the depth's queue is full: nobody will compute it: give the row up, and let nobody wait
+              diag(S, DIAG_QUEUE_FULL);
+              const uint32_t row = __ldcg(&S.cx.jobs[j].row_acc) & 0x7FFFFFFFu;
+              if (!(atomicOr(&S.row_flags[row], ROW_BROKEN) & ROW_BROKEN)) stat_add(S, CNT_STAT_CAPERR, 1u);
+              atomicExch(&S.counters[CNT_ERR], 1u);
+              fill_publish(S, j, rq.frame1, rq.code, G.eq_of_byte[byte[u]], V_DEAD);
+              t = SS_DEAD;
+            }
           }
-          if (ld_acquire(&q[Q_OUT]) == 0u) {
-            got = 2;
-            break;
-          }
-          if (polls > limit || ((polls & 63u) == 63u && ld_acquire(&S.counters[CNT_BAR_ERR]))) {
-            if (polls > limit) diag(S, DIAG_WAIT_QUEUE);
-            got = 3;
-            break;
-          }
-          __nanosleep(polls < 8u ? 100 : 500);  // many warps read the same counters: back off
         }
+        st[node[u]] = t;
+        any_alive |= (t != SS_DEAD);
       }
-      got = __shfl_sync(FULL, got, 0);
-      if (got != 1) {
-        abandoned = got == 3;
-        break;
-      }
-      const uint4 e = __ldcg(S.cx.queue + ticket);
-      if (lane == 0) {
-        uint32_t* st = wk.stack();
-        st[0] = e.x;
-        st[1] = (e.y & 0xFFFFu) | (e.z << 16);
-        st[2] = (e.y >> 16) == 0xFFFFu ? NOF : (e.y >> 16);
-      }
-      wk.held = 1;
-      __syncwarp();
-    }
-    // ---- depth first through what this warp holds
-    while (wk.held) {
-      const uint32_t k = --wk.held;
-      __syncwarp();
-      const uint32_t* st = wk.stack();
-      const uint32_t node = st[3u * k], cj_ = st[3u * k + 1u], fr_ = st[3u * k + 2u];
-      __syncwarp();
-      walk_expand(wk, cj_ >> 16, node, cj_ & 0xFFFFu, fr_);
-      wk.share();
     }
     __syncwarp();
-    if (lane == 0) {
-      __threadfence();
-      atomicSub(&q[Q_OUT], 1u);
+    if (__any_sync(FULL, any_alive) && lane == 0) atomicOr(&S.counters[CNT_LEVEL_ALIVE + L], 1u);
+    // ---- this CTA's part of the pass is done: its warps serve the queued transitions by ticket while
+    // the other CTAs finish (see sweep_kernel)
+    if (!pass_arrive(S, pass_phase)) return;
+    const uint32_t all_passed = pass_phase * gridDim.x;
+    const uint32_t takers = (expect_req > 4u * gridDim.x) ? (uint32_t)SWEEP_WARPS : 8u;
+    bool have_ticket = false, gave_up = false;
+    uint32_t ticket = 0;
+    for (uint32_t polls = 0; warp < takers;) {
+      if (!have_ticket) {
+        if (lane == 0) ticket = atomicAdd(&S.counters[CNT_LEVEL_TAKEN + L], 1u);
+        ticket = __shfl_sync(FULL, ticket, 0);
+        have_ticket = true;
+      }
+      uint32_t passed = 0, queued = 0;
+      if (lane == 0) {  // in this order: once all have passed, the number queued is final
+        passed = ld_acquire(&S.counters[CNT_PASS_DONE]) >= all_passed ? 1u : 0u;
+        queued = min(ld_acquire(&S.counters[CNT_LEVEL_REQ + L]), req_half);
+      }
+      passed = __shfl_sync(FULL, passed, 0);
+      queued = __shfl_sync(FULL, queued, 0);
+      if (ticket >= queued) {
+        if (passed) break;
+        if (++polls > poll_limit(S, 21)) {
+          gave_up = true;
+          if (lane == 0) diag(S, DIAG_WAIT_QUEUE);
+        }
+        if ((polls & 63u) == 0u && lane == 0 && ld_acquire(&S.counters[CNT_BAR_ERR])) gave_up = true;
+        gave_up = __any_sync(FULL, gave_up);
+        if (gave_up) break;
+        __nanosleep(polls < 16u ? 40 : 200);
+        continue;
+      }
+      polls = 0;
+      unsigned long long rq0 = 0, rq1 = 0;
+      if (lane == 0) {  // the entry is written right after its number was drawn: wait for it to land
+        const unsigned long long want = (gen << 48) | ((unsigned long long)L << 40) | 1ull;
+        for (uint32_t spin = 0; spin < poll_limit(S, 22); ++spin) {
+          rq0 = ld_acquire64(&S.cx.req2[req_base + ticket].x);
+          if (rq0 == want) break;
+          rq0 = 0;
+        }
+        if (rq0) rq1 = __ldcg(&S.cx.req2[req_base + ticket].y);
+      }
+      rq0 = __shfl_sync(FULL, rq0, 0);
+      rq1 = __shfl_sync(FULL, rq1, 0);
+      have_ticket = false;
+      if (rq0 == 0) {
+        if (lane == 0) diag(S, DIAG_WAIT_QUEUE);
+        gave_up = true;
+        break;
+      }
+      const uint32_t j = (uint32_t)(rq1 >> 32), frame1 = (uint32_t)(rq1 >> 24) & 0xFFu, code = (uint32_t)(rq1 >> 8) & 0xFFFFu, pb = (uint32_t)rq1 & 0xFFu;
+      const CtxJob cj = S.cx.jobs[j];
+      uint32_t in_frame = frame1 ? frame1 - 1u : NOF;  // the frame whose sets the parent's items may name
+      if (frame1 == 0u && code != CODE_CHART) {      // a set of the walk's own knows the frame it lives in
+        const uint32_t salt = __ldcg(A.recs + ((size_t)j * A.cap + (code - LBASE)) * A.rec_words + AR_SALT);
+        in_frame = salt ? salt - 1u : NOF;
+      }
+      const uint32_t r = wk.step(cj, j, code == CODE_CHART ? cj.m - 1u : code, in_frame, pb);
+      uint32_t val = V_DEAD;
+      if (r != T_DEAD) {
+        val = r;
+        // is the new set a root in its own right?  Looked up before anybody can see the set
+        uint32_t fr = 0;
+        if (lane == 0) fr = ld_acquire(A.recs + ((size_t)j * A.cap + r) * A.rec_words + AR_FRAME);
+        fr = __shfl_sync(FULL, fr, 0);
+        if (fr == 0u) resolve_frame(wk, cj, j, r);
+      }
+      if (lane == 0) fill_publish(S, j, frame1, code, G.eq_of_byte[pb], val);
     }
+    if (gave_up && lane == 0) atomicExch(&S.counters[CNT_BAR_ERR], 1u);
+    __shared__ uint32_t lvl_s[3];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      lvl_s[0] = ld_acquire(&S.counters[CNT_LEVEL_ALIVE + L]);
+      lvl_s[1] = ld_acquire(&S.counters[CNT_BAR_ERR]);
+      lvl_s[2] = ld_acquire(&S.counters[CNT_LEVEL_REQ + L]);
+    }
+    __syncthreads();
+    const bool alive = lvl_s[0] != 0u;
+    if (lvl_s[1]) return;
+    expect_req = lvl_s[2];
+    last_level = L;
+    if (!alive) break;  // nothing survives this depth in any job
   }
-  if (abandoned && lane == 0) atomicExch(&S.counters[CNT_BAR_ERR], 1u);
+  {
+    uint32_t abandoned = 0;
+    if (lane == 0) abandoned = ld_acquire(&S.counters[CNT_BAR_ERR]);
+    if (__shfl_sync(FULL, abandoned, 0) != 0u) return;  // the masks are zeroed when they are published
+  }
   if (wk.big_mode) hset_clear_all(sw.w.hset, sw.w.hset_mask);
   if (lane == 0) {
     if (sw.n_computed | sw.n_created) {
@@ -1220,17 +931,73 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) ctx_kernel(GrammarDev Gg,
       stat_add(S, CNT_STAT_CTX_STATES, sw.n_created);
       stat_add64(S, CNT_STAT_STEP_CYCLES, sw.cycles);
     }
-    if (wk.n_frontier) stat_add(S, CNT_STAT_FRONTIER, wk.n_frontier);
-    if (wk.n_nodes) stat_add(S, CNT_STAT_TASKS, wk.n_nodes);
-    if (wk.n_tasks) stat_add(S, CNT_STAT_SHARED_NODES, wk.n_tasks);
     if (wk.n_frames) stat_add(S, CNT_STAT_FRAMES, wk.n_frames);
+  }
+  // ---- mask words: 32 tokens per warp pass, one ballot per word (token t is valid iff the node where its
+  // bytes end was reached alive; EOS iff the chart is accepting)
+  const uint32_t Wm = G.Wm;
+  constexpr uint32_t MW = 6;
+  const uint32_t visited_end = __ldg(&G.lvl_off[last_level + 1]);
+  for (uint32_t c0 = gw; c0 < n_jobs * Wm; c0 += MW * GW) {
+    uint32_t node[MW], s_[MW], dst[MW];
+    bool valid[MW], eos_ok[MW];
+#pragma unroll
+    for (uint32_t u = 0; u < MW; ++u) {
+      const uint32_t c = c0 + u * GW;
+      valid[u] = c < n_jobs * Wm;
+      const uint32_t tok = (c % Wm) * 32 + lane;
+      node[u] = (valid[u] && tok < G.V) ? __ldg(&G.tok_node[tok]) : 0xFFFFFFFEu;
+      dst[u] = (valid[u] && lane == 0) ? (uint32_t)__ldcg(&S.cx.jobs[__ldg(&S.cx.fjobs[c / Wm])].mrow) : 0u;
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < MW; ++u) {
+      const uint32_t c = c0 + u * GW;
+      s_[u] = SS_DEAD;
+      eos_ok[u] = false;
+      if (node[u] == 0xFFFFFFFFu) {  // a token without bytes: only EOS can be valid
+        const uint32_t tok = (c % Wm) * 32 + lane;
+        eos_ok[u] = ((int32_t)tok == G.eos) && (__ldcg(&S.cx.jobs[__ldg(&S.cx.fjobs[c / Wm])].row_acc) >> 31) != 0u;
+      } else if (node[u] < visited_end) {
+        s_[u] = __ldcg(S.cx.st32 + (size_t)(c / Wm) * stride + node[u]);
+      }
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < MW; ++u) {
+      if (!valid[u]) continue;  // (uniform)
+      const uint32_t c = c0 + u * GW;
+      const uint32_t ji = c / Wm, wd = c % Wm;
+      uint32_t s = s_[u];
+      if (s == SS_PENDING) {  // a leaf that waited for a transition: its parent is final by now
+        const uint32_t j = __ldg(&S.cx.fjobs[ji]);
+        const uint32_t* st = S.cx.st32 + (size_t)ji * stride;
+        const uint32_t start = __ldcg(&S.cx.jobs[j].pad[0]) ? ((1u << 16) | RBASE) : CODE_CHART;
+        const uint32_t p = __ldg(&G.parent[node[u]]);
+        const uint32_t p_state = (p == 0) ? start : __ldcg(st + p);
+        const uint32_t nbyte = __ldg(&G.node_byte[node[u]]);
+        FillReq rq;
+        uint32_t t2 = (p_state == SS_DEAD || p_state == SS_PENDING) ? SS_DEAD : fill_next(G, S, j, p_state, nbyte, false, rq);
+        for (uint32_t spin = 0; t2 == SS_PENDING && spin < poll_limit(S, 21); ++spin) {
+          __nanosleep(40);
+          t2 = fill_next(G, S, j, p_state, nbyte, false, rq);
+        }
+        if (t2 == SS_PENDING || p_state == SS_PENDING) {
+          diag(S, DIAG_WAIT_VALUE);
+          const uint32_t row = __ldcg(&S.cx.jobs[j].row_acc) & 0x7FFFFFFFu;
+          if (!(atomicOr(&S.row_flags[row], ROW_BROKEN) & ROW_BROKEN)) stat_add(S, CNT_STAT_CAPERR, 1u);
+          t2 = SS_DEAD;
+        }
+        s = t2;
+      }
+      const uint32_t word = __ballot_sync(FULL, s != SS_DEAD || eos_ok[u]);
+      if (lane == 0) S.mask_rows[(size_t)dst[u] * Wm + wd] = word;
+    }
   }
 }
 
 // ===================================================================================== launchers
 
 cudaError_t configure_walk_kernels() {
-  return cudaFuncSetAttribute((const void*)ctx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+  return cudaFuncSetAttribute((const void*)fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
 }
 
 void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_sweep,
@@ -1254,8 +1021,13 @@ void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStr
     launch_sweep(G, R, sweep_grid, st);
     collect_kernel<<<S.B, COLLECT_THREADS, 0, st>>>(G, S);
   }
-  ctx_init_kernel<<<std::min<uint32_t>(S.B, 148u), 1024, 0, st>>>(G, S);
-  ctx_kernel<<<(unsigned)sweep_grid, SWEEP_WARPS * 32, S.au.smem_bytes, st>>>(G, S);
+  job_setup_kernel<<<std::min<uint32_t>(S.B, 296u), 256, 0, st>>>(G, S);
+  {  // (launched cooperatively: its thread blocks wait for one another between the trie's depths)
+    GrammarDev g = G;
+    StateDev s = S;
+    void* args[] = {&g, &s};
+    cudaLaunchCooperativeKernel((const void*)fill_kernel, dim3((unsigned)sweep_grid), dim3(SWEEP_WARPS * 32), args, S.au.smem_bytes, st);
+  }
   if (after_sweep) cudaEventRecord(after_sweep, st);
   launch_publish(S, st);
 }

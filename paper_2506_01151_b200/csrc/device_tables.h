@@ -50,6 +50,7 @@ enum : uint32_t {
   CNT_N_STATES = 0,
   CNT_N_MASK_ROWS = 1,
   CNT_N_JOBS = 2,
+  CNT_N_FJOBS = 3,      // jobs that go through the level sweep of the fill
   CNT_ERR = 4,          // sticky: some device routine hit a capacity limit
   CNT_AUTO_ITEMS = 5,   // top of the automaton's item pool (words), reset by every fill
   CNT_POOL_LO = 6,      // 64-bit pool top (words) lives in slots 6,7 (8-byte aligned)
@@ -79,12 +80,12 @@ enum : uint32_t {
   CNT_STAT_ROOT_SWEEPS = 150,  // 64-bit: roots whose context-independent part was swept
   CNT_STAT_JOBS_ROOT = 152,    // 64-bit: computed rows that started from a swept root
   CNT_STAT_JOBS_PLAIN = 154,   // 64-bit: computed rows that walked the whole trie themselves
-  CNT_STAT_FRONTIER = 156,     // 64-bit: frontier entries looked at
-  CNT_STAT_TASKS = 158,        // 64-bit: node expansions queued
+  CNT_STAT_JOBS_MASK = 156,    // 64-bit: computed rows answered by their root's mask row alone
+  CNT_STAT_SPARE = 158,
   CNT_STAT_ABORTS = 160,       // 64-bit: fills abandoned because a bounded wait ran out
   CNT_STAT_STEP_CYCLES = 162,  // 64-bit: SM cycles spent inside Earley steps of the fill (summed over warps)
   CNT_STAT_ADV_WORDS = 164,    // 64-bit: chart words read and written by advance
-  CNT_STAT_SHARED_NODES = 182, // 64-bit: nodes handed from one warp to the others through the queue
+  CNT_STAT_SPARE2 = 182,
   CNT_STAT_FRAMES = 184,       // 64-bit: frames made (sets of a walk recognised as roots)
   CNT_DIAG = 166,              // [16] where capacity errors and expired waits came from (see DIAG_*)
   CNT_TOTAL = 186
@@ -141,11 +142,11 @@ constexpr uint32_t AR_ITEMS = 0, AR_N = 1, AR_HASH = 2, AR_NK = 3, AR_SCAN = 4, 
 // of its scanned / completed items become placeholders 0..k-1 (ascending), the set's own index
 // becomes k.  The trie sweep over the root's one-set chart, in which a completion that would have
 // to read a placeholder set answers T_CTX instead, yields
-//   - the tokens valid whatever the rest of the chart holds (one mask row per root),
-//   - the frontier: every trie node whose transition is the first T_CTX on its path, with the
-//     Earley set of its parent,
-//   - the Earley sets met on the way ("region": item lists only), which a sequence's own walk reads
-//     with the placeholders bound to its chart's set indices.
+//   - the tokens valid whatever the rest of the chart holds (one mask row per root) and the number of
+//     trie nodes at which the chart would have been needed (none: the row is the whole answer),
+//   - the Earley sets met on the way (the root's "region": their items, which an Earley step of a
+//     sequence reads with the placeholders bound to its chart's set indices) and the transitions
+//     between them, one 16-bit entry per (set, byte class).
 // Origin codes inside a sequence's walk: [0, LBASE) a set of its chart, [LBASE, RBASE) a set the
 // walk made, [RBASE, ORIGIN_SELF) set (code - RBASE) of the root's region (0 = the root set).
 constexpr uint32_t LBASE = 0x800u, RBASE = 0x8000u;
@@ -169,8 +170,6 @@ struct RootDev {
   uint32_t* charts;      // pool of one-set charts, the key of a root (the scanned / completed items come first)
   uint32_t charts_cap;
   uint32_t* ci_rows;     // [max_roots][Wm]
-  uint2* frontier;       // pool: x = node, y = parent's region set | byte class << 16
-  uint32_t fr_cap;
   uint2* states;         // pool: per region set x = first item (in `items`), y = item count
   uint32_t st_cap;
   uint32_t* items;       // pool
@@ -178,17 +177,6 @@ struct RootDev {
   uint16_t* trans;       // pool: per region set one entry per byte class: the set reached, R_DEAD or R_CTX
   uint32_t tr_cap;
   uint32_t* tops;        // [TOP_N] tops of the pools
-  // What a root's region makes of the subtree of a trie node, when the walk of some row stands at that
-  // node in the root set: the tokens below that are valid whatever the chart holds, and the nodes where
-  // the chart is needed again (node, region set | byte class << 16).  Computed once per (root, node)
-  // by whoever needs it first, then shared by all rows and fills.
-  unsigned long long* mkey;  // [m_mask + 1] (root + 1) << 32 | node, 0 = empty
-  uint32_t* mval;            // [m_mask + 1] 0 while it is being computed, then entry + 1
-  uint32_t m_mask;
-  uint4* ment;               // pool: x = first word in mdata, y = tokens, z = frontier entries (two words each, after the tokens)
-  uint32_t me_cap;
-  uint32_t* mdata;           // pool
-  uint32_t md_cap;
   // roots made by a walk (a set it met had no entry yet): swept by the next fill
   uint32_t* pending;         // [pend_cap] root ids
   uint32_t pend_cap;
@@ -207,8 +195,7 @@ struct CtxJob {
   uint32_t row_acc;      // row | accepting << 31
   uint32_t root;         // root id or ROOT_NONE (the walk starts at the trie's first level from the chart's last set)
   uint32_t P;            // placeholders of the root
-  uint32_t fr_off, fr_n; // frontier entries (or first node / node count of depth 1 when root is ROOT_NONE)
-  uint32_t st_off;       // the region's sets in RootDev::states
+  uint32_t spare[3];
   int32_t mrow;          // mask row to write
   uint32_t pad[2];
 };
@@ -228,21 +215,19 @@ constexpr uint32_t NOFRAME = 0xffffffffu;
 constexpr uint32_t AR_FRAME = 12;     // word of a walk's set record: 0 not looked up yet, NOFRAME, or frame + 1 (the frame it opens)
 constexpr uint32_t AR_SALT = 13;      // word of a set record: 0, or frame + 1 (the frame the set lives in)
 
-constexpr uint32_t CT_SLOTS = 1024;  // per job: remembered transitions out of region sets (power of two)
-enum : uint32_t { Q_TAIL = 0, Q_HEAD = 32, Q_OUT = 64, Q_CHUNK = 96, Q_CHUNKS = 97, Q_WORDS = 128 };
+constexpr uint32_t CT_SLOTS = 4096;  // per job: remembered transitions out of region sets (power of two)
 
 struct CtxDev {
-  uint32_t* job_root;          // [B] root of job j (ROOT_NONE: none)
   uint16_t* bind;              // [B][max_ph] the chart set each placeholder stands for
   CtxJob* jobs;                // [B]
   unsigned long long* ctab;    // [B][CT_SLOTS] generation << 48 | (frame + 1) << 40 | set code << 24 | byte class << 16 | value
-  uint32_t* chunk_off;         // [B + 1] first chunk (32 frontier entries) of each job
-  uint4* queue;                // [q_cap] x: node, y: set the node leads to, z: job, w: tag (generation << 16 | 1), written last
-  uint32_t q_cap;
-  uint32_t* qctr;              // [Q_WORDS] tail, head, outstanding work, next chunk: one 128-byte line each
+  uint32_t* fjobs;             // [B] the jobs that go through the level sweep
   Frame* frames;               // [B][MAXF]
   uint16_t* fbind;             // [B][MAXF][max_ph] what each frame's placeholders stand for (sets of the chart)
   uint32_t* frame_ctr;         // [B] frames of the job so far
+  uint32_t* st32;              // [B][st_stride] the fill's level sweep: the set each trie node leads to (see fill_kernel)
+  ulonglong2* req2;            // [req2_cap] its queue of transitions to compute, two halves for odd and even depths
+  uint32_t req2_cap;
 };
 
 struct StateDev {

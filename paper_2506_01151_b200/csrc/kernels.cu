@@ -274,6 +274,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
   if (threadIdx.x < CNT_LAST_LEVEL + 1 - CNT_LEVEL_TAKEN) S.counters[CNT_LEVEL_TAKEN + threadIdx.x] = 0u;
   if (threadIdx.x == 0) {
     S.counters[CNT_N_JOBS] = 0u;
+    S.counters[CNT_N_FJOBS] = 0u;
     S.counters[CNT_AUTO_ITEMS] = 0u;
   }
   if (S.rt.counters) {  // the root sweep of this fill starts from clean counters, too
@@ -363,57 +364,6 @@ __device__ __forceinline__ JobCtx job_ctx(const StateDev& S, uint32_t j) {
   if (S.ctx_mode) J.cap = min(J.cap, ORIGIN_SELF - 16u - RBASE);  // a root's sets are named RBASE + id later on
   J.st = A.st + (size_t)j * A.st_stride;
   return J;
-}
-
-// How often a bounded wait polls before it gives up: 2^dflt times, or 2^poll_limit_shift when the state
-// was created with a limit of its own (tests use a tiny one to take the give-up path).
-__device__ __forceinline__ uint32_t poll_limit(const StateDev& S, uint32_t dflt) {
-  return 1u << (S.poll_limit_shift ? S.poll_limit_shift : dflt);
-}
-
-// All CTAs of the (cooperatively launched) grid meet here.  Returns false if the sweep must be
-// abandoned: some CTA waited longer than the limit, which only a fault elsewhere can cause.
-__device__ __forceinline__ bool grid_barrier(const StateDev& S, uint32_t& phase) {
-  __shared__ uint32_t ok_s;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    ++phase;
-    __threadfence();
-    atomicAdd(&S.counters[CNT_BAR], 1u);
-    const uint32_t target = phase * gridDim.x;
-    uint32_t ok = 1u;
-    for (uint32_t polls = 0;; ++polls) {
-      if (ld_acquire(&S.counters[CNT_BAR]) >= target) break;
-      if (polls > poll_limit(S, 24) || ld_acquire(&S.counters[CNT_BAR_ERR])) {
-        if (polls > poll_limit(S, 24)) diag(S, DIAG_WAIT_GRID);
-        atomicExch(&S.counters[CNT_BAR_ERR], 1u);
-        ok = 0u;
-        break;
-      }
-      __nanosleep(40);
-    }
-    __threadfence();
-    ok_s = ok;
-  }
-  __syncthreads();
-  const bool ok = ok_s != 0u;
-  __syncthreads();
-  return ok;
-}
-
-// A CTA reports that its part of a depth's pass is done (its writes are visible to whoever then sees
-// the count) and goes on without waiting.  Returns false if the sweep is being abandoned.
-__device__ __forceinline__ bool pass_arrive(const StateDev& S, uint32_t& phase) {
-  __shared__ uint32_t go_s;
-  __syncthreads();
-  ++phase;  // (every thread keeps the count: the warps compare it with the global one on their own)
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(&S.counters[CNT_PASS_DONE], 1u);
-    go_s = ld_acquire(&S.counters[CNT_BAR_ERR]) == 0u ? 1u : 0u;
-  }
-  __syncthreads();
-  return go_s != 0u;
 }
 
 // What the Earley set at `node` is, given that its mark says "pending": the transition it waited

@@ -104,7 +104,11 @@ struct SweepWarp {
   unsigned long long cycles = 0;           // SM cycles inside step()
   uint32_t chunk_at = 0, chunk_left = 0;   // this warp's private piece of the item pool (lane 0's copy counts)
   uint32_t gen = 1;                        // this fill's generation of the per-job hashes
-  uint32_t salt = 0;                       // told apart by it: sets with equal items that mean different things (see Frame)
+  // Sets whose items name sets outside the chart (origin codes from region_base on: a frame's sets, or sets
+  // of the walk's own, which may name a frame's sets in turn) mean different things in different frames:
+  // such a set carries the frame as its "salt" and equals only sets with the same salt.  A set whose
+  // origins all lie in the chart is the same set wherever it is met.
+  uint32_t salt = 0, region_base = 0xffffffffu, eff_salt = 0;
 
   // A new set of job J with the items w.cur[0..n), the first nk of them its kernel: its id or T_FAIL.
   __device__ uint32_t create_set(const JobCtx& J, uint32_t n, uint32_t nk, uint32_t hash) {
@@ -144,7 +148,7 @@ struct SweepWarp {
       else if (i == AR_N) v2 = n;
       else if (i == AR_HASH) v2 = hash;
       else if (i == AR_NK) v2 = nk;
-      else if (i == AR_SALT) v2 = salt;
+      else if (i == AR_SALT) v2 = eff_salt;
       else if (i >= AR_SCAN && i < AR_SCAN + 8) v2 = tmp8[i - AR_SCAN];
       else if (i >= AR_TRANS) v2 = T_UNKNOWN;
       rec[i] = v2;
@@ -161,7 +165,7 @@ struct SweepWarp {
   __device__ __forceinline__ bool same_set(const JobCtx& J, uint32_t sid, uint32_t nk, uint32_t hash, Member member) {
     const uint32_t lane = lane_id();
     const uint32_t* rec = J.recs + (size_t)sid * S.au.rec_words;
-    if (__ldcg(rec + AR_HASH) != hash || __ldcg(rec + AR_NK) != nk || __ldcg(rec + AR_SALT) != salt) return false;
+    if (__ldcg(rec + AR_HASH) != hash || __ldcg(rec + AR_NK) != nk || __ldcg(rec + AR_SALT) != eff_salt) return false;
     const uint32_t* items = S.au.items + __ldcg(rec + AR_ITEMS);
     bool ok = true;
     for (uint32_t base = 0; base < nk; base += 32) {
@@ -252,7 +256,8 @@ struct SweepWarp {
     const uint32_t nk = small_drop_completed(G, w, n, mine);
     uint32_t h = lane < nk ? mix32(mine) : 0u;
     for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
-    h = mix32(h + nk * 0x9E3779B9u + salt * 0x85EBCA77u);
+    eff_salt = __any_sync(FULL, lane < nk && (mine >> 16) >= region_base && (mine >> 16) != ORIGIN_SELF) ? salt : 0u;
+    h = mix32(h + nk * 0x9E3779B9u + eff_salt * 0x85EBCA77u);
     auto member = [&](uint32_t x, bool valid) {  // the kernel sits one item per lane
       bool found = false;
       for (uint32_t i = 0; i < nk; ++i)
@@ -300,15 +305,18 @@ struct SweepWarp {
     }
     // the kernel: the items that are not completed; all of cur[0..hashed) are in the uniqueness hash
     uint32_t nk = 0, h = 0;
+    bool reg = false;
     for (uint32_t base = 0; base < hashed; base += 32) {
       const uint32_t i = base + lane;
       const uint32_t it = i < hashed ? w.cur[i] : 0u;
       const bool keep = i < hashed && (G.info[it & 0xFFFFu] >> INFO_KIND_SHIFT) != KIND_END;
       if (keep) h += mix32(it);
+      if (keep && (it >> 16) >= region_base && (it >> 16) != ORIGIN_SELF) reg = true;
       nk += __popc(__ballot_sync(FULL, keep));
     }
     for (int d = 16; d > 0; d >>= 1) h += __shfl_xor_sync(FULL, h, d);
-    h = mix32(h + nk * 0x9E3779B9u + salt * 0x85EBCA77u);
+    eff_salt = __any_sync(FULL, reg) ? salt : 0u;
+    h = mix32(h + nk * 0x9E3779B9u + eff_salt * 0x85EBCA77u);
     auto member = [&](uint32_t x, bool valid) { return !valid || hset_contains(w.hset, w.hset_mask, x); };
     const uint32_t id = lookup_set(J, nk, h, member);
     if (id != T_FAIL) {
@@ -357,5 +365,57 @@ struct SweepWarp {
     return r;
   }
 };
+
+// How often a bounded wait polls before it gives up: 2^dflt times, or 2^poll_limit_shift when the state
+// was created with a limit of its own (tests use a tiny one to take the give-up path).
+__device__ __forceinline__ uint32_t poll_limit(const StateDev& S, uint32_t dflt) {
+  return 1u << (S.poll_limit_shift ? S.poll_limit_shift : dflt);
+}
+
+// All CTAs of the (cooperatively launched) grid meet here.  Returns false if the sweep must be
+// abandoned: some CTA waited longer than the limit, which only a fault elsewhere can cause.
+__device__ __forceinline__ bool grid_barrier(const StateDev& S, uint32_t& phase) {
+  __shared__ uint32_t ok_s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    ++phase;
+    __threadfence();
+    atomicAdd(&S.counters[CNT_BAR], 1u);
+    const uint32_t target = phase * gridDim.x;
+    uint32_t ok = 1u;
+    for (uint32_t polls = 0;; ++polls) {
+      if (ld_acquire(&S.counters[CNT_BAR]) >= target) break;
+      if (polls > poll_limit(S, 24) || ld_acquire(&S.counters[CNT_BAR_ERR])) {
+        if (polls > poll_limit(S, 24)) diag(S, DIAG_WAIT_GRID);
+        atomicExch(&S.counters[CNT_BAR_ERR], 1u);
+        ok = 0u;
+        break;
+      }
+      __nanosleep(40);
+    }
+    __threadfence();
+    ok_s = ok;
+  }
+  __syncthreads();
+  const bool ok = ok_s != 0u;
+  __syncthreads();
+  return ok;
+}
+
+// A CTA reports that its part of a depth's pass is done (its writes are visible to whoever then sees
+// the count) and goes on without waiting.  Returns false if the sweep is being abandoned.
+__device__ __forceinline__ bool pass_arrive(const StateDev& S, uint32_t& phase) {
+  __shared__ uint32_t go_s;
+  __syncthreads();
+  ++phase;  // (every thread keeps the count: the warps compare it with the global one on their own)
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(&S.counters[CNT_PASS_DONE], 1u);
+    go_s = ld_acquire(&S.counters[CNT_BAR_ERR]) == 0u ? 1u : 0u;
+  }
+  __syncthreads();
+  return go_s != 0u;
+}
+
 
 }  // namespace fmt
