@@ -3,9 +3,12 @@
 (row resets the stream asks for, fmt_state_advance with the chosen tokens, fmt_fill_and_apply on
 that step's logits).  Metric: vocab-mask token-checks per second = batch * V * steps / time.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--repeats R] [--passes P] [--impl ours|reference]
 
-With --gpus N > 1 the script is launched by torch.distributed.run, one rank per GPU; every rank
+The K timed steps are repeated R times, every repeat from empty caches and a fresh replay of the
+prefixes and the W warm-up steps; the line's value is the median repeat, with CUDA events around
+every step (latency_ms).  After that the same token stream is run P - 1 more times with the caches
+kept (passes).  With --gpus N > 1 the script is launched by torch.distributed.run, one rank per GPU; every rank
 runs the same workload on its own replica of the tables (sequences are independent, so the path
 shards by sequence with no collective on the data path); time is the max over ranks.
 --impl reference times the CPU oracle on the host cores instead (a deliberately slow baseline).
@@ -31,11 +34,8 @@ import workloads  # noqa: E402
 
 METRIC = "vocab-mask token-checks/s"
 UNIT = "token-checks/s"
-DEFAULT_CONFIG = 3
+DEFAULT_CONFIG = 5
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (config 3 only; taken on the kernels as committed with those summaries)
-NCU_TRAFFIC_BYTES = {3: {"sweep_kernel": 3.6e6, "gather_apply_kernel": 7.9e6, "advance_kernel": 1.6e5}}
 
 
 # --------------------------------------------------------------------------- small helpers
@@ -123,13 +123,18 @@ class ClockSampler:
             self._stop.wait(0.004 if self._nvml is not None else 0.2)
 
     def start(self):
+        self._stop.clear()
         self._thread = threading.Thread(target=self._run, daemon=True)
         self._thread.start()
 
-    def stop(self) -> dict:
+    def pause(self):
         self._stop.set()
         if self._thread:
             self._thread.join(timeout=6)
+            self._thread = None
+
+    def stop(self) -> dict:
+        self.pause()
         return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": max(self.mx) if self.mx else None,
                 "reasons": sorted(self.reasons), "samples": len(self.sm), "source": self.source}
 
@@ -155,14 +160,15 @@ def aggregate_over_ranks(elapsed_ms: float, units: float, dist=None):
 class Driver:
     """Owns the library objects and the device buffers of one replica and runs steps."""
 
-    def __init__(self, w: workloads.Workload, device, ring_bytes: int = int(1.6 * L2_BYTES)):
+    def __init__(self, w: workloads.Workload, device, roots: bool = False, ring_bytes: int = int(1.6 * L2_BYTES)):
         import torch
 
         import paper_2506_01151_b200 as fmt
 
         self.torch, self.fmt, self.w, self.device = torch, fmt, w, device
         self.grammar = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
-        self.state = fmt.State(self.grammar, w.batch)
+        self.state = fmt.State(self.grammar, w.batch, roots=roots)
+        self.roots = roots
         self.stream = torch.cuda.current_stream(device)
         B, V = w.batch, w.V
         self.status = torch.zeros(B, dtype=torch.int32, device=device)
@@ -180,6 +186,7 @@ class Driver:
         g.manual_seed(2506_01151)
         self.ring = (torch.randn((self.n_ring, B, V), generator=g, device=device, dtype=torch.float32) * 2.0).to(torch.bfloat16)
         self.launches = 0
+        self.events = []
 
     def feed_prefix(self):
         for p in range(self.prefix.shape[0]):
@@ -195,7 +202,62 @@ class Driver:
         self.state.advance(self.tokens[i], self.status, stream=s)
         lg = self.ring[i % self.n_ring] if logits is None else logits
         self.state.fill_and_apply(lg, self.fmt.BF16, stream=s)
-        self.launches += 5  # advance; plan, sweep, publish, mask+apply
+        # advance; plan, [entry look-up (2), sweep of new entries, its collection, job set-up], trie sweep, publish, mask+apply
+        self.launches += 10 if self.roots else 5
+
+    def restart(self, warmup: int, clear_caches: bool):
+        """Back to the start of the token stream: all rows reset, prefixes fed, `warmup` untimed steps."""
+        s = self.stream.cuda_stream
+        if clear_caches:
+            self.state.cache_clear(stream=s)
+            self.state.ci_cache_clear(stream=s)
+        self.state.reset(stream=s)
+        self.feed_prefix()
+        for i in range(warmup):
+            self.step(i)
+        self.torch.cuda.synchronize(self.device)
+
+    def timed(self, start: int, n: int):
+        """Steps start .. start+n-1 with an event after every step, on the stream the kernels run on:
+        total milliseconds and the n per-step durations."""
+        torch = self.torch
+        while len(self.events) < n + 1:
+            self.events.append(torch.cuda.Event(enable_timing=True))
+        ev = self.events
+        ev[0].record(self.stream)
+        for k in range(n):
+            self.step(start + k)
+            ev[k + 1].record(self.stream)
+        torch.cuda.synchronize(self.device)
+        return ev[0].elapsed_time(ev[n]), [ev[k].elapsed_time(ev[k + 1]) for k in range(n)]
+
+
+def percentile(xs, q):
+    s = sorted(xs)
+    return s[min(len(s) - 1, int(q * len(s)))]
+
+
+def stat_delta(a, b, keys):
+    return {k: b[k] - a[k] for k in keys}
+
+
+STAT_KEYS = ["fills", "fills_computed", "fills_from_cache", "fills_shared", "rows_mask_only", "rows_from_root", "rows_plain",
+             "root_sweeps", "sweep_transitions", "sweep_states", "walk_transitions", "walk_states", "walk_frames",
+             "big_mode_units", "steps_advanced", "advances_cached", "earley_step_cycles", "capacity_errors", "fills_aborted"]
+
+
+def read_traffic(config: int, kernel: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel` on workload `config`, from the
+    table of ncu captures kept under profiles/ (None if there is no line for it)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                p = line.split("#")[0].split()
+                if len(p) >= 3 and p[0] == str(config) and p[1] == kernel:
+                    return float(p[2])
+    except OSError:
+        pass
+    return None
 
 
 def run_ours(args):
@@ -211,45 +273,54 @@ def run_ours(args):
     device = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
-    K, W = args.steps, args.warmup
+    K, W, R = args.steps, args.warmup, max(1, args.repeats)
     w = workloads.build(args.config, steps=K + W, batch=args.batch)
-    drv = Driver(w, device)
-    drv.feed_prefix()
-    for i in range(W):
-        drv.step(i)
-    torch.cuda.synchronize(device)
-    stats0 = drv.state.stats()
-    drv.launches = 0
-
-    # ---- timed region: device-resident inputs
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize(device)
-    sampler = ClockSampler(local)
-    sampler.start()
-    drv.state.set_profiling(True)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(drv.stream)
-    for i in range(W, W + K):
-        drv.step(i)
-    e1.record(drv.stream)
-    torch.cuda.synchronize(device)
-    if world > 1:
-        dist.barrier()
-    elapsed_ms = e0.elapsed_time(e1)
-    clocks = sampler.stop()
-    prof = drv.state.read_profile()
-    drv.state.set_profiling(False)
-    launches = drv.launches
-    stats1 = drv.state.stats()
+    drv = Driver(w, device, roots=args.roots)
     units = float(w.batch) * w.V * K
-    t_ms, total_units = aggregate_over_ranks(elapsed_ms, units, dist if world > 1 else None)
+    sampler = ClockSampler(local)
 
-    # ---- cold fills: the same steps with the state cache emptied before every fill
-    cold = None
-    e2e = None
+    # ---- R repeats of the same work: empty caches, prefixes, W untimed steps, then EXACTLY K timed steps
+    reps = []
+    for r in range(R):
+        drv.restart(W, clear_caches=r > 0)  # (the first repeat starts from a new state: its caches are empty)
+        stats0 = drv.state.stats()
+        drv.launches = 0
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+        sampler.start()
+        drv.state.read_profile()
+        drv.state.set_profiling(True)
+        total_ms, per_step = drv.timed(W, K)
+        if world > 1:
+            dist.barrier()
+        sampler.pause()
+        prof = drv.state.read_profile()
+        drv.state.set_profiling(False)
+        t_ms, total_units = aggregate_over_ranks(total_ms, units, dist if world > 1 else None)
+        reps.append({"t_ms": t_ms, "units": total_units, "per_step": per_step, "prof": prof, "launches": drv.launches,
+                     "stats": stat_delta(stats0, drv.state.stats(), STAT_KEYS)})
+    clocks = sampler.stop()
+    # ---- once more, untimed, with the cycle counter read around every Earley step (it slows the sweeps a little)
+    drv.restart(W, clear_caches=True)
+    stats0 = drv.state.stats()
+    drv.state.set_profiling(True, step_cycles=True)
+    drv.timed(W, K)
+    prof_cyc = drv.state.read_profile()
+    drv.state.set_profiling(False)
+    st_cyc = stat_delta(stats0, drv.state.stats(), STAT_KEYS)
+    order = sorted(range(R), key=lambda r: reps[r]["t_ms"])
+    med = reps[order[(R - 1) // 2]]  # the median repeat (the lower one of two) is the one reported in full
+    t_ms, total_units, prof, st = med["t_ms"], med["units"], med["prof"], med["stats"]
+
+    cold = cold_all = e2e = passes = None
+    stats_end = drv.state.stats()
     if rank == 0:
-        cold = measure_cold(drv, w, W, min(K, 32))
+        if world == 1 and args.passes > 1:
+            passes = measure_passes(drv, W, K, args.passes, med)
+        stats_end = drv.state.stats()
+        cold = measure_cold(drv, w, W, min(K, 16), clear_ci=False)
+        cold_all = measure_cold(drv, w, W, min(K, 16), clear_ci=True)
         e2e = measure_e2e(drv, w, W, min(K, 64))
     if world > 1:
         dist.barrier()
@@ -261,52 +332,90 @@ def run_ours(args):
     info = drv.grammar.info()
     peak, peak_kind = measured_peaks()
     B, V, Wm = w.batch, w.V, info.mask_words
-    # algorithmic bytes per launch of each kernel kind: what the method itself must move through HBM
+    sm_mhz = clocks["sm_mhz"] or 1900.0
+    # ---- algorithmic bytes per launch of each kind of kernel: what the method itself must move through HBM
     trie_bytes = info.trie_nodes * (1 + 4 + 1) + 4 * V  # node byte, parent, depth; token -> node
-    jobs = stats1["fills_computed"] - stats0["fills_computed"]
-    walk_bytes_per_launch = trie_bytes + (jobs / max(1, K)) * (4 * Wm + 2048)
-    apply_bytes_per_launch = B * (4 * Wm + 2 * V)
+    jobs = st["fills_computed"]
+    sweep_jobs = st["rows_from_root"] + st["rows_plain"]
+    sweep_bytes = trie_bytes + (sweep_jobs / max(1, K)) * (4 * Wm + 2048)  # + per job: its mask row and its chart
+    apply_rw = B * (4 * Wm + 2 * 2 * V)   # mask words read, logits read and written
+    apply_wo = B * (4 * Wm + 2 * V)       # if the logits only had to be written
     kinds = {
-        "sweep_kernel": (prof["sweep_ms"], prof["sweep_launches"], walk_bytes_per_launch),
-        "gather_apply_kernel": (prof["apply_ms"], prof["apply_launches"], apply_bytes_per_launch),
+        "fill_kernel": (prof["sweep_ms"], prof["sweep_launches"], sweep_bytes),
+        "sweep_kernel (new entries)": (prof["roots_ms"], prof["roots_launches"], trie_bytes),
+        "gather_apply_kernel": (prof["apply_ms"], prof["apply_launches"], apply_rw),
         "advance_kernel": (prof["advance_ms"], prof["advance_launches"], B * 2 * 4 * 256),
     }
     dom = max(kinds, key=lambda k: kinds[k][0])
     d_ms, d_n, d_bytes = kinds[dom]
     avg_ms = d_ms / max(1, d_n)
     achieved = d_bytes / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else 0.0
+    # ---- the other bound of the trie sweep: Earley steps.  Each step is one warp's work; the sweep kernels keep
+    # `resident_warps` warps on the GPU, so steps * cycles per step / (resident warps * SM clock) is the time the
+    # sweeps would take if every warp did nothing but Earley steps from start to end.
+    steps_earley = st_cyc["sweep_transitions"] + st_cyc["walk_transitions"]
+    resident_warps = 148 * 24
+    earley_ms = st_cyc["earley_step_cycles"] / (resident_warps * sm_mhz * 1e3) if steps_earley else 0.0
+    sweeps_ms = prof_cyc["sweep_ms"] + prof_cyc["roots_ms"]
+    second = {
+        "bound": "latency (Earley steps)", "earley_steps_per_step": steps_earley / K,
+        "earley_steps_per_computed_row": steps_earley / max(1, st_cyc["fills_computed"]),
+        "cycles_per_earley_step": st_cyc["earley_step_cycles"] / max(1, steps_earley), "resident_warps": resident_warps,
+        "sm_mhz": sm_mhz, "all_warps_busy_ms_per_step": earley_ms / K, "sweeps_ms_per_step": sweeps_ms / K,
+        "frac": earley_ms / sweeps_ms if sweeps_ms > 0 else None,
+        "what": "measured in a run of its own (reading the cycle counter around every step slows the sweeps): warp-cycles "
+                "spent inside Earley steps / (resident warps x SM clock) = the sweeps' time if no warp ever waited for a "
+                "trie level, a queue or a barrier; frac = that time / the sweeps' time in the same run",
+    }
+    floor_rw = (apply_rw + trie_bytes) / (peak * 1e9) * 1e3
+    floor_wo = (apply_wo + trie_bytes) / (peak * 1e9) * 1e3
+    ms_step = t_ms / K
     roofline = {
         "bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "traffic": NCU_TRAFFIC_BYTES.get(args.config, {}).get(dom), "peak_source": peak_kind + " copy bandwidth", "avg_launch_us": avg_ms * 1e3,
-        "bytes_per_launch": d_bytes,
+        "traffic": read_traffic(args.config, dom.split()[0]), "peak_source": peak_kind + " copy bandwidth",
+        "avg_launch_us": avg_ms * 1e3, "bytes_per_launch": d_bytes,
         "per_kernel_ms": {k: v[0] for k, v in kinds.items()},
-        "hbm_floor_us_per_step": (apply_bytes_per_launch + trie_bytes) / (peak * 1e9) * 1e6,
-        "step_frac_of_hbm_floor": ((apply_bytes_per_launch + trie_bytes) / (peak * 1e9) * 1e3) / (t_ms / K),
+        "per_kernel_ms_per_step": {k: v[0] / K for k, v in kinds.items()},
+        "hbm_floor_ms_per_step": {"read_write": floor_rw, "write_only": floor_wo,
+                                  "what": "trie once + mask words + logits (read and written | written only) at the peak"},
+        "step_frac_of_hbm_floor": {"read_write": floor_rw / ms_step, "write_only": floor_wo / ms_step},
+        "gather_apply_gbs": apply_rw / (prof["apply_ms"] / max(1, prof["apply_launches"]) * 1e-3) / 1e9 if prof["apply_ms"] > 0 else None,
+        "second_bound": second,
     }
-    fills = stats1["fills"] - stats0["fills"]
+    ms_list = [r["t_ms"] / K for r in reps]
+    fills = max(1, st["fills"])
+    states = max(1, stats_end["states_cached"])
     out = {
         "metric": METRIC, "value": total_units / (t_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": t_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
         "data": "synthetic",
         "config": {"workload": w.name, "config": args.config, "batch": B, "vocab": V, "logits": "bf16",
                    "l2": "logits cycle through a ring of %d buffers (%.0f MB) > 126 MB L2" % (drv.n_ring, drv.n_ring * B * V * 2 / 1e6),
-                   "state_cache": "on (the paper's state cache; cold numbers under 'cold')",
+                   "state_cache": "on, empty at the start of every repeat (the paper's state cache; per-pass numbers under 'passes')",
+                   "context_independent_cache": "on" if drv.roots else "off",
                    "parallelism": "replicas" if world > 1 else "single"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-        "cache": {"fills": fills, "computed": jobs,
-                  "from_cache": stats1["fills_from_cache"] - stats0["fills_from_cache"],
-                  "shared": stats1["fills_shared"] - stats0["fills_shared"],
-                  "hit_rate": 1.0 - jobs / max(1, fills), "states_cached": stats1["states_cached"],
-                  "chart_items_max": stats1["chart_items_max"], "chart_sets_max": stats1["chart_sets_max"],
-                  "capacity_errors": stats1["capacity_errors"],
-                  "sweep_transitions": stats1["sweep_transitions"] - stats0["sweep_transitions"],
-                  "sweep_states": stats1["sweep_states"] - stats0["sweep_states"],
-                  "big_mode": stats1["big_mode_units"] - stats0["big_mode_units"],
-                  "advances": stats1["steps_advanced"] - stats0["steps_advanced"],
-                  "advances_from_cache": stats1["advances_cached"] - stats0["advances_cached"]},
-        "cold": cold,
+        "repeats": {"n": R, "ms_per_step": ms_list, "median": statistics.median(ms_list), "min": min(ms_list), "max": max(ms_list),
+                    "what": "each repeat: caches emptied, prefixes fed, W untimed steps, K timed steps; value = the median repeat"},
+        "latency_ms": {"p50": percentile(med["per_step"], 0.50), "p90": percentile(med["per_step"], 0.90),
+                       "p99": percentile(med["per_step"], 0.99), "max": max(med["per_step"]), "min": min(med["per_step"]),
+                       "what": "per decoding step (advance + fill + masking of B rows), CUDA events around every step of the median repeat"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": med["launches"], "roofline": roofline,
+        "cache": {"fills": st["fills"], "computed": jobs, "from_state_cache": st["fills_from_cache"], "shared_within_fill": st["fills_shared"],
+                  "hit_rate": 1.0 - jobs / fills,
+                  "computed_by": {"context_independent_row_only": st["rows_mask_only"], "sweep_in_frames": st["rows_from_root"],
+                                  "sweep_from_chart": st["rows_plain"]},
+                  "new_entries_swept": st["root_sweeps"], "entries": stats_end["roots"],
+                  "earley_steps": {"rows": st["walk_transitions"], "new_entries": st["sweep_transitions"]},
+                  "states_cached": stats_end["states_cached"], "chart_items_max": stats_end["chart_items_max"],
+                  "chart_sets_max": stats_end["chart_sets_max"], "capacity_errors": stats_end["capacity_errors"],
+                  "fills_aborted": stats_end["fills_aborted"], "big_mode": st["big_mode_units"],
+                  "advances": st["steps_advanced"], "advances_from_cache": st["advances_cached"]},
+        "memory": {"device_bytes": stats_end["device_bytes"], "states_cached": stats_end["states_cached"],
+                   "state_pool_bytes_used": 4 * stats_end["pool_words_used"], "mask_rows_cached": stats_end["mask_rows_cached"],
+                   "bytes_per_cached_state": (4 * stats_end["pool_words_used"] + 4 * Wm * stats_end["mask_rows_cached"]) / states},
+        "passes": passes, "cold": cold, "cold_all": cold_all,
         "grammar": {"nonterminals": info.n_nonterminals, "rules": info.n_rules, "dotted": info.n_dotted,
-                    "trie_nodes": info.trie_nodes, "byte_classes": info.n_byte_classes},
+                    "trie_nodes": info.trie_nodes, "trie_depth": info.trie_depth, "byte_classes": info.n_byte_classes},
     }
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, W, budget_s=args.cpu_seconds)
@@ -317,27 +426,51 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def measure_cold(drv: "Driver", w, start: int, n: int):
-    """ms per fill when every row's mask is recomputed (state cache emptied before each fill)."""
+def measure_passes(drv: "Driver", W: int, K: int, n_passes: int, first):
+    """The same token stream again and again with the caches kept: pass 1 is a repeat from empty caches, pass p
+    finds what passes 1..p-1 left."""
+    out = [{"pass": 1, "ms_per_step": first["t_ms"] / K, "hit_rate": 1.0 - first["stats"]["fills_computed"] / max(1, first["stats"]["fills"]),
+            "computed": first["stats"]["fills_computed"], "new_entries_swept": first["stats"]["root_sweeps"],
+            "earley_steps": first["stats"]["walk_transitions"] + first["stats"]["sweep_transitions"],
+            "p50_ms": percentile(first["per_step"], 0.5), "p99_ms": percentile(first["per_step"], 0.99)}]
+    # the last repeat has left the caches as one pass leaves them
+    for p in range(2, n_passes + 1):
+        drv.restart(W, clear_caches=False)
+        s0 = drv.state.stats()
+        total_ms, per_step = drv.timed(W, K)
+        d = stat_delta(s0, drv.state.stats(), STAT_KEYS)
+        out.append({"pass": p, "ms_per_step": total_ms / K, "hit_rate": 1.0 - d["fills_computed"] / max(1, d["fills"]),
+                    "computed": d["fills_computed"], "new_entries_swept": d["root_sweeps"],
+                    "earley_steps": d["walk_transitions"] + d["sweep_transitions"],
+                    "p50_ms": percentile(per_step, 0.5), "p99_ms": percentile(per_step, 0.99)})
+    return out
+
+
+def measure_cold(drv: "Driver", w, start: int, n: int, clear_ci: bool):
+    """ms per fill when every row's mask is recomputed: the state cache is emptied before each fill, and with
+    `clear_ci` the cache of context-independent entries too."""
     torch = drv.torch
     s = drv.stream.cuda_stream
     mask = torch.zeros((w.batch, drv.grammar.mask_words), dtype=torch.int32, device=drv.device)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    total = 0.0
-    drv.state.read_profile()
-    drv.state.set_profiling(True)
+    times = []
+    s0 = drv.state.stats()
     for i in range(n):
         drv.state.cache_clear(stream=s)
+        if clear_ci:
+            drv.state.ci_cache_clear(stream=s)
         e0.record(drv.stream)
         drv.state.fill_mask(mask, stream=s)
         e1.record(drv.stream)
         torch.cuda.synchronize(drv.device)
-        total += e0.elapsed_time(e1)
-    prof = drv.state.read_profile()
-    drv.state.set_profiling(False)
-    return {"fills": n, "ms_per_fill": total / n, "sweep_ms_per_fill": prof["sweep_ms"] / max(1, prof["sweep_launches"]),
-            "token_checks_per_s": w.batch * w.V / (total / n * 1e-3),
-            "what": "fmt_fill_mask with the state cache emptied before each call: every distinct row state walks the trie"}
+        times.append(e0.elapsed_time(e1))
+    d = stat_delta(s0, drv.state.stats(), STAT_KEYS)
+    return {"fills": n, "ms_per_fill": statistics.median(times), "min": min(times), "max": max(times),
+            "rows_computed_per_fill": d["fills_computed"] / n,
+            "earley_steps_per_computed_row": (d["walk_transitions"] + d["sweep_transitions"]) / max(1, d["fills_computed"]),
+            "token_checks_per_s": w.batch * w.V / (statistics.median(times) * 1e-3),
+            "what": "fmt_fill_mask with the state cache emptied before each call%s: every distinct row state is computed"
+                    % (" and the context-independent entries too" if clear_ci else ", context-independent entries kept")}
 
 
 def measure_e2e(drv: "Driver", w, start: int, n: int):
@@ -478,6 +611,9 @@ def main():
     ap.add_argument("--config", type=int, default=DEFAULT_CONFIG)
     ap.add_argument("--batch", type=int, default=None, help="override the config's batch size (not the headline workload)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--repeats", type=int, default=5, help="repeats of the timed K steps, each from empty caches (value = the median)")
+    ap.add_argument("--passes", type=int, default=10, help="passes over the token stream with the caches kept (1 GPU only; 0 or 1: none)")
+    ap.add_argument("--roots", action="store_true", help="switch the cache of context-independent entries on (off by default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()

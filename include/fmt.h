@@ -72,8 +72,13 @@ typedef struct {
   uint64_t pool_words;        /* uint32 words of chart storage for the cache (default 64 Mi) */
   uint32_t sweep_states;       /* distinct Earley sets one mask computation may create while it
                                  sweeps the vocabulary (default: 4 Mi / batch, within 2048..32768) */
-  uint32_t roots_disable;      /* 1: no context-independent mask cache: every computed row walks the
-                                 whole vocabulary trie against its own chart */
+  uint32_t roots_enable;       /* 1: keep the context-independent mask cache (Section 4.3): last Earley sets
+                                 with their origins made anonymous, each swept once over the vocabulary, so
+                                 that rows in the same situation share table look-ups and run Earley steps
+                                 only where the answer depends on their own chart.  Off by default: it cuts
+                                 the Earley steps per computed row several times but costs about 1 GB of
+                                 device memory and, on the workloads measured, more time per fill than it
+                                 saves (each trie depth still waits for its slowest step) */
   uint32_t max_roots;          /* entries of the context-independent mask cache (default 4096; each
                                  holds one mask row of ceil(V/32) words) */
   uint32_t root_max_items;     /* a last Earley set with more items than this gets no entry (default and maximum 1024) */
@@ -268,13 +273,18 @@ fmt_status fmt_state_copy_counters(fmt_state* s, int which, uint32_t* out, size_
 fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream);
 
 /* Kernel timing with CUDA events on the caller's stream (no counterpart in the paper: a
- * measurement aid).  While enabled, every fmt_state_advance, the trie-sweep kernel of every fill
- * and every logits-masking kernel of this state is bracketed by a pair of events (up to 16384
- * pairs per kind, later launches are not timed).  fmt_state_read_profile synchronizes those
- * events, adds up the elapsed times and forgets them. */
+ * measurement aid).  While enabled, every fmt_state_advance, both halves of every fill (first the work
+ * on context-independent entries: finding each row's entry and sweeping the new ones; then the trie
+ * sweep of the rows) and every logits-masking kernel of this state are bracketed by pairs of events (up
+ * to 16384 pairs per kind, later launches are not timed).  fmt_state_read_profile synchronizes those
+ * events, adds up the elapsed times and forgets them.  `enable` is a set of bits: 1 = those events;
+ * 2 = count the SM cycles that warps spend inside Earley steps (fmt_stats.earley_step_cycles; reading
+ * the cycle counter around every step slows the sweeps by several per cent, so it is a switch). */
 typedef struct {
   double advance_ms, sweep_ms, apply_ms;
   uint64_t advance_launches, sweep_launches, apply_launches;
+  double roots_ms;         /* the fills' work on context-independent entries */
+  uint64_t roots_launches;
 } fmt_profile;
 fmt_status fmt_state_set_profiling(fmt_state* s, int enable);
 fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);

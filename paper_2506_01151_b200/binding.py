@@ -41,7 +41,7 @@ class StateOptions(C.Structure):
     _fields_ = [
         ("cache_disable", C.c_uint32), ("max_states", C.c_uint32), ("max_mask_rows", C.c_uint32),
         ("chart_words", C.c_uint32), ("pool_words", C.c_uint64), ("sweep_states", C.c_uint32),
-        ("roots_disable", C.c_uint32), ("max_roots", C.c_uint32), ("root_max_items", C.c_uint32),
+        ("roots_enable", C.c_uint32), ("max_roots", C.c_uint32), ("root_max_items", C.c_uint32),
         ("root_max_origins", C.c_uint32), ("wait_limit_log2", C.c_uint32),
     ]
 
@@ -68,7 +68,8 @@ class Stats(C.Structure):
 
 class Profile(C.Structure):
     _fields_ = [("advance_ms", C.c_double), ("sweep_ms", C.c_double), ("apply_ms", C.c_double),
-                ("advance_launches", C.c_uint64), ("sweep_launches", C.c_uint64), ("apply_launches", C.c_uint64)]
+                ("advance_launches", C.c_uint64), ("sweep_launches", C.c_uint64), ("apply_launches", C.c_uint64),
+                ("roots_ms", C.c_double), ("roots_launches", C.c_uint64)]
 
 
 _lib = None
@@ -202,7 +203,7 @@ class State:
 
     def __init__(self, grammar: Grammar, batch: int, stream=None, cache: bool = True, max_states: int = 0,
                  max_mask_rows: int = 0, pool_words: int = 0, chart_words: int = 0, sweep_states: int = 0,
-                 roots: bool = True, max_roots: int = 0, root_max_items: int = 0, root_max_origins: int = 0,
+                 roots: bool = False, max_roots: int = 0, root_max_items: int = 0, root_max_origins: int = 0,
                  wait_limit_log2: int = 0):
         self.grammar = grammar
         self.batch = batch
@@ -213,7 +214,7 @@ class State:
         opt.pool_words = pool_words
         opt.chart_words = chart_words
         opt.sweep_states = sweep_states
-        opt.roots_disable = 0 if roots else 1
+        opt.roots_enable = 1 if roots else 0
         opt.max_roots = max_roots
         opt.root_max_items = root_max_items
         opt.root_max_origins = root_max_origins
@@ -298,8 +299,9 @@ class State:
         _check(lib().fmt_state_copy_chart(self._h, row, buf.ctypes.data, n.value, C.byref(n), _ptr(stream)))
         return buf
 
-    def set_profiling(self, on: bool):
-        _check(lib().fmt_state_set_profiling(self._h, 1 if on else 0))
+    def set_profiling(self, on: bool, step_cycles: bool = False):
+        """Kernel timing with CUDA events; `step_cycles` also counts the SM cycles inside Earley steps."""
+        _check(lib().fmt_state_set_profiling(self._h, (1 if on else 0) | (2 if step_cycles else 0)))
 
     def read_profile(self) -> dict:
         out = Profile()

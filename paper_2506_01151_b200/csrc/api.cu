@@ -72,12 +72,12 @@ struct fmt_grammar {
   DeviceBuffers bufs;
 };
 
-// CUDA-event pairs around the three kinds of kernels, filled while profiling is enabled.
+// CUDA-event pairs around the four kinds of work, filled while profiling is enabled.
 struct Profiler {
   static constexpr size_t kMaxPairs = 16384;
   bool on = false;
-  std::vector<cudaEvent_t> a[3], b[3];  // 0 advance, 1 trie sweep, 2 logits masking
-  size_t used[3] = {0, 0, 0};
+  std::vector<cudaEvent_t> a[4], b[4];  // 0 advance, 1 trie sweep of the fill, 2 logits masking, 3 the fill's work on roots
+  size_t used[4] = {0, 0, 0, 0};
   bool next(int kind, cudaEvent_t* before, cudaEvent_t* after) {
     *before = *after = nullptr;
     if (!on || used[kind] >= kMaxPairs) return false;
@@ -97,7 +97,7 @@ struct Profiler {
     return true;
   }
   ~Profiler() {
-    for (int k = 0; k < 3; ++k) {
+    for (int k = 0; k < 4; ++k) {
       for (auto e : a[k]) cudaEventDestroy(e);
       for (auto e : b[k]) cudaEventDestroy(e);
     }
@@ -125,8 +125,8 @@ static cudaError_t next_generations(fmt_state* s, cudaStream_t st) {
   if (s->next_gen + 1u > 65534u) {
     e = cudaMemsetAsync(d.au.hash, 0, (size_t)d.B * (d.au.hash_mask + 1u) * 4, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(d.au.req, 0, (size_t)d.au.req_cap * 8, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(d.cx.ctab, 0, (size_t)d.B * CT_SLOTS * 8, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(d.cx.req2, 0, (size_t)d.cx.req2_cap * 16, st);
+    if (e == cudaSuccess && d.rt.on) e = cudaMemsetAsync(d.cx.ctab, 0, (size_t)d.B * CT_SLOTS * 8, st);
+    if (e == cudaSuccess && d.rt.on) e = cudaMemsetAsync(d.cx.req2, 0, (size_t)d.cx.req2_cap * 16, st);
     s->next_gen = 1;
   }
   d.gen = s->next_gen;
@@ -345,7 +345,7 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   au.items_cap = 128u << 20;
   d.poll_limit_shift = (opt && opt->wait_limit_log2) ? std::min(opt->wait_limit_log2, 30u) : 0u;
   RootDev& rt = d.rt;
-  rt.on = (opt && opt->roots_disable) ? 0u : 1u;
+  rt.on = (opt && opt->roots_enable) ? 1u : 0u;
   rt.max_roots = (opt && opt->max_roots) ? opt->max_roots : 4096u;
   rt.max_items = (opt && opt->root_max_items) ? std::min(opt->root_max_items, 1024u) : 1024u;
   rt.max_ph = (opt && opt->root_max_origins) ? std::min(opt->root_max_origins, 1024u) : 16u;
@@ -398,31 +398,33 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   au.req_cap = 1u << 20;
   AL(au.req, au.req_cap, 0);
   AL(au.job_info, batch, 0);
-  AL(rt.hash, rh, 0);
-  AL(rt.info, (size_t)rt.max_roots * RI_WORDS, 0);
   AL(rt.n_roots, 4, 0);
-  AL(rt.charts, rt.charts_cap, 0);
-  AL(rt.ci_rows, (size_t)rt.max_roots * g->dev.Wm, 0);
-  AL(rt.states, rt.st_cap, 0);
-  AL(rt.items, rt.it_cap, 0);
-  AL(rt.trans, rt.tr_cap, 0);
   AL(rt.tops, TOP_N, 0);
-  AL(rt.pending, rt.pend_cap, 0);
   AL(rt.counters, CNT_TOTAL, 0);
-  AL(rt.rj_chart, batch, 0);
-  AL(rt.rj_mask, batch, 0);
-  AL(rt.rj_flags, batch, 0);
-  AL(rt.rj_jobs, batch, 0);
-  AL(d.cx.bind, (size_t)batch * rt.max_ph, 0);
-  AL(d.cx.jobs, batch, 0);
-  AL(d.cx.ctab, (size_t)batch * CT_SLOTS, 0);
-  AL(d.cx.fjobs, batch, 0);
-  AL(d.cx.frames, (size_t)batch * MAXF, 0);
-  AL(d.cx.fbind, (size_t)batch * MAXF * rt.max_ph, 0);
-  AL(d.cx.frame_ctr, batch, 0);
-  AL(d.cx.st32, (size_t)batch * au.st_stride, 0xFF);
-  d.cx.req2_cap = 1u << 20;
-  AL(d.cx.req2, d.cx.req2_cap, 0);
+  if (rt.on) {  // the cache of context-independent entries and the frames of the rows' sweeps
+    AL(rt.hash, rh, 0);
+    AL(rt.info, (size_t)rt.max_roots * RI_WORDS, 0);
+    AL(rt.charts, rt.charts_cap, 0);
+    AL(rt.ci_rows, (size_t)rt.max_roots * g->dev.Wm, 0);
+    AL(rt.states, rt.st_cap, 0);
+    AL(rt.items, rt.it_cap, 0);
+    AL(rt.trans, rt.tr_cap, 0);
+    AL(rt.pending, rt.pend_cap, 0);
+    AL(rt.rj_chart, batch, 0);
+    AL(rt.rj_mask, batch, 0);
+    AL(rt.rj_flags, batch, 0);
+    AL(rt.rj_jobs, batch, 0);
+    AL(d.cx.bind, (size_t)batch * rt.max_ph, 0);
+    AL(d.cx.jobs, batch, 0);
+    AL(d.cx.ctab, (size_t)batch * CT_SLOTS, 0);
+    AL(d.cx.fjobs, batch, 0);
+    AL(d.cx.frames, (size_t)batch * MAXF, 0);
+    AL(d.cx.fbind, (size_t)batch * MAXF * rt.max_ph, 0);
+    AL(d.cx.frame_ctr, batch, 0);
+    AL(d.cx.st32, (size_t)batch * au.st_stride, 0xFF);
+    d.cx.req2_cap = 1u << 20;
+    AL(d.cx.req2, d.cx.req2_cap, 0);
+  }
   AL(s->init_state_dev, 4, 0xFF);
   AL(s->result_dev, 4, 0);
   AL(s->query_dev, (size_t)batch * 16, 0);
@@ -482,10 +484,11 @@ fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, 
   if (!s || !mask_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
   if (stride_words < s->g->dev.Wm) return fail(FMT_ERR_INVALID_ARG, "stride_words is smaller than ceil(V/32)");
   cudaStream_t st = (cudaStream_t)stream;
-  cudaEvent_t w0, w1;
+  cudaEvent_t w0, w1, r0 = nullptr, r1 = nullptr;
+  if (s->dev.rt.on) s->prof.next(3, &r0, &r1);
   s->prof.next(1, &w0, &w1);
   if (cudaError_t e = next_generations(s, st)) return cuda_fail(e, "fmt_fill_mask");
-  launch_fill(s->g->dev, s->dev, s->sweep_grid, st, w0, w1);
+  launch_fill(s->g->dev, s->dev, s->sweep_grid, st, r0, r1, w0, w1);
   launch_gather(s->g->dev, s->dev, mask_dev, stride_words, st);
   return launched("fmt_fill_mask");
 }
@@ -508,11 +511,12 @@ fmt_status fmt_fill_and_apply(fmt_state* s, uint32_t* mask_dev_or_null, size_t s
     return fail(FMT_ERR_INVALID_ARG, "stride_words is smaller than ceil(V/32)");
   if (row_stride_elems < s->g->dev.V) return fail(FMT_ERR_INVALID_ARG, "row_stride_elems is smaller than V");
   cudaStream_t st = (cudaStream_t)stream;
-  cudaEvent_t w0, w1, a0, a1;
+  cudaEvent_t w0, w1, a0, a1, r0 = nullptr, r1 = nullptr;
+  if (s->dev.rt.on) s->prof.next(3, &r0, &r1);
   s->prof.next(1, &w0, &w1);
   s->prof.next(2, &a0, &a1);
   if (cudaError_t e = next_generations(s, st)) return cuda_fail(e, "fmt_fill_and_apply");
-  launch_fill(s->g->dev, s->dev, s->sweep_grid, st, w0, w1);
+  launch_fill(s->g->dev, s->dev, s->sweep_grid, st, r0, r1, w0, w1);
   if (a0) cudaEventRecord(a0, st);
   launch_gather_apply(s->g->dev, s->dev, logits_dev, (int)dtype, row_stride_elems, mask_dev_or_null, stride_words, st);
   if (a1) cudaEventRecord(a1, st);
@@ -540,6 +544,7 @@ fmt_status fmt_state_ci_cache_clear(fmt_state* s, void* stream) {
   if (!s) return fail(FMT_ERR_INVALID_ARG, "NULL state");
   cudaStream_t st = (cudaStream_t)stream;
   RootDev& r = s->dev.rt;
+  if (!r.on) return FMT_OK;  // (the state was created without that cache)
   cudaError_t e = cudaMemsetAsync(r.hash, 0, ((size_t)r.hash_mask + 1) * 4, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(r.n_roots, 0, 4, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(r.tops, 0, TOP_N * 4, st);
@@ -601,14 +606,15 @@ fmt_status fmt_state_copy_chart(fmt_state* s, uint32_t row, uint32_t* out, size_
 
 fmt_status fmt_state_set_profiling(fmt_state* s, int enable) {
   if (!s) return fail(FMT_ERR_INVALID_ARG, "NULL state");
-  s->prof.on = enable != 0;
+  s->prof.on = (enable & 1) != 0;
+  s->dev.time_steps = (enable & 2) ? 1u : 0u;
   return FMT_OK;
 }
 
 fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out) {
   if (!s || !out) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
-  double ms[3] = {0, 0, 0};
-  for (int k = 0; k < 3; ++k) {
+  double ms[4] = {0, 0, 0, 0};
+  for (int k = 0; k < 4; ++k) {
     for (size_t i = 0; i < s->prof.used[k]; ++i) {
       cudaError_t e = cudaEventSynchronize(s->prof.b[k][i]);
       float t = 0.f;
@@ -619,7 +625,8 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out) {
   }
   out->advance_ms = ms[0], out->sweep_ms = ms[1], out->apply_ms = ms[2];
   out->advance_launches = s->prof.used[0], out->sweep_launches = s->prof.used[1], out->apply_launches = s->prof.used[2];
-  s->prof.used[0] = s->prof.used[1] = s->prof.used[2] = 0;
+  out->roots_ms = ms[3], out->roots_launches = s->prof.used[3];
+  s->prof.used[0] = s->prof.used[1] = s->prof.used[2] = s->prof.used[3] = 0;
   return FMT_OK;
 }
 
@@ -660,9 +667,10 @@ fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   out->sweep_states = u64(CNT_STAT_LOCAL);
   out->advances_cached = u64(CNT_STAT_ADV_HIT);
   out->rows_from_root = u64(CNT_STAT_JOBS_ROOT);
-  out->rows_plain = u64(CNT_STAT_JOBS_PLAIN);
-  out->walk_transitions = u64(CNT_STAT_CTX_TRANS);
-  out->walk_states = u64(CNT_STAT_CTX_STATES);
+  out->rows_plain = s->dev.rt.on ? u64(CNT_STAT_JOBS_PLAIN) : u64(CNT_STAT_COMPUTED);  // (without that cache every computed row is swept from its chart)
+  // (rows swept from their chart's last set without frames count their steps in the sweep's own slots)
+  out->walk_transitions = u64(CNT_STAT_CTX_TRANS) + u64(CNT_STAT_TRANS);
+  out->walk_states = u64(CNT_STAT_CTX_STATES) + u64(CNT_STAT_LOCAL);
   out->rows_mask_only = u64(CNT_STAT_JOBS_MASK);
   out->walk_frames = u64(CNT_STAT_FRAMES);
   out->root_sweeps = u64(CNT_STAT_ROOT_SWEEPS);

@@ -1000,10 +1000,18 @@ cudaError_t configure_walk_kernels() {
   return cudaFuncSetAttribute((const void*)fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
 }
 
-void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_sweep,
-                 cudaEvent_t after_sweep) {
+void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_roots,
+                 cudaEvent_t after_roots, cudaEvent_t before_sweep, cudaEvent_t after_sweep) {
   launch_plan(G, S, st);
-  if (before_sweep) cudaEventRecord(before_sweep, st);
+  if (!S.rt.on) {
+    // without the cache of context-independent entries every row is swept from its chart's last set
+    if (before_sweep) cudaEventRecord(before_sweep, st);
+    launch_sweep(G, S, sweep_grid, st);
+    if (after_sweep) cudaEventRecord(after_sweep, st);
+    launch_publish(S, st);
+    return;
+  }
+  if (before_roots) cudaEventRecord(before_roots, st);
   const unsigned job_blocks = (unsigned)std::min<uint32_t>((S.B + ROOT_WARPS - 1) / ROOT_WARPS, 296u);
   pending_kernel<<<1, 32, 0, st>>>(S);
   root_kernel<<<job_blocks, ROOT_WARPS * 32, 0, st>>>(G, S);
@@ -1021,6 +1029,8 @@ void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStr
     launch_sweep(G, R, sweep_grid, st);
     collect_kernel<<<S.B, COLLECT_THREADS, 0, st>>>(G, S);
   }
+  if (after_roots) cudaEventRecord(after_roots, st);
+  if (before_sweep) cudaEventRecord(before_sweep, st);
   job_setup_kernel<<<std::min<uint32_t>(S.B, 296u), 256, 0, st>>>(G, S);
   {  // (launched cooperatively: its thread blocks wait for one another between the trie's depths)
     GrammarDev g = G;

@@ -236,6 +236,7 @@ struct StateDev {
   uint32_t gen;               // generation of the sweep's per-job hashes and queue tags (1 .. 65535)
   uint32_t gen_ctx;           // generation of the context-dependent walk's tables
   uint32_t poll_limit_shift;  // bounded waits give up after 2^shift polls
+  uint32_t time_steps;        // count the SM cycles spent inside Earley steps (costs a few per cent of the sweep)
   uint32_t chart_words;       // capacity of one private chart buffer
   uint32_t cache_on;
   uint32_t max_states, ht_mask, max_mask_rows;

@@ -112,42 +112,6 @@ __device__ __forceinline__ uint32_t scan_into_cur(const GrammarDev& G, const War
   return min(w.ctr[W_NCUR], w.cur_cap);
 }
 
-// The sets that one wave of completed items sends the warp to.  Lane c holds a completed item of
-// non-terminal X that began in set o (or none): the first lane of every distinct (X, o) looks the set up, the
-// others get length 0.  `incl` is the running total of the lengths, so that position t of the
-// concatenation of all those sets belongs to the first lane whose `incl` exceeds t.
-struct WaveSets {
-  const uint32_t* ptr;
-  uint32_t len, incl, total;
-  __device__ __forceinline__ uint32_t owner(uint32_t t) const {
-    uint32_t c = 0;
-#pragma unroll
-    for (uint32_t d = 16; d > 0; d >>= 1)
-      if (__shfl_sync(FULL, incl, c + d - 1u) <= t) c += d;
-    return c;
-  }
-};
-
-template <class View>
-__device__ __forceinline__ WaveSets wave_sets(const View& view, bool done_item, uint32_t X, uint32_t o) {
-  const uint32_t lane = lane_id();
-  const unsigned long long key = done_item ? (((unsigned long long)o << 32) | X) : ((1ull << 63) | lane);
-  const uint32_t same = __match_any_sync(FULL, key);  // (every lane takes part: not under the && below)
-  const bool leader = done_item && (uint32_t)(__ffs(same) - 1) == lane;
-  WaveSets ws;
-  ws.ptr = nullptr;
-  ws.len = 0;
-  if (leader) view(o, ws.ptr, ws.len);
-  ws.incl = ws.len;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const uint32_t up = __shfl_up_sync(FULL, ws.incl, d);
-    if ((int)lane >= d) ws.incl += up;
-  }
-  ws.total = __shfl_sync(FULL, ws.incl, 31);
-  return ws;
-}
-
 // Complete (Section 3.2) to a fixpoint over cur, starting at item index `head`.  `view(o, ptr, len)`
 // yields the items of set o and `view.fix(item, o)` rewrites an item read from set o into the
 // naming used by the set under construction (identity for plain charts).  Completed items whose origin is the set itself are not processed:
@@ -175,22 +139,19 @@ __device__ __forceinline__ void complete_fixpoint(const GrammarDev& G, const War
     }
     if (have && kind == KIND_END && (it & 0xFFFFu) == ITEM_ACCEPT) w.ctr[W_ACCEPT] = 1u;
     bool done_item = have && kind == KIND_END && (it >> 16) != cur_index && (it & 0xFFFFu) != ITEM_ACCEPT;  // (nothing waits for the augmented start symbol)
-    if (__any_sync(FULL, done_item)) {
-      // All completions of the wave at once: one lane per distinct (non-terminal, origin) looks its set
-      // up, then the waiting items of all those sets are spread evenly over the lanes.
-      const WaveSets ws = wave_sets(view, done_item, inf & INFO_ARG_MASK, it >> 16);
-      for (uint32_t base = 0; base < ws.total; base += 32) {
-        const uint32_t t = base + lane;
-        const bool valid = t < ws.total;
-        const uint32_t c = ws.owner(valid ? t : 0u);
-        const uint32_t k = t - __shfl_sync(FULL, ws.incl - ws.len, c);
-        const uint32_t* sp = (const uint32_t*)__shfl_sync(FULL, (unsigned long long)ws.ptr, c);
-        const uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, c), o = __shfl_sync(FULL, it >> 16, c);
-        if (valid) {
-          const uint32_t wi = sp[k];
-          const uint32_t winf = G.info[wi & 0xFFFFu];
-          if ((winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X) add_item(G, w, view.fix(wi, o) + 1u);
-        }
+    uint32_t bal = __ballot_sync(FULL, done_item);
+    while (bal) {
+      int src = __ffs(bal) - 1;
+      bal &= bal - 1;
+      uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, src);
+      uint32_t o = __shfl_sync(FULL, it >> 16, src);
+      const uint32_t* sp;
+      uint32_t sl;
+      view(o, sp, sl);
+      for (uint32_t k = lane; k < sl; k += 32) {
+        uint32_t wi = sp[k];
+        uint32_t winf = G.info[wi & 0xFFFFu];
+        if ((winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X) add_item(G, w, view.fix(wi, o) + 1u);
       }
       __syncwarp();
     }
@@ -351,17 +312,18 @@ __device__ __forceinline__ uint32_t small_scan_complete(const GrammarDev& G, con
     uint32_t bal = __ballot_sync(FULL, have && kind == KIND_END && (mine >> 16) != cur_index && (mine & 0xFFFFu) != ITEM_ACCEPT);
     const uint32_t it = mine;
     head = n;
-    if (bal) {
-      const WaveSets ws = wave_sets(view, (bal >> lane) & 1u, inf & INFO_ARG_MASK, it >> 16);
-      for (uint32_t base = 0; base < ws.total; base += 32) {
-        const uint32_t t = base + lane;
-        const bool valid = t < ws.total;
-        const uint32_t c = ws.owner(valid ? t : 0u);
-        const uint32_t k = t - __shfl_sync(FULL, ws.incl - ws.len, c);
-        const uint32_t* sp = (const uint32_t*)__shfl_sync(FULL, (unsigned long long)ws.ptr, c);
-        const uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, c), o = __shfl_sync(FULL, it >> 16, c);
-        const uint32_t wi = valid ? sp[k] : 0u;
-        const uint32_t winf = valid ? G.info[wi & 0xFFFFu] : 0u;
+    while (bal) {
+      const int src = __ffs(bal) - 1;
+      bal &= bal - 1;
+      const uint32_t X = __shfl_sync(FULL, inf & INFO_ARG_MASK, src);
+      const uint32_t o = __shfl_sync(FULL, it >> 16, src);
+      const uint32_t* sp;
+      uint32_t sl;
+      view(o, sp, sl);
+      for (uint32_t base = 0; base < sl; base += 32) {
+        const uint32_t k = base + lane;
+        const uint32_t wi = k < sl ? sp[k] : 0u;
+        const uint32_t winf = k < sl ? G.info[wi & 0xFFFFu] : 0u;
         const bool match = (winf >> INFO_KIND_SHIFT) == KIND_NT && (winf & INFO_ARG_MASK) == X;
         const uint32_t cand = view.fix(wi, o) + 1u;
         const uint32_t skip = match ? (G.info[cand & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;

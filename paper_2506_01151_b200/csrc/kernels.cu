@@ -491,7 +491,8 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32, 1) sweep_kernel(GrammarDev G
           // one 256-bit test rejects most bytes without touching the transition table
           if ((__ldcg(rec + AR_SCAN + (byte[u] >> 5)) >> (byte[u] & 31u)) & 1u) {
             uint32_t* slot = J.recs + (size_t)p_state * A.rec_words + AR_TRANS + G.eq_of_byte[byte[u]];
-            t = ld_acquire(slot);
+            t = __ldcg(slot);  // (a final value is final; anything else is read again, in order)
+            if (t == T_UNKNOWN || t == T_PENDING) t = ld_acquire(slot);
             if (t == T_UNKNOWN) {
               t = atomicCAS(slot, T_UNKNOWN, T_PENDING);
               if (t == T_UNKNOWN) {  // ours to queue

@@ -20,8 +20,8 @@ void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* token
 void launch_plan(const GrammarDev& G, const StateDev& S, cudaStream_t st);
 void launch_publish(const StateDev& S, cudaStream_t st);
 cudaError_t configure_walk_kernels();
-void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_sweep = nullptr,
-                 cudaEvent_t after_sweep = nullptr);
+void launch_fill(const GrammarDev& G, const StateDev& S, int sweep_grid, cudaStream_t st, cudaEvent_t before_roots = nullptr,
+                 cudaEvent_t after_roots = nullptr, cudaEvent_t before_sweep = nullptr, cudaEvent_t after_sweep = nullptr);
 void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t stride_words, cudaStream_t st);
 void launch_apply(const uint32_t* mask, size_t stride_words, void* logits, int dtype, uint32_t batch, uint32_t V,
                   size_t row_stride, cudaStream_t st);

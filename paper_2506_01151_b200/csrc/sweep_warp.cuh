@@ -338,7 +338,7 @@ struct SweepWarp {
   template <class View>
   __device__ uint32_t step(const JobCtx& J, const View& view, const uint32_t* pitems, uint32_t plen, uint32_t pcode,
                            uint32_t byte, bool small_ok) {
-    const long long t0 = clock64();
+    const long long t0 = S.time_steps ? clock64() : 0;
     view.ctx_reset(w);
     uint32_t r = small_ok ? compute_small(J, view, pitems, plen, pcode, byte) : T_RETRY;
     if (r == T_RETRY) {
@@ -346,7 +346,7 @@ struct SweepWarp {
       r = compute_general(J, view, pitems, plen, pcode, byte);
     }
     if (r != T_FAIL) ++n_computed;
-    cycles += (unsigned long long)(clock64() - t0);
+    if (S.time_steps) cycles += (unsigned long long)(clock64() - t0);
     return r;
   }
 

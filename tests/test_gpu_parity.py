@@ -83,9 +83,16 @@ def test_config1_without_cache():
     assert stats["fills_from_cache"] == 0 and (q["state_id"] == -1).all()
 
 
-def test_config2_small_vocab_every_step():
+# Every reduced case runs both ways: each row swept from its own chart (the default), and with the
+# cache of context-independent entries (Section 4.3) that lets rows share table look-ups.
+BOTH_WAYS = pytest.mark.parametrize("roots", [False, True], ids=["from_chart", "ci_cache"])
+
+
+@BOTH_WAYS
+def test_config2_small_vocab_every_step(roots):
     w = workloads.build(2, V=4000, batch=4, steps=96)
-    run_workload(w, check_steps=set(range(w.steps)), fused_every=16)
+    stats, _ = run_workload(w, check_steps=set(range(w.steps)), fused_every=16, roots=roots)
+    assert (stats["roots"] > 0) == roots and (stats["rows_from_root"] + stats["rows_mask_only"] > 0) == roots
 
 
 def test_config2_full():
@@ -94,19 +101,22 @@ def test_config2_full():
     assert stats["fills_from_cache"] + stats["fills_shared"] > 0  # pruned charts repeat (state cache)
 
 
-def test_config3_reduced():
+@BOTH_WAYS
+def test_config3_reduced(roots):
     w = workloads.build(3, V=20000, batch=8, steps=160)
-    run_workload(w, check_steps=set(range(0, 160, 8)), fused_every=40)
+    run_workload(w, check_steps=set(range(0, 160, 8)), fused_every=40, roots=roots)
 
 
-def test_config4_reduced():
+@BOTH_WAYS
+def test_config4_reduced(roots):
     w = workloads.build(4, V=20000, batch=8, steps=128)
-    run_workload(w, check_steps=set(range(0, 128, 8)), fused_every=32)
+    run_workload(w, check_steps=set(range(0, 128, 8)), fused_every=32, roots=roots)
 
 
-def test_config5_reduced():
+@BOTH_WAYS
+def test_config5_reduced(roots):
     w = workloads.build(5, V=20000, batch=8, steps=32, prefix_scale=0.25)
-    run_workload(w, check_steps=set(range(0, 32, 4)), fused_every=16)
+    run_workload(w, check_steps=set(range(0, 32, 4)), fused_every=16, roots=roots)
 
 
 # ---- full sizes, in the launch configuration the benchmark times; masks compared on sampled steps
@@ -125,6 +135,12 @@ def test_config3_full_size_sampled_steps():
 def test_config4_full_size_sampled_steps():
     w = workloads.build(4)
     run_workload(w, check_steps=_sampled(w.steps, 16), fused_every=128, check_prefix_mask=False)
+
+
+def test_config3_full_size_with_the_context_independent_cache():
+    w = workloads.build(3, steps=192)
+    stats, _ = run_workload(w, check_steps=_sampled(w.steps, 24), check_prefix_mask=False, roots=True)
+    assert stats["rows_from_root"] > 0.8 * stats["fills_computed"] and stats["root_sweeps"] > 0 and stats["fills_aborted"] == 0
 
 
 def test_config5_full_size_sampled_rows_and_steps():

@@ -53,7 +53,7 @@ def test_rows_with_different_charts_share_the_context_independent_part():
     w = workloads.build(2, V=6000, batch=2, steps=4)
     g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
     og, ov = oracle.Grammar(w.ebnf, w.start), oracle.Vocab(w.vocab, w.eos)
-    st = fmt.State(g, 2, cache=False)  # no state cache: every fill computes both rows
+    st = fmt.State(g, 2, cache=False, roots=True)  # no state cache: every fill computes both rows
     seqs = [oracle.Sequence_(og) for _ in range(2)]
     _feed_bytes(st, seqs, [list(b'{"a": "x'), []])
     got = _mask_of(st, g, 2)
@@ -215,7 +215,8 @@ def test_rows_sharing_a_broken_computation_get_no_guessed_mask():
     assert s["capacity_errors"] > 0 or s["roots"] > 0  # 16 sets are not enough for JSON unless the root carries the work
 
 
-def test_a_wait_that_runs_out_gives_up_cleanly():
+@pytest.mark.parametrize("roots", [False, True], ids=["from_chart", "ci_cache"])
+def test_a_wait_that_runs_out_gives_up_cleanly(roots):
     """Every wait inside the fill's kernels is a poll with a limit.  With a limit of two polls the
     waits run out although nothing is wrong: the fill must come back, report itself aborted and
     hand out all-zero masks (never a wrong bit); with the default limits the next fill is exact."""
@@ -224,7 +225,7 @@ def test_a_wait_that_runs_out_gives_up_cleanly():
     w = workloads.build(2, V=6000, batch=4, steps=4)
     g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
     og, ov = oracle.Grammar(w.ebnf, w.start), oracle.Vocab(w.vocab, w.eos)
-    st = fmt.State(g, 4, cache=False)
+    st = fmt.State(g, 4, cache=False, roots=roots)
     seqs = [oracle.Sequence_(og) for _ in range(4)]
     _feed_bytes(st, seqs, [list(b'{"a": "x'), list(b"[1, 2"), list(b'{"k": tr'), list(b"[[")])
     want = np.stack([s.mask(ov) for s in seqs])
