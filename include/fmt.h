@@ -297,7 +297,7 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
  * whose device memory is entirely owned by a caching allocator or handed out up front, a
  * real-time or library context where an allocation may synchronize the device or fail under
  * memory pressure, a plugin that may only launch kernels.  fmt_fill_mask itself never allocates,
- * but it needs an fmt_state, whose creation allocates hundreds of megabytes.  This call needs no
+ * but it needs an fmt_state, whose creation allocates gigabytes (fmt_stats.device_bytes).  This call needs no
  * fmt_state: it sweeps the vocabulary trie for charts the caller already holds in device memory
  * (in the layout fmt_state_copy_chart documents) and uses a fixed scratch array that is part of
  * the loaded library image (about 55 MB of device memory on every GPU that loads the library,
@@ -310,9 +310,12 @@ fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
  *   n              number of charts, at most FMT_NOALLOC_MAX_CHARTS, and n x (trie nodes of the
  *                  vocabulary) at most 8 Mi (beyond either limit: FMT_ERR_CAPACITY)
  *   mask_dev       device output, n rows of exactly ceil(V/32) words (dense, no extra stride)
- *   status_dev     device output or NULL, n int32: FMT_OK, FMT_ERR_INVALID_ARG (the chart's header
- *                  does not fit its slot) or FMT_ERR_CAPACITY (the Earley sets met while sweeping the
- *                  vocabulary outgrew the fixed scratch; that row's mask is all-zero)
+ *   status_dev     device output or NULL, n int32: FMT_OK, FMT_ERR_INVALID_ARG (the chart does not fit
+ *                  its slot, its sets' offsets decrease, or an item names a dotted rule or a set that
+ *                  does not exist; such a chart is not swept and its mask is all-zero) or
+ *                  FMT_ERR_CAPACITY (the Earley sets met while sweeping the vocabulary outgrew the
+ *                  fixed scratch, or a bounded wait inside the sweep ran out, which gives up every
+ *                  chart of the call; that row's mask is all-zero)
  *
  * The first call on each device looks up the scratch array's device address and raises the
  * kernels' shared-memory limit; make that first call outside any stream capture.  Every call on

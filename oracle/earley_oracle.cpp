@@ -458,7 +458,7 @@ struct Item {
   }
 };
 
-struct ItemSet {  // "each state set maintains only unique states" (Section 3.2)
+struct ItemSet {  // an Earley set holds every item at most once (Section 3.2)
   std::vector<Item> items;
   std::unordered_set<uint64_t> seen;
   static uint64_t key(const Item& it) {
@@ -807,7 +807,7 @@ int orc_max_threads() {
 #endif
 }
 
-// Section 3.3: "sets the logits of invalid tokens to -inf".  dtype 0 = bfloat16, 1 = float32.
+// Section 3.3: the logit of every token the mask rules out becomes -inf.  dtype 0 = bfloat16, 1 = float32.
 // Valid entries are left untouched bit for bit.
 void orc_apply_mask(const uint32_t* mask, size_t stride_words, void* logits, int dtype, uint32_t batch, uint32_t V,
                     size_t row_stride_elems) {

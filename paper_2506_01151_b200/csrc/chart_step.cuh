@@ -2,8 +2,8 @@
 //   Scan -> Complete (fixpoint) -> Predict; after the token's last byte: Compact (Section 4.2.3),
 // which leaves exactly the chart that compacting after every byte would leave (an item needed at
 // the end was needed at every step before), at a fraction of the work,
-// and the state cache: the pruned chart, densely renumbered, is the cache key ("multiple
-// different input token sequences can correspond to the same pruned Earley states", Section 5.2).
+// and the state cache: the pruned chart, densely renumbered, is the cache key (Section 5.2: token
+// sequences that differ may still end in one and the same pruned chart, and then share an entry).
 //
 // Compact keeps, besides the unfinished items of the new last set, exactly the items a later
 // Complete can still read: an item (Y -> mu . A nu, o') of an earlier set o stays iff a kept item

@@ -903,12 +903,13 @@ static size_t adv_smem_bytes(const GrammarDev& G) {
 static size_t init_smem_bytes() { return (size_t)ADV_WARP_WORDS * 4; }
 // Dynamic shared memory of the sweep for a grammar: per-warp scratch plus, if they fit the
 // budget, the item-info / byte-class / byte-class-number tables.
+constexpr uint32_t SWEEP_SMEM_LIMIT = 224 * 1024;  // what the sweep kernels opt in to
 void sweep_layout(const GrammarDev& G, uint32_t* smem_bytes, uint32_t* tables_in_smem) {
   const uint32_t ntw = (2u * G.Nw + 7u) & ~7u;
   const uint32_t warp_words = SWEEP_CUR + SWEEP_HSET + ntw + W_CTRS + 8;
   uint32_t bytes = SWEEP_WARPS * warp_words * 4u;
   const uint32_t tab = G.hot_words * 4u;
-  *tables_in_smem = tab <= HOT_TABLE_BYTES ? 1u : 0u;
+  *tables_in_smem = (tab <= HOT_TABLE_BYTES && bytes + tab <= SWEEP_SMEM_LIMIT) ? 1u : 0u;
   if (*tables_in_smem) bytes += tab;
   *smem_bytes = bytes;
 }
@@ -918,7 +919,7 @@ cudaError_t configure_kernels() {
   cudaError_t e;
   if ((e = opt_in_smem((const void*)init_kernel, init_smem_bytes())) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)advance_kernel, (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + HOT_TABLE_BYTES)) != cudaSuccess) return e;
-  if ((e = opt_in_smem((const void*)sweep_kernel, 224 * 1024)) != cudaSuccess) return e;
+  if ((e = opt_in_smem((const void*)sweep_kernel, SWEEP_SMEM_LIMIT)) != cudaSuccess) return e;
   return configure_walk_kernels();
 }
 

@@ -67,7 +67,7 @@ __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scrat
                                        uint32_t n, uint32_t* mask) {
   const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t nth = (size_t)gridDim.x * blockDim.x;
-  if (tid < CNT_TOTAL) S.counters[tid] = (tid == CNT_HASH_GEN) ? 1u : 0u;  // the hashes are cleared below: every call is generation 1
+  if (tid < CNT_TOTAL) S.counters[tid] = 0u;  // (the sweep's generation is 1 in every call: the hashes and the queue are cleared below)
   if (tid < n) {
     const uint32_t r = (uint32_t)tid;
     const uint32_t* ch = charts + off.v[r];
@@ -91,7 +91,29 @@ __global__ void noalloc_prepare_kernel(GrammarDev G, StateDev S, uint32_t* scrat
     big[(i / NA_HSET_SLOTS) * per_warp + NA_ARENA_ITEMS + (i % NA_HSET_SLOTS)] = 0xffffffffu;
 }
 
-// One thread: the job list holds the charts whose header was accepted.
+// One CTA per chart whose header was accepted: the rest of the chart.  The sweep indexes its tables
+// with what the chart says, so every word is checked here: the sets' offsets must not decrease, every
+// item must name a dotted rule of this grammar and start in a set of this chart.
+__global__ void noalloc_validate_kernel(GrammarDev G, uint32_t* scratch, const uint32_t* charts, Offsets off, uint32_t n) {
+  const uint32_t r = blockIdx.x;
+  if (r >= n || scratch[NA_OFF_BAD + r]) return;
+  const uint32_t* ch = charts + off.v[r];
+  const uint32_t m = ch[CH_SETS], items = ch[CH_ITEMS];
+  const uint32_t* set_off = ch + CH_HDR;
+  const uint32_t* it = set_off + m + 1;
+  bool bad = false;
+  for (uint32_t i = threadIdx.x; i < m; i += blockDim.x) {
+    const uint32_t a = set_off[i], b = set_off[i + 1];
+    if (a > b || b > items || (i == 0 && a != 0u)) bad = true;
+  }
+  for (uint32_t k = threadIdx.x; k < items; k += blockDim.x) {
+    const uint32_t x = it[k];
+    if ((x & 0xFFFFu) >= G.D || (x >> 16) >= m) bad = true;
+  }
+  if (bad) scratch[NA_OFF_BAD + r] = 1u;  // (every writer writes the same value)
+}
+
+// One thread: the job list holds the charts that passed both checks.
 __global__ void noalloc_jobs_kernel(StateDev S, const uint32_t* scratch, uint32_t n) {
   if (blockIdx.x != 0 || threadIdx.x != 0) return;
   uint32_t j = 0;
@@ -105,7 +127,8 @@ __global__ void noalloc_finish_kernel(GrammarDev G, StateDev S, const uint32_t* 
   const uint32_t r = blockIdx.x;
   if (r >= n) return;
   const bool bad = scratch[NA_OFF_BAD + r] != 0u;
-  const bool broken = (S.row_flags[r] & ROW_BROKEN) != 0u;
+  // a sweep that gave up on a wait leaves no mask to trust, whichever chart it was at
+  const bool broken = (S.row_flags[r] & ROW_BROKEN) != 0u || S.counters[CNT_BAR_ERR] != 0u;
   if (broken)
     for (uint32_t i = threadIdx.x; i < G.Wm; i += blockDim.x) mask[(size_t)r * G.Wm + i] = 0u;
   if (status && threadIdx.x == 0) status[r] = bad ? FMT_ERR_INVALID_ARG : (broken ? FMT_ERR_CAPACITY : FMT_OK);
@@ -192,6 +215,7 @@ extern "C" fmt_status fmt_fill_mask_noalloc(const fmt_grammar* g, const uint32_t
   sweep_layout(*G, &S.au.smem_bytes, &S.au.tables_in_smem);
   cudaStream_t st = (cudaStream_t)stream;
   noalloc_prepare_kernel<<<256, 256, 0, st>>>(*G, S, scratch, charts_dev, off, n, mask_dev);
+  noalloc_validate_kernel<<<n, 256, 0, st>>>(*G, scratch, charts_dev, off, n);
   noalloc_jobs_kernel<<<1, 32, 0, st>>>(S, scratch, n);
   launch_sweep(*G, S, (int)NA_GRID, st);
   noalloc_finish_kernel<<<n, 128, 0, st>>>(*G, S, scratch, n, mask_dev, status_dev);
