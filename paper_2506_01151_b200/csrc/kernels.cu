@@ -751,9 +751,8 @@ __global__ void gather_kernel(GrammarDev G, StateDev S, uint32_t* out, size_t st
   }
 }
 
-// logits[t] = -inf where bit t is 0, for one row.  Each thread takes one mask word (32 tokens:
-// 64 bytes of bf16, 128 bytes of fp32) at a time and handles it in groups of 8 tokens with 16-byte
-// accesses when the row is 16-byte aligned, else token by token.  Groups whose 8 tokens are all
+// logits[t] = -inf where bit t is 0, for one row, in groups of 8 tokens with 16-byte accesses when the
+// row is 16-byte aligned, else token by token.  Groups whose 8 tokens are all
 // valid are not touched; groups whose 8 tokens are all invalid are stored without being read.
 template <typename T>
 __device__ __forceinline__ void apply_group(T* p, uint32_t bits) {  // 8 tokens at p, 16-byte aligned
@@ -795,20 +794,29 @@ __device__ __forceinline__ void apply_row(const uint32_t* mask_row, int32_t spec
   const bool aligned = (reinterpret_cast<uintptr_t>(logits) & 15u) == 0;
   const uint32_t words = (V + 31) / 32;
   const T neg = sizeof(T) == 2 ? (T)0xFF80u : (T)0xFF800000u;
-  for (uint32_t wd = tid; wd < words; wd += nthreads) {
-    uint32_t word = 0;
-    if (mask_row) word = __ldg(&mask_row[wd]);
-    else if (special == MASK_EOS_ONLY && eos >= 0 && wd == ((uint32_t)eos >> 5)) word = 1u << ((uint32_t)eos & 31u);
-    if (mask_out) mask_out[wd] = word;
-    if (word == 0xFFFFFFFFu) continue;
-    const uint32_t t0 = wd * 32;
-    if (aligned && t0 + 32 <= V) {
-#pragma unroll
-      for (uint32_t gq = 0; gq < 4; ++gq) {
-        const uint32_t bits = (word >> (8 * gq)) & 0xFFu;
-        if (bits != 0xFFu) apply_group<T>(logits + t0 + 8 * gq, bits);
-      }
-    } else {
+  auto word_at = [&](uint32_t wd) -> uint32_t {
+    if (mask_row) return __ldg(&mask_row[wd]);
+    return (special == MASK_EOS_ONLY && eos >= 0 && wd == ((uint32_t)eos >> 5)) ? 1u << ((uint32_t)eos & 31u) : 0u;
+  };
+  if (mask_out)
+    for (uint32_t wd = tid; wd < words; wd += nthreads) mask_out[wd] = word_at(wd);
+  if (aligned) {
+    // consecutive lanes take consecutive groups of 8 tokens (16 bytes of bf16, 32 of fp32): every access of a
+    // warp covers one contiguous piece of the row; four lanes share a mask word
+    const uint32_t groups = V / 8;
+#pragma unroll 4
+    for (uint32_t gq = tid; gq < groups; gq += nthreads) {
+      const uint32_t bits = (word_at(gq >> 2) >> (8u * (gq & 3u))) & 0xFFu;
+      if (bits != 0xFFu) apply_group<T>(logits + (size_t)gq * 8, bits);
+    }
+    if (tid == 0)
+      for (uint32_t t = groups * 8; t < V; ++t)
+        if (!((word_at(t >> 5) >> (t & 31u)) & 1u)) logits[t] = neg;
+  } else {
+    for (uint32_t wd = tid; wd < words; wd += nthreads) {
+      const uint32_t word = word_at(wd);
+      if (word == 0xFFFFFFFFu) continue;
+      const uint32_t t0 = wd * 32;
       for (uint32_t i = 0; i < 32 && t0 + i < V; ++i)
         if (!((word >> i) & 1u)) logits[t0 + i] = neg;
     }
@@ -958,13 +966,13 @@ void launch_gather(const GrammarDev& G, const StateDev& S, uint32_t* out, size_t
 void launch_apply(const uint32_t* mask, size_t stride_words, void* logits, int dtype, uint32_t batch, uint32_t V,
                   size_t row_stride, cudaStream_t st) {
   if (batch == 0 || V == 0) return;
-  dim3 grid((unsigned)std::min<uint32_t>(((V + 31) / 32 + 255) / 256, 64), batch);
+  dim3 grid((unsigned)std::max<uint32_t>(1u, std::min<uint32_t>((V / 8 + 1023) / 1024, 64)), batch);
   if (dtype == FMT_BF16) apply_kernel<uint16_t><<<grid, 256, 0, st>>>(mask, stride_words, (uint16_t*)logits, V, row_stride);
   else apply_kernel<uint32_t><<<grid, 256, 0, st>>>(mask, stride_words, (uint32_t*)logits, V, row_stride);
 }
 void launch_gather_apply(const GrammarDev& G, const StateDev& S, void* logits, int dtype, size_t row_stride,
                          uint32_t* mask_out, size_t stride_words, cudaStream_t st) {
-  dim3 grid((unsigned)std::min<uint32_t>(((G.V + 31) / 32 + 255) / 256, 64), S.B);
+  dim3 grid((unsigned)std::max<uint32_t>(1u, std::min<uint32_t>((G.V / 8 + 1023) / 1024, 64)), S.B);  // about four groups of 8 tokens per thread
   if (dtype == FMT_BF16)
     gather_apply_kernel<uint16_t><<<grid, 256, 0, st>>>(G, S, (uint16_t*)logits, row_stride, mask_out, stride_words);
   else
