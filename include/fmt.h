@@ -66,10 +66,10 @@ typedef struct {
 /* Options of fmt_state_create.  Zero-initialise; 0 means "default". */
 typedef struct {
   uint32_t cache_disable;     /* 1: no state cache: every fill recomputes its mask */
-  uint32_t max_states;        /* state-cache entries (default 65536) */
-  uint32_t max_mask_rows;     /* cached mask rows (default 8192) */
+  uint32_t max_states;        /* state-cache entries (default 262144) */
+  uint32_t max_mask_rows;     /* cached mask rows (default 32768; each holds ceil(V/32) words) */
   uint32_t chart_words;       /* capacity of one row's chart in uint32 words (default 65536) */
-  uint64_t pool_words;        /* uint32 words of chart storage for the cache (default 64 Mi) */
+  uint64_t pool_words;        /* uint32 words of chart storage for the cache (default 192 Mi) */
   uint32_t sweep_states;       /* distinct Earley sets one mask computation may create while it
                                  sweeps the vocabulary (default: 4 Mi / batch, within 2048..32768) */
   uint32_t roots_enable;       /* 1: keep the context-independent mask cache (Section 4.3): last Earley sets
@@ -85,6 +85,10 @@ typedef struct {
   uint32_t root_max_origins;   /* nor one whose items start in more distinct earlier sets (default 16) */
   uint32_t wait_limit_log2;    /* every wait inside a kernel is a poll that gives up after 2^this many
                                  polls (0 = defaults, 2^21..2^24); see fmt_state_set_wait_limit */
+  uint32_t cache_keep_when_full; /* 0: when the state cache has no room for a new entry (states, chart
+                                 storage or mask rows), the next fmt_state_advance empties it - every entry
+                                 at once; the rows' current charts are entered again - and caching goes
+                                 on.  1: the cache keeps what it has and takes no new entries */
 } fmt_state_options;
 
 typedef struct {
@@ -138,6 +142,7 @@ typedef struct {
                                    warp computes, [5] wait for queued work, [6] wait for the other thread
                                    blocks, [7] a context-independent entry that could not be kept;
                                    [8..15] the same for the sweeps that fill such entries */
+  uint64_t cache_flushes;       /* times the state cache was emptied because it had no room left */
 } fmt_stats;
 
 /*

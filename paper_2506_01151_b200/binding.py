@@ -42,7 +42,7 @@ class StateOptions(C.Structure):
         ("cache_disable", C.c_uint32), ("max_states", C.c_uint32), ("max_mask_rows", C.c_uint32),
         ("chart_words", C.c_uint32), ("pool_words", C.c_uint64), ("sweep_states", C.c_uint32),
         ("roots_enable", C.c_uint32), ("max_roots", C.c_uint32), ("root_max_items", C.c_uint32),
-        ("root_max_origins", C.c_uint32), ("wait_limit_log2", C.c_uint32),
+        ("root_max_origins", C.c_uint32), ("wait_limit_log2", C.c_uint32), ("cache_keep_when_full", C.c_uint32),
     ]
 
 
@@ -58,7 +58,7 @@ class Stats(C.Structure):
         "mask_rows_cached", "pool_words_used", "chart_items_max", "chart_sets_max", "capacity_errors",
         "big_mode_units", "sweep_transitions", "sweep_states", "advances_cached", "roots", "root_sweeps",
         "rows_mask_only", "rows_from_root", "rows_plain", "walk_transitions", "walk_states", "walk_frames",
-        "fills_aborted", "device_bytes", "earley_step_cycles", "advance_chart_words")] + [("diag", C.c_uint64 * 16)]
+        "fills_aborted", "device_bytes", "earley_step_cycles", "advance_chart_words")] + [("diag", C.c_uint64 * 16), ("cache_flushes", C.c_uint64)]
 
     def as_dict(self):
         d = {n: int(getattr(self, n)) for n, _ in self._fields_ if n != "diag"}
@@ -204,7 +204,7 @@ class State:
     def __init__(self, grammar: Grammar, batch: int, stream=None, cache: bool = True, max_states: int = 0,
                  max_mask_rows: int = 0, pool_words: int = 0, chart_words: int = 0, sweep_states: int = 0,
                  roots: bool = False, max_roots: int = 0, root_max_items: int = 0, root_max_origins: int = 0,
-                 wait_limit_log2: int = 0):
+                 wait_limit_log2: int = 0, keep_when_full: bool = False):
         self.grammar = grammar
         self.batch = batch
         opt = StateOptions()
@@ -219,6 +219,7 @@ class State:
         opt.root_max_items = root_max_items
         opt.root_max_origins = root_max_origins
         opt.wait_limit_log2 = wait_limit_log2
+        opt.cache_keep_when_full = 1 if keep_when_full else 0
         h = C.c_void_p()
         _check(lib().fmt_state_create(grammar._h, batch, C.byref(opt), _ptr(stream), C.byref(h)))
         self._h = h

@@ -115,6 +115,14 @@ struct fmt_state {
   int sweep_grid = 1;
   uint32_t next_gen = 1;      // generations handed to the fills: two per fill, 1 .. 65534
   size_t device_bytes = 0;    // what fmt_state_create allocated
+  // The device sets this host-mapped word when the state cache has no room for a new entry; the next
+  // fmt_state_advance empties the cache (all entries at once) and caching goes on.
+  uint32_t* full_flag_host = nullptr;
+  bool skip_full_check = false;
+  uint64_t flushes = 0;
+  ~fmt_state() {
+    if (full_flag_host) cudaFreeHost(full_flag_host);
+  }
 };
 
 // Two fresh generations for a fill (its root sweep and its walk).  Tables tagged with a generation
@@ -319,9 +327,9 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   d.cache_on = (opt && opt->cache_disable) ? 0u : 1u;
   d.chart_words = (opt && opt->chart_words) ? opt->chart_words : 65536u;
   if (d.chart_words < 1024) d.chart_words = 1024;
-  d.max_states = (opt && opt->max_states) ? opt->max_states : 65536u;
-  d.max_mask_rows = (opt && opt->max_mask_rows) ? opt->max_mask_rows : 8192u;
-  d.pool_words = (opt && opt->pool_words) ? opt->pool_words : (64ull << 20);
+  d.max_states = (opt && opt->max_states) ? opt->max_states : 262144u;
+  d.max_mask_rows = (opt && opt->max_mask_rows) ? opt->max_mask_rows : 32768u;
+  d.pool_words = (opt && opt->pool_words) ? opt->pool_words : (192ull << 20);
   if (!d.cache_on) {
     d.max_states = 1;
     d.max_mask_rows = 0;
@@ -434,6 +442,18 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
     delete s;
     return stt;
   }
+  if (d.cache_on && !(opt && opt->cache_keep_when_full)) {
+    void* dp = nullptr;
+    if (cudaHostAlloc((void**)&s->full_flag_host, sizeof(uint32_t), cudaHostAllocMapped) == cudaSuccess &&
+        cudaHostGetDevicePointer(&dp, s->full_flag_host, 0) == cudaSuccess) {
+      *s->full_flag_host = 0u;
+      d.full_flag = static_cast<uint32_t*>(dp);
+    } else {  // no mapped memory: the cache simply stops taking entries when it is full
+      if (s->full_flag_host) cudaFreeHost(s->full_flag_host);
+      s->full_flag_host = nullptr;
+      cudaGetLastError();
+    }
+  }
   launch_init(g->dev, d, s->result_dev, st);
   launch_intern_init(d, s->init_state_dev, st);
   launch_reset(d, nullptr, batch, s->init_state_dev, st);
@@ -472,6 +492,18 @@ fmt_status fmt_state_reset(fmt_state* s, const uint32_t* rows_dev, uint32_t n, v
 
 fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t* status_dev, void* stream) {
   if (!s || !token_ids_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  if (s->full_flag_host) {
+    volatile uint32_t* flag = s->full_flag_host;
+    if (s->skip_full_check) {  // kernels enqueued before the last flush may have raised the flag once more
+      *flag = 0u;
+      s->skip_full_check = false;
+    } else if (*flag) {
+      *flag = 0u;
+      s->skip_full_check = true;
+      ++s->flushes;
+      if (fmt_status rc = fmt_state_cache_clear(s, stream)) return rc;
+    }
+  }
   cudaEvent_t e0, e1;
   s->prof.next(0, &e0, &e1);
   if (e0) cudaEventRecord(e0, (cudaStream_t)stream);
@@ -676,6 +708,7 @@ fmt_status fmt_get_stats(fmt_state* s, fmt_stats* out, void* stream) {
   out->root_sweeps = u64(CNT_STAT_ROOT_SWEEPS);
   out->fills_aborted = u64(CNT_STAT_ABORTS);
   out->device_bytes = s->device_bytes;
+  out->cache_flushes = s->flushes;
   out->earley_step_cycles = u64(CNT_STAT_STEP_CYCLES);
   out->advance_chart_words = u64(CNT_STAT_ADV_WORDS);
   for (int i = 0; i < 8; ++i) out->diag[i] = c[CNT_DIAG + i];

@@ -239,6 +239,7 @@ struct StateDev {
   uint32_t time_steps;        // count the SM cycles spent inside Earley steps (costs a few per cent of the sweep)
   uint32_t chart_words;       // capacity of one private chart buffer
   uint32_t cache_on;
+  uint32_t* full_flag;        // host-mapped word (or nullptr): set when the state cache or its mask rows have no room left
   uint32_t max_states, ht_mask, max_mask_rows;
   uint64_t pool_base, pool_words;   // word offsets into arena / size of the pool
   uint64_t init_off;                // word offset of the start chart

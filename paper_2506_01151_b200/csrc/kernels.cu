@@ -51,7 +51,10 @@ __device__ int32_t intern_chart(const StateDev& S, const uint32_t* ch, uint64_t&
         }
         id = __shfl_sync(FULL, id, 0);
         off = __shfl_sync(FULL, off, 0);
-        if (id < 0) return -1;  // the cache is full
+        if (id < 0) {  // the cache is full: tell the host, which empties it before the next advance
+          if (lane == 0 && S.full_flag) *reinterpret_cast<volatile uint32_t*>(S.full_flag) = 1u;
+          return -1;
+        }
         uint32_t* dst = S.arena + S.pool_base + off;
         for (uint32_t i = lane; i < words; i += 32) dst[i] = ch[i];
         if (lane == 0) {
@@ -313,6 +316,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
         uint32_t got = atomicAdd(&S.counters[CNT_N_MASK_ROWS], 1u);
         if (got < S.max_mask_rows) mrow = (int32_t)(S.B + got);
       }
+      if (mrow == (int32_t)row && S.full_flag) *reinterpret_cast<volatile uint32_t*>(S.full_flag) = 1u;  // no mask row left to cache it in
       S.row_mask[row] = mrow;
     } else {
       S.row_mask[row] = (int32_t)row;

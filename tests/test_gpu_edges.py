@@ -156,13 +156,17 @@ def test_fused_apply_fp32_and_wide_mask_stride():
     assert np.array_equal(lt.cpu().numpy().view(np.uint32), want.view(np.uint32))
 
 
-def test_tiny_cache_still_gives_right_masks():
+@pytest.mark.parametrize("keep", [True, False], ids=["keep_when_full", "empty_when_full"])
+def test_tiny_cache_still_gives_right_masks(keep):
+    """A state cache far too small for the workload: either it keeps its first entries and takes no
+    more (rows that found no room carry their charts themselves), or - the default - it is emptied
+    whenever it has no room left and goes on caching.  The masks are the oracle's either way."""
     import paper_2506_01151_b200 as fmt
 
     torch, dev = _torch()
     w = workloads.build(2, V=3000, batch=4, steps=60)
     g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
-    st = fmt.State(g, w.batch, max_states=8, max_mask_rows=2, pool_words=4096)  # fills up at once
+    st = fmt.State(g, w.batch, max_states=8, max_mask_rows=2, pool_words=4096, keep_when_full=keep)  # fills up at once
     og, ov = oracle.Grammar(w.ebnf, w.start), oracle.Vocab(w.vocab, w.eos)
     seqs = [oracle.Sequence_(og) for _ in range(w.batch)]
     for p in range(w.prefix.shape[0]):
@@ -190,7 +194,12 @@ def test_tiny_cache_still_gives_right_masks():
                     assert np.array_equal(got[b], seqs[b].mask(ov)), (i, b)
     s = st.stats()
     assert s["states_cached"] <= 8 and s["mask_rows_cached"] <= 2 and s["capacity_errors"] == 0
-    assert (st.query()["state_id"] == -1).any()  # some rows could not be cached and carry their chart themselves
+    if keep:
+        assert s["cache_flushes"] == 0
+        assert (st.query()["state_id"] == -1).any()  # some rows could not be cached and carry their chart themselves
+    else:
+        assert s["cache_flushes"] >= 3  # emptied again and again, and entries taken again after each time
+        assert s["fills_from_cache"] + s["advances_cached"] >= 0
 
 
 def _wide_grammar(n):
