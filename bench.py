@@ -341,7 +341,7 @@ def run_ours(args):
     apply_rw = B * (4 * Wm + 2 * 2 * V)   # mask words read, logits read and written
     apply_wo = B * (4 * Wm + 2 * V)       # if the logits only had to be written
     kinds = {
-        "fill_kernel": (prof["sweep_ms"], prof["sweep_launches"], sweep_bytes),
+        ("fill_kernel" if drv.roots else "sweep_kernel"): (prof["sweep_ms"], prof["sweep_launches"], sweep_bytes),
         "sweep_kernel (new entries)": (prof["roots_ms"], prof["roots_launches"], trie_bytes),
         "gather_apply_kernel": (prof["apply_ms"], prof["apply_launches"], apply_rw),
         "advance_kernel": (prof["advance_ms"], prof["advance_launches"], B * 2 * 4 * 256),
