@@ -225,6 +225,26 @@ fmt_status fmt_state_reset(fmt_state* s, const uint32_t* rows_dev, uint32_t n, v
 fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t* status_dev, void* stream);
 
 /*
+ * Jump-ahead: per row, the run of bytes that every continuation of the row's text must begin with.
+ * (Section 5.1 evaluates a JSON-Schema task, where keys, quotes and punctuation between the values are
+ * fixed by the schema; the paper names no such call.  A server may append the run's tokens without
+ * sampling.)  As long as the text so far is not a sentence of the grammar (EOS is not valid) and exactly
+ * one byte can follow it, that byte joins the run and the row's chart is stepped over it, in scratch
+ * memory: the row itself does not change.
+ *   bytes_dev     device output, row r's run at bytes_dev[r * stride_bytes ..]; bytes beyond the run's
+ *                 length are left as they were
+ *   stride_bytes  >= max_len
+ *   len_dev       device output, [batch] uint32: the run's length, 0 .. max_len; 0 for finished or
+ *                 broken rows.  A run that reaches max_len, or whose Earley sets outgrow the scratch,
+ *                 is cut there: every prefix of a forced run is forced, so a shorter answer is still right
+ *   max_len       at most FMT_MAX_FORCED_BYTES (larger values are clamped); call again after advancing
+ *                 the row for longer runs
+ */
+#define FMT_MAX_FORCED_BYTES 32
+fmt_status fmt_state_forced_bytes(fmt_state* s, uint8_t* bytes_dev, size_t stride_bytes, uint32_t* len_dev, uint32_t max_len,
+                                  void* stream);
+
+/*
  * Write the mask of every row (Sections 3.3, 4.1): mask_dev[row * stride_words + w].
  * stride_words >= ceil(V/32).  Rows whose pruned chart is in the state cache copy the cached
  * mask; the others sweep the vocabulary trie.

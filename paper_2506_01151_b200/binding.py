@@ -21,7 +21,7 @@ BF16, FP32 = 0, 1
 
 EXPORTS = [
     "fmt_compile", "fmt_json_schema_to_ebnf", "fmt_compile_json_schema", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table",
-    "fmt_state_create", "fmt_state_destroy", "fmt_state_reset", "fmt_state_advance", "fmt_fill_mask",
+    "fmt_state_create", "fmt_state_destroy", "fmt_state_reset", "fmt_state_advance", "fmt_state_forced_bytes", "fmt_fill_mask",
     "fmt_apply_mask", "fmt_fill_and_apply", "fmt_state_cache_clear", "fmt_state_ci_cache_clear", "fmt_state_set_wait_limit", "fmt_state_copy_counters", "fmt_state_query", "fmt_state_copy_chart", "fmt_get_stats",
     "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_fill_mask_noalloc", "fmt_last_error",
 ]
@@ -92,6 +92,7 @@ def lib():
         L.fmt_state_destroy.restype = None
         L.fmt_state_reset.argtypes = [vp, vp, u32, vp]
         L.fmt_state_advance.argtypes = [vp, vp, vp, vp]
+        L.fmt_state_forced_bytes.argtypes = [vp, vp, sz, vp, u32, vp]
         L.fmt_fill_mask.argtypes = [vp, vp, sz, vp]
         L.fmt_apply_mask.argtypes = [vp, sz, vp, C.c_int, u32, u32, sz, vp]
         L.fmt_fill_and_apply.argtypes = [vp, vp, sz, vp, C.c_int, sz, vp]
@@ -241,6 +242,11 @@ class State:
 
     def advance(self, token_ids_dev, status_dev=None, stream=None):
         _check(lib().fmt_state_advance(self._h, _ptr(token_ids_dev), _ptr(status_dev), _ptr(stream)))
+
+    def forced_bytes(self, bytes_dev, len_dev, max_len: int = 32, stride_bytes: Optional[int] = None, stream=None):
+        """fmt_state_forced_bytes: per row the bytes every continuation must begin with (uint8 [batch, stride], uint32 [batch])."""
+        stride = stride_bytes if stride_bytes is not None else int(bytes_dev.shape[-1])
+        _check(lib().fmt_state_forced_bytes(self._h, _ptr(bytes_dev), stride, _ptr(len_dev), max_len, _ptr(stream)))
 
     def fill_mask(self, mask_dev, stride_words: Optional[int] = None, stream=None):
         stride = self.grammar.mask_words if stride_words is None else stride_words

@@ -512,6 +512,15 @@ fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t
   return launched("fmt_state_advance");
 }
 
+fmt_status fmt_state_forced_bytes(fmt_state* s, uint8_t* bytes_dev, size_t stride_bytes, uint32_t* len_dev, uint32_t max_len,
+                                  void* stream) {
+  if (!s || !bytes_dev || !len_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  if (max_len > FMT_MAX_FORCED_BYTES) max_len = FMT_MAX_FORCED_BYTES;
+  if (stride_bytes < max_len) return fail(FMT_ERR_INVALID_ARG, "stride_bytes is smaller than max_len");
+  launch_forced(s->g->dev, s->dev, bytes_dev, stride_bytes, len_dev, max_len, (cudaStream_t)stream);
+  return launched("fmt_state_forced_bytes");
+}
+
 fmt_status fmt_fill_mask(fmt_state* s, uint32_t* mask_dev, size_t stride_words, void* stream) {
   if (!s || !mask_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
   if (stride_words < s->g->dev.Wm) return fail(FMT_ERR_INVALID_ARG, "stride_words is smaller than ceil(V/32)");

@@ -167,12 +167,18 @@ struct TokenView {
 // is garbage), -1 (a capacity limit was hit) or -2 (the arena for the token's sets is too small:
 // the caller may retry with a larger one).  src and dst must not overlap.  `arena` (arena_cap
 // items, a power of two if the last set is to be sorted in place) holds the token's sets.
+//
+// With `forced_out` set, the bytes are not given but found: as long as the text so far is not a sentence and
+// exactly one byte can follow, that byte is taken (and written to forced_out); `len` is then the longest run
+// looked for, nothing is compacted or written to dst, and the return value is the length of the run.
 __device__ int token_step(const GrammarDev& G, AdvScratch& s, const uint32_t* src, const uint8_t* bytes, uint32_t len,
-                          uint32_t* dst, uint32_t dst_cap, uint32_t* arena, uint32_t arena_cap) {
+                          uint32_t* dst, uint32_t dst_cap, uint32_t* arena, uint32_t arena_cap,
+                          uint8_t* forced_out = nullptr) {
   const uint32_t lane = lane_id();
   const uint32_t m = src[CH_SETS];
   const uint32_t n_items = src[CH_ITEMS];
-  if (m == 0 || m + len + MAX_TOKEN_BYTES + 4 > ADV_MAX_SETS || n_items > ADV_MAX_ITEMS || len > MAX_TOKEN_BYTES) return -1;
+  if (m == 0 || m + len + MAX_TOKEN_BYTES + 4 > ADV_MAX_SETS || n_items > ADV_MAX_ITEMS || len > MAX_TOKEN_BYTES)
+    return forced_out ? 0 : -1;
   // small charts are read from shared memory from here on
   const uint32_t src_words = src[CH_WORDS];
   __syncwarp();
@@ -188,17 +194,31 @@ __device__ int token_step(const GrammarDev& G, AdvScratch& s, const uint32_t* sr
   __syncwarp();
   // ---- per byte: Scan, Complete, Predict; the new set is appended to the arena
   uint32_t top = 0;
-  bool accepting = false;
+  bool accepting = forced_out != nullptr && (src[CH_FLAGS] & CHART_ACCEPTING) != 0u;
   const uint32_t* prev = sitems + soff[m - 1];
   uint32_t prev_len = soff[m] - soff[m - 1];
   for (uint32_t L = 1; L <= len; ++L) {
-    if (top + 64 > arena_cap) return -2;
+    if (top + 64 > arena_cap) return forced_out ? (int)(L - 1) : -2;
+    uint32_t byte;
+    if (forced_out) {  // is the next byte forced?
+      if (accepting) return (int)(L - 1);  // the text may end here
+      scannable_bytes(G, prev, prev_len, s.pairs);
+      uint32_t wd = lane < 8 ? s.pairs[lane] : 0u;
+      uint32_t cnt = __popc(wd);
+      for (int dd = 16; dd > 0; dd >>= 1) cnt += __shfl_xor_sync(FULL, cnt, dd);
+      if (cnt != 1u) return (int)(L - 1);
+      const uint32_t has = __ballot_sync(FULL, wd != 0u);
+      const int src_lane = __ffs(has) - 1;
+      byte = (uint32_t)src_lane * 32u + (uint32_t)(__ffs(__shfl_sync(FULL, wd, src_lane)) - 1);
+      __syncwarp();
+    } else {
+      byte = __ldg(&bytes[L - 1]);
+    }
     s.w.cur = arena + top;
     s.w.cur_cap = arena_cap - top;
     __syncwarp();
     if (lane < W_CTRS) s.w.ctr[lane] = 0u;
     __syncwarp();
-    const uint32_t byte = __ldg(&bytes[L - 1]);
     const uint32_t index = m - 1 + L;
     uint32_t n;
     // sets of up to 32 scanned and completed items (nearly all) are built in lanes ...
@@ -206,39 +226,41 @@ __device__ int token_step(const GrammarDev& G, AdvScratch& s, const uint32_t* sr
     const uint32_t ns = (prev_len <= 96u) ? small_scan_complete(G, s.w, view, prev, prev_len, byte, index,
                                                                  [](uint32_t it) { return it; }, mine, accepting)
                                            : SMALL_OVERFLOW;
-    if (ns == 0) return 0;
+    if (ns == 0) return forced_out ? (int)(L - 1) : 0;
     if (ns != SMALL_OVERFLOW) {
       const uint32_t nk = small_drop_completed(G, s.w, ns, mine);
       if (lane == 0) s.w.ctr[W_NCUR] = nk;
       predict_into_cur(G, s.w, index);
-      if (s.w.ctr[W_OVERFLOW]) return -2;
+      if (s.w.ctr[W_OVERFLOW]) return forced_out ? (int)(L - 1) : -2;
       n = min(s.w.ctr[W_NCUR], s.w.cur_cap);
     } else {  // ... larger ones with the uniqueness hash
       n = scan_into_cur(G, s.w, prev, prev_len, byte);
       if (s.w.ctr[W_OVERFLOW]) {
         hset_clear_all(s.w.hset, s.w.hset_mask);
-        return -2;
+        return forced_out ? (int)(L - 1) : -2;
       }
-      if (n == 0) return 0;
+      if (n == 0) return forced_out ? (int)(L - 1) : 0;
       complete_fixpoint(G, s.w, view, index, 0u);
       uint32_t hashed = min(s.w.ctr[W_NCUR], s.w.cur_cap);
       if (s.w.ctr[W_OVERFLOW]) {
         hset_clear_all(s.w.hset, s.w.hset_mask);
         clear_nt(G, s.w);
-        return -2;
+        return forced_out ? (int)(L - 1) : -2;
       }
       hset_clear_items(s.w, hashed);
       accepting = s.w.ctr[W_ACCEPT] != 0u;
       predict_into_cur(G, s.w, index);
-      if (s.w.ctr[W_OVERFLOW]) return -2;
+      if (s.w.ctr[W_OVERFLOW]) return forced_out ? (int)(L - 1) : -2;
       n = drop_completed(G, s.w, min(s.w.ctr[W_NCUR], s.w.cur_cap));
     }
     prev = arena + top;
     prev_len = n;
     top += n;
     if (lane == 0) lvl_off[L + 1] = top;
+    if (forced_out && lane == 0) forced_out[L - 1] = (uint8_t)byte;  // (the step went through: the byte counts)
     __syncwarp();
   }
+  if (forced_out) return (int)len;
   // ---- Compact once: which items of the earlier sets can a later Complete still read?
   const uint32_t last = m - 1 + len;           // index of the last set
   const uint32_t last_at = lvl_off[len];       // its first item in the arena

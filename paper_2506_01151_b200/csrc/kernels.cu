@@ -268,6 +268,37 @@ __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev G
   finish(FMT_OK);
 }
 
+// ===================================================================================== forced bytes
+//
+// Per row, the run of bytes that every continuation of the row's text must begin with (the keys and
+// punctuation a JSON schema fixes, Section 5.1's JSON-Schema task): as long as the text is not a
+// sentence and the last Earley set can scan exactly one byte, that byte is taken and the chart is
+// stepped over it.  Nothing of the row changes: the sets made on the way live in the warp's scratch.
+__global__ void __launch_bounds__(ADV_WARPS * 32, 1) forced_kernel(GrammarDev Gg, StateDev S, uint8_t* bytes_out,
+                                                                   size_t stride, uint32_t* len_out, uint32_t max_len) {
+  extern __shared__ __align__(16) uint32_t smem[];
+  const uint32_t warp = threadIdx.x >> 5, lane = lane_id();
+  const uint32_t row = blockIdx.x * ADV_WARPS + warp;
+  GrammarDev G = Gg;
+  if (Gg.hot_words * 4u <= HOT_TABLE_BYTES) {
+    G = stage_hot_tables(Gg, smem + (size_t)ADV_WARPS * ADV_WARP_WORDS);
+    __syncthreads();
+  }
+  if (row >= S.B) return;
+  AdvScratch s = adv_scratch(smem + (size_t)warp * ADV_WARP_WORDS);
+  int n = 0;
+  if (!(S.row_flags[row] & (ROW_FINISHED | ROW_BROKEN)) && max_len > 0) {
+    hset_clear_all(s.w.hset, s.w.hset_mask);
+    for (uint32_t i = lane; i < ADV_NT_WORDS; i += 32) s.w.nt[i] = 0u;
+    __syncwarp();
+    const uint32_t* cur = S.arena + S.row_chart[row];
+    n = token_step(G, s, cur, nullptr, min(max_len, MAX_TOKEN_BYTES), nullptr, 0u, s.w.cur, ADV_CUR_CAP,
+                   bytes_out + (size_t)row * stride);
+    if (n < 0) n = 0;
+  }
+  if (lane == 0) len_out[row] = (uint32_t)n;
+}
+
 // ===================================================================================== fill: plan
 
 // One block decides, row by row, where each mask comes from: the state cache, another row of
@@ -931,6 +962,7 @@ cudaError_t configure_kernels() {
   cudaError_t e;
   if ((e = opt_in_smem((const void*)init_kernel, init_smem_bytes())) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)advance_kernel, (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + HOT_TABLE_BYTES)) != cudaSuccess) return e;
+  if ((e = opt_in_smem((const void*)forced_kernel, (size_t)ADV_WARPS * ADV_WARP_WORDS * 4 + HOT_TABLE_BYTES)) != cudaSuccess) return e;
   if ((e = opt_in_smem((const void*)sweep_kernel, SWEEP_SMEM_LIMIT)) != cudaSuccess) return e;
   return configure_walk_kernels();
 }
@@ -948,6 +980,10 @@ void launch_intern_init(const StateDev& S, int32_t* init_state_dev, cudaStream_t
 void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const int32_t* init_state_dev, cudaStream_t st) {
   if (n == 0) return;
   reset_kernel<<<(n + 127) / 128, 128, 0, st>>>(S, rows_dev, n, init_state_dev);
+}
+void launch_forced(const GrammarDev& G, const StateDev& S, uint8_t* bytes_out, size_t stride, uint32_t* len_out,
+                   uint32_t max_len, cudaStream_t st) {
+  forced_kernel<<<(S.B + ADV_WARPS - 1) / ADV_WARPS, ADV_WARPS * 32, adv_smem_bytes(G), st>>>(G, S, bytes_out, stride, len_out, max_len);
 }
 void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st) {
   advance_kernel<<<(S.B + ADV_WARPS - 1) / ADV_WARPS, ADV_WARPS * 32, adv_smem_bytes(G), st>>>(G, S, tokens, status);

@@ -17,6 +17,8 @@ void launch_init(const GrammarDev& G, const StateDev& S, int32_t* result_dev, cu
 void launch_intern_init(const StateDev& S, int32_t* init_state_dev, cudaStream_t st);
 void launch_reset(const StateDev& S, const uint32_t* rows_dev, uint32_t n, const int32_t* init_state_dev, cudaStream_t st);
 void launch_advance(const GrammarDev& G, const StateDev& S, const int32_t* tokens, int32_t* status, cudaStream_t st);
+void launch_forced(const GrammarDev& G, const StateDev& S, uint8_t* bytes_out, size_t stride, uint32_t* len_out, uint32_t max_len,
+                   cudaStream_t st);
 void launch_plan(const GrammarDev& G, const StateDev& S, cudaStream_t st);
 void launch_publish(const StateDev& S, cudaStream_t st);
 cudaError_t configure_walk_kernels();

@@ -247,3 +247,74 @@ def test_a_wait_that_runs_out_gives_up_cleanly(roots):
         assert seqs[b].advance(bytes([c]))
     assert np.array_equal(_mask_of(st, g, 4), np.stack([s.mask(ov) for s in seqs]))
     assert st.stats()["capacity_errors"] == 0
+
+
+def _oracle_forced_run(seq, limit):
+    """Brute force on the oracle: while the text is not a sentence and exactly one of the 256 bytes
+    can follow, take it."""
+    run = []
+    s = seq.clone()
+    while len(run) < limit and not s.accepting:
+        ok = [b for b in range(256) if s.check(bytes([b]))]
+        if len(ok) != 1:
+            break
+        run.append(ok[0])
+        assert s.advance(bytes(ok))
+    return run
+
+
+def test_forced_bytes_equal_the_oracles_brute_force():
+    """Jump-ahead on the JSON-Schema workload (keys and punctuation are fixed by the schema): after
+    every step, each row's run equals the oracle's, found byte by byte over all 256 bytes; and the
+    run is the common prefix of every valid token's bytes."""
+    import paper_2506_01151_b200 as fmt
+
+    torch, dev = _torch()
+    w = workloads.build(3, V=6000, batch=6, steps=48)
+    g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
+    og, ov = oracle.Grammar(w.ebnf, w.start), oracle.Vocab(w.vocab, w.eos)
+    st = fmt.State(g, w.batch)
+    seqs = [oracle.Sequence_(og) for _ in range(w.batch)]
+    for p in range(w.prefix.shape[0]):
+        assert all(x == 0 for x in _advance(st, [int(x) for x in w.prefix[p]]))
+    for b in range(w.batch):
+        assert seqs[b].advance(w.prefix_bytes[b])
+    out = torch.full((w.batch, 32), 0xEE, dtype=torch.uint8, device=dev)
+    lens = torch.full((w.batch,), 99, dtype=torch.int32, device=dev)
+    longest, nonzero = 0, 0
+    for i in range(w.steps):
+        r = np.nonzero(w.reset_before[i])[0]
+        if len(r):
+            st.reset(torch.from_numpy(r.astype(np.int32)).to(dev))
+            for b in r:
+                seqs[int(b)] = oracle.Sequence_(og)
+        _advance(st, [int(x) for x in w.tokens[i]])
+        fin = [int(w.tokens[i, b]) == w.eos for b in range(w.batch)]
+        for b in range(w.batch):
+            t = int(w.tokens[i, b])
+            if t != w.eos and t >= 0:
+                assert seqs[b].advance(w.vocab[t])
+        before = [st.chart_words(b).tolist() for b in range(w.batch)]
+        out.fill_(0xEE)
+        st.forced_bytes(out, lens, 32)
+        got_len, got = lens.cpu().numpy(), out.cpu().numpy()
+        assert [st.chart_words(b).tolist() for b in range(w.batch)] == before  # the rows did not move
+        for b in range(w.batch):
+            if fin[b]:
+                assert got_len[b] == 0
+                continue
+            want = _oracle_forced_run(seqs[b], 32)
+            assert got[b, : got_len[b]].tolist() == want, (i, b, bytes(want))
+            assert (got[b, got_len[b]:] == 0xEE).all()
+            longest = max(longest, len(want))
+            nonzero += len(want) > 0
+            if want and i % 8 == 0:  # every valid token agrees with the run as far as both go
+                m = seqs[b].mask(ov)
+                for t in np.nonzero(oracle.bits(m, len(w.vocab)))[0][:200]:
+                    tb = w.vocab[int(t)]
+                    k = min(len(tb), len(want))
+                    assert list(tb[:k]) == want[:k], (i, b, tb)
+    assert longest >= 4 and nonzero >= 10  # key literals give real runs
+    # a shorter limit cuts the run, it does not change it
+    st.forced_bytes(out, lens, 3)
+    assert (lens.cpu().numpy() <= 3).all()
