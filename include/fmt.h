@@ -60,7 +60,15 @@ typedef struct fmt_state fmt_state;
 typedef struct {
   uint32_t host_only;        /* 1: build the tables on the host only (no device needed; the
                                 grammar can be inspected but no state can be created) */
-  uint32_t reserved[7];
+  uint32_t no_dfa_terminals; /* 1: keep every non-terminal as rules.  By default a non-terminal whose language is
+                                regular (everything it reaches recurses only at the right end, or only at the left
+                                end, of its rules - what `*` and `+` turn into) and that is used from a rule that
+                                is not, is compiled into one deterministic automaton over the bytes (Section 4.1:
+                                terminals as regular languages run as state machines): inside it an Earley item is
+                                "automaton state q, begun in set o", a byte is one table look-up, and Predict and
+                                Complete run only where the automaton begins and where it accepts.  The language
+                                and the masks are the same either way; pruned charts differ in their items */
+  uint32_t reserved[6];
 } fmt_compile_options;
 
 /* Options of fmt_state_create.  Zero-initialise; 0 means "default". */
@@ -104,6 +112,8 @@ typedef struct {
   uint32_t n_byte_classes;   /* bytes fall into this many classes that no grammar terminal tells apart */
   uint32_t n_empty_tokens;   /* tokens with no bytes (EOS included) */
   uint32_t start_nullable;   /* 1 if the empty string is a sentence */
+  uint32_t n_automata;       /* regular non-terminals that run as deterministic automata (Section 4.1) */
+  uint32_t n_automaton_states; /* their states, all together (each is one dotted-rule id, counted in n_dotted) */
 } fmt_grammar_info;
 
 typedef struct {
@@ -189,12 +199,23 @@ fmt_status fmt_compile_json_schema(const char* schema, size_t schema_len, const 
 fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out);
 
 /*
+ * Run automaton k (0 .. fmt_grammar_info.n_automata - 1; see fmt_compile_options.no_dfa_terminals) over
+ * `bytes` on the host, for inspection and tests: *accepted = 1 iff the bytes are a sentence of the regular
+ * non-terminal the automaton stands for, whose name (as in the grammar text; helper non-terminals made
+ * by `*`, `+`, `?` and groups carry a `~`) is copied to name_out, NUL-terminated, if name_out is not NULL.
+ */
+fmt_status fmt_grammar_automaton_match(const fmt_grammar* g, uint32_t k, const uint8_t* bytes, size_t len, int* accepted,
+                                       char* name_out, size_t name_cap);
+
+/*
  * Copy one host-side table of the compiled grammar, for inspection and tests.
  *   which: 0 trie child_off [T+1] u32   1 trie node_byte [T] u8    2 trie parent [T] u32
  *          3 trie tok_off [T+1] u32     4 trie tok_ids u32         5 level offsets [depth+2] u32
  *          6 nullable flags [N] u8      7 item info [D] u32        8 item lhs [D] u16
  *          9 tok_node [V] u32 (node where a token ends, 0xFFFFFFFF if it has no bytes)
  *         10 byte class of each byte [256] u8
+ *         11 automata: transitions [states][byte classes] u16 (target state | 0x4000 target has transitions |
+ *            0x8000 target accepts, 0xFFFF none)   12 accepting flag per state u8   13 start state per automaton u32
  * Writes min(cap_bytes, size) bytes to `out` (may be NULL) and the full size to *size_bytes.
  */
 fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, size_t cap_bytes, size_t* size_bytes);

@@ -20,7 +20,7 @@ ERR_OOM, ERR_CUDA, ERR_CAPACITY, ERR_TOKEN_REJECTED, ERR_FINISHED = 5, 6, 7, 8, 
 BF16, FP32 = 0, 1
 
 EXPORTS = [
-    "fmt_compile", "fmt_json_schema_to_ebnf", "fmt_compile_json_schema", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table",
+    "fmt_compile", "fmt_json_schema_to_ebnf", "fmt_compile_json_schema", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table", "fmt_grammar_automaton_match",
     "fmt_state_create", "fmt_state_destroy", "fmt_state_reset", "fmt_state_advance", "fmt_state_forced_bytes", "fmt_fill_mask",
     "fmt_apply_mask", "fmt_fill_and_apply", "fmt_state_cache_clear", "fmt_state_ci_cache_clear", "fmt_state_set_wait_limit", "fmt_state_copy_counters", "fmt_state_query", "fmt_state_copy_chart", "fmt_get_stats",
     "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_fill_mask_noalloc", "fmt_last_error",
@@ -34,7 +34,7 @@ class FmtError(RuntimeError):
 
 
 class CompileOptions(C.Structure):
-    _fields_ = [("host_only", C.c_uint32), ("reserved", C.c_uint32 * 7)]
+    _fields_ = [("host_only", C.c_uint32), ("no_dfa_terminals", C.c_uint32), ("reserved", C.c_uint32 * 6)]
 
 
 class StateOptions(C.Structure):
@@ -49,7 +49,7 @@ class StateOptions(C.Structure):
 class GrammarInfo(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in (
         "n_nonterminals", "n_rules", "n_dotted", "n_classes", "n_nullable", "vocab_size", "mask_words",
-        "trie_nodes", "trie_depth", "n_byte_classes", "n_empty_tokens", "start_nullable")]
+        "trie_nodes", "trie_depth", "n_byte_classes", "n_empty_tokens", "start_nullable", "n_automata", "n_automaton_states")]
 
 
 class Stats(C.Structure):
@@ -87,6 +87,7 @@ def lib():
         L.fmt_grammar_destroy.restype = None
         L.fmt_grammar_get_info.argtypes = [vp, C.POINTER(GrammarInfo)]
         L.fmt_grammar_copy_table.argtypes = [vp, C.c_int, vp, sz, C.POINTER(sz)]
+        L.fmt_grammar_automaton_match.argtypes = [vp, u32, C.c_char_p, sz, C.POINTER(C.c_int), C.c_char_p, sz]
         L.fmt_state_create.argtypes = [vp, u32, C.POINTER(StateOptions), vp, C.POINTER(vp)]
         L.fmt_state_destroy.argtypes = [vp]
         L.fmt_state_destroy.restype = None
@@ -129,7 +130,7 @@ def _ptr(x) -> Optional[int]:
 
 
 _TABLE_DTYPES = {0: np.uint32, 1: np.uint8, 2: np.uint32, 3: np.uint32, 4: np.uint32, 5: np.uint32, 6: np.uint8,
-                 7: np.uint32, 8: np.uint16, 9: np.uint32, 10: np.uint8}
+                 7: np.uint32, 8: np.uint16, 9: np.uint32, 10: np.uint8, 11: np.uint16, 12: np.uint8, 13: np.uint32}
 
 
 def json_schema_to_ebnf(schema) -> str:
@@ -146,7 +147,7 @@ class Grammar:
     """fmt_compile: grammar text + vocabulary -> device tables and byte trie."""
 
     @classmethod
-    def from_json_schema(cls, schema, vocab: Sequence[bytes], eos: int = -1, host_only: bool = False) -> "Grammar":
+    def from_json_schema(cls, schema, vocab: Sequence[bytes], eos: int = -1, host_only: bool = False, dfa: bool = True) -> "Grammar":
         """fmt_compile_json_schema: the instances of a JSON schema as the grammar."""
         self = cls.__new__(cls)
         src = schema.encode("utf-8") if isinstance(schema, str) else bytes(schema)
@@ -155,6 +156,7 @@ class Grammar:
         blob = np.frombuffer(b"".join(vocab) + b"\0", dtype=np.uint8).copy()
         opt = CompileOptions()
         opt.host_only = 1 if host_only else 0
+        opt.no_dfa_terminals = 0 if dfa else 1
         h = C.c_void_p()
         _check(lib().fmt_compile_json_schema(src, len(src), blob.ctypes.data, offs.ctypes.data, len(vocab), eos,
                                              C.byref(opt), C.byref(h)))
@@ -164,13 +166,14 @@ class Grammar:
         self.mask_words = (self.V + 31) // 32
         return self
 
-    def __init__(self, ebnf, start: str, vocab: Sequence[bytes], eos: int = -1, host_only: bool = False):
+    def __init__(self, ebnf, start: str, vocab: Sequence[bytes], eos: int = -1, host_only: bool = False, dfa: bool = True):
         src = ebnf.encode("latin-1") if isinstance(ebnf, str) else bytes(ebnf)
         offs = np.zeros(len(vocab) + 1, dtype=np.uint64)
         offs[1:] = np.cumsum([len(t) for t in vocab], dtype=np.uint64)
         blob = np.frombuffer(b"".join(vocab) + b"\0", dtype=np.uint8).copy()
         opt = CompileOptions()
         opt.host_only = 1 if host_only else 0
+        opt.no_dfa_terminals = 0 if dfa else 1
         h = C.c_void_p()
         _check(lib().fmt_compile(src, len(src), start.encode(), blob.ctypes.data, offs.ctypes.data, len(vocab), eos,
                                  C.byref(opt), C.byref(h)))
@@ -190,6 +193,18 @@ class Grammar:
         out = GrammarInfo()
         _check(lib().fmt_grammar_get_info(self._h, C.byref(out)))
         return out
+
+    def automaton_name(self, k: int) -> str:
+        name = C.create_string_buffer(256)
+        acc = C.c_int()
+        _check(lib().fmt_grammar_automaton_match(self._h, k, b"", 0, C.byref(acc), name, 256))
+        return name.value.decode("latin-1")
+
+    def automaton_accepts(self, k: int, data: bytes) -> bool:
+        """fmt_grammar_automaton_match: is `data` a sentence of the regular non-terminal automaton k stands for?"""
+        acc = C.c_int()
+        _check(lib().fmt_grammar_automaton_match(self._h, k, bytes(data), len(data), C.byref(acc), None, 0))
+        return bool(acc.value)
 
     def table(self, which: int) -> np.ndarray:
         n = C.c_size_t()

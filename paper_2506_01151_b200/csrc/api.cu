@@ -168,7 +168,7 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
   fmt_grammar* g = new (std::nothrow) fmt_grammar;
   if (!g) return fail(FMT_ERR_OOM, "out of host memory");
   try {
-    compile_grammar(ebnf, ebnf_len, start_rule, g->host);
+    compile_grammar(ebnf, ebnf_len, start_rule, g->host, !(opt && opt->no_dfa_terminals));
     static const uint8_t none = 0;
     build_trie(vocab_bytes ? vocab_bytes : &none, vocab_offsets, V, eos_token_id, g->host);
     if (eos_token_id >= 0 && vocab_offsets[eos_token_id + 1] != vocab_offsets[eos_token_id])
@@ -213,6 +213,12 @@ fmt_status fmt_compile(const char* ebnf, size_t ebnf_len, const char* start_rule
       d.nt_closure = d.hot_block + o_clo;
       d.direct_off = d.hot_block + o_doff;
       d.direct_items = reinterpret_cast<const uint16_t*>(d.hot_block + o_dit);
+    }
+    d.dfa_first = h.dfa_first;
+    if (h.dfa_states) {
+      UP(dfa_trans);
+      UP(dfa_done);
+      UP(dfa_scan);
     }
     UP(node_byte);
     UP(parent);
@@ -284,6 +290,30 @@ fmt_status fmt_grammar_get_info(const fmt_grammar* g, fmt_grammar_info* out) {
   out->n_byte_classes = h.n_eq;
   out->n_empty_tokens = h.n_empty;
   out->start_nullable = h.start_nullable ? 1u : 0u;
+  out->n_automata = (uint32_t)h.dfa_nt.size();
+  out->n_automaton_states = h.dfa_states;
+  return FMT_OK;
+}
+
+fmt_status fmt_grammar_automaton_match(const fmt_grammar* g, uint32_t k, const uint8_t* bytes, size_t len, int* accepted,
+                                       char* name_out, size_t name_cap) {
+  if (!g || !accepted || (!bytes && len)) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
+  const HostTables& h = g->host;
+  if (k >= h.dfa_nt.size()) return fail(FMT_ERR_INVALID_ARG, "no such automaton");
+  if (name_out && name_cap) {
+    const std::string& nm = h.nt_names[h.dfa_nt[k]];
+    const size_t n = std::min(nm.size(), name_cap - 1);
+    memcpy(name_out, nm.data(), n);
+    name_out[n] = 0;
+  }
+  uint32_t q = h.dfa_start[k];
+  *accepted = 0;
+  for (size_t i = 0; i < len; ++i) {
+    const uint16_t t = h.dfa_trans[(size_t)q * h.n_eq + h.eq_of_byte[bytes[i]]];
+    if (t == 0xFFFFu) return FMT_OK;
+    q = t & 0x3FFFu;
+  }
+  *accepted = h.dfa_accept[q] ? 1 : 0;
   return FMT_OK;
 }
 
@@ -304,6 +334,9 @@ fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, si
     case 8: src = h.lhs.data(), n = (size_t)h.D * 2; break;
     case 9: src = h.tok_node.data(), n = h.tok_node.size() * 4; break;
     case 10: src = h.eq_of_byte.data(), n = 256; break;
+    case 11: src = h.dfa_trans.data(), n = h.dfa_trans.size() * 2; break;
+    case 12: src = h.dfa_accept.data(), n = h.dfa_accept.size(); break;
+    case 13: src = h.dfa_start.data(), n = h.dfa_start.size() * 4; break;
     default: return fail(FMT_ERR_INVALID_ARG, "unknown table");
   }
   *size_bytes = n;

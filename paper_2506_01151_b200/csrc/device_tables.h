@@ -17,6 +17,11 @@ struct GrammarDev {
   const uint32_t* nt_closure;    // [N][Nw]
   const uint32_t* direct_off;    // [N+1]
   const uint16_t* direct_items;
+  // regular non-terminals run as automata: item id dfa_first + g is automaton state g
+  uint32_t dfa_first;
+  const uint16_t* dfa_trans;     // [states][n_eq] target | 0x4000 target has transitions | 0x8000 target accepts, or 0xFFFF
+  const uint16_t* dfa_done;      // [states] completed item of the state's non-terminal
+  const uint32_t* dfa_scan;      // [states][8] bytes with a transition
   const uint8_t* node_byte;      // [T]
   const uint32_t* parent;        // [T]
   const uint8_t* node_depth;     // [T]

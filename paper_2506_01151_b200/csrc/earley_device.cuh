@@ -99,6 +99,34 @@ __device__ __forceinline__ bool class_has(const GrammarDev& G, uint32_t cls, uin
   return (G.class_bits[cls * 8u + (byte >> 5)] >> (byte & 31u)) & 1u;
 }
 
+// What scanning `byte` makes of item `it` (Section 3.2's Scan; `inf` = its info word): up to two items.
+// An item before a terminal that matches moves its dot.  An item inside an automaton (a regular
+// non-terminal, Section 4.1) follows the automaton's transition: it becomes the next state's item if that
+// state has transitions of its own, and the completed item of the non-terminal if that state accepts (a
+// state that accepts and leads nowhere is thus never an item: a finished automaton is dropped at once).
+struct Scanned {
+  uint32_t a, b;   // the items (valid if has_a / has_b)
+  bool has_a, has_b;
+};
+__device__ __forceinline__ Scanned scan_item(const GrammarDev& G, uint32_t it, uint32_t inf, uint32_t byte) {
+  Scanned r{0u, 0u, false, false};
+  const uint32_t kind = inf >> INFO_KIND_SHIFT;
+  if (kind == KIND_TERM) {
+    r.has_a = class_has(G, inf & INFO_ARG_MASK, byte);
+    r.a = it + 1u;
+  } else if (kind == KIND_DFA) {
+    const uint32_t g = inf & INFO_ARG_MASK;
+    const uint32_t t = __ldg(&G.dfa_trans[(size_t)g * G.n_eq + G.eq_of_byte[byte]]);
+    if (t != 0xFFFFu) {
+      r.has_a = (t & 0x4000u) != 0u;
+      r.a = (it & 0xFFFF0000u) | (G.dfa_first + (t & 0x3FFFu));
+      r.has_b = (t & 0x8000u) != 0u;
+      r.b = (it & 0xFFFF0000u) | __ldg(&G.dfa_done[g]);
+    }
+  }
+  return r;
+}
+
 // Scan (Section 3.2): items of `set` whose post-dot terminal matches `byte`, dot advanced, go
 // into cur.  Returns the number of items in cur afterwards (uniform over the warp).
 __device__ __forceinline__ uint32_t scan_into_cur(const GrammarDev& G, const WarpCtx& w, const uint32_t* set,
@@ -106,7 +134,9 @@ __device__ __forceinline__ uint32_t scan_into_cur(const GrammarDev& G, const War
   for (uint32_t k = lane_id(); k < len; k += 32) {
     uint32_t it = set[k];
     uint32_t inf = G.info[it & 0xFFFFu];
-    if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) add_item(G, w, it + 1u);
+    const Scanned sc = scan_item(G, it, inf, byte);
+    if (sc.has_a) add_item(G, w, sc.a);
+    if (sc.has_b) add_item(G, w, sc.b);
   }
   __syncwarp();
   return min(w.ctr[W_NCUR], w.cur_cap);
@@ -291,11 +321,13 @@ __device__ __forceinline__ uint32_t small_scan_complete(const GrammarDev& G, con
   for (uint32_t base = 0; base < len; base += 32) {
     const uint32_t k = base + lane;
     uint32_t it = k < len ? set[k] : 0u;
-    const uint32_t inf = k < len ? G.info[it & 0xFFFFu] : 0u;
-    const bool hit = (inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte);
+    const uint32_t inf = k < len ? G.info[it & 0xFFFFu] : 0u;  // (info word 0 is a non-terminal item: scans nothing)
     it = rename(it);
-    const uint32_t skip = hit ? (G.info[(it + 1u) & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
-    if (__any_sync(FULL, hit)) n = append_small(it + 1u, hit, skip, n, mine);
+    const Scanned sc = scan_item(G, it, k < len ? inf : (KIND_NT << INFO_KIND_SHIFT), byte);
+    const uint32_t skip_a = sc.has_a ? (G.info[sc.a & 0xFFFFu] >> INFO_SKIP_SHIFT) & INFO_SKIP_MASK : 0u;
+    if (__any_sync(FULL, sc.has_a)) n = append_small(sc.a, sc.has_a, skip_a, n, mine);
+    if (n > 32u) return SMALL_OVERFLOW;
+    if (__any_sync(FULL, sc.has_b)) n = append_small(sc.b, sc.has_b, 0u, n, mine);  // (a completed item has nothing to skip)
     if (n > 32u) return SMALL_OVERFLOW;
   }
   if (n == 0) return 0;
@@ -395,8 +427,10 @@ __device__ __forceinline__ void scannable_bytes(const GrammarDev& G, const uint3
   for (int i = 0; i < 8; ++i) acc[i] = 0u;
   for (uint32_t k = lane_id(); k < len; k += 32) {
     uint32_t inf = G.info[set[k] & 0xFFFFu];
-    if ((inf >> INFO_KIND_SHIFT) == KIND_TERM) {
-      const uint4* p = reinterpret_cast<const uint4*>(G.class_bits + (inf & INFO_ARG_MASK) * 8u);
+    const uint32_t kind = inf >> INFO_KIND_SHIFT;
+    if (kind == KIND_TERM || kind == KIND_DFA) {
+      const uint4* p = reinterpret_cast<const uint4*>(kind == KIND_TERM ? G.class_bits + (inf & INFO_ARG_MASK) * 8u
+                                                                        : G.dfa_scan + (size_t)(inf & INFO_ARG_MASK) * 8u);
       uint4 a = p[0], b = p[1];
       acc[0] |= a.x, acc[1] |= a.y, acc[2] |= a.z, acc[3] |= a.w;
       acc[4] |= b.x, acc[5] |= b.y, acc[6] |= b.z, acc[7] |= b.w;

@@ -325,11 +325,304 @@ class Parser {
   }
 };
 
+// ------------------------------------------------------------------------------------ regular non-terminals -> DFAs
+//
+// Section 4.1 models terminals as regular languages run as finite-state machines inside the chart.
+// Here the grammar text has no separate lexical level, so the regular parts are found: a
+// non-terminal is regular when, in everything it can reach, recursion is only ever at the right end
+// of a rule or only ever at the left end (within each group of mutually recursive non-terminals;
+// `*` and `+` are desugared into exactly such rules).  A regular non-terminal that is used from a
+// non-regular rule becomes one deterministic automaton over the byte classes; the Earley items inside
+// it are "automaton state q, started in set o" and a byte costs one table look-up, with no Predict and
+// no Complete until the automaton accepts (then it completes like any non-terminal).
+
+struct Nfa {
+  std::vector<std::vector<int>> eps;
+  std::vector<std::vector<std::pair<int, int>>> edge;  // (byte class, target)
+  int add() {
+    eps.emplace_back();
+    edge.emplace_back();
+    return (int)eps.size() - 1;
+  }
+};
+
+struct OneDfa {
+  int nt = -1;                       // the non-terminal it stands for (builder numbering)
+  uint32_t n_states = 0;             // state 0 is the start state
+  std::vector<int> trans;            // [n_states][n_eq] target state or -1
+  std::vector<char> accepting;       // [n_states]
+};
+
+struct RegularInfo {
+  std::vector<int> scc_of;           // per non-terminal
+  std::vector<std::vector<int>> scc_members;
+  std::vector<int> scc_kind;         // 0 not regular, 1 no recursion, 2 right-linear, 3 left-linear
+  std::vector<char> regular;         // per non-terminal
+};
+
+constexpr size_t NFA_STATE_CAP = 60000, DFA_STATE_CAP = 6000;
+
+class DfaBuilder {
+ public:
+  DfaBuilder(const std::vector<Production>& rules, size_t n_nt, const std::vector<Bits256>& classes,
+             const std::vector<uint8_t>& eq_of_byte, uint32_t n_eq)
+      : rules_(rules), n_nt_(n_nt), classes_(classes), n_eq_(n_eq) {
+    by_lhs_.resize(n_nt);
+    for (size_t i = 0; i < rules.size(); ++i) by_lhs_[rules[i].lhs].push_back((int)i);
+    rep_.assign(n_eq, 0);
+    for (int b = 255; b >= 0; --b) rep_[eq_of_byte[b]] = (uint8_t)b;
+    classify();
+  }
+  const RegularInfo& info() const { return info_; }
+
+  // The automaton of regular non-terminal x, minimised; false if it outgrows the caps.
+  bool build(int x, OneDfa& out) {
+    Nfa n;
+    too_big_ = false;
+    const int s = n.add(), t = n.add();
+    instantiate(n, x, s, t);
+    if (too_big_) return false;
+    return determinise(n, s, t, out) && (out.nt = x, true);
+  }
+
+ private:
+  const std::vector<Production>& rules_;
+  size_t n_nt_;
+  const std::vector<Bits256>& classes_;
+  uint32_t n_eq_;
+  std::vector<std::vector<int>> by_lhs_;
+  std::vector<uint8_t> rep_;  // one byte of every equivalence class
+  RegularInfo info_;
+  bool too_big_ = false;
+
+  // ---- strongly connected components of "A uses B" (Tarjan, iterative enough for grammar sizes: recursion depth = chain length)
+  void classify() {
+    const int n = (int)n_nt_;
+    info_.scc_of.assign(n, -1);
+    std::vector<int> index(n, -1), low(n, 0), stack;
+    std::vector<char> on(n, 0);
+    int counter = 0;
+    struct Frame {
+      int v;
+      size_t rule, sym;
+    };
+    for (int root = 0; root < n; ++root) {
+      if (index[root] >= 0 || by_lhs_[root].empty()) continue;
+      std::vector<Frame> call{{root, 0, 0}};
+      index[root] = low[root] = counter++;
+      stack.push_back(root), on[root] = 1;
+      while (!call.empty()) {
+        Frame& f = call.back();
+        bool descended = false;
+        while (f.rule < by_lhs_[f.v].size() && !descended) {
+          const Production& p = rules_[by_lhs_[f.v][f.rule]];
+          while (f.sym < p.rhs.size()) {
+            const int w = p.rhs[f.sym++];
+            if (w < 0 || by_lhs_[w].empty()) continue;
+            if (index[w] < 0) {
+              index[w] = low[w] = counter++;
+              stack.push_back(w), on[w] = 1;
+              call.push_back({w, 0, 0});
+              descended = true;
+              break;
+            }
+            if (on[w]) low[f.v] = std::min(low[f.v], index[w]);
+          }
+          if (!descended) ++f.rule, f.sym = 0;
+        }
+        if (descended) continue;
+        const int v = f.v;
+        call.pop_back();
+        if (!call.empty()) low[call.back().v] = std::min(low[call.back().v], low[v]);
+        if (low[v] == index[v]) {
+          const int id = (int)info_.scc_members.size();
+          info_.scc_members.emplace_back();
+          for (;;) {
+            const int w = stack.back();
+            stack.pop_back(), on[w] = 0;
+            info_.scc_of[w] = id;
+            info_.scc_members[id].push_back(w);
+            if (w == v) break;
+          }
+        }
+      }
+    }
+    // components come out callees first: a component's kind and whether all it uses is regular
+    const int m = (int)info_.scc_members.size();
+    info_.scc_kind.assign(m, 0);
+    info_.regular.assign(n, 0);
+    for (int c = 0; c < m; ++c) {
+      bool right_ok = true, left_ok = true, recursive = false, uses_ok = true;
+      for (int a : info_.scc_members[c])
+        for (int r : by_lhs_[a]) {
+          const Production& p = rules_[r];
+          int inside = 0;
+          for (size_t k = 0; k < p.rhs.size(); ++k) {
+            const int w = p.rhs[k];
+            if (w < 0) continue;
+            if (info_.scc_of[w] == c) {
+              ++inside;
+              if (k + 1 != p.rhs.size()) right_ok = false;
+              if (k != 0) left_ok = false;
+            } else if (!info_.regular[w]) {
+              uses_ok = false;
+            }
+          }
+          if (inside) recursive = true;
+          if (inside > 1) right_ok = left_ok = false;
+        }
+      int kind = 0;
+      if (uses_ok) kind = !recursive ? 1 : right_ok ? 2 : left_ok ? 3 : 0;
+      info_.scc_kind[c] = kind;
+      for (int a : info_.scc_members[c]) info_.regular[a] = kind != 0;
+    }
+  }
+
+  // ---- Thompson-style construction: non-terminal x between NFA states `from` and `to`
+  void chain(Nfa& n, int a, const std::vector<int>& syms, size_t lo, size_t hi, int b) {
+    if (too_big_) return;
+    if (lo == hi) {
+      n.eps[a].push_back(b);
+      return;
+    }
+    int cur = a;
+    for (size_t k = lo; k < hi; ++k) {
+      const int nxt = (k + 1 == hi) ? b : n.add();
+      if (syms[k] < 0) n.edge[cur].push_back({~syms[k], nxt});
+      else instantiate(n, syms[k], cur, nxt);
+      cur = nxt;
+    }
+  }
+  void instantiate(Nfa& n, int x, int from, int to) {
+    if (n.eps.size() > NFA_STATE_CAP) too_big_ = true;
+    if (too_big_) return;
+    const int c = info_.scc_of[x];
+    const int kind = info_.scc_kind[c];
+    if (kind == 1) {
+      for (int r : by_lhs_[x]) chain(n, from, rules_[r].rhs, 0, rules_[r].rhs.size(), to);
+      return;
+    }
+    // one NFA state per member of the component, private to this instance
+    std::map<int, int> st;
+    for (int a : info_.scc_members[c]) st[a] = n.add();
+    if (kind == 2) {  // right-linear: state of A = "an A is about to start"; whoever ends, ends the instance
+      n.eps[from].push_back(st[x]);
+      for (int a : info_.scc_members[c])
+        for (int r : by_lhs_[a]) {
+          const std::vector<int>& rhs = rules_[r].rhs;
+          const bool tail = !rhs.empty() && rhs.back() >= 0 && info_.scc_of[rhs.back()] == c;
+          if (tail) chain(n, st[a], rhs, 0, rhs.size() - 1, st[rhs.back()]);
+          else chain(n, st[a], rhs, 0, rhs.size(), to);
+        }
+    } else {  // left-linear: state of A = "an A has just ended"
+      n.eps[st[x]].push_back(to);
+      for (int a : info_.scc_members[c])
+        for (int r : by_lhs_[a]) {
+          const std::vector<int>& rhs = rules_[r].rhs;
+          const bool head = !rhs.empty() && rhs.front() >= 0 && info_.scc_of[rhs.front()] == c;
+          if (head) chain(n, st[rhs.front()], rhs, 1, rhs.size(), st[a]);
+          else chain(n, from, rhs, 0, rhs.size(), st[a]);
+        }
+    }
+  }
+
+  // ---- subset construction over the byte equivalence classes, then Moore minimisation
+  bool determinise(const Nfa& n, int start, int final_state, OneDfa& out) {
+    const size_t C = classes_.size();
+    std::vector<std::vector<char>> has(C);  // has[c][e]: class c contains the bytes of equivalence class e
+    auto closure = [&](std::vector<int>& set) {
+      std::vector<int> work = set;
+      std::vector<char> in(n.eps.size(), 0);
+      for (int s : set) in[s] = 1;
+      while (!work.empty()) {
+        const int s = work.back();
+        work.pop_back();
+        for (int t : n.eps[s])
+          if (!in[t]) in[t] = 1, set.push_back(t), work.push_back(t);
+      }
+      std::sort(set.begin(), set.end());
+    };
+    std::map<std::vector<int>, int> ids;
+    std::vector<std::vector<int>> sets;
+    std::vector<int> first{start};
+    closure(first);
+    ids[first] = 0;
+    sets.push_back(first);
+    std::vector<int> trans;
+    for (size_t q = 0; q < sets.size(); ++q) {
+      trans.resize((q + 1) * n_eq_, -1);
+      for (uint32_t e = 0; e < n_eq_; ++e) {
+        const uint32_t byte = rep_[e];
+        std::vector<int> next;
+        for (int s : sets[q])
+          for (auto& ed : n.edge[s]) {
+            const int c = ed.first;
+            if ((classes_[c][byte >> 5] >> (byte & 31)) & 1u) next.push_back(ed.second);
+          }
+        if (next.empty()) continue;
+        std::sort(next.begin(), next.end());
+        next.erase(std::unique(next.begin(), next.end()), next.end());
+        closure(next);
+        auto it = ids.find(next);
+        if (it == ids.end()) {
+          if (sets.size() >= DFA_STATE_CAP) return false;
+          it = ids.emplace(next, (int)sets.size()).first;
+          sets.push_back(next);
+        }
+        trans[q * n_eq_ + e] = it->second;
+      }
+    }
+    (void)has;
+    const size_t S = sets.size();
+    std::vector<char> acc(S, 0);
+    for (size_t q = 0; q < S; ++q) acc[q] = std::binary_search(sets[q].begin(), sets[q].end(), final_state);
+    // Moore: split blocks until every block's members agree on the block of every successor
+    std::vector<int> block(S);
+    for (size_t q = 0; q < S; ++q) block[q] = acc[q];
+    for (size_t n_blocks = 0;;) {
+      std::map<std::vector<int>, int> sig_ids;
+      std::vector<int> nb(S);
+      for (size_t q = 0; q < S; ++q) {
+        std::vector<int> sig(n_eq_ + 1);
+        sig[0] = block[q];
+        for (uint32_t e = 0; e < n_eq_; ++e) sig[e + 1] = trans[q * n_eq_ + e] < 0 ? -1 : block[trans[q * n_eq_ + e]];
+        auto it = sig_ids.find(sig);
+        if (it == sig_ids.end()) it = sig_ids.emplace(std::move(sig), (int)sig_ids.size()).first;
+        nb[q] = it->second;
+      }
+      block.swap(nb);
+      if (sig_ids.size() == n_blocks) break;
+      n_blocks = sig_ids.size();
+    }
+    // number the blocks from the start state's, in order of discovery
+    std::vector<int> new_id(S, -1), order;
+    std::vector<int> block_id(S, -1);  // block -> new id
+    auto take = [&](int q) {
+      if (block_id[block[q]] < 0) block_id[block[q]] = (int)order.size(), order.push_back(q);
+    };
+    take(0);
+    for (size_t i = 0; i < order.size(); ++i)
+      for (uint32_t e = 0; e < n_eq_; ++e)
+        if (trans[(size_t)order[i] * n_eq_ + e] >= 0) take(trans[(size_t)order[i] * n_eq_ + e]);
+    out.n_states = (uint32_t)order.size();
+    out.trans.assign((size_t)out.n_states * n_eq_, -1);
+    out.accepting.assign(out.n_states, 0);
+    for (size_t i = 0; i < order.size(); ++i) {
+      out.accepting[i] = acc[order[i]];
+      for (uint32_t e = 0; e < n_eq_; ++e) {
+        const int t = trans[(size_t)order[i] * n_eq_ + e];
+        out.trans[i * n_eq_ + e] = t < 0 ? -1 : block_id[block[t]];
+      }
+    }
+    return true;
+  }
+};
+
 }  // namespace
 
 // ------------------------------------------------------------------------------------ tables
 
-void compile_grammar(const char* text, size_t len, const std::string& start, HostTables& out) {
+void compile_grammar(const char* text, size_t len, const std::string& start, HostTables& out, bool dfa_terminals) {
   GrammarBuilder b;
   int aug = b.nt("$");
   b.defined[aug] = 1;
@@ -387,12 +680,74 @@ void compile_grammar(const char* text, size_t len, const std::string& start, Hos
       if (ok) nullable[p.lhs] = 1, again = true;
     }
   }
+  // bytes are equivalent when every byte class of the grammar contains both or neither
+  out.eq_of_byte.assign(256, 0);
+  {
+    std::vector<char> used(b.classes.size(), 0);
+    for (auto& p : rules)
+      for (int s : p.rhs)
+        if (s < 0) used[~s] = 1;
+    std::map<std::vector<uint8_t>, uint32_t> seen;
+    for (int byte = 0; byte < 256; ++byte) {
+      std::vector<uint8_t> member;
+      for (size_t c = 0; c < b.classes.size(); ++c)
+        if (used[c]) member.push_back((b.classes[c][byte >> 5] >> (byte & 31)) & 1u);
+      auto it = seen.find(member);
+      if (it == seen.end()) it = seen.emplace(member, (uint32_t)seen.size()).first;
+      out.eq_of_byte[byte] = (uint8_t)it->second;
+    }
+    out.n_eq = (uint32_t)seen.size();
+  }
+  // regular non-terminals used from non-regular rules become automata (see DfaBuilder)
+  std::vector<OneDfa> dfas;
+  std::vector<int> dfa_of(n_all, -1);
+  if (dfa_terminals) {
+    DfaBuilder db(rules, n_all, b.classes, out.eq_of_byte, out.n_eq);
+    const RegularInfo& ri = db.info();
+    std::vector<char> wanted(n_all, 0);
+    for (auto& p : rules)
+      if (p.lhs == aug || !ri.regular[p.lhs])
+        for (int s : p.rhs)
+          if (s >= 0 && s != aug && ri.regular[s]) wanted[s] = 1;
+    size_t total_states = 0;
+    for (size_t x = 0; x < n_all; ++x) {
+      if (!wanted[x]) continue;
+      OneDfa one;
+      if (!db.build((int)x, one)) continue;                        // too large: stays a set of rules
+      if (total_states + one.n_states > 16000) continue;           // (state numbers have 14 bits)
+      total_states += one.n_states;
+      dfa_of[x] = (int)dfas.size();
+      dfas.push_back(std::move(one));
+    }
+    if (!dfas.empty()) {  // their rules go, and with them whatever only they used
+      std::vector<Production> left;
+      for (auto& p : rules)
+        if (dfa_of[p.lhs] < 0) left.push_back(p);
+      std::vector<char> r2(n_all, 0);
+      r2[aug] = 1;
+      for (bool again = true; again;) {
+        again = false;
+        for (auto& p : left)
+          if (r2[p.lhs])
+            for (int s : p.rhs)
+              if (s >= 0 && !r2[s]) r2[s] = 1, again = dfa_of[s] < 0 || again;
+      }
+      rules.clear();
+      for (auto& p : left)
+        if (r2[p.lhs]) rules.push_back(p);
+      for (size_t x = 0; x < n_all; ++x)
+        if (dfa_of[x] >= 0 && !r2[x]) dfa_of[x] = -2;  // (built but no longer used: cannot happen, kept for safety)
+    }
+  }
   // renumber non-terminals ($ = 0) and byte classes (only those still used)
   std::vector<int> nt_new(n_all, -1);
   int N = 0;
   nt_new[aug] = N++;
   for (auto& p : rules)
     if (nt_new[p.lhs] < 0) nt_new[p.lhs] = N++;
+  for (auto& p : rules)
+    for (int s : p.rhs)
+      if (s >= 0 && nt_new[s] < 0) nt_new[s] = N++;  // (non-terminals that are automata have no rules)
   std::vector<int> cls_new(b.classes.size(), -1);
   int C = 0;
   for (auto& p : rules)
@@ -404,6 +759,14 @@ void compile_grammar(const char* text, size_t len, const std::string& start, Hos
     if (!p.rhs.empty()) solid.push_back(p);
   size_t D = 0;
   for (auto& p : solid) D += p.rhs.size() + 1;
+  // after the rule positions: one item id per automaton state, then one "done" id per automaton
+  const size_t D_rules = D;
+  size_t S_total = 0;
+  std::vector<int> used_dfas;
+  for (size_t x = 0; x < n_all; ++x)
+    if (dfa_of[x] >= 0) used_dfas.push_back((int)x);
+  for (int x : used_dfas) S_total += dfas[dfa_of[x]].n_states;
+  D += S_total + used_dfas.size();
   if (D > 65535 || N > (int)MAX_NONTERMINALS || C > 65535)
     throw CompileError{FMT_ERR_CAPACITY, "grammar too large: more than 65535 dotted rules or classes, or 4096 non-terminals"};
 
@@ -427,24 +790,51 @@ void compile_grammar(const char* text, size_t len, const std::string& start, Hos
     if (cls_new[c] >= 0)
       for (int w = 0; w < 8; ++w) out.class_bits[(size_t)cls_new[c] * 8 + w] = b.classes[c][w];
 
-  // bytes are equivalent when every byte class contains both or neither: they scan the same items
-  {
-    std::map<std::vector<uint8_t>, uint32_t> seen;
-    out.eq_of_byte.assign(256, 0);
-    for (int byte = 0; byte < 256; ++byte) {
-      std::vector<uint8_t> member((size_t)C);
-      for (int c = 0; c < C; ++c) member[c] = (out.class_bits[(size_t)c * 8 + (byte >> 5)] >> (byte & 31)) & 1u;
-      auto it = seen.find(member);
-      if (it == seen.end()) it = seen.emplace(member, (uint32_t)seen.size()).first;
-      out.eq_of_byte[byte] = (uint8_t)it->second;
-    }
-    out.n_eq = (uint32_t)seen.size();
-  }
-
   out.info.assign(D, 0);
   out.lhs.assign(D, 0);
   out.skip.assign(D, 0);
   std::vector<std::vector<uint32_t>> first_item(N);  // start item of each rule, per non-terminal
+  // the automata: item id dfa_first + g is "state g" (all automata's states numbered in a row), the ids
+  // after them are the completed items of the non-terminals they stand for
+  out.dfa_first = (uint32_t)D_rules;
+  out.dfa_states = (uint32_t)S_total;
+  out.dfa_trans.assign(S_total * out.n_eq, 0xFFFFu);
+  out.dfa_done.assign(S_total, 0);
+  out.dfa_scan.assign(S_total * 8, 0);
+  out.dfa_accept.assign(S_total, 0);
+  out.dfa_nt.clear();
+  out.dfa_start.clear();
+  {
+    uint32_t g0 = 0;
+    for (size_t j = 0; j < used_dfas.size(); ++j) {
+      const OneDfa& a = dfas[dfa_of[used_dfas[j]]];
+      const int L = nt_new[used_dfas[j]];
+      const uint32_t done_id = (uint32_t)(D_rules + S_total + j);
+      out.dfa_nt.push_back((uint32_t)L);
+      out.dfa_start.push_back(g0);
+      first_item[L].push_back(out.dfa_first + g0);
+      out.info[done_id] = (KIND_END << INFO_KIND_SHIFT) | (uint32_t)L;
+      out.lhs[done_id] = (uint16_t)L;
+      for (uint32_t q = 0; q < a.n_states; ++q) {
+        const uint32_t g = g0 + q;
+        out.info[out.dfa_first + g] = (KIND_DFA << INFO_KIND_SHIFT) | g;
+        out.lhs[out.dfa_first + g] = (uint16_t)L;
+        out.dfa_done[g] = (uint16_t)done_id;
+        out.dfa_accept[g] = (uint8_t)a.accepting[q];
+        for (uint32_t e = 0; e < out.n_eq; ++e) {
+          const int t = a.trans[(size_t)q * out.n_eq + e];
+          if (t < 0) continue;
+          bool alive = false;  // a state nothing leaves is never made an item: a finished automaton is dropped at once
+          for (uint32_t e2 = 0; e2 < out.n_eq; ++e2) alive = alive || a.trans[(size_t)t * out.n_eq + e2] >= 0;
+          out.dfa_trans[(size_t)g * out.n_eq + e] =
+              (uint16_t)((g0 + (uint32_t)t) | (alive ? 0x4000u : 0u) | (a.accepting[t] ? 0x8000u : 0u));
+          for (int byte = 0; byte < 256; ++byte)
+            if (out.eq_of_byte[byte] == e) out.dfa_scan[(size_t)g * 8 + (byte >> 5)] |= 1u << (byte & 31);
+        }
+      }
+      g0 += a.n_states;
+    }
+  }
   uint32_t d = 0;
   for (auto& p : solid) {  // solid[0] is $ -> start, so items 0 and 1 are the start and accept items
     int L = nt_new[p.lhs];
@@ -461,7 +851,7 @@ void compile_grammar(const char* text, size_t len, const std::string& start, Hos
       }
     }
   }
-  for (uint32_t i = (uint32_t)D; i-- > 0;)
+  for (uint32_t i = (uint32_t)D_rules; i-- > 0;)
     if ((out.info[i] >> INFO_KIND_SHIFT) == KIND_NT && (out.info[i] & INFO_NULLABLE))
       out.skip[i] = (uint8_t)std::min<uint32_t>(255u, 1u + out.skip[i + 1]);
   for (uint32_t i = 0; i < (uint32_t)D; ++i) out.info[i] |= (uint32_t)out.skip[i] << INFO_SKIP_SHIFT;

@@ -12,7 +12,8 @@ namespace fmt {
 //   END : argument = left-hand side        (dot at the end of the rule)
 //   TERM: argument = byte-class id         (post-dot symbol is a terminal)
 //   NT  : argument = non-terminal id       (post-dot symbol is a non-terminal)
-enum : uint32_t { KIND_END = 0u, KIND_TERM = 1u, KIND_NT = 2u };
+//   DFA : argument = automaton state      (the item is inside a regular non-terminal run as an automaton)
+enum : uint32_t { KIND_END = 0u, KIND_TERM = 1u, KIND_NT = 2u, KIND_DFA = 3u };
 constexpr uint32_t INFO_KIND_SHIFT = 30;
 constexpr uint32_t INFO_NULLABLE = 1u << 29;
 constexpr uint32_t INFO_ARG_MASK = 0xFFFFu;
@@ -41,6 +42,16 @@ struct HostTables {
                                        // leading nullable symbols, completed items left out
   std::vector<uint8_t> eq_of_byte;     // [256] bytes that belong to the same byte classes share a number
   uint32_t n_eq = 0;                   // how many such equivalence classes of bytes there are
+  // regular non-terminals run as deterministic automata (Section 4.1's regular terminals): item id
+  // dfa_first + g is state g; dfa_trans[g][byte class] = target state | 0x4000 (the target has transitions
+  // of its own) | 0x8000 (the target accepts), or 0xFFFF
+  uint32_t dfa_first = 0, dfa_states = 0;
+  std::vector<uint16_t> dfa_trans;     // [dfa_states][n_eq]
+  std::vector<uint16_t> dfa_done;      // [dfa_states] id of the completed item of the state's non-terminal
+  std::vector<uint32_t> dfa_scan;      // [dfa_states][8] bytes with a transition
+  std::vector<uint8_t> dfa_accept;     // [dfa_states]
+  std::vector<uint32_t> dfa_nt;        // per automaton: its non-terminal
+  std::vector<uint32_t> dfa_start;     // per automaton: its start state
   std::vector<uint8_t> nullable;       // [N]
   std::vector<std::string> nt_names;   // [N]
   // ---- vocabulary trie in CSR form, nodes in breadth-first order (root = 0)
@@ -62,7 +73,7 @@ struct HostTables {
 std::string json_schema_to_ebnf(const char* schema, size_t len);
 
 // Both throw CompileError.
-void compile_grammar(const char* text, size_t len, const std::string& start, HostTables& out);
+void compile_grammar(const char* text, size_t len, const std::string& start, HostTables& out, bool dfa_terminals = true);
 void build_trie(const uint8_t* bytes, const uint64_t* offs, uint32_t V, int32_t eos, HostTables& out);
 
 }  // namespace fmt

@@ -283,7 +283,9 @@ struct SweepWarp {
     for (uint32_t k = lane; k < plen; k += 32) {
       const uint32_t it = pitems[k];
       const uint32_t inf = G.info[it & 0xFFFFu];
-      if ((inf >> INFO_KIND_SHIFT) == KIND_TERM && class_has(G, inf & INFO_ARG_MASK, byte)) add_item(G, w, view.fix(it, pcode) + 1u);
+      const Scanned sc = scan_item(G, view.fix(it, pcode), inf, byte);
+      if (sc.has_a) add_item(G, w, sc.a);
+      if (sc.has_b) add_item(G, w, sc.b);
     }
     __syncwarp();
     if (w.ctr[W_OVERFLOW]) {

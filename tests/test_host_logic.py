@@ -97,7 +97,7 @@ def test_grammar_reduction_and_nullability():
     dead ::= dead "q"
     unused ::= "z"
     '''
-    g = fmt.Grammar(text, "s", [b"a", b""], eos=1, host_only=True)
+    g = fmt.Grammar(text, "s", [b"a", b""], eos=1, host_only=True, dfa=False)  # (the rules as written: no automata)
     info = g.info()
     nullable = g.table(6)
     assert info.start_nullable == 1
