@@ -553,6 +553,30 @@ def cpu_baseline(w, start: int, budget_s: float = 15.0):
 
     rows = min(w.batch, 16)
     g, vocab, seqs, advance = oracle_sample(w, start, rows)
+    # the same rows with the oracle's CPU Compact (Section 4.2.3), for the sizes of pruned against full charts
+    n_pruned = min(rows, 4)
+    pruned = []
+    for b in range(n_pruned):
+        s = oracle.Sequence_(g, pruned=True)
+        s.advance(w.prefix_bytes[b])
+        pruned.append(s)
+    for i in range(start):
+        for b in range(n_pruned):
+            if w.reset_before[i, b]:
+                pruned[b] = oracle.Sequence_(g, pruned=True)
+            t = int(w.tokens[i, b])
+            if t != w.eos and t >= 0:
+                pruned[b].advance(w.vocab[t])
+    sizes = {"full_items_max": 0, "full_sets_max": 0, "pruned_items_max": 0, "pruned_sets_max": 0}
+
+    def note_sizes():
+        for b in range(n_pruned):
+            sizes["full_items_max"] = max(sizes["full_items_max"], seqs[b].total_items)
+            sizes["full_sets_max"] = max(sizes["full_sets_max"], seqs[b].num_sets)
+            sizes["pruned_items_max"] = max(sizes["pruned_items_max"], pruned[b].total_items)
+            sizes["pruned_sets_max"] = max(sizes["pruned_sets_max"], pruned[b].num_sets)
+
+    note_sizes()
     t0 = time.perf_counter()
     masks = 0
     i = start
@@ -563,8 +587,18 @@ def cpu_baseline(w, start: int, budget_s: float = 15.0):
             masks += 1
         i += 1
     dt = time.perf_counter() - t0
+    for k in range(start, i):  # (outside the timed part) the pruned copies follow, then both are measured
+        for b in range(n_pruned):
+            if w.reset_before[k, b]:
+                pruned[b] = oracle.Sequence_(g, pruned=True)
+            t = int(w.tokens[k, b])
+            if t != w.eos and t >= 0:
+                pruned[b].advance(w.vocab[t])
+    note_sizes()
+    sizes["what"] = ("items and Earley sets of the oracle's charts for %d of the sampled rows, full chart against the chart "
+                     "after the oracle's Compact (the paper's maximum-memory comparison)" % n_pruned)
     return {"value": masks * w.V / dt, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
-            "ms_per_row_mask": dt / max(1, masks) * 1e3,
+            "ms_per_row_mask": dt / max(1, masks) * 1e3, "chart_sizes": sizes,
             "sample": "%d rows x %d steps of %s: advance + full-vocabulary mask per row, OpenMP over tokens" % (rows, i - start, w.name)}
 
 
