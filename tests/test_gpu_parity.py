@@ -9,7 +9,7 @@ from helpers import OracleBatch, describe_diff
 pytestmark = pytest.mark.gpu
 
 
-def run_workload(w, check_steps, rows=None, cache=True, fused_every=0, check_prefix_mask=True, **state_kw):
+def run_workload(w, check_steps, rows=None, cache=True, fused_every=0, check_prefix_mask=True, dfa=True, **state_kw):
     """Feed the workload through the library and the oracle; compare statuses every step and
     masks (all rows in `rows`) at the steps in `check_steps`.  Returns the library's stats."""
     import torch
@@ -17,7 +17,7 @@ def run_workload(w, check_steps, rows=None, cache=True, fused_every=0, check_pre
     import paper_2506_01151_b200 as fmt
 
     dev = torch.device("cuda:0")
-    g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
+    g = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos, dfa=dfa)
     st = fmt.State(g, w.batch, cache=cache, **state_kw)
     ob = OracleBatch(w)
     rows = list(range(w.batch)) if rows is None else rows
@@ -117,6 +117,16 @@ def test_config4_reduced(roots):
 def test_config5_reduced(roots):
     w = workloads.build(5, V=20000, batch=8, steps=32, prefix_scale=0.25)
     run_workload(w, check_steps=set(range(0, 32, 4)), fused_every=16, roots=roots)
+
+
+@pytest.mark.parametrize("config", [2, 3, 4, 5])
+def test_reduced_configs_with_every_non_terminal_kept_as_rules(config):
+    """By default regular non-terminals run as automata (Section 4.1); with that switched off the
+    same masks must come out of rules alone."""
+    kw = {2: dict(V=4000, batch=4, steps=64), 3: dict(V=20000, batch=8, steps=96), 4: dict(V=20000, batch=8, steps=64),
+          5: dict(V=20000, batch=8, steps=24, prefix_scale=0.25)}[config]
+    w = workloads.build(config, **kw)
+    run_workload(w, check_steps=set(range(0, w.steps, 4)), fused_every=16, dfa=False)
 
 
 # ---- full sizes, in the launch configuration the benchmark times; masks compared on sampled steps
