@@ -74,8 +74,7 @@ enum : uint32_t {
   CNT_BAR_ERR = 31,     // a block gave up waiting at the barrier
   CNT_LEVEL_ALIVE = 32, // [MAX_TOKEN_BYTES + 2] per trie depth: some node of some job was alive
   CNT_LEVEL_REQ = 68,   // [MAX_TOKEN_BYTES + 2] per trie depth: transitions queued for computation
-  CNT_HASH_GEN = 104,   // generation of the sweep's per-job hashes (1 .. 65535), advanced by every fill
-  CNT_HASH_CLEAR = 105, // this fill starts the generations over: the sweep clears the hashes first
+  CNT_HASH_GEN = 104,   // (the depth counters that every fill clears end here; the fills' generations are handed out by the host)
   CNT_STAT_ADV_HIT = 106,  // 64-bit: advances answered by the transition cache
   CNT_LEVEL_TAKEN = 108,   // [MAX_TOKEN_BYTES + 2] per trie depth: tickets drawn for the queued transitions
   CNT_PASS_DONE = 144,     // CTAs that have finished their part of a depth's pass (summed over the depths)
@@ -86,11 +85,9 @@ enum : uint32_t {
   CNT_STAT_JOBS_ROOT = 152,    // 64-bit: computed rows that started from a swept root
   CNT_STAT_JOBS_PLAIN = 154,   // 64-bit: computed rows that walked the whole trie themselves
   CNT_STAT_JOBS_MASK = 156,    // 64-bit: computed rows answered by their root's mask row alone
-  CNT_STAT_SPARE = 158,
   CNT_STAT_ABORTS = 160,       // 64-bit: fills abandoned because a bounded wait ran out
   CNT_STAT_STEP_CYCLES = 162,  // 64-bit: SM cycles spent inside Earley steps of the fill (summed over warps)
   CNT_STAT_ADV_WORDS = 164,    // 64-bit: chart words read and written by advance
-  CNT_STAT_SPARE2 = 182,
   CNT_STAT_FRAMES = 184,       // 64-bit: frames made (sets of a walk recognised as roots)
   CNT_DIAG = 166,              // [16] where capacity errors and expired waits came from (see DIAG_*)
   CNT_TOTAL = 186
@@ -158,10 +155,10 @@ constexpr uint32_t LBASE = 0x800u, RBASE = 0x8000u;
 constexpr uint32_t ROOT_NONE = 0xffffffffu;
 enum : uint32_t { ROOT_NEW = 0, ROOT_READY = 1, ROOT_FAILED = 2 };
 enum : uint32_t {  // words of a root's directory entry
-  RI_STATUS = 0, RI_P = 1, RI_NK = 2, RI_N = 3, RI_HASH = 4, RI_CHART = 5, RI_FR_OFF = 6, RI_FR_N = 7,
+  RI_STATUS = 0, RI_P = 1, RI_NK = 2, RI_N = 3, RI_HASH = 4, RI_CHART = 5, RI_FR_N = 7,
   RI_ST_OFF = 8, RI_NSTATES = 9, RI_TR_OFF = 10, RI_WORDS = 16
 };
-enum : uint32_t { TOP_CHARTS = 0, TOP_FRONTIER = 1, TOP_STATES = 2, TOP_ITEMS = 3, TOP_TRANS = 4, TOP_MENT = 5, TOP_MDATA = 6, TOP_PENDING = 7, TOP_N = 8 };
+enum : uint32_t { TOP_CHARTS = 0, TOP_STATES = 2, TOP_ITEMS = 3, TOP_TRANS = 4, TOP_PENDING = 7, TOP_N = 8 };
 constexpr uint16_t R_DEAD = 0xFFFFu, R_CTX = 0xFFFEu;  // values of a region's transition table besides set numbers
 
 struct RootDev {
