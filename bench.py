@@ -160,14 +160,14 @@ def aggregate_over_ranks(elapsed_ms: float, units: float, dist=None):
 class Driver:
     """Owns the library objects and the device buffers of one replica and runs steps."""
 
-    def __init__(self, w: workloads.Workload, device, roots: bool = False, ring_bytes: int = int(1.6 * L2_BYTES)):
+    def __init__(self, w: workloads.Workload, device, roots: bool = False, cache: bool = True, ring_bytes: int = int(1.6 * L2_BYTES)):
         import torch
 
         import paper_2506_01151_b200 as fmt
 
         self.torch, self.fmt, self.w, self.device = torch, fmt, w, device
         self.grammar = fmt.Grammar(w.ebnf, w.start, w.vocab, w.eos)
-        self.state = fmt.State(self.grammar, w.batch, roots=roots)
+        self.state = fmt.State(self.grammar, w.batch, roots=roots, cache=cache)
         self.roots = roots
         self.stream = torch.cuda.current_stream(device)
         B, V = w.batch, w.V
@@ -295,10 +295,12 @@ def run_ours(args):
         if world > 1:
             dist.barrier()
         sampler.pause()
+        series = {name: [float(x) for x in drv.state.read_profile_series(kind)]
+                  for kind, name in ((0, "advance"), (1, "sweep"), (2, "masking"))}
         prof = drv.state.read_profile()
         drv.state.set_profiling(False)
         t_ms, total_units = aggregate_over_ranks(total_ms, units, dist if world > 1 else None)
-        reps.append({"t_ms": t_ms, "units": total_units, "per_step": per_step, "prof": prof, "launches": drv.launches,
+        reps.append({"t_ms": t_ms, "units": total_units, "per_step": per_step, "prof": prof, "launches": drv.launches, "series": series,
                      "stats": stat_delta(stats0, drv.state.stats(), STAT_KEYS)})
     clocks = sampler.stop()
     # ---- once more, untimed, with the cycle counter read around every Earley step (it slows the sweeps a little)
@@ -313,7 +315,7 @@ def run_ours(args):
     med = reps[order[(R - 1) // 2]]  # the median repeat (the lower one of two) is the one reported in full
     t_ms, total_units, prof, st = med["t_ms"], med["units"], med["prof"], med["stats"]
 
-    cold = cold_all = e2e = passes = None
+    cold = cold_all = e2e = passes = cache_off = None
     stats_end = drv.state.stats()
     if rank == 0:
         if world == 1 and args.passes > 1:
@@ -322,6 +324,8 @@ def run_ours(args):
         cold = measure_cold(drv, w, W, min(K, 16), clear_ci=False)
         cold_all = measure_cold(drv, w, W, min(K, 16), clear_ci=True)
         e2e = measure_e2e(drv, w, W, min(K, 64))
+        if world == 1:
+            cache_off = measure_cache_off(w, device, W, min(K, 32))
     if world > 1:
         dist.barrier()
     if rank != 0:
@@ -399,6 +403,8 @@ def run_ours(args):
         "latency_ms": {"p50": percentile(med["per_step"], 0.50), "p90": percentile(med["per_step"], 0.90),
                        "p99": percentile(med["per_step"], 0.99), "max": max(med["per_step"]), "min": min(med["per_step"]),
                        "what": "per decoding step (advance + fill + masking of B rows), CUDA events around every step of the median repeat"},
+        "kernel_latency_ms": {name: ({"p50": percentile(xs, 0.5), "p99": percentile(xs, 0.99), "max": max(xs), "launches": len(xs)} if xs else None)
+                              for name, xs in med["series"].items()},
         "clocks": clocks, "e2e": e2e, "gpu_launches": med["launches"], "roofline": roofline,
         "cache": {"fills": st["fills"], "computed": jobs, "from_state_cache": st["fills_from_cache"], "shared_within_fill": st["fills_shared"],
                   "hit_rate": 1.0 - jobs / fills,
@@ -413,7 +419,7 @@ def run_ours(args):
         "memory": {"device_bytes": stats_end["device_bytes"], "states_cached": stats_end["states_cached"],
                    "state_pool_bytes_used": 4 * stats_end["pool_words_used"], "mask_rows_cached": stats_end["mask_rows_cached"],
                    "bytes_per_cached_state": (4 * stats_end["pool_words_used"] + 4 * Wm * stats_end["mask_rows_cached"]) / states},
-        "passes": passes, "cold": cold, "cold_all": cold_all,
+        "passes": passes, "cold": cold, "cold_all": cold_all, "cache_off": cache_off,
         "grammar": {"nonterminals": info.n_nonterminals, "rules": info.n_rules, "dotted": info.n_dotted,
                     "trie_nodes": info.trie_nodes, "trie_depth": info.trie_depth, "byte_classes": info.n_byte_classes},
     }
@@ -443,6 +449,24 @@ def measure_passes(drv: "Driver", W: int, K: int, n_passes: int, first):
                     "computed": d["fills_computed"], "new_entries_swept": d["root_sweeps"],
                     "earley_steps": d["walk_transitions"] + d["sweep_transitions"],
                     "p50_ms": percentile(per_step, 0.5), "p99_ms": percentile(per_step, 0.99)})
+    return out
+
+
+def measure_cache_off(w, device, W: int, n: int):
+    """The same steps on a state created without the state cache (Section 5.2 switched off): every fill
+    computes every row that is not finished."""
+    import torch
+
+    drv = Driver(w, device, cache=False)
+    drv.restart(W, clear_caches=False)
+    total_ms, per_step = drv.timed(W, n)
+    st = drv.state.stats()
+    out = {"steps": n, "ms_per_step": total_ms / n, "p50_ms": percentile(per_step, 0.5), "p99_ms": percentile(per_step, 0.99),
+           "token_checks_per_s": w.batch * w.V * n / (total_ms * 1e-3), "fills_from_cache": st["fills_from_cache"],
+           "what": "advance + fill + masking per step with fmt_state_options.cache_disable = 1"}
+    drv.state.close()
+    del drv
+    torch.cuda.empty_cache()
     return out
 
 
@@ -595,10 +619,13 @@ def cpu_baseline(w, start: int, budget_s: float = 15.0):
             if t != w.eos and t >= 0:
                 pruned[b].advance(w.vocab[t])
     note_sizes()
+    t1 = time.perf_counter()
+    seqs[0].mask(vocab, threads=1)
+    single = w.V / (time.perf_counter() - t1)
     sizes["what"] = ("items and Earley sets of the oracle's charts for %d of the sampled rows, full chart against the chart "
                      "after the oracle's Compact (the paper's maximum-memory comparison)" % n_pruned)
     return {"value": masks * w.V / dt, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
-            "ms_per_row_mask": dt / max(1, masks) * 1e3, "chart_sizes": sizes,
+            "ms_per_row_mask": dt / max(1, masks) * 1e3, "single_thread_value": single, "chart_sizes": sizes,
             "sample": "%d rows x %d steps of %s: advance + full-vocabulary mask per row, OpenMP over tokens" % (rows, i - start, w.name)}
 
 

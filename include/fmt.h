@@ -342,6 +342,10 @@ typedef struct {
 } fmt_profile;
 fmt_status fmt_state_set_profiling(fmt_state* s, int enable);
 fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out);
+/* The same measurements launch by launch, before fmt_state_read_profile forgets them: kind 0 advance,
+ * 1 trie sweep, 2 logits masking, 3 the fills' work on context-independent entries.  Writes up to `cap`
+ * durations in milliseconds to ms_out (may be NULL) and the number recorded to *n. */
+fmt_status fmt_state_read_profile_series(fmt_state* s, int kind, float* ms_out, size_t cap, size_t* n);
 
 /*
  * Masks for up to FMT_NOALLOC_MAX_CHARTS pruned charts without any memory allocation.

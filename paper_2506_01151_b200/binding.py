@@ -23,7 +23,7 @@ EXPORTS = [
     "fmt_compile", "fmt_json_schema_to_ebnf", "fmt_compile_json_schema", "fmt_grammar_destroy", "fmt_grammar_get_info", "fmt_grammar_copy_table", "fmt_grammar_automaton_match",
     "fmt_state_create", "fmt_state_destroy", "fmt_state_reset", "fmt_state_advance", "fmt_state_forced_bytes", "fmt_fill_mask",
     "fmt_apply_mask", "fmt_fill_and_apply", "fmt_state_cache_clear", "fmt_state_ci_cache_clear", "fmt_state_set_wait_limit", "fmt_state_copy_counters", "fmt_state_query", "fmt_state_copy_chart", "fmt_get_stats",
-    "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_fill_mask_noalloc", "fmt_last_error",
+    "fmt_state_set_profiling", "fmt_state_read_profile", "fmt_state_read_profile_series", "fmt_fill_mask_noalloc", "fmt_last_error",
 ]
 
 
@@ -106,6 +106,7 @@ def lib():
         L.fmt_get_stats.argtypes = [vp, C.POINTER(Stats), vp]
         L.fmt_state_set_profiling.argtypes = [vp, C.c_int]
         L.fmt_state_read_profile.argtypes = [vp, C.POINTER(Profile)]
+        L.fmt_state_read_profile_series.argtypes = [vp, C.c_int, vp, sz, C.POINTER(sz)]
         L.fmt_fill_mask_noalloc.argtypes = [vp, vp, vp, u32, vp, vp, vp]
         L.fmt_last_error.restype = C.c_char_p
         for name in EXPORTS:
@@ -324,6 +325,14 @@ class State:
     def set_profiling(self, on: bool, step_cycles: bool = False):
         """Kernel timing with CUDA events; `step_cycles` also counts the SM cycles inside Earley steps."""
         _check(lib().fmt_state_set_profiling(self._h, (1 if on else 0) | (2 if step_cycles else 0)))
+
+    def read_profile_series(self, kind: int) -> np.ndarray:
+        """Per-launch durations (ms) of one kind of kernel (0 advance, 1 sweep, 2 masking, 3 entries); call before read_profile."""
+        n = C.c_size_t()
+        _check(lib().fmt_state_read_profile_series(self._h, kind, None, 0, C.byref(n)))
+        buf = np.zeros(max(n.value, 1), dtype=np.float32)
+        _check(lib().fmt_state_read_profile_series(self._h, kind, buf.ctypes.data, n.value, C.byref(n)))
+        return buf[: n.value]
 
     def read_profile(self) -> dict:
         out = Profile()

@@ -685,6 +685,17 @@ fmt_status fmt_state_set_profiling(fmt_state* s, int enable) {
   return FMT_OK;
 }
 
+fmt_status fmt_state_read_profile_series(fmt_state* s, int kind, float* ms_out, size_t cap, size_t* n) {
+  if (!s || !n || kind < 0 || kind > 3) return fail(FMT_ERR_INVALID_ARG, "bad argument");
+  *n = s->prof.used[kind];
+  for (size_t i = 0; i < s->prof.used[kind] && i < cap && ms_out; ++i) {
+    cudaError_t e = cudaEventSynchronize(s->prof.b[kind][i]);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms_out[i], s->prof.a[kind][i], s->prof.b[kind][i]);
+    if (e != cudaSuccess) return cuda_fail(e, "fmt_state_read_profile_series");
+  }
+  return FMT_OK;
+}
+
 fmt_status fmt_state_read_profile(fmt_state* s, fmt_profile* out) {
   if (!s || !out) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
   double ms[4] = {0, 0, 0, 0};
