@@ -94,9 +94,13 @@ typedef struct {
   uint32_t wait_limit_log2;    /* every wait inside a kernel is a poll that gives up after 2^this many
                                  polls (0 = defaults, 2^21..2^24); see fmt_state_set_wait_limit */
   uint32_t cache_keep_when_full; /* 0: when the state cache has no room for a new entry (states, chart
-                                 storage or mask rows), the next fmt_state_advance empties it - every entry
-                                 at once; the rows' current charts are entered again - and caching goes
-                                 on.  1: the cache keeps what it has and takes no new entries */
+                                 storage or mask rows), the next fmt_state_advance turns it over: the cache's
+                                 storage exists twice, the other copy becomes the one in use, the rows' current
+                                 charts are entered again, and so is - with its mask row - every entry that was
+                                 found again at least once after it was made (a second chance for what is in
+                                 use; what was met once goes).  max_states, max_mask_rows and pool_words are the
+                                 capacities of ONE copy.  1: one copy only; when it is full the cache keeps
+                                 what it has and takes no new entries */
 } fmt_state_options;
 
 typedef struct {
@@ -152,7 +156,7 @@ typedef struct {
                                    warp computes, [5] wait for queued work, [6] wait for the other thread
                                    blocks, [7] a context-independent entry that could not be kept;
                                    [8..15] the same for the sweeps that fill such entries */
-  uint64_t cache_flushes;       /* times the state cache was emptied because it had no room left */
+  uint64_t cache_flushes;       /* times the state cache was turned over because it had no room left */
 } fmt_stats;
 
 /*

@@ -117,6 +117,16 @@ struct fmt_state {
   size_t device_bytes = 0;    // what fmt_state_create allocated
   // The device sets this host-mapped word when the state cache has no room for a new entry; the next
   // fmt_state_advance empties the cache (all entries at once) and caching goes on.
+  // Two generations of cache storage (chart pool, per-entry tables, mask rows): emptying the cache switches to
+  // the other one and carries over the entries that were found again after they were made.
+  int generation = 0;
+  uint64_t* st_off2[2] = {nullptr, nullptr};
+  int32_t* st_mask2[2] = {nullptr, nullptr};
+  uint8_t* st_ref2[2] = {nullptr, nullptr};
+  uint64_t pool_base2[2] = {0, 0};
+  uint32_t mrow_base2[2] = {0, 0};
+  uint32_t* old_count_dev = nullptr;
+  uint64_t survivors_runs = 0;
   uint32_t* full_flag_host = nullptr;
   bool skip_full_check = false;
   uint64_t flushes = 0;
@@ -373,6 +383,13 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   d.ht_mask = ht - 1;
   d.init_off = (uint64_t)batch * 3u * d.chart_words;
   d.pool_base = d.init_off + d.chart_words;
+  d.pool_lo = d.pool_base;
+  const bool two_gens = d.cache_on && !(opt && opt->cache_keep_when_full);
+  s->pool_base2[0] = d.pool_base;
+  s->pool_base2[1] = d.pool_base + (two_gens ? d.pool_words : 0);
+  s->mrow_base2[0] = batch;
+  s->mrow_base2[1] = batch + (two_gens ? d.max_mask_rows : 0);
+  d.mrow_base = batch;
   d.big_arena_items = 1u << 16;
   d.big_hset_slots = 1u << 14;
   AutoDev& au = d.au;
@@ -412,16 +429,24 @@ fmt_status fmt_state_create(const fmt_grammar* g, uint32_t batch, const fmt_stat
   s->sweep_grid = std::max(1, per_sm * sms);
   const size_t big_words = (size_t)s->sweep_grid * sweep_warps() * ((size_t)d.big_arena_items + d.big_hset_slots);
 #define AL(ptr, count, fill) if (e == cudaSuccess) e = s->bufs.alloc((size_t)(count), &(ptr), (fill))
-  AL(d.arena, d.pool_base + d.pool_words, 0);
+  AL(d.arena, d.pool_base + d.pool_words * (two_gens ? 2 : 1), 0);
   AL(d.row_chart, batch, 0);
   AL(d.row_buf, batch, 0xFF);
   AL(d.row_state, batch, 0xFF);
   AL(d.row_flags, batch, 0);
   AL(d.row_mask, batch, 0xFF);
   AL(d.ht, ht, 0);
-  AL(d.st_off, d.max_states, 0);
-  AL(d.st_mask, d.max_states, 0xFF);
-  AL(d.mask_rows, ((size_t)batch + d.max_mask_rows) * g->dev.Wm, 0);
+  AL(s->st_off2[0], d.max_states, 0);
+  AL(s->st_mask2[0], d.max_states, 0xFF);
+  AL(s->st_ref2[0], d.max_states, 0);
+  if (two_gens) {
+    AL(s->st_off2[1], d.max_states, 0);
+    AL(s->st_mask2[1], d.max_states, 0xFF);
+    AL(s->st_ref2[1], d.max_states, 0);
+  }
+  AL(s->old_count_dev, 4, 0);
+  d.st_off = s->st_off2[0], d.st_mask = s->st_mask2[0], d.st_ref = s->st_ref2[0];
+  AL(d.mask_rows, ((size_t)batch + (size_t)d.max_mask_rows * (two_gens ? 2 : 1)) * g->dev.Wm, 0);
   uint32_t trn = 1024;
   while (trn < d.max_states * 4u) trn <<= 1;
   d.tr_mask = trn - 1;
@@ -523,6 +548,8 @@ fmt_status fmt_state_reset(fmt_state* s, const uint32_t* rows_dev, uint32_t n, v
   return launched("fmt_state_reset");
 }
 
+static fmt_status cache_turn_over(fmt_state* s, cudaStream_t st);
+
 fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t* status_dev, void* stream) {
   if (!s || !token_ids_dev) return fail(FMT_ERR_INVALID_ARG, "NULL argument");
   if (s->full_flag_host) {
@@ -534,7 +561,7 @@ fmt_status fmt_state_advance(fmt_state* s, const int32_t* token_ids_dev, int32_t
       *flag = 0u;
       s->skip_full_check = true;
       ++s->flushes;
-      if (fmt_status rc = fmt_state_cache_clear(s, stream)) return rc;
+      if (fmt_status rc = cache_turn_over(s, (cudaStream_t)stream)) return rc;
     }
   }
   cudaEvent_t e0, e1;
@@ -609,9 +636,35 @@ fmt_status fmt_state_cache_clear(fmt_state* s, void* stream) {
   if (e == cudaSuccess) e = cudaMemsetAsync(d.tr_val, 0x80, ((size_t)d.tr_mask + 1) * 4, st);
   // counters: states, mask rows, jobs, work, error flag, pool top
   if (e == cudaSuccess) e = cudaMemsetAsync(d.counters, 0, 8 * 4, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.st_ref, 0, d.max_states, st);
   if (e != cudaSuccess) return cuda_fail(e, "fmt_state_cache_clear");
   launch_reintern(d, s->init_state_dev, st);
   return launched("fmt_state_cache_clear");
+}
+
+// The cache has no room left: switch to the other generation of its storage, enter the rows' current charts
+// again and carry over every entry that was found again after it was made, with its mask row.
+static fmt_status cache_turn_over(fmt_state* s, cudaStream_t st) {
+  if (!s->st_off2[1]) return fmt_state_cache_clear(s, st);
+  const StateDev old = s->dev;
+  StateDev& d = s->dev;
+  launch_evacuate(old, st);  // rows whose chart lives in the cache's storage take it along
+  cudaError_t e = cudaMemcpyAsync(s->old_count_dev, old.counters + CNT_N_STATES, 4, cudaMemcpyDeviceToDevice, st);
+  s->generation ^= 1;
+  const int gi = s->generation;
+  d.st_off = s->st_off2[gi], d.st_mask = s->st_mask2[gi], d.st_ref = s->st_ref2[gi];
+  d.pool_base = s->pool_base2[gi];
+  d.mrow_base = s->mrow_base2[gi];
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.ht, 0, ((size_t)d.ht_mask + 1) * 4, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.tr_key, 0, ((size_t)d.tr_mask + 1) * 8, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.tr_val, 0x80, ((size_t)d.tr_mask + 1) * 4, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.counters, 0, 8 * 4, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.st_ref, 0, d.max_states, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d.st_mask, 0xFF, (size_t)d.max_states * 4, st);
+  if (e != cudaSuccess) return cuda_fail(e, "emptying the state cache");
+  launch_reintern(d, s->init_state_dev, st);
+  launch_survivors(s->g->dev, old, d, s->old_count_dev, st);
+  return launched("emptying the state cache");
 }
 
 fmt_status fmt_state_ci_cache_clear(fmt_state* s, void* stream) {

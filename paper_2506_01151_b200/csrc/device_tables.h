@@ -243,7 +243,10 @@ struct StateDev {
   uint32_t cache_on;
   uint32_t* full_flag;        // host-mapped word (or nullptr): set when the state cache or its mask rows have no room left
   uint32_t max_states, ht_mask, max_mask_rows;
-  uint64_t pool_base, pool_words;   // word offsets into arena / size of the pool
+  uint64_t pool_base, pool_words;   // word offsets into arena / size of the pool (the generation in use)
+  uint64_t pool_lo;                 // where chart storage of the cache begins (both generations lie above it)
+  uint32_t mrow_base;               // first cached mask row of the generation in use (an index into mask_rows)
+  uint8_t* st_ref;                  // [max_states] the entry was found again after it was made (it survives the next emptying)
   uint64_t init_off;                // word offset of the start chart
   uint32_t* arena;            // [B*3 private buffers][start chart][pool]
   uint64_t* row_chart;        // [B] word offset of the row's current chart

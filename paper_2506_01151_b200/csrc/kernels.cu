@@ -85,6 +85,7 @@ __device__ int32_t intern_chart(const StateDev& S, const uint32_t* ch, uint64_t&
         if (__ldcg(other + i) != ch[i]) same = false;
     same = __all_sync(FULL, same);
     if (same) {
+      if (lane == 0 && S.st_ref) S.st_ref[sid] = 1;  // (found again)
       off_out = poff;
       return (int32_t)sid;
     }
@@ -207,6 +208,7 @@ __global__ void __launch_bounds__(ADV_WARPS * 32, 1) advance_kernel(GrammarDev G
     if (known >= 0 && (uint32_t)known < S.max_states) {
       if (lane == 0) {
         S.row_state[row] = known;
+        S.st_ref[known] = 1;
         S.row_chart[row] = ld_cg64(&S.st_off[known]);
         S.row_buf[row] = 255;
         stat_add(S, CNT_STAT_ADV, 1u);
@@ -332,6 +334,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
     if (sid >= 0) {
       int32_t old = atomicCAS(&S.st_mask[sid], -1, -2 - (int32_t)row);
       if (old >= 0) {  // cached
+        S.st_ref[sid] = 1;  // (used again: it outlives the next emptying of the cache)
         S.row_mask[row] = old;
         stat_add(S, CNT_STAT_CACHED, 1u);
         continue;
@@ -345,7 +348,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(GrammarDev G, StateDev S) {
       int32_t mrow = (int32_t)row;
       if (ld_acquire(&S.counters[CNT_N_MASK_ROWS]) < S.max_mask_rows) {
         uint32_t got = atomicAdd(&S.counters[CNT_N_MASK_ROWS], 1u);
-        if (got < S.max_mask_rows) mrow = (int32_t)(S.B + got);
+        if (got < S.max_mask_rows) mrow = (int32_t)(S.mrow_base + got);
       }
       if (mrow == (int32_t)row && S.full_flag) *reinterpret_cast<volatile uint32_t*>(S.full_flag) = 1u;  // no mask row left to cache it in
       S.row_mask[row] = mrow;
@@ -885,7 +888,7 @@ __global__ void evacuate_kernel(StateDev S) {
   if (row >= S.B) return;
   const uint64_t off = S.row_chart[row];
   __syncthreads();
-  if (off >= S.pool_base) {
+  if (off >= S.pool_lo) {
     const uint32_t* src = S.arena + off;
     uint32_t* dst = private_buf(S, row, 0);
     const uint32_t words = src[CH_WORDS];
@@ -920,6 +923,35 @@ __global__ void __launch_bounds__(32) reintern_kernel(StateDev S, int32_t* init_
 __global__ void fix_init_rows_kernel(StateDev S, const int32_t* init_state) {
   const uint32_t row = blockIdx.x * blockDim.x + threadIdx.x;
   if (row < S.B && S.row_chart[row] == S.init_off) S.row_state[row] = *init_state;
+}
+
+// Emptying the cache with survivors (see fmt_state_create's cache_keep_when_full): `Old` is the cache as it
+// was - its charts, mask rows and tables are still intact in the other half of the storage -, S the emptied
+// one.  Every entry of Old that was found again after it was made is entered into S, with its mask row.
+__global__ void __launch_bounds__(32) survivors_kernel(GrammarDev G, StateDev Old, StateDev S, const uint32_t* old_count) {
+  const uint32_t id = blockIdx.x * gridDim.y + blockIdx.y;
+  if (id >= min(*old_count, Old.max_states) || !Old.st_ref[id]) return;
+  const uint32_t lane = lane_id();
+  uint64_t off;
+  const int32_t nid = intern_chart(S, Old.arena + Old.st_off[id], off);
+  if (nid < 0) return;  // no room: it goes after all
+  const int32_t orow = Old.st_mask[id];
+  if (orow < (int32_t)Old.B) return;  // no mask was kept for it
+  uint32_t nrow = 0;
+  if (lane == 0) {
+    nrow = 0xFFFFFFFFu;
+    if (S.st_mask[nid] == -1 && ld_acquire(&S.counters[CNT_N_MASK_ROWS]) < S.max_mask_rows) {
+      const uint32_t got = atomicAdd(&S.counters[CNT_N_MASK_ROWS], 1u);
+      if (got < S.max_mask_rows) nrow = S.mrow_base + got;
+    }
+  }
+  nrow = __shfl_sync(FULL, nrow, 0);
+  if (nrow == 0xFFFFFFFFu) return;
+  const uint32_t* src = Old.mask_rows + (size_t)orow * G.Wm;
+  uint32_t* dst = S.mask_rows + (size_t)nrow * G.Wm;
+  for (uint32_t i = lane; i < G.Wm; i += 32) dst[i] = src[i];
+  __syncwarp();
+  if (lane == 0) S.st_mask[nid] = (int32_t)nrow;
 }
 
 __global__ void query_kernel(StateDev S, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets, uint32_t* n_items,
@@ -1022,6 +1054,11 @@ void launch_evacuate(const StateDev& S, cudaStream_t st) { evacuate_kernel<<<S.B
 void launch_reintern(const StateDev& S, int32_t* init_state_dev, cudaStream_t st) {
   reintern_kernel<<<S.B + 1, 32, 0, st>>>(S, init_state_dev);
   fix_init_rows_kernel<<<(S.B + 127) / 128, 128, 0, st>>>(S, init_state_dev);
+}
+void launch_survivors(const GrammarDev& G, const StateDev& Old, const StateDev& S, const uint32_t* old_count, cudaStream_t st) {
+  const uint32_t n = Old.max_states;
+  dim3 grid((n + 255) / 256, 256);
+  survivors_kernel<<<grid, 32, 0, st>>>(G, Old, S, old_count);
 }
 void launch_query(const StateDev& S, uint8_t* a, uint8_t* f, uint32_t* ns, uint32_t* ni, int32_t* sid, cudaStream_t st) {
   query_kernel<<<(S.B + 127) / 128, 128, 0, st>>>(S, a, f, ns, ni, sid);

@@ -30,6 +30,7 @@ void launch_apply(const uint32_t* mask, size_t stride_words, void* logits, int d
 void launch_gather_apply(const GrammarDev& G, const StateDev& S, void* logits, int dtype, size_t row_stride,
                          uint32_t* mask_out, size_t stride_words, cudaStream_t st);
 void launch_evacuate(const StateDev& S, cudaStream_t st);
+void launch_survivors(const GrammarDev& G, const StateDev& Old, const StateDev& S, const uint32_t* old_count, cudaStream_t st);
 void launch_reintern(const StateDev& S, int32_t* init_state_dev, cudaStream_t st);
 void launch_query(const StateDev& S, uint8_t* accepting, uint8_t* finished, uint32_t* n_sets, uint32_t* n_items,
                   int32_t* state_id, cudaStream_t st);

@@ -355,3 +355,31 @@ def test_advance_transition_cache_replays_exactly():
     replayed = s1["steps_advanced"] - s0["steps_advanced"]
     assert replayed > 0 and s1["advances_cached"] - s0["advances_cached"] == replayed
     assert s1["states_cached"] == s0["states_cached"]
+
+
+def test_entries_in_use_survive_when_the_cache_turns_over():
+    """A cache of 8 entries; row 1 meets a new chart at every step (right recursion keeps its history), row 0
+    is sent back to the start at every step.  The cache fills up and is turned over again and again; the start
+    state, found again every time, must keep its mask through every turn-over: it is computed exactly once."""
+    import paper_2506_01151_b200 as fmt
+
+    torch, dev = _torch()
+    text = 's ::= "a" s | "b"'
+    vocab = [b"a", b"b", b"ab", b"aab", b""]
+    g = fmt.Grammar(text, "s", vocab, 4, dfa=False)
+    og, ov = oracle.Grammar(text, "s"), oracle.Vocab(vocab, 4)
+    st = fmt.State(g, 2, max_states=8, max_mask_rows=8, pool_words=1 << 16)
+    seq1 = oracle.Sequence_(og)
+    start_mask = oracle.Sequence_(og).mask(ov)
+    row0 = torch.tensor([0], dtype=torch.int32, device=dev)
+    for i in range(40):
+        assert _advance(st, [0, 0]) == [0, 0]  # both rows take "a"
+        assert seq1.advance(b"a")
+        st.reset(row0)
+        got = _mask_of(st, g, 2)
+        assert np.array_equal(got[0], start_mask) and np.array_equal(got[1], seq1.mask(ov)), i
+    s = st.stats()
+    assert s["cache_flushes"] >= 3 and s["capacity_errors"] == 0
+    # 40 new charts for row 1, and the start state once (its first fill): every other fill of row 0 was a hit
+    assert s["fills_computed"] == 41, s["fills_computed"]
+    assert s["fills_from_cache"] == 39
