@@ -228,9 +228,10 @@ fmt_status fmt_grammar_copy_table(const fmt_grammar* g, int which, void* out, si
  * Create `batch` sequences, all at the start of the grammar (Earley set S[0], Section 3.2).
  * Runs a small kernel on `stream` and synchronizes it once.  opt may be NULL.
  * Device memory: everything the state will ever use is allocated here (fmt_stats.device_bytes reports it;
- * no later call allocates).  With the default options it is about 2.7 GB for batch 8 and 4-5 GB for
- * batch 64-256 with a 128 K-152 K vocabulary: 0.8 GB of chart storage for the state cache (pool_words),
- * max_mask_rows x ceil(V/32) words of cached masks (0.5-0.6 GB), batch x 3 private chart buffers of
+ * no later call allocates).  With the default options it is about 3.7 GB for batch 8 and 5.3-6.5 GB for
+ * batch 64-256 with a 128 K-152 K vocabulary: 2 x 0.8 GB of chart storage for the state cache (pool_words,
+ * two generations: see cache_keep_when_full), 2 x max_mask_rows x ceil(V/32) words of cached masks
+ * (2 x 0.5-0.6 GB), batch x 3 private chart buffers of
  * chart_words words, and the fills' working tables (per row a table of up to sweep_states Earley sets,
  * one 16-bit entry per row and trie node, a 0.5 GB pool for the sets' items); the context-independent
  * cache (roots_enable) adds about 1 GB.  A cached state costs its chart (0.8-3.4 KB in the measured
