@@ -421,7 +421,8 @@ def run_ours(args):
                    "bytes_per_cached_state": (4 * stats_end["pool_words_used"] + 4 * Wm * stats_end["mask_rows_cached"]) / states},
         "passes": passes, "cold": cold, "cold_all": cold_all, "cache_off": cache_off,
         "grammar": {"nonterminals": info.n_nonterminals, "rules": info.n_rules, "dotted": info.n_dotted,
-                    "trie_nodes": info.trie_nodes, "trie_depth": info.trie_depth, "byte_classes": info.n_byte_classes},
+                    "trie_nodes": info.trie_nodes, "trie_depth": info.trie_depth, "byte_classes": info.n_byte_classes,
+                    "automata": info.n_automata, "automaton_states": info.n_automaton_states},
     }
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(w, W, budget_s=args.cpu_seconds)
